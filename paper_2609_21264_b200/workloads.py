@@ -1,0 +1,128 @@
+"""Seeded synthetic workloads shared by the tests, the benchmark and the smoke check.
+
+This module holds the workload shapes and the input generator only -- none of
+the attention arithmetic.  It depends on numpy alone, so both the CPU oracle's
+tests and the CUDA path's tests can draw identical inputs from it.
+
+Inputs are i.i.d. Gaussian, as in the paper's numerical-stability protocol
+(Section 5.5: entries of Q, K, V drawn from N(0, sigma^2)), rounded to bf16 with
+round-to-nearest-even.  The bf16 *bit patterns* (uint16) are the inputs of
+record: the oracle widens them exactly and the GPU consumes them as they are.
+
+The shapes stand in for the paper's Table 6 (attention shapes of public LLM
+configurations, synthetic data); no dataset or trained weight is involved.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, replace
+
+import numpy as np
+
+DEFAULT_SEED = 20260921
+_TENSOR_ID = {"Q": 1, "K": 2, "V": 3}
+
+
+@dataclass(frozen=True)
+class Workload:
+    """One attention problem: shapes, mask mode, scale and input recipe."""
+    name: str
+    B: int
+    Hq: int
+    Hkv: int
+    Sq: int
+    Sk: int
+    dqk: int
+    dv: int
+    causal: bool
+    scale: float
+    sigma: float = 1.0
+    k_mult: float = 1.0   # K is multiplied by this (exact in bf16 for powers of two)
+    seed: int = DEFAULT_SEED
+
+    def shapes(self):
+        return ((self.B, self.Hq, self.Sq, self.dqk),
+                (self.B, self.Hkv, self.Sk, self.dqk),
+                (self.B, self.Hkv, self.Sk, self.dv),
+                (self.B, self.Hq, self.Sq, self.dv))
+
+    def with_(self, **kw) -> "Workload":
+        return replace(self, **kw)
+
+
+def _w(name, B, Hq, Hkv, S, dqk, dv, causal, k_mult=1.0, idx=0):
+    return Workload(name, B, Hq, Hkv, S, S, dqk, dv, causal, 1.0 / math.sqrt(dqk),
+                    1.0, k_mult, DEFAULT_SEED + idx)
+
+
+# The five benchmark configurations (index = position in the baseline's list).
+CONFIGS = (
+    _w("bert_base_mha_s512", 1, 12, 12, 512, 64, 64, False, idx=0),
+    _w("llama3_8b_gqa_s2048", 1, 32, 8, 2048, 128, 128, True, idx=1),
+    _w("llama2_7b_mha_b4_s8192", 4, 32, 32, 8192, 128, 128, True, k_mult=2.0, idx=2),
+    _w("deepseek_v2_mha_s4096_d192_128", 1, 128, 128, 4096, 192, 128, True, idx=3),
+    _w("long_context_gqa_s131072", 1, 32, 8, 131072, 128, 128, True, idx=4),
+)
+
+
+def config(index_or_name) -> Workload:
+    if isinstance(index_or_name, int):
+        return CONFIGS[index_or_name]
+    for c in CONFIGS:
+        if c.name == index_or_name:
+            return c
+    raise KeyError(index_or_name)
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 to bf16 (nearest, ties to even); returns uint16 bit patterns."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    rounded = u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))
+    return (rounded >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f64(h: np.ndarray) -> np.ndarray:
+    """Exact widening of bf16 bit patterns to float64."""
+    w = (np.ascontiguousarray(h, dtype=np.uint16).astype(np.uint32) << np.uint32(16))
+    return w.view(np.float32).astype(np.float64)
+
+
+def gaussian_bf16(shape, seed: int, tensor: str, sigma: float = 1.0, mult: float = 1.0) -> np.ndarray:
+    """bf16 bit patterns of mult * bf16(sigma * N(0,1)), counter-based (Philox) per (seed, tensor)."""
+    key = np.array([np.uint64(seed), np.uint64(_TENSOR_ID[tensor])], dtype=np.uint64)
+    gen = np.random.Generator(np.random.Philox(key=key))
+    x = gen.standard_normal(size=shape, dtype=np.float32)
+    if sigma != 1.0:
+        x *= np.float32(sigma)
+    bits = f32_to_bf16_bits(x)
+    if mult != 1.0:
+        # multiply the already rounded values; exact when mult is a power of two
+        y = (bits.astype(np.uint32) << np.uint32(16)).view(np.float32) * np.float32(mult)
+        bits = f32_to_bf16_bits(y)
+    return bits
+
+
+def make_inputs(w: Workload):
+    """(Q, K, V) as uint16 arrays of bf16 bit patterns with the workload's shapes."""
+    qs, ks, vs, _ = w.shapes()
+    Q = gaussian_bf16(qs, w.seed, "Q", w.sigma)
+    K = gaussian_bf16(ks, w.seed, "K", w.sigma, w.k_mult)
+    V = gaussian_bf16(vs, w.seed, "V", w.sigma)
+    return Q, K, V
+
+
+def sample_rows(w: Workload, n_random: int, seed: int = 0, heads=None) -> np.ndarray:
+    """(b, hq, i) triples: tile-boundary rows plus random rows, for sampled checks."""
+    rng = np.random.default_rng(seed)
+    fixed = [0, 1, 127, 128, 129, w.Sq // 2 - 1, w.Sq // 2, w.Sq - 1]
+    fixed = sorted({i for i in fixed if 0 <= i < w.Sq})
+    hs = list(range(w.Hq)) if heads is None else list(heads)
+    rows = []
+    for b in range(w.B):
+        for h in hs:
+            for i in fixed:
+                rows.append((b, h, i))
+    for _ in range(n_random):
+        rows.append((int(rng.integers(w.B)), int(hs[int(rng.integers(len(hs)))]),
+                     int(rng.integers(w.Sq))))
+    return np.asarray(rows, dtype=np.int64)

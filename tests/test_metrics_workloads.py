@@ -1,0 +1,77 @@
+"""Host logic: the throughput metric's convention, work/traffic counts, input generator."""
+import json
+import os
+
+import numpy as np
+
+from paper_2609_21264_b200 import metrics as M
+from paper_2609_21264_b200 import workloads as W
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def test_metric_convention_matches_the_paper_tables():
+    g = json.load(open(os.path.join(GOLDEN, "paper_throughput.json")))
+    for r in g["rows"]:
+        f = M.flops_paper(1, r["H"], r["S"], r["S"], r["d"], r["d"])
+        gflops = M.tflops_gemm(f, r["seconds"]) * 1e3
+        assert abs(gflops / r["gflops"] - 1.0) < r["rel_tol"], r
+
+
+def test_visible_pairs_against_enumeration():
+    for Sq in range(1, 9):
+        for Sk in range(1, 9):
+            full = sum(1 for i in range(Sq) for j in range(Sk))
+            caus = sum(1 for i in range(Sq) for j in range(Sk) if j <= i + Sk - Sq)
+            assert M.visible_pairs(Sq, Sk, False) == full
+            assert M.visible_pairs(Sq, Sk, True) == caus, (Sq, Sk)
+
+
+def test_work_and_traffic_of_the_five_configs():
+    # figures of the hot-path scope table
+    exp = [(8.053e8, 8.053e8, 3.17e6), (6.872e10, 3.438e10, 42.2e6), (4.398e12, 2.1993e12, 1.078e9),
+           (1.3744e12, 6.874e11, 673e6), (2.8147e14, 1.4074e14, 2.70e9)]
+    for c, (fp, fa, by) in zip(W.CONFIGS, exp):
+        assert abs(M.flops_paper(c.B, c.Hq, c.Sq, c.Sk, c.dqk, c.dv) / fp - 1) < 1e-3
+        assert abs(M.flops_algorithmic(c.B, c.Hq, c.Sq, c.Sk, c.dqk, c.dv, c.causal) / fa - 1) < 1e-3
+        assert abs(M.bytes_compulsory(c.B, c.Hq, c.Hkv, c.Sq, c.Sk, c.dqk, c.dv) / by - 1) < 2e-3
+
+
+def test_roofline_picks_the_slower_side():
+    t, bound = M.roofline_seconds(10**12, 10**6, 1000.0, 1000.0)
+    assert bound == "tensor" and abs(t - 1e-3) < 1e-12
+    t, bound = M.roofline_seconds(10**6, 10**9, 1000.0, 1000.0)
+    assert bound == "hbm" and abs(t - 1e-3) < 1e-12
+
+
+def test_bf16_rounding_is_nearest_even():
+    import torch
+    x = np.random.default_rng(0).standard_normal(100000).astype(np.float32) * 3
+    x[:4] = [1.00390625, 1.01171875, -1.00390625, 0.0]   # exact ties: to even
+    bits = W.f32_to_bf16_bits(x)
+    ref = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(bits, ref)
+    back = W.bf16_bits_to_f64(bits)
+    np.testing.assert_array_equal(back, torch.from_numpy(x).to(torch.bfloat16).double().numpy())
+
+
+def test_generator_is_seeded_and_shaped():
+    w = W.config(0)
+    Q, K, V = W.make_inputs(w)
+    Q2, K2, V2 = W.make_inputs(w)
+    assert Q.dtype == np.uint16 and Q.shape == (1, 12, 512, 64) and V.shape == (1, 12, 512, 64)
+    np.testing.assert_array_equal(Q, Q2)
+    assert not np.array_equal(Q, K) and not np.array_equal(K, V)
+    q = W.bf16_bits_to_f64(Q)
+    assert abs(q.mean()) < 0.01 and abs(q.std() - 1.0) < 0.01
+    w3 = W.config(2).with_(B=1, Hq=2, Hkv=2, Sq=256, Sk=256)
+    _, K3, _ = W.make_inputs(w3)
+    assert abs(W.bf16_bits_to_f64(K3).std() - 2.0) < 0.02      # K scaled by 2
+    assert W.make_inputs(w.with_(seed=7))[0].tobytes() != Q.tobytes()
+
+
+def test_sample_rows_are_in_range():
+    w = W.config(4)
+    rows = W.sample_rows(w, 32, seed=1, heads=[0, 31])
+    assert rows.shape[1] == 3 and (rows[:, 2] < w.Sq).all() and (rows[:, 1] < w.Hq).all()
+    assert {0, 127, 128, w.Sq - 1} <= set(rows[:, 2].tolist())
