@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the fused attention forward pass on B200 (one JSON line on stdout).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config IDX] [--impl reference]
+
+A step is one pass of the whole hot path (one `fa_forward` launch) over one
+batch of the workload.  `value` is effective-GEMM throughput (Section 5.1 of the
+paper: 2*H*Lq*Lk*(dk+dv)/T) counted over VISIBLE (query, key) pairs only; the
+paper's own convention (full Lq*Lk rectangle even when causal) is reported as
+`value_paper_convention`.  Inputs are synthetic Gaussians already resident in
+HBM; several input sets are rotated so that the footprint between two uses of
+the same set exceeds L2.  `e2e` is the same metric through `fa_forward_host`
+with pinned host buffers (copies inside the timed region).
+
+`--impl reference` times the fp64 CPU oracle instead (a deliberately slow
+program; parity and the roofline fraction are the headline, not that ratio).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_21264_b200 import launch, metrics, workloads  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+# Paper, Table 6: Llama-3 8B shape (32/8 heads, d=128, causal, S=2048) on XDNA 2: 34076 us.
+PAPER_SECONDS = {"llama3_8b_gqa_s2048": 34076e-6}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (None = not captured for that workload).
+NCU_DRAM_BYTES_PER_LAUNCH = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self.error = None
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {
+                getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+                getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+                getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+                getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            }
+            get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
+            while not self._stop.is_set():
+                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                mask = get_reasons(h)
+                for bit, name in names.items():
+                    if bit and (mask & bit):
+                        self.reasons.add(name)
+                time.sleep(self.period)
+        except Exception as ex:  # pragma: no cover
+            self.error = repr(ex)
+
+    def stop(self):
+        self._stop.set()
+        self.join(timeout=2.0)
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s),
+                **({"error": self.error} if self.error else {})}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+def make_device_sets(w, n_sets, device):
+    """n_sets independent (Q, K, V, O, lse) sets of synthetic bf16 Gaussians on the device."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(w.seed)
+    qs, ks, vs, os_ = w.shapes()
+    sets = []
+    for _ in range(n_sets):
+        q = (torch.randn(qs, generator=g, device=device, dtype=torch.float32) * w.sigma).to(torch.bfloat16)
+        k = (torch.randn(ks, generator=g, device=device, dtype=torch.float32) * w.sigma).to(torch.bfloat16)
+        if w.k_mult != 1.0:
+            k = k * w.k_mult
+        v = (torch.randn(vs, generator=g, device=device, dtype=torch.float32) * w.sigma).to(torch.bfloat16)
+        o = torch.empty(os_, device=device, dtype=torch.bfloat16)
+        lse = torch.empty(os_[:3], device=device, dtype=torch.float32)
+        sets.append((q.contiguous(), k.contiguous(), v.contiguous(), o, lse))
+    return sets
+
+
+def workload_numbers(w):
+    fl_alg = metrics.flops_algorithmic(w.B, w.Hq, w.Sq, w.Sk, w.dqk, w.dv, w.causal)
+    fl_pap = metrics.flops_paper(w.B, w.Hq, w.Sq, w.Sk, w.dqk, w.dv)
+    nbytes = metrics.bytes_compulsory(w.B, w.Hq, w.Hkv, w.Sq, w.Sk, w.dqk, w.dv)
+    return fl_alg, fl_pap, nbytes
+
+
+def n_sets_for(w):
+    _, _, nbytes = workload_numbers(w)
+    return max(2, min(16, -(-2 * L2_BYTES // nbytes))) if nbytes < 2 * L2_BYTES else 1
+
+
+def run_device_timed(binding, h, w, sets, steps, warmup, world):
+    """Time `steps` launches (after `warmup`) with CUDA events on the launching stream; seconds."""
+    import torch
+    stream = torch.cuda.current_stream()
+
+    def one(i):
+        q, k, v, o, lse = sets[i % len(sets)]
+        st = binding.fa_forward(h, q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(),
+                                w.B, w.Hq, w.Hkv, w.Sq, w.Sk, w.dqk, w.dv, w.causal, w.scale,
+                                stream.cuda_stream)
+        if st != binding.FA_OK:
+            raise binding.FaError(st, "fa_forward")
+
+    for i in range(warmup):
+        one(i)
+    torch.cuda.synchronize()
+    launch.barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = binding.fa_launch_count(h)
+    e0.record(stream)
+    for i in range(steps):
+        one(warmup + i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    launch.barrier(world)
+    st, detail = binding.fa_last_status(h)
+    if st != binding.FA_OK:
+        raise binding.FaError(st, "device status (site 0x%x)" % detail)
+    return e0.elapsed_time(e1) * 1e-3, binding.fa_launch_count(h) - n0
+
+
+def run_e2e_timed(binding, h, w, steps, warmup, world):
+    """Same metric through fa_forward_host: pinned host buffers, copies inside the timed region."""
+    import numpy as np
+    import torch
+    Q, K, V = workloads.make_inputs(w)
+    pin = [torch.from_numpy(a.view(np.int16)).pin_memory() for a in (Q, K, V)]
+    o = torch.empty(w.shapes()[3], dtype=torch.int16).pin_memory()
+    lse = torch.empty(w.shapes()[3][:3], dtype=torch.float32).pin_memory()
+    stream = torch.cuda.current_stream()
+
+    def one():
+        st = binding.fa_forward_host(h, pin[0].data_ptr(), pin[1].data_ptr(), pin[2].data_ptr(), o.data_ptr(),
+                                     lse.data_ptr(), w.B, w.Hq, w.Hkv, w.Sq, w.Sk, w.dqk, w.dv, w.causal,
+                                     w.scale, stream.cuda_stream)
+        if st != binding.FA_OK:
+            raise binding.FaError(st, "fa_forward_host")
+
+    for _ in range(max(1, warmup)):
+        one()
+    torch.cuda.synchronize()
+    launch.barrier(world)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()                       # synchronises the stream itself before returning
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    launch.barrier(world)
+    h2d = sum(int(t.numel()) * t.element_size() for t in pin)
+    d2h = int(o.numel()) * 2 + int(lse.numel()) * 4
+    return dt, h2d, d2h, float(lse.double().mean())
+
+
+def oracle_timed(w, budget_s=20.0):
+    """The fp64 oracle on the host cores over a bounded sample of query rows of the workload."""
+    import numpy as np
+    import oracle
+    Q, K, V = workloads.make_inputs(w)
+    rng = np.random.default_rng(0)
+    threads = oracle.num_threads()
+
+    def rows_sample(n):
+        return np.stack([rng.integers(w.B, size=n), rng.integers(w.Hq, size=n), rng.integers(w.Sq, size=n)],
+                        axis=1).astype(np.int64)
+
+    def pairs_of(rows):
+        i = rows[:, 2]
+        vis = np.minimum(w.Sk, np.maximum(0, i + (w.Sk - w.Sq) + 1)) if w.causal else np.full(len(i), w.Sk)
+        return int(vis.sum())
+
+    probe = rows_sample(64 * threads)
+    t0 = time.perf_counter()
+    oracle.attention(Q, K, V, causal=w.causal, scale=w.scale, rows=probe)
+    dt = time.perf_counter() - t0
+    rate = pairs_of(probe) / max(dt, 1e-6)                   # visible pairs per second
+    total_pairs = w.B * w.Hq * metrics.visible_pairs(w.Sq, w.Sk, w.causal)
+    if total_pairs / rate <= budget_s:
+        t0 = time.perf_counter()
+        oracle.attention(Q, K, V, causal=w.causal, scale=w.scale)
+        dt = time.perf_counter() - t0
+        pairs, sample = total_pairs, "whole workload (%d rows)" % (w.B * w.Hq * w.Sq)
+    else:
+        n = max(threads, int(budget_s * rate / (total_pairs / (w.B * w.Hq * w.Sq))))
+        rows = rows_sample(n)
+        t0 = time.perf_counter()
+        oracle.attention(Q, K, V, causal=w.causal, scale=w.scale, rows=rows)
+        dt = time.perf_counter() - t0
+        pairs, sample = pairs_of(rows), "%d random query rows of the workload" % n
+    flops = 2 * pairs * (w.dqk + w.dv)
+    return {"value": flops / dt / 1e12, "unit": "TFLOP_GEMM/s", "cores": threads, "kind": "oracle",
+            "sample": sample, "seconds": dt}
+
+
+def config_dict(w, extra=None):
+    d = {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "Sq": w.Sq, "Sk": w.Sk, "dqk": w.dqk,
+         "dv": w.dv, "causal": w.causal, "scale": w.scale, "inputs": "bf16 N(0,1), seeded",
+         "flop_convention": "value counts visible (i,j) pairs only; value_paper_convention counts Sq*Sk"}
+    if extra:
+        d.update(extra)
+    return d
+
+
+def run_reference(args, w, rank, world):
+    """Reference arm: the CPU oracle, rank 0 only."""
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    Q, K, V = workloads.make_inputs(w)
+    threads = oracle.num_threads()
+    rows_total = w.B * w.Hq * w.Sq
+    rng = np.random.default_rng(0)
+    # size one step so that steps+warmup steps end within ~2 minutes
+    probe = np.stack([rng.integers(w.B, size=256), rng.integers(w.Hq, size=256), rng.integers(w.Sq, size=256)],
+                     axis=1).astype(np.int64)
+    t0 = time.perf_counter()
+    oracle.attention(Q, K, V, causal=w.causal, scale=w.scale, rows=probe)
+    per_row = (time.perf_counter() - t0) / 256
+    budget_per_step = 120.0 / max(1, args.steps + args.warmup)
+    n = int(min(rows_total, max(threads, budget_per_step / per_row)))
+    whole = n >= rows_total
+    rows = None if whole else np.stack([rng.integers(w.B, size=n), rng.integers(w.Hq, size=n),
+                                        rng.integers(w.Sq, size=n)], axis=1).astype(np.int64)
+    if whole:
+        pairs = w.B * w.Hq * metrics.visible_pairs(w.Sq, w.Sk, w.causal)
+    else:
+        i = rows[:, 2]
+        pairs = int((np.minimum(w.Sk, np.maximum(0, i + (w.Sk - w.Sq) + 1)) if w.causal
+                     else np.full(n, w.Sk)).sum())
+    for _ in range(args.warmup):
+        oracle.attention(Q, K, V, causal=w.causal, scale=w.scale, rows=rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.attention(Q, K, V, causal=w.causal, scale=w.scale, rows=rows)
+    dt = time.perf_counter() - t0
+    value = 2 * pairs * (w.dqk + w.dv) * args.steps / dt / 1e12
+    sample = "whole workload" if whole else "%d random query rows per step" % n
+    line = {"impl": "reference", "metric": "attention_fwd_tflop_gemm_per_s", "value": value,
+            "unit": "TFLOP_GEMM/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(w),
+            "cpu_baseline": {"value": value, "unit": "TFLOP_GEMM/s", "cores": threads, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "TFLOP_GEMM/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--config", type=int, default=1, help="index into the five benchmark configurations")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the short timing of the other configs")
+    args = ap.parse_args()
+    w = workloads.config(args.config)
+
+    if args.impl == "reference":
+        rank, world, _ = launch.env_rank()
+        args.steps = args.steps if args.steps is not None else 3
+        args.warmup = args.warmup if args.warmup is not None else 1
+        run_reference(args, w, rank, world)
+        return
+
+    import torch
+    from paper_2609_21264_b200 import binding
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    rank, world, local = launch.init_process_group("nccl")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world != args.gpus and rank == 0:
+        print("warning: --gpus %d but WORLD_SIZE=%d" % (args.gpus, world), file=sys.stderr)
+
+    fl_alg, fl_pap, nbytes = workload_numbers(w)
+    default_steps = max(20, min(2000, int(0.25 / max(fl_alg / 1.0e15, 1e-5))))
+    steps = args.steps if args.steps is not None else default_steps
+    warmup = args.warmup if args.warmup is not None else max(3, min(50, steps // 10))
+    warmup = max(3, warmup)
+
+    h = binding.fa_create(device=local)
+    n_sets = n_sets_for(w)
+    sets = make_device_sets(w, n_sets, device)
+
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    seconds, launches = run_device_timed(binding, h, w, sets, steps, warmup, world)
+    clocks = sampler.stop()
+    seconds = launch.max_over_ranks(seconds, world, device)
+    t_step = seconds / steps
+
+    peaks = load_peaks()
+    long_step = t_step > 5e-3
+    peak_tf = peaks["bf16_tflops_sustained"] if long_step else peaks["bf16_tflops"]
+    t_roof, bound = metrics.roofline_seconds(fl_alg, nbytes, peak_tf, peaks["hbm_gbs"])
+    if bound == "tensor":
+        achieved, peak, unit = fl_alg / t_step / 1e12, peak_tf, "TFLOP/s"
+    else:
+        achieved, peak, unit = nbytes / t_step / 1e9, peaks["hbm_gbs"], "GB/s"
+    roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+                "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(w.name),
+                "peak_source": "%s (%s)" % (peaks["source"], "sustained" if long_step else "burst"),
+                "kernel": binding.fa_last_kernel_name(h), "algorithmic_flops_per_launch": fl_alg,
+                "compulsory_bytes_per_launch": nbytes, "avg_launch_us": t_step * 1e6,
+                "t_roof_us": t_roof * 1e6,
+                "frac_of_nominal_2250_tflops": fl_alg / t_step / 2.25e15}
+
+    value = world * fl_alg / t_step / 1e12
+    line = {"metric": "attention_fwd_tflop_gemm_per_s", "value": value, "unit": "TFLOP_GEMM/s",
+            "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": t_step * 1e3,
+            "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": (PAPER_SECONDS[w.name] / t_step if (w.name in PAPER_SECONDS and world == 1) else None),
+            "dtype": "bf16", "data": "synthetic",
+            "config": config_dict(w, {"l2": "rotating %d input sets (%.0f MB in total, L2 is 126 MB)"
+                                      % (n_sets, n_sets * nbytes / 1e6) if n_sets > 1 else
+                                      "one input set of %.0f MB (larger than the 126 MB L2)" % (nbytes / 1e6),
+                                      "parallelism": "replicas x%d, no collective" % world}),
+            "value_paper_convention": world * fl_pap / t_step / 1e12,
+            "paper_context": "3.62 TFLOP_GEMM/s on XDNA 2 (paper's headline, other hardware and shape)",
+            "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches)}
+
+    if not args.no_e2e:
+        e2e_steps = max(3, min(steps, 50))
+        dt, h2d, d2h, _ = run_e2e_timed(binding, h, w, e2e_steps, 3, world)
+        dt = launch.max_over_ranks(dt, world, device)
+        line["e2e"] = {"value": world * fl_alg * e2e_steps / dt / 1e12, "unit": "TFLOP_GEMM/s",
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                       "ms_per_step": dt / e2e_steps * 1e3}
+
+    if not args.no_sweep and world == 1:
+        per = []
+        del sets
+        torch.cuda.empty_cache()
+        for idx, wc in enumerate(workloads.CONFIGS):
+            fa, fp, nb = workload_numbers(wc)
+            ss = make_device_sets(wc, n_sets_for(wc), device)
+            k = max(5, min(200, int(0.3 / max(fa / 1.0e15, 1e-5))))
+            sec, _ = run_device_timed(binding, h, wc, ss, k, 3, 1)
+            t = sec / k
+            pk = peaks["bf16_tflops_sustained"] if t > 5e-3 else peaks["bf16_tflops"]
+            tr, bd = metrics.roofline_seconds(fa, nb, pk, peaks["hbm_gbs"])
+            per.append({"config": idx, "workload": wc.name, "us": t * 1e6, "tflops_algorithmic": fa / t / 1e12,
+                        "tflops_paper_convention": fp / t / 1e12, "bound": bd, "roofline_frac": tr / t,
+                        "frac_of_nominal_2250": fa / t / 2.25e15, "steps": k})
+            del ss
+            torch.cuda.empty_cache()
+        line["per_config"] = per
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = oracle_timed(w)
+
+    binding.fa_destroy(h)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    launch.destroy(world)
+
+
+if __name__ == "__main__":
+    main()

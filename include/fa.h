@@ -1,0 +1,144 @@
+/*
+ * fa.h -- C ABI of the B200 (sm_100a) fused attention forward library.
+ *
+ * The library computes, for every batch b, query head hq and query row i,
+ *
+ *     O[b,hq,i,:] = softmax_j( scale * <Q[b,hq,i,:], K[b,kvh,j,:]> ) . V[b,kvh,:,:]
+ *     lse[b,hq,i] = ln sum_j exp( scale * <Q[b,hq,i,:], K[b,kvh,j,:]> )
+ *
+ * which is Eq. 1 of the paper (scaled dot-product attention, Section 2.1)
+ * replicated over heads, evaluated by the fused online-softmax recurrence of
+ * Algorithm 1 (running row maximum u, running row sum s, unnormalised
+ * accumulator G', one division at the end), so that the Sq x Sk score matrix
+ * never leaves the SM.  `causal` selects the mask step of Algorithm 1: key j is
+ * visible to query i iff j <= i + (Sk - Sq) (for Sq == Sk: a token sees itself
+ * and its predecessors).  Grouped-query attention (Section 4.4): query head hq
+ * reads kv head kvh = hq / (Hq / Hkv).  Data are bfloat16 as in the paper's
+ * evaluation (Section 5.1); scores, the softmax state and both accumulators
+ * are fp32.  lse is not a paper output: it carries the (u, s) pair that
+ * Algorithm 1 returns, as u + ln s, in natural-log units of the scaled scores.
+ *
+ * Layouts (row-major, contiguous, no padding):
+ *     Q   [B, Hq,  Sq, dqk]  bf16        K [B, Hkv, Sk, dqk] bf16
+ *     V   [B, Hkv, Sk, dv ]  bf16        O [B, Hq,  Sq, dv ] bf16
+ *     lse [B, Hq,  Sq]       fp32
+ * Rows with no visible key (possible only when causal and Sq > Sk) get
+ * O = 0 and lse = -inf.
+ *
+ * Supported head sizes: (dqk, dv) in {(64,64), (128,128), (192,128)}.
+ *
+ * Threading: a handle must not be used from two host threads at once.
+ * All functions return a status code; nothing throws, aborts or prints.
+ */
+#ifndef FA_B200_H_
+#define FA_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fa_handle fa_handle; /* opaque; created by fa_create, freed by fa_destroy */
+
+typedef enum fa_status {
+    FA_OK = 0,
+    FA_ERR_INVALID_ARG = 1,    /* NULL/misaligned pointer, non-positive size, Hq % Hkv != 0, bad scale */
+    FA_ERR_UNSUPPORTED = 2,    /* head sizes or extents the kernels do not cover                     */
+    FA_ERR_CUDA = 3,           /* a CUDA runtime/driver call failed (launch, copy, allocation)       */
+    FA_ERR_DEVICE_TIMEOUT = 4, /* a bounded device-side wait ran out; the results are invalid        */
+    FA_ERR_NO_DEVICE = 5,      /* no CUDA device, or the device is not compute capability 10.x       */
+    FA_ERR_OOM = 6             /* host or device allocation failed                                   */
+} fa_status;
+
+/* fa_config.flags: run the serialised cross-check kernel (one tile in flight, no overlap
+ * between loads, MMAs and softmax) instead of the pipelined one.  Same results up to
+ * rounding order; much slower.  Meant for tests. */
+#define FA_FLAG_SERIAL_KERNEL 1u
+
+/* Optional creation parameters.  Zero-initialise, set struct_size = sizeof(fa_config). */
+typedef struct fa_config {
+    uint32_t struct_size;     /* sizeof(fa_config) of the caller's header                      */
+    int32_t device;           /* CUDA device ordinal; -1 = the calling thread's current device */
+    uint32_t flags;           /* bitwise OR of FA_FLAG_*; other bits must be 0                 */
+    uint32_t wait_limit_ms;   /* limit of every device-side wait; 0 = default (2000 ms)        */
+} fa_config;
+
+/*
+ * Create a handle bound to one device.  `cfg` may be NULL (defaults, current
+ * device).  The handle owns a small status word (pinned host memory mapped to
+ * the device), a cache of TMA tensor maps keyed by (pointer, shape), and the
+ * staging buffers of fa_forward_host.  Allocates; call outside stream capture.
+ */
+fa_status fa_create(fa_handle** out, const fa_config* cfg);
+
+/*
+ * Fused attention forward (Eq. 1 evaluated by Algorithm 1; causal mask,
+ * GQA head sharing and lse as described at the top of this file).
+ *
+ *   Q, K, V  device pointers to bf16, 16-byte aligned, layouts as above; read only.
+ *   O        device pointer to bf16, 16-byte aligned; every element is overwritten.
+ *   lse      device pointer to fp32, 4-byte aligned, or NULL to skip it.
+ *   B, Hq, Hkv, Sq, Sk, dqk, dv   extents; all > 0; Hq % Hkv == 0.  Sq and Sk need
+ *            not be multiples of the 128-row tile.
+ *   causal   0 = every key visible; non-zero = key j visible iff j <= i + (Sk - Sq).
+ *   scale    multiplier of the dot products; 0.0f selects 1/sqrt(dqk) (Eq. 1).
+ *            Must be finite and >= 0.
+ *   stream   a cudaStream_t (NULL = the legacy default stream) of the handle's device.
+ *
+ * The call is asynchronous: it validates, enqueues the kernel on `stream` and
+ * returns.  The caller owns all buffers and keeps them alive until the stream
+ * has passed the kernel; O must not alias an input.  The library does not
+ * synchronise and does not allocate device memory here.  Argument and launch
+ * errors are returned at once; a device-side timeout shows up in
+ * fa_last_status after the caller has synchronised the stream.
+ */
+fa_status fa_forward(fa_handle* h,
+                     const void* Q, const void* K, const void* V,
+                     void* O, float* lse,
+                     int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv,
+                     int causal, float scale, void* stream);
+
+/*
+ * The same operation with HOST buffers (same layouts and types): copies Q, K, V
+ * to staging memory owned by the handle, runs fa_forward, copies O (and lse if
+ * not NULL) back, all on `stream`, and synchronises `stream` before returning.
+ * Pinned host buffers give the full copy bandwidth; pageable ones work.  The
+ * staging buffers grow on demand (device allocation on the first call and
+ * whenever a larger problem arrives) and are freed by fa_destroy.
+ */
+fa_status fa_forward_host(fa_handle* h,
+                          const void* Q_host, const void* K_host, const void* V_host,
+                          void* O_host, float* lse_host,
+                          int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv,
+                          int causal, float scale, void* stream);
+
+/*
+ * Device-side status of the kernels launched through `h` so far: FA_OK, or
+ * FA_ERR_DEVICE_TIMEOUT if any bounded wait (mbarrier, TMEM allocation) ran
+ * out since the handle was created or the status was last read (reading
+ * clears it).  Synchronises nothing: meaningful after the caller has
+ * synchronised the stream(s) it launched on.  `detail`, if not NULL, receives
+ * a diagnostic word (role and barrier that gave up; 0 when FA_OK).
+ */
+fa_status fa_last_status(fa_handle* h, uint32_t* detail);
+
+/* Free everything the handle owns.  fa_destroy(NULL) returns FA_OK. */
+fa_status fa_destroy(fa_handle* h);
+
+/* Static, NUL-terminated description of a status code. */
+const char* fa_strerror(fa_status s);
+
+/*
+ * Introspection used by tests and the benchmark: number of kernel launches
+ * issued through the handle so far, and the name of the kernel variant the
+ * last fa_forward selected (static string; "" before the first call).
+ */
+uint64_t fa_launch_count(const fa_handle* h);
+const char* fa_last_kernel_name(const fa_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FA_B200_H_ */

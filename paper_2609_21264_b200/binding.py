@@ -1,0 +1,142 @@
+"""ctypes binding of the C ABI in ``include/fa.h`` -- argument marshalling only.
+
+Function names and argument order follow the header.  Pointers are plain
+integers (``tensor.data_ptr()``, ``stream.cuda_stream``); `forward` is a small
+convenience that takes torch tensors, allocates O and lse with torch (device
+memory plumbing) and calls `fa_forward`.  There is no fallback: if the library
+is missing or the call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+from . import build as _build
+
+FA_OK = 0
+FA_ERR_INVALID_ARG = 1
+FA_ERR_UNSUPPORTED = 2
+FA_ERR_CUDA = 3
+FA_ERR_DEVICE_TIMEOUT = 4
+FA_ERR_NO_DEVICE = 5
+FA_ERR_OOM = 6
+FA_FLAG_SERIAL_KERNEL = 1
+
+EXPORTS = ("fa_create", "fa_forward", "fa_forward_host", "fa_last_status", "fa_destroy",
+           "fa_strerror", "fa_launch_count", "fa_last_kernel_name")
+
+
+class FaError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__("%s: %s (status %d)" % (what, fa_strerror(status), status))
+        self.status = status
+
+
+class fa_config(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("device", ctypes.c_int32),
+                ("flags", ctypes.c_uint32), ("wait_limit_ms", ctypes.c_uint32)]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB_PATH
+
+
+def load():
+    """Load libfa_b200.so (built in-tree by ``build.build()``); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise ImportError("CUDA library %s is missing; run `python -m paper_2609_21264_b200.build` "
+                          "(there is no CPU fallback)" % path)
+    lib = ctypes.CDLL(path)
+    vp, i32, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    lib.fa_create.restype = i32
+    lib.fa_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(fa_config)]
+    fwd_args = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, f32, vp]
+    lib.fa_forward.restype = i32
+    lib.fa_forward.argtypes = fwd_args
+    lib.fa_forward_host.restype = i32
+    lib.fa_forward_host.argtypes = fwd_args
+    lib.fa_last_status.restype = i32
+    lib.fa_last_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.fa_destroy.restype = i32
+    lib.fa_destroy.argtypes = [vp]
+    lib.fa_strerror.restype = ctypes.c_char_p
+    lib.fa_strerror.argtypes = [i32]
+    lib.fa_launch_count.restype = ctypes.c_uint64
+    lib.fa_launch_count.argtypes = [vp]
+    lib.fa_last_kernel_name.restype = ctypes.c_char_p
+    lib.fa_last_kernel_name.argtypes = [vp]
+    _lib = lib
+    return lib
+
+
+def fa_strerror(status: int) -> str:
+    return load().fa_strerror(int(status)).decode()
+
+
+def fa_create(device: int = -1, flags: int = 0, wait_limit_ms: int = 0) -> int:
+    """Returns an opaque handle (integer address).  Raises FaError on failure."""
+    cfg = fa_config(ctypes.sizeof(fa_config), device, flags, wait_limit_ms)
+    out = ctypes.c_void_p()
+    st = load().fa_create(ctypes.byref(out), ctypes.byref(cfg))
+    if st != FA_OK:
+        raise FaError(st, "fa_create")
+    return out.value
+
+
+def fa_forward(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, stream=0) -> int:
+    """Raw call with device pointers as integers; returns the status code."""
+    return load().fa_forward(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv,
+                             int(bool(causal)), float(scale), stream)
+
+
+def fa_forward_host(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, stream=0) -> int:
+    """Raw call with HOST pointers as integers; returns the status code."""
+    return load().fa_forward_host(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv,
+                                  int(bool(causal)), float(scale), stream)
+
+
+def fa_last_status(h):
+    """(status, detail) of the device-side status word; clears it."""
+    detail = ctypes.c_uint32(0)
+    st = load().fa_last_status(h, ctypes.byref(detail))
+    return st, detail.value
+
+
+def fa_destroy(h) -> int:
+    return load().fa_destroy(h)
+
+
+def fa_launch_count(h) -> int:
+    return int(load().fa_launch_count(h))
+
+
+def fa_last_kernel_name(h) -> str:
+    return load().fa_last_kernel_name(h).decode()
+
+
+def forward(h, q, k, v, *, causal: bool, scale: float = 0.0, out=None, lse=None, want_lse=True):
+    """Attention forward on torch CUDA tensors (bf16, contiguous, [B,H,S,d]); returns (O, lse)."""
+    import torch
+    for t in (q, k, v):
+        if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or t.dim() != 4:
+            raise ValueError("q, k, v must be contiguous 4-D bf16 CUDA tensors")
+    B, Hq, Sq, dqk = q.shape
+    _, Hkv, Sk, dv = v.shape
+    if out is None:
+        out = torch.empty((B, Hq, Sq, dv), dtype=torch.bfloat16, device=q.device)
+    if lse is None and want_lse:
+        lse = torch.empty((B, Hq, Sq), dtype=torch.float32, device=q.device)
+    stream = torch.cuda.current_stream(q.device).cuda_stream
+    st = fa_forward(h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                    lse.data_ptr() if lse is not None else None,
+                    B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, stream)
+    if st != FA_OK:
+        raise FaError(st, "fa_forward")
+    return out, lse

@@ -1,0 +1,327 @@
+// Host side of the C ABI declared in include/fa.h: argument checks, TMA tensor
+// maps, kernel selection and launch.  No torch types, no CPU fallback.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/fa.h"
+#include "fa_common.cuh"
+#include "fa_fwd_simple.cuh"
+
+namespace {
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                   const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct MapEntry {
+    const void* ptr;
+    int d, S, BH, box_rows;
+    uint64_t stamp;
+    CUtensorMap map;
+};
+
+constexpr int kMapCacheSize = 16;
+
+}  // namespace
+
+struct fa_handle {
+    int device = 0;
+    uint32_t flags = 0;
+    uint32_t* status_host = nullptr;   // pinned + mapped: [0] status, [1] wait site
+    uint32_t* status_dev = nullptr;
+    unsigned long long wait_limit_ns = 2000ull * 1000000ull;
+    EncodeTiledFn encode = nullptr;
+    std::vector<MapEntry> maps;
+    uint64_t stamp = 0;
+    uint64_t launches = 0;
+    const char* last_kernel = "";
+    void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // Q K V O lse
+    size_t stage_cap[5] = {0, 0, 0, 0, 0};
+    bool attr_done[8] = {false, false, false, false, false, false, false, false};
+};
+
+namespace {
+
+class DeviceGuard {
+  public:
+    explicit DeviceGuard(int want) {
+        if (cudaGetDevice(&prev_) != cudaSuccess) prev_ = -1;
+        if (prev_ != want) { ok_ = (cudaSetDevice(want) == cudaSuccess); changed_ = ok_; }
+    }
+    ~DeviceGuard() { if (changed_ && prev_ >= 0) cudaSetDevice(prev_); }
+    bool ok() const { return ok_; }
+  private:
+    int prev_ = -1;
+    bool ok_ = true;
+    bool changed_ = false;
+};
+
+// bf16 tensor [BH, S, d] (row-major) seen as a 3-D TMA tensor (d, S, BH); box =
+// 64 columns x box_rows rows, 128-byte swizzle, out-of-range rows read as zero.
+fa_status get_map(fa_handle* h, const void* ptr, int d, int S, long long BH, int box_rows,
+                  const CUtensorMap** out) {
+    for (auto& e : h->maps) {
+        if (e.ptr == ptr && e.d == d && e.S == S && e.BH == BH && e.box_rows == box_rows) {
+            e.stamp = ++h->stamp;
+            *out = &e.map;
+            return FA_OK;
+        }
+    }
+    MapEntry ne;
+    memset(&ne, 0, sizeof ne);
+    ne.ptr = ptr; ne.d = d; ne.S = S; ne.BH = static_cast<int>(BH); ne.box_rows = box_rows;
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(S),
+                                static_cast<cuuint64_t>(BH)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2ull,
+                                   static_cast<cuuint64_t>(d) * 2ull * static_cast<cuuint64_t>(S)};
+    const cuuint32_t box[3] = {static_cast<cuuint32_t>(fa::kChunkCols),
+                               static_cast<cuuint32_t>(box_rows), 1u};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    const CUresult r = h->encode(&ne.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr),
+                                 dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return FA_ERR_CUDA;
+    ne.stamp = ++h->stamp;
+    if (static_cast<int>(h->maps.size()) < kMapCacheSize) {
+        h->maps.push_back(ne);
+        *out = &h->maps.back().map;
+    } else {
+        size_t victim = 0;
+        for (size_t i = 1; i < h->maps.size(); ++i)
+            if (h->maps[i].stamp < h->maps[victim].stamp) victim = i;
+        h->maps[victim] = ne;
+        *out = &h->maps[victim].map;
+    }
+    return FA_OK;
+}
+
+template <typename Kernel>
+fa_status ensure_smem_attr(fa_handle* h, int slot, Kernel kernel, int bytes) {
+    if (h->attr_done[slot]) return FA_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return FA_ERR_CUDA;
+    }
+    h->attr_done[slot] = true;
+    return FA_OK;
+}
+
+template <int DQK, int DV>
+fa_status launch_simple(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
+                        const CUtensorMap& mv, const fa::FwdParams& p, cudaStream_t st) {
+    using Cfg = fa::SimpleCfg<DQK, DV>;
+    // ask for more than half of the SM's shared memory so that one CTA owns the SM's TMEM
+    const int smem = Cfg::kSmemBytes > 120 * 1024 ? Cfg::kSmemBytes : 120 * 1024;
+    auto kernel = fa::fa_fwd_simple_kernel<DQK, DV>;
+    fa_status s = ensure_smem_attr(h, slot, kernel, smem);
+    if (s != FA_OK) return s;
+    dim3 grid(p.n_q_tiles, p.Hq, p.B);
+    kernel<<<grid, 128, smem, st>>>(mq, mk, mv, p);
+    if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
+    h->launches += 1;
+    return FA_OK;
+}
+
+bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
+
+fa_status check_args(const void* Q, const void* K, const void* V, const void* O, const float* lse,
+                     int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, float scale,
+                     bool device_ptrs) {
+    if (!Q || !K || !V || !O) return FA_ERR_INVALID_ARG;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || dqk <= 0 || dv <= 0)
+        return FA_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0) return FA_ERR_INVALID_ARG;
+    if (!isfinite(scale) || scale < 0.f) return FA_ERR_INVALID_ARG;
+    if (device_ptrs) {
+        if (misaligned(Q, 16) || misaligned(K, 16) || misaligned(V, 16) || misaligned(O, 16))
+            return FA_ERR_INVALID_ARG;
+        if (lse && misaligned(lse, 4)) return FA_ERR_INVALID_ARG;
+    }
+    const bool dims_ok = (dqk == 64 && dv == 64) || (dqk == 128 && dv == 128) || (dqk == 192 && dv == 128);
+    if (!dims_ok) return FA_ERR_UNSUPPORTED;
+    const long long n_q_tiles = (static_cast<long long>(Sq) + fa::kTileM - 1) / fa::kTileM;
+    if (Hq > 65535 || B > 65535 || n_q_tiles > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+    if (static_cast<long long>(B) * Hq > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+    return FA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* fa_strerror(fa_status s) {
+    switch (s) {
+        case FA_OK: return "success";
+        case FA_ERR_INVALID_ARG: return "invalid argument";
+        case FA_ERR_UNSUPPORTED: return "unsupported head sizes or extents";
+        case FA_ERR_CUDA: return "CUDA call failed";
+        case FA_ERR_DEVICE_TIMEOUT: return "device-side wait ran out";
+        case FA_ERR_NO_DEVICE: return "no usable CUDA device (need compute capability 10.x)";
+        case FA_ERR_OOM: return "out of memory";
+    }
+    return "unknown status";
+}
+
+fa_status fa_create(fa_handle** out, const fa_config* cfg) {
+    if (!out) return FA_ERR_INVALID_ARG;
+    *out = nullptr;
+    int device = -1;
+    uint32_t flags = 0, limit_ms = 0;
+    if (cfg) {
+        if (cfg->struct_size < sizeof(fa_config)) return FA_ERR_INVALID_ARG;
+        device = cfg->device;
+        flags = cfg->flags;
+        limit_ms = cfg->wait_limit_ms;
+        if (flags & ~FA_FLAG_SERIAL_KERNEL) return FA_ERR_INVALID_ARG;
+    }
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || count <= 0) {
+        cudaGetLastError();
+        return FA_ERR_NO_DEVICE;
+    }
+    if (device < 0) {
+        if (cudaGetDevice(&device) != cudaSuccess) return FA_ERR_NO_DEVICE;
+    }
+    if (device >= count) return FA_ERR_INVALID_ARG;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess)
+        return FA_ERR_CUDA;
+    if (major != 10) return FA_ERR_NO_DEVICE;
+
+    fa_handle* h = new (std::nothrow) fa_handle();
+    if (!h) return FA_ERR_OOM;
+    h->device = device;
+    h->flags = flags;
+    if (limit_ms) h->wait_limit_ns = static_cast<unsigned long long>(limit_ms) * 1000000ull;
+    h->maps.reserve(kMapCacheSize);
+
+    DeviceGuard guard(device);
+    if (!guard.ok()) { delete h; return FA_ERR_CUDA; }
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn) {
+        cudaGetLastError();
+        delete h;
+        return FA_ERR_CUDA;
+    }
+    h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    if (cudaHostAlloc(reinterpret_cast<void**>(&h->status_host), 16, cudaHostAllocMapped) != cudaSuccess) {
+        cudaGetLastError();
+        delete h;
+        return FA_ERR_OOM;
+    }
+    memset(h->status_host, 0, 16);
+    if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&h->status_dev), h->status_host, 0) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFreeHost(h->status_host);
+        delete h;
+        return FA_ERR_CUDA;
+    }
+    *out = h;
+    return FA_OK;
+}
+
+fa_status fa_destroy(fa_handle* h) {
+    if (!h) return FA_OK;
+    DeviceGuard guard(h->device);
+    fa_status s = FA_OK;
+    for (int i = 0; i < 5; ++i)
+        if (h->stage[i] && cudaFree(h->stage[i]) != cudaSuccess) s = FA_ERR_CUDA;
+    if (h->status_host && cudaFreeHost(h->status_host) != cudaSuccess) s = FA_ERR_CUDA;
+    delete h;
+    return s;
+}
+
+fa_status fa_last_status(fa_handle* h, uint32_t* detail) {
+    if (!h) return FA_ERR_INVALID_ARG;
+    volatile uint32_t* sw = h->status_host;
+    const uint32_t code = sw[0];
+    const uint32_t who = sw[1];
+    if (detail) *detail = code ? who : 0u;
+    if (code) { sw[0] = 0; sw[1] = 0; }
+    return code == 0 ? FA_OK : (code == FA_ERR_DEVICE_TIMEOUT ? FA_ERR_DEVICE_TIMEOUT : FA_ERR_CUDA);
+}
+
+uint64_t fa_launch_count(const fa_handle* h) { return h ? h->launches : 0; }
+const char* fa_last_kernel_name(const fa_handle* h) { return h ? h->last_kernel : ""; }
+
+fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, void* O, float* lse,
+                     int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal,
+                     float scale, void* stream) {
+    if (!h) return FA_ERR_INVALID_ARG;
+    fa_status s = check_args(Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, scale, true);
+    if (s != FA_OK) return s;
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return FA_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (scale == 0.f) scale = 1.f / sqrtf(static_cast<float>(dqk));
+
+    const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr;
+    if ((s = get_map(h, Q, dqk, Sq, static_cast<long long>(B) * Hq, fa::kTileM, &mq)) != FA_OK) return s;
+    CUtensorMap map_q = *mq;   // copies: a later insertion may evict or move cache entries
+    if ((s = get_map(h, K, dqk, Sk, static_cast<long long>(B) * Hkv, fa::kTileN, &mk)) != FA_OK) return s;
+    CUtensorMap map_k = *mk;
+    if ((s = get_map(h, V, dv, Sk, static_cast<long long>(B) * Hkv, fa::kTileN, &mv)) != FA_OK) return s;
+    CUtensorMap map_v = *mv;
+
+    fa::FwdParams p;
+    p.O = static_cast<__nv_bfloat16*>(O);
+    p.lse = lse;
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Sk = Sk;
+    p.causal = causal ? 1 : 0;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
+    p.status = h->status_dev;
+    p.wait_limit_ns = h->wait_limit_ns;
+
+    h->last_kernel = "fa_fwd_simple";
+    if (dqk == 64) return launch_simple<64, 64>(h, 0, map_q, map_k, map_v, p, st);
+    if (dqk == 128) return launch_simple<128, 128>(h, 1, map_q, map_k, map_v, p, st);
+    return launch_simple<192, 128>(h, 2, map_q, map_k, map_v, p, st);
+}
+
+fa_status fa_forward_host(fa_handle* h, const void* Qh, const void* Kh, const void* Vh, void* Oh,
+                          float* lse_h, int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv,
+                          int causal, float scale, void* stream) {
+    if (!h) return FA_ERR_INVALID_ARG;
+    fa_status s = check_args(Qh, Kh, Vh, Oh, lse_h, B, Hq, Hkv, Sq, Sk, dqk, dv, scale, false);
+    if (s != FA_OK) return s;
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return FA_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t nq = static_cast<size_t>(B) * Hq * Sq;
+    const size_t nk = static_cast<size_t>(B) * Hkv * Sk;
+    const size_t bytes[5] = {nq * dqk * 2, nk * dqk * 2, nk * dv * 2, nq * dv * 2, nq * 4};
+    for (int i = 0; i < 5; ++i) {
+        if (h->stage_cap[i] >= bytes[i]) continue;
+        if (h->stage[i]) { cudaFree(h->stage[i]); h->stage[i] = nullptr; h->stage_cap[i] = 0; }
+        if (cudaMalloc(&h->stage[i], bytes[i]) != cudaSuccess) { cudaGetLastError(); return FA_ERR_OOM; }
+        h->stage_cap[i] = bytes[i];
+    }
+    const void* src[3] = {Qh, Kh, Vh};
+    for (int i = 0; i < 3; ++i)
+        if (cudaMemcpyAsync(h->stage[i], src[i], bytes[i], cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return FA_ERR_CUDA;
+    s = fa_forward(h, h->stage[0], h->stage[1], h->stage[2], h->stage[3],
+                   lse_h ? static_cast<float*>(h->stage[4]) : nullptr,
+                   B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, stream);
+    if (s != FA_OK) return s;
+    if (cudaMemcpyAsync(Oh, h->stage[3], bytes[3], cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return FA_ERR_CUDA;
+    if (lse_h && cudaMemcpyAsync(lse_h, h->stage[4], bytes[4], cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return FA_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return FA_ERR_CUDA;
+    return FA_OK;
+}
+
+}  // extern "C"

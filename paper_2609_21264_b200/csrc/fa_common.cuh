@@ -1,0 +1,50 @@
+// Types shared by the attention forward kernels and the host-side launcher.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace fa {
+
+constexpr int kTileM = 128;       // query rows per tile (one TMEM lane per row)
+constexpr int kTileN = 128;       // keys per K/V tile
+constexpr int kChunkCols = 64;    // bf16 columns per 128-byte swizzled smem row
+constexpr int kChunkBytes = kTileN * kChunkCols * 2;   // one 128-row x 64-col chunk = 16 KB
+
+// "who" codes recorded when a bounded wait gives up: (role << 8) | barrier id.
+enum WaitSite : uint32_t {
+    kSiteSimpleQ = 0x0101, kSiteSimpleK = 0x0102, kSiteSimpleV = 0x0103, kSiteSimpleMma = 0x0104,
+    kSiteLoadKvEmpty = 0x0201, kSiteLoadQEmpty = 0x0202,
+    kSiteMmaQFull = 0x0301, kSiteMmaKvFull = 0x0302, kSiteMmaPFull = 0x0303,
+    kSiteMmaOReady = 0x0304, kSiteMmaSFree = 0x0305,
+    kSiteSoftmaxSFull = 0x0401, kSiteSoftmaxPFree = 0x0402, kSiteSoftmaxCorrFree = 0x0403,
+    kSiteCorrScale = 0x0501, kSiteCorrPvDone = 0x0502, kSiteCorrFinal = 0x0503,
+    kSiteEpiOFull = 0x0601,
+};
+
+struct FwdParams {
+    __nv_bfloat16* O;         // [B, Hq, Sq, dv]
+    float* lse;               // [B, Hq, Sq] or nullptr
+    int B, Hq, Hkv, Sq, Sk;
+    int causal;
+    float scale_log2;         // scale * log2(e): scores are handled in log2 units
+    int n_q_tiles;            // ceil(Sq / 128)
+    uint32_t* status;         // [0] = fa_status, [1] = wait site; mapped host memory
+    unsigned long long wait_limit_ns;
+};
+
+// Number of K/V tiles a query tile starting at row i0 (covering `rows` rows) has to visit.
+// Key j is visible to query i iff j <= i + (Sk - Sq) in causal mode.
+__host__ __device__ inline int kv_tiles_for_q_tile(int i0, int rows, int Sq, int Sk, int causal) {
+    int last_key = Sk - 1;
+    if (causal) {
+        int last_row = i0 + rows - 1;
+        if (last_row > Sq - 1) last_row = Sq - 1;
+        const int lim = last_row + (Sk - Sq);
+        if (lim < last_key) last_key = lim;
+    }
+    return last_key < 0 ? 0 : last_key / kTileN + 1;
+}
+
+}  // namespace fa
