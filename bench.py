@@ -55,7 +55,7 @@ class ClockSampler(threading.Thread):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
-        self._stop = threading.Event()
+        self._halt = threading.Event()
         self.error = None
 
     def run(self):
@@ -72,7 +72,7 @@ class ClockSampler(threading.Thread):
             }
             get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
                 getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
-            while not self._stop.is_set():
+            while not self._halt.is_set():
                 self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
                 mask = get_reasons(h)
                 for bit, name in names.items():
@@ -83,7 +83,7 @@ class ClockSampler(threading.Thread):
             self.error = repr(ex)
 
     def stop(self):
-        self._stop.set()
+        self._halt.set()
         self.join(timeout=2.0)
         s = sorted(self.samples)
         return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
