@@ -12,6 +12,7 @@
 
 #include "../../include/fa.h"
 #include "fa_common.cuh"
+#include "fa_fwd_pipelined.cuh"
 #include "fa_fwd_simple.cuh"
 
 namespace {
@@ -126,6 +127,21 @@ fa_status launch_simple(fa_handle* h, int slot, const CUtensorMap& mq, const CUt
     if (s != FA_OK) return s;
     dim3 grid(p.n_q_tiles, p.Hq, p.B);
     kernel<<<grid, 128, smem, st>>>(mq, mk, mv, p);
+    if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
+    h->launches += 1;
+    return FA_OK;
+}
+
+template <int DQK, int DV>
+fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
+                           const CUtensorMap& mv, const fa::FwdParams& p, cudaStream_t st) {
+    constexpr int smem = fa::pipe_smem_bytes<DQK, DV>();
+    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+    auto kernel = fa::fa_fwd_pipelined_kernel<DQK, DV>;
+    fa_status s = ensure_smem_attr(h, slot, kernel, smem);
+    if (s != FA_OK) return s;
+    dim3 grid((p.n_q_tiles + 1) / 2, p.Hq, p.B);
+    kernel<<<grid, fa::PipeCfg<DQK, DV>::kThreads, smem, st>>>(mq, mk, mv, p);
     if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
     h->launches += 1;
     return FA_OK;
@@ -284,6 +300,12 @@ fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, 
     p.status = h->status_dev;
     p.wait_limit_ns = h->wait_limit_ns;
 
+    if (!(h->flags & FA_FLAG_SERIAL_KERNEL)) {
+        h->last_kernel = "fa_fwd_pipelined";
+        if (dqk == 64) return launch_pipelined<64, 64>(h, 3, map_q, map_k, map_v, p, st);
+        if (dqk == 128) return launch_pipelined<128, 128>(h, 4, map_q, map_k, map_v, p, st);
+        return launch_pipelined<192, 128>(h, 5, map_q, map_k, map_v, p, st);
+    }
     h->last_kernel = "fa_fwd_simple";
     if (dqk == 64) return launch_simple<64, 64>(h, 0, map_q, map_k, map_v, p, st);
     if (dqk == 128) return launch_simple<128, 128>(h, 1, map_q, map_k, map_v, p, st);

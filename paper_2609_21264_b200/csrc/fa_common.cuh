@@ -21,6 +21,7 @@ enum WaitSite : uint32_t {
     kSiteSoftmaxSFull = 0x0401, kSiteSoftmaxPFree = 0x0402, kSiteSoftmaxCorrFree = 0x0403,
     kSiteCorrScale = 0x0501, kSiteCorrPvDone = 0x0502, kSiteCorrFinal = 0x0503,
     kSiteEpiOFull = 0x0601,
+    kSiteSmemAlign = 0x0701,
 };
 
 struct FwdParams {

@@ -1,0 +1,427 @@
+// Pipelined, warp-specialised attention forward kernel for sm_100a.
+//
+// One CTA owns two adjacent 128-row query tiles of one (batch, query head) and
+// walks the K/V tiles they can see.  Roles:
+//   warps 0-3   softmax of query tile 0 (one TMEM lane = one query row per thread), then its
+//               final normalisation and stores
+//   warps 4-7   softmax of query tile 1
+//   warps 8-11  correction: rescale of the O accumulators when a reference maximum moved
+//   warp  12    MMA issue (one thread): S_t = Q_t K_j^T and O_t += P_t V_j with tcgen05
+//   warp  13    TMA loads of Q_t, K_j, V_j into mbarrier-guarded shared-memory rings
+//   warps 14-15 idle (they keep the fourth warpgroup complete)
+// While one softmax warpgroup works on S_t(j), the tensor core runs the MMAs of
+// the other tile, so the exponentials overlap the contractions.
+//
+// The recurrence is Algorithm 1 with fp32 state: running row maximum u, running
+// row sum s, unnormalised accumulator G' in TMEM, P rounded to bf16 before the
+// second contraction, one division at the end (Section 2.1).  Two deviations in
+// evaluation order, neither changing the result beyond rounding:
+//   * the scale 1/sqrt(dk) is folded into the exponent (exp2((g - u) * scale *
+//     log2 e)) instead of being applied to Q, so Q is never re-rounded;
+//   * the reference maximum u is only advanced when the row maximum grew by more
+//     than 2^8 in the exponent, so the rescale r = exp(u' - u) of G' is skipped
+//     on most tiles; G' and s are always expressed against the same u, and the
+//     final G'/s and lse = u + ln s are unchanged.
+// TMEM: S_0 [0,128) S_1 [128,256) O_0 [256,256+dv) O_1 [384,384+dv); bf16 P_t
+// overlays the first 64 columns of S_t.
+#pragma once
+
+#include <math.h>
+
+#include "fa_common.cuh"
+#include "ptx.cuh"
+
+namespace fa {
+
+template <int DQK, int DV>
+struct PipeCfg {
+    static constexpr int kQChunks = DQK / kChunkCols;
+    static constexpr int kVChunks = DV / kChunkCols;
+    static constexpr int kQBytes = kQChunks * kChunkBytes;    // one query tile
+    static constexpr int kKBytes = kQBytes;
+    static constexpr int kVBytes = kVChunks * kChunkBytes;
+    static constexpr int kKStages = (DQK == 192) ? 2 : (DQK == 128 ? 3 : 4);
+    static constexpr int kVStages = (DQK == 192) ? 1 : (DQK == 128 ? 2 : 4);
+    static constexpr int kTileBytes = 2 * kQBytes + kKStages * kKBytes + kVStages * kVBytes;
+    static constexpr int kTmemCols = 512;
+    static constexpr int kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 384;
+    static constexpr int kThreads = 512;
+};
+
+constexpr float kRescaleThresholdLog2 = 8.0f;
+
+struct PipeShared {
+    uint64_t q_full[2];
+    uint64_t k_full[4], k_empty[4];
+    uint64_t v_full[4], v_empty[4];
+    uint64_t s_full[2];      // MMA -> softmax: S_t(j) is in TMEM
+    uint64_t p_full[2];      // softmax + correction -> MMA: P_t(j) written, O_t rescaled
+    uint64_t scale_full[2];  // softmax -> correction: alpha of iteration j published
+    uint64_t o_final[2];     // MMA -> softmax: last PV of tile t done, O_t is final
+    float alpha[2][2][kTileM];   // [tile][j & 1][row]
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+template <int DQK, int DV>
+constexpr int pipe_smem_bytes() {
+    return PipeCfg<DQK, DV>::kTileBytes + static_cast<int>(sizeof(PipeShared));
+}
+
+template <int DQK, int DV>
+__global__ void __launch_bounds__(512, 1)
+fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
+                        const __grid_constant__ CUtensorMap tm_k,
+                        const __grid_constant__ CUtensorMap tm_v,
+                        const FwdParams p) {
+    using Cfg = PipeCfg<DQK, DV>;
+    using namespace ptx;
+    constexpr int NK = Cfg::kKStages;
+    constexpr int NV = Cfg::kVStages;
+
+    // All shared memory is dynamic: the swizzled tiles first (they need a 1024-byte aligned
+    // base), the barriers and hand-off buffers behind them.
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    PipeShared& sh = *reinterpret_cast<PipeShared*>(smem_raw + Cfg::kTileBytes);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+
+    const uint32_t smem_base = smem_addr(smem_raw);
+    if ((smem_base & 1023u) != 0u) {          // uniform over the CTA; nothing has been set up yet
+        if (tid == 0 && p.status) {
+            volatile uint32_t* sw = p.status;
+            sw[1] = kSiteSmemAlign;
+            sw[0] = 3u;                       // FA_ERR_CUDA
+            __threadfence_system();
+        }
+        return;
+    }
+    const uint32_t sQ = smem_base;                               // two tiles
+    const uint32_t sK = sQ + 2 * Cfg::kQBytes;                   // NK stages
+    const uint32_t sV = sK + NK * Cfg::kKBytes;                  // NV stages
+
+    const int pair = static_cast<int>(gridDim.x) - 1 - static_cast<int>(blockIdx.x);   // heavy first
+    const int hq = blockIdx.y;
+    const int b = blockIdx.z;
+    const int kvh = hq / (p.Hq / p.Hkv);
+    const int q_idx = b * p.Hq + hq;
+    const int kv_idx = b * p.Hkv + kvh;
+    const int off = p.Sk - p.Sq;
+
+    int i0[2], n_kv[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        i0[t] = (2 * pair + t) * kTileM;
+        n_kv[t] = (i0[t] < p.Sq) ? kv_tiles_for_q_tile(i0[t], kTileM, p.Sq, p.Sk, p.causal) : 0;
+    }
+    const int n_max = n_kv[0] > n_kv[1] ? n_kv[0] : n_kv[1];
+
+    // ---------------------------------------------------------------- setup
+    if (tid == 0) {
+        sh.abort_flag = 0;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(smem_addr(&sh.q_full[t]), 1);
+            mbar_init(smem_addr(&sh.s_full[t]), 1);
+            mbar_init(smem_addr(&sh.p_full[t]), 8);       // 4 softmax warps + 4 correction warps
+            mbar_init(smem_addr(&sh.scale_full[t]), 4);
+            mbar_init(smem_addr(&sh.o_final[t]), 1);
+        }
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(smem_addr(&sh.k_full[s]), 1);
+            mbar_init(smem_addr(&sh.k_empty[s]), 1);
+            mbar_init(smem_addr(&sh.v_full[s]), 1);
+            mbar_init(smem_addr(&sh.v_empty[s]), 1);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 12) {
+        tmem_alloc(smem_addr(&sh.tmem_base), Cfg::kTmemCols);
+        tmem_relinquish_alloc_permit();
+    }
+    if (warp == 13 && lane == 0) {
+        prefetch_tensormap(&tm_q);
+        prefetch_tensormap(&tm_k);
+        prefetch_tensormap(&tm_v);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+
+    const uint32_t tmem_base = sh.tmem_base;
+    WaitCtx wctx{&sh.abort_flag, p.status, p.wait_limit_ns};
+    const float c = p.scale_log2;
+
+    if (warp < 8) {
+        // ============================================================ softmax of tile t
+        const int t = warp >> 2;
+        const int row = tid & (kTileM - 1);
+        const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1) + lane_sel;
+        const uint32_t bar_s = smem_addr(&sh.s_full[t]);
+        const uint32_t bar_p = smem_addr(&sh.p_full[t]);
+        const uint32_t bar_scale = smem_addr(&sh.scale_full[t]);
+        const int i_glob = i0[t] + row;
+        int kmax_row = p.Sk - 1;
+        if (p.causal && i_glob + off < kmax_row) kmax_row = i_glob + off;
+        const float tau_raw = kRescaleThresholdLog2 / c;
+
+        float m_ref = -INFINITY;   // reference maximum, raw score units
+        float l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_kv[t]; ++j) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_s, j & 1, wctx, kSiteSoftmaxSFull));
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int j0 = j * kTileN;
+            const bool need_mask = (j0 + kTileN - 1 > kmax_row);
+
+            // pass 1: row maximum of the raw scores
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c4 = 0; c4 < 4; ++c4) {
+                uint32_t r[32];
+                tmem_ld_x32(tS + c4 * 32, r);
+                tc_wait_ld();
+                if (need_mask) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (j0 + c4 * 32 + e > kmax_row) r[e] = 0xff800000u;   // -inf
+                }
+                float a0 = mx, a1 = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    a0 = fmax3(a0, __uint_as_float(r[e]), __uint_as_float(r[e + 1]));
+                    a1 = fmax3(a1, __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                }
+                mx = fmaxf(a0, a1);
+            }
+            // advance the reference maximum only when the row maximum grew by more than the threshold
+            float alpha = 1.f;
+            if (mx > m_ref + tau_raw) {
+                alpha = exp2_approx((m_ref - mx) * c);    // r = exp(u' - u); 0 on the first tile
+                m_ref = mx;
+            }
+            sh.alpha[t][j & 1][row] = alpha;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_scale);
+
+            const float mc = (m_ref == -INFINITY) ? 0.f : m_ref * c;
+            // pass 2: exponentials, row sum, bf16 P back to TMEM (over the first half of S)
+            float rowsum0 = 0.f, rowsum1 = 0.f;
+#pragma unroll 1
+            for (int c4 = 0; c4 < 4; ++c4) {
+                uint32_t r[32];
+                tmem_ld_x32(tS + c4 * 32, r);
+                tc_wait_ld();
+                if (need_mask) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (j0 + c4 * 32 + e > kmax_row) r[e] = 0xff800000u;
+                }
+                uint32_t pk[16];
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    const float p0 = exp2_approx(fmaf(__uint_as_float(r[e]), c, -mc));
+                    const float p1 = exp2_approx(fmaf(__uint_as_float(r[e + 1]), c, -mc));
+                    rowsum0 += p0;
+                    rowsum1 += p1;
+                    pk[e / 2] = pack_bf16x2(p0, p1);
+                }
+                tmem_st_x16(tS + c4 * 16, pk);
+            }
+            l = l * alpha + (rowsum0 + rowsum1);
+            tc_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_p);
+        }
+        // epilogue: O = G' / s (bf16), lse = u * scale + ln s
+        if (ok && i0[t] < p.Sq) {
+            __nv_bfloat16* o_row = p.O + (static_cast<size_t>(q_idx) * p.Sq + i_glob) * DV;
+            if (n_kv[t] == 0) {       // no key visible to any row of this tile
+                if (i_glob < p.Sq) {
+                    const uint4 z = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                    for (int v = 0; v < DV / 8; ++v) reinterpret_cast<uint4*>(o_row)[v] = z;
+                    if (p.lse) p.lse[static_cast<size_t>(q_idx) * p.Sq + i_glob] = -INFINITY;
+                }
+            } else if (__all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.o_final[t]), 0, wctx, kSiteEpiOFull))) {
+                tc_fence_after_sync();
+                const float inv_l = (l > 0.f) ? (1.f / l) : 0.f;
+                if (p.lse && i_glob < p.Sq) {
+                    p.lse[static_cast<size_t>(q_idx) * p.Sq + i_glob] =
+                        (l > 0.f) ? (m_ref * c * 0.6931471805599453f + logf(l)) : -INFINITY;
+                }
+                const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1) + lane_sel;
+#pragma unroll 1
+                for (int cc = 0; cc < DV / 32; ++cc) {
+                    uint32_t r[32];
+                    tmem_ld_x32(tO + cc * 32, r);
+                    tc_wait_ld();
+                    if (i_glob < p.Sq) {
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2)
+                            pk[e / 2] = pack_bf16x2(__uint_as_float(r[e]) * inv_l,
+                                                    __uint_as_float(r[e + 1]) * inv_l);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            reinterpret_cast<uint4*>(o_row + cc * 32)[v] =
+                                make_uint4(pk[4 * v], pk[4 * v + 1], pk[4 * v + 2], pk[4 * v + 3]);
+                    }
+                }
+            }
+        }
+    } else if (warp < 12) {
+        // ============================================================ correction of the O accumulators
+        const int row = tid & (kTileM - 1);
+        const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        bool ok = true;
+        for (int j = 0; j < n_max && ok; ++j) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                if (j >= n_kv[t] || !ok) continue;
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.scale_full[t]), j & 1, wctx,
+                                                       kSiteCorrScale));
+                if (!ok) break;
+                const float alpha = sh.alpha[t][j & 1][row];
+                if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                    tc_fence_after_sync();
+                    const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1) + lane_sel;
+#pragma unroll 1
+                    for (int cc = 0; cc < DV / 32; ++cc) {
+                        uint32_t r[32];
+                        tmem_ld_x32(tO + cc * 32, r);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+                        tmem_st_x32(tO + cc * 32, r);
+                    }
+                    tc_wait_st();
+                    tc_fence_before_sync();
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_addr(&sh.p_full[t]));
+            }
+        }
+    } else if (warp == 12) {
+        // ============================================================ MMA issue
+        if (lane == 0 && n_max > 0) {
+            constexpr uint32_t kIdescQK = make_idesc_bf16_f32(kTileM, kTileN, false, false);
+            constexpr uint32_t kIdescPV = make_idesc_bf16_f32(kTileM, DV, false, true);
+            auto issue_qk = [&](int t, int stage) {
+                const uint32_t q_base = sQ + t * Cfg::kQBytes;
+                const uint32_t k_base = sK + stage * Cfg::kKBytes;
+                const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1);
+#pragma unroll
+                for (int k = 0; k < DQK / 16; ++k) {
+                    const uint32_t koff = (k / 4) * kChunkBytes + (k % 4) * 32;
+                    mma_ss(tS, make_smem_desc_sw128(q_base + koff, 16, 1024),
+                           make_smem_desc_sw128(k_base + koff, 16, 1024), kIdescQK, k > 0 ? 1u : 0u);
+                }
+            };
+            auto issue_pv = [&](int t, int stage, bool accumulate) {
+                const uint32_t v_base = sV + stage * Cfg::kVBytes;
+                const uint32_t tP = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1);
+                const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1);
+#pragma unroll
+                for (int kk = 0; kk < kTileN / 16; ++kk) {
+                    mma_ts(tO, tP + kk * 8, make_smem_desc_sw128(v_base + kk * 2048, kChunkBytes, 1024),
+                           kIdescPV, (accumulate || kk > 0) ? 1u : 0u);
+                }
+            };
+            bool ok = mbar_wait(smem_addr(&sh.k_full[0]), 0, wctx, kSiteMmaKvFull);
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                if (n_kv[t] == 0 || !ok) continue;
+                ok = mbar_wait(smem_addr(&sh.q_full[t]), 0, wctx, kSiteMmaQFull);
+                if (!ok) break;
+                tc_fence_after_sync();
+                issue_qk(t, 0);
+                tc_commit(smem_addr(&sh.s_full[t]));
+            }
+            if (ok) tc_commit(smem_addr(&sh.k_empty[0]));
+            for (int j = 0; j < n_max && ok; ++j) {
+                const int sv = j % NV;
+                const int sk = (j + 1) % NK;
+                ok = mbar_wait(smem_addr(&sh.v_full[sv]), (j / NV) & 1, wctx, kSiteMmaKvFull);
+                bool k_ready = false;
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (j >= n_kv[t] || !ok) continue;
+                    ok = mbar_wait(smem_addr(&sh.p_full[t]), j & 1, wctx, kSiteMmaPFull);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue_pv(t, sv, j > 0);
+                    if (j + 1 < n_kv[t]) {
+                        if (!k_ready) {
+                            ok = mbar_wait(smem_addr(&sh.k_full[sk]), ((j + 1) / NK) & 1, wctx, kSiteMmaKvFull);
+                            if (!ok) break;
+                            tc_fence_after_sync();
+                            k_ready = true;
+                        }
+                        issue_qk(t, sk);
+                        tc_commit(smem_addr(&sh.s_full[t]));
+                    } else {
+                        tc_commit(smem_addr(&sh.o_final[t]));
+                    }
+                }
+                if (!ok) break;
+                tc_commit(smem_addr(&sh.v_empty[sv]));
+                if (j + 1 < n_max) tc_commit(smem_addr(&sh.k_empty[sk]));
+            }
+        }
+    } else if (warp == 13) {
+        // ============================================================ TMA loads
+        if (lane == 0 && n_max > 0) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                if (n_kv[t] == 0) continue;
+                const uint32_t bar = smem_addr(&sh.q_full[t]);
+                mbar_arrive_expect_tx(bar, Cfg::kQBytes);
+#pragma unroll
+                for (int cc = 0; cc < Cfg::kQChunks; ++cc)
+                    tma_load_3d(sQ + t * Cfg::kQBytes + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols,
+                                i0[t], q_idx);
+            }
+            bool ok = true;
+            for (int j = 0; j < n_max && ok; ++j) {
+                const int j0 = j * kTileN;
+                {
+                    const int s = j % NK;
+                    ok = mbar_wait(smem_addr(&sh.k_empty[s]), ((j / NK) & 1) ^ 1, wctx, kSiteLoadKvEmpty);
+                    if (!ok) break;
+                    const uint32_t bar = smem_addr(&sh.k_full[s]);
+                    mbar_arrive_expect_tx(bar, Cfg::kKBytes);
+#pragma unroll
+                    for (int cc = 0; cc < Cfg::kQChunks; ++cc)
+                        tma_load_3d(sK + s * Cfg::kKBytes + cc * kChunkBytes, &tm_k, bar, cc * kChunkCols,
+                                    j0, kv_idx);
+                }
+                {
+                    const int s = j % NV;
+                    ok = mbar_wait(smem_addr(&sh.v_empty[s]), ((j / NV) & 1) ^ 1, wctx, kSiteLoadKvEmpty);
+                    if (!ok) break;
+                    const uint32_t bar = smem_addr(&sh.v_full[s]);
+                    mbar_arrive_expect_tx(bar, Cfg::kVBytes);
+#pragma unroll
+                    for (int cc = 0; cc < Cfg::kVChunks; ++cc)
+                        tma_load_3d(sV + s * Cfg::kVBytes + cc * kChunkBytes, &tm_v, bar, cc * kChunkCols,
+                                    j0, kv_idx);
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown (all warps)
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 12) tmem_dealloc(tmem_base, Cfg::kTmemCols);
+}
+
+}  // namespace fa
