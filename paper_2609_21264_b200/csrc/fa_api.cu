@@ -47,6 +47,9 @@ struct fa_handle {
     void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // Q K V O lse
     size_t stage_cap[5] = {0, 0, 0, 0, 0};
     bool attr_done[8] = {false, false, false, false, false, false, false, false};
+#ifdef FA_TRACE
+    long long* trace = nullptr;
+#endif
 };
 
 namespace {
@@ -299,6 +302,9 @@ fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, 
     p.n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
     p.status = h->status_dev;
     p.wait_limit_ns = h->wait_limit_ns;
+#ifdef FA_TRACE
+    p.trace = h->trace;
+#endif
 
     if (!(h->flags & FA_FLAG_SERIAL_KERNEL)) {
         h->last_kernel = "fa_fwd_pipelined";
@@ -345,5 +351,14 @@ fa_status fa_forward_host(fa_handle* h, const void* Qh, const void* Kh, const vo
     if (cudaStreamSynchronize(st) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
 }
+
+#ifdef FA_TRACE
+// Debug builds only: device buffer of kTraceRoles*kTraceIters*kTraceEvents int64 clock stamps.
+fa_status fa_debug_set_trace(fa_handle* h, void* device_buffer) {
+    if (!h) return FA_ERR_INVALID_ARG;
+    h->trace = static_cast<long long*>(device_buffer);
+    return FA_OK;
+}
+#endif
 
 }  // extern "C"

@@ -33,7 +33,21 @@ struct FwdParams {
     int n_q_tiles;            // ceil(Sq / 128)
     uint32_t* status;         // [0] = fa_status, [1] = wait site; mapped host memory
     unsigned long long wait_limit_ns;
+#ifdef FA_TRACE
+    long long* trace;         // [role][iteration][event] SM clock stamps of CTA (0,0,0); debug builds only
+#endif
 };
+
+#ifdef FA_TRACE
+constexpr int kTraceIters = 64, kTraceEvents = 16, kTraceRoles = 4;   // roles: softmax0, softmax1, mma, corr
+#define FA_TRACE_STAMP(role, iter, ev)                                                          \
+    do {                                                                                        \
+        if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (iter) < kTraceIters) \
+            p.trace[((role) * kTraceIters + (iter)) * kTraceEvents + (ev)] = clock64();         \
+    } while (0)
+#else
+#define FA_TRACE_STAMP(role, iter, ev) do { } while (0)
+#endif
 
 // Number of K/V tiles a query tile starting at row i0 (covering `rows` rows) has to visit.
 // Key j is visible to query i iff j <= i + (Sk - Sq) in causal mode.

@@ -48,14 +48,21 @@ struct PipeCfg {
     static constexpr int kThreads = 512;
 };
 
+template <int V>
+struct IntC { static constexpr int value = V; };
+
 constexpr float kRescaleThresholdLog2 = 8.0f;
+// Registers per thread after the per-role reallocation (512 threads start with 128 each):
+// 256 softmax threads x 192 + 128 correction threads x 64 + 128 other threads x 64 = 65536.
+constexpr int kRegsSoftmax = 192, kRegsCorrection = 64, kRegsOther = 64;
 
 struct PipeShared {
     uint64_t q_full[2];
     uint64_t k_full[4], k_empty[4];
     uint64_t v_full[4], v_empty[4];
     uint64_t s_full[2];      // MMA -> softmax: S_t(j) is in TMEM
-    uint64_t p_full[2];      // softmax + correction -> MMA: P_t(j) written, O_t rescaled
+    uint64_t p_half[2];      // softmax + correction -> MMA: keys 0..63 of P_t(j) written, O_t rescaled
+    uint64_t p_full[2];      // softmax -> MMA: all of P_t(j) written
     uint64_t scale_full[2];  // softmax -> correction: alpha of iteration j published
     uint64_t o_final[2];     // MMA -> softmax: last PV of tile t done, O_t is final
     float alpha[2][2][kTileM];   // [tile][j & 1][row]
@@ -110,13 +117,11 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int kv_idx = b * p.Hkv + kvh;
     const int off = p.Sk - p.Sq;
 
-    int i0[2], n_kv[2];
-#pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        i0[t] = (2 * pair + t) * kTileM;
-        n_kv[t] = (i0[t] < p.Sq) ? kv_tiles_for_q_tile(i0[t], kTileM, p.Sq, p.Sk, p.causal) : 0;
-    }
-    const int n_max = n_kv[0] > n_kv[1] ? n_kv[0] : n_kv[1];
+    // per-tile scalars (no arrays: a runtime-indexed array would live in local memory)
+    const int i0_0 = (2 * pair) * kTileM, i0_1 = i0_0 + kTileM;
+    const int nkv_0 = (i0_0 < p.Sq) ? kv_tiles_for_q_tile(i0_0, kTileM, p.Sq, p.Sk, p.causal) : 0;
+    const int nkv_1 = (i0_1 < p.Sq) ? kv_tiles_for_q_tile(i0_1, kTileM, p.Sq, p.Sk, p.causal) : 0;
+    const int n_max = nkv_0 > nkv_1 ? nkv_0 : nkv_1;
 
     // ---------------------------------------------------------------- setup
     if (tid == 0) {
@@ -125,7 +130,8 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         for (int t = 0; t < 2; ++t) {
             mbar_init(smem_addr(&sh.q_full[t]), 1);
             mbar_init(smem_addr(&sh.s_full[t]), 1);
-            mbar_init(smem_addr(&sh.p_full[t]), 8);       // 4 softmax warps + 4 correction warps
+            mbar_init(smem_addr(&sh.p_half[t]), 8);       // 4 softmax warps + 4 correction warps
+            mbar_init(smem_addr(&sh.p_full[t]), 4);       // 4 softmax warps
             mbar_init(smem_addr(&sh.scale_full[t]), 4);
             mbar_init(smem_addr(&sh.o_final[t]), 1);
         }
@@ -157,14 +163,18 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
 
     if (warp < 8) {
         // ============================================================ softmax of tile t
+        setmaxnreg_inc<kRegsSoftmax>();
         const int t = warp >> 2;
         const int row = tid & (kTileM - 1);
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1) + lane_sel;
         const uint32_t bar_s = smem_addr(&sh.s_full[t]);
         const uint32_t bar_p = smem_addr(&sh.p_full[t]);
+        const uint32_t bar_ph = smem_addr(&sh.p_half[t]);
         const uint32_t bar_scale = smem_addr(&sh.scale_full[t]);
-        const int i_glob = i0[t] + row;
+        const int i0_t = t == 0 ? i0_0 : i0_1;
+        const int nkv_t = t == 0 ? nkv_0 : nkv_1;
+        const int i_glob = i0_t + row;
         int kmax_row = p.Sk - 1;
         if (p.causal && i_glob + off < kmax_row) kmax_row = i_glob + off;
         const float tau_raw = kRescaleThresholdLog2 / c;
@@ -172,32 +182,40 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         float m_ref = -INFINITY;   // reference maximum, raw score units
         float l = 0.f;
         bool ok = true;
-        for (int j = 0; j < n_kv[t]; ++j) {
+        for (int j = 0; j < nkv_t; ++j) {
             ok = __all_sync(0xffffffffu, mbar_wait(bar_s, j & 1, wctx, kSiteSoftmaxSFull));
             if (!ok) break;
             tc_fence_after_sync();
+            if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(t, j, 0);
             const int j0 = j * kTileN;
             const bool need_mask = (j0 + kTileN - 1 > kmax_row);
 
-            // pass 1: row maximum of the raw scores
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int c4 = 0; c4 < 4; ++c4) {
-                uint32_t r[32];
-                tmem_ld_x32(tS + c4 * 32, r);
-                tc_wait_ld();
-                if (need_mask) {
+            // the whole score row in registers: four loads in flight, one wait
+            uint32_t s[kTileN];
+            tmem_ld_x32(tS + 0, s + 0);
+            tmem_ld_x32(tS + 32, s + 32);
+            tmem_ld_x32(tS + 64, s + 64);
+            tmem_ld_x32(tS + 96, s + 96);
+            tc_wait_ld();
+            if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(t, j, 1);
+            if (need_mask) {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (j0 + c4 * 32 + e > kmax_row) r[e] = 0xff800000u;   // -inf
-                }
-                float a0 = mx, a1 = -INFINITY;
+                for (int e = 0; e < kTileN; ++e)
+                    if (j0 + e > kmax_row) s[e] = 0xff800000u;   // -inf
+            }
+            float mx;
+            {
+                float a[8];
 #pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    a0 = fmax3(a0, __uint_as_float(r[e]), __uint_as_float(r[e + 1]));
-                    a1 = fmax3(a1, __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                for (int q = 0; q < 8; ++q) a[q] = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < kTileN; e += 16) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        a[q] = fmax3(a[q], __uint_as_float(s[e + 2 * q]), __uint_as_float(s[e + 2 * q + 1]));
                 }
-                mx = fmaxf(a0, a1);
+                mx = fmaxf(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]));
+                mx = fmax3(mx, a[6], a[7]);
             }
             // advance the reference maximum only when the row maximum grew by more than the threshold
             float alpha = 1.f;
@@ -208,41 +226,62 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             sh.alpha[t][j & 1][row] = alpha;
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_scale);
+            if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(t, j, 2);
 
             const float mc = (m_ref == -INFINITY) ? 0.f : m_ref * c;
-            // pass 2: exponentials, row sum, bf16 P back to TMEM (over the first half of S)
-            float rowsum0 = 0.f, rowsum1 = 0.f;
-#pragma unroll 1
-            for (int c4 = 0; c4 < 4; ++c4) {
-                uint32_t r[32];
-                tmem_ld_x32(tS + c4 * 32, r);
-                tc_wait_ld();
-                if (need_mask) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (j0 + c4 * 32 + e > kmax_row) r[e] = 0xff800000u;
-                }
-                uint32_t pk[16];
+            // Exponentials in place (packed FMA for the argument), row sum, bf16 P back to TMEM
+            // over the first half of S.  The exponentials of chunk q+1 are issued before chunk q
+            // is summed, converted and stored, so the MUFU pipe does not drain between chunks.
+            const float2 c2 = make_float2(c, c);
+            const float2 nmc2 = make_float2(-mc, -mc);
+            float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
+            auto exp_chunk = [&](int q) {
 #pragma unroll
                 for (int e = 0; e < 32; e += 2) {
-                    const float p0 = exp2_approx(fmaf(__uint_as_float(r[e]), c, -mc));
-                    const float p1 = exp2_approx(fmaf(__uint_as_float(r[e + 1]), c, -mc));
-                    rowsum0 += p0;
-                    rowsum1 += p1;
-                    pk[e / 2] = pack_bf16x2(p0, p1);
+                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[q * 32 + e]),
+                                                            __uint_as_float(s[q * 32 + e + 1])), c2, nmc2);
+                    s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
+                    s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
                 }
-                tmem_st_x16(tS + c4 * 16, pk);
-            }
-            l = l * alpha + (rowsum0 + rowsum1);
+            };
+            auto emit_chunk = [&](int q) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    const float2 v0 = make_float2(__uint_as_float(s[q * 32 + e]), __uint_as_float(s[q * 32 + e + 1]));
+                    const float2 v1 = make_float2(__uint_as_float(s[q * 32 + e + 2]), __uint_as_float(s[q * 32 + e + 3]));
+                    sum_a = __fadd2_rn(sum_a, v0);
+                    sum_b = __fadd2_rn(sum_b, v1);
+                    pk[e / 2] = pack_bf16x2(v0.x, v0.y);
+                    pk[e / 2 + 1] = pack_bf16x2(v1.x, v1.y);
+                }
+                tmem_st_x16(tS + q * 16, pk);
+            };
+            exp_chunk(0);
+            exp_chunk(1);
+            emit_chunk(0);
+            exp_chunk(2);
+            emit_chunk(1);
+            // first half of P (keys 0..63) is in flight: let the MMA warp start O += P V early
+            tc_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_ph);
+            exp_chunk(3);
+            emit_chunk(2);
+            emit_chunk(3);
+            l = l * alpha + ((sum_a.x + sum_a.y) + (sum_b.x + sum_b.y));
+            if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(t, j, 3);
             tc_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_p);
+            if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(t, j, 4);
         }
         // epilogue: O = G' / s (bf16), lse = u * scale + ln s
-        if (ok && i0[t] < p.Sq) {
+        if (ok && i0_t < p.Sq) {
             __nv_bfloat16* o_row = p.O + (static_cast<size_t>(q_idx) * p.Sq + i_glob) * DV;
-            if (n_kv[t] == 0) {       // no key visible to any row of this tile
+            if (nkv_t == 0) {         // no key visible to any row of this tile
                 if (i_glob < p.Sq) {
                     const uint4 z = make_uint4(0, 0, 0, 0);
 #pragma unroll
@@ -278,17 +317,19 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         }
     } else if (warp < 12) {
         // ============================================================ correction of the O accumulators
+        setmaxnreg_dec<kRegsCorrection>();
         const int row = tid & (kTileM - 1);
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
         bool ok = true;
         for (int j = 0; j < n_max && ok; ++j) {
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
-                if (j >= n_kv[t] || !ok) continue;
+                if (j >= (t == 0 ? nkv_0 : nkv_1) || !ok) continue;
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.scale_full[t]), j & 1, wctx,
                                                        kSiteCorrScale));
                 if (!ok) break;
                 const float alpha = sh.alpha[t][j & 1][row];
+                if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(3, j, t * 4 + 0);
                 if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
                     tc_fence_after_sync();
                     const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1) + lane_sel;
@@ -306,88 +347,123 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                     tc_fence_before_sync();
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_addr(&sh.p_full[t]));
+                if (lane == 0) mbar_arrive(smem_addr(&sh.p_half[t]));
+                if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(3, j, t * 4 + 1);
             }
         }
     } else if (warp == 12) {
         // ============================================================ MMA issue
+        setmaxnreg_dec<kRegsOther>();
         if (lane == 0 && n_max > 0) {
             constexpr uint32_t kIdescQK = make_idesc_bf16_f32(kTileM, kTileN, false, false);
             constexpr uint32_t kIdescPV = make_idesc_bf16_f32(kTileM, DV, false, true);
-            auto issue_qk = [&](int t, int stage) {
-                const uint32_t q_base = sQ + t * Cfg::kQBytes;
-                const uint32_t k_base = sK + stage * Cfg::kKBytes;
+            // Descriptor words are built once.  Per MMA only the 14-bit start-address field of the
+            // low word moves (shared-memory addresses stay below 2^18, so no carry leaves it).
+            constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // sbo, version, swizzle
+            const uint32_t q_lo0 = ((sQ & 0x3FFFFu) >> 4) | (1u << 16);
+            const uint32_t q_lo1 = q_lo0 + (Cfg::kQBytes >> 4);
+            const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
+            const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((static_cast<uint32_t>(kChunkBytes) >> 4) << 16);
+            auto desc = [](uint32_t lo) -> uint64_t {
+                return (static_cast<uint64_t>(kDescHi) << 32) | lo;
+            };
+            auto issue_qk = [&](auto tc, int stage) {
+                constexpr int t = decltype(tc)::value;
+                const uint32_t qlo = (t == 0) ? q_lo0 : q_lo1;
+                const uint32_t klo = k_lo0 + stage * (Cfg::kKBytes >> 4);
                 const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1);
 #pragma unroll
                 for (int k = 0; k < DQK / 16; ++k) {
-                    const uint32_t koff = (k / 4) * kChunkBytes + (k % 4) * 32;
-                    mma_ss(tS, make_smem_desc_sw128(q_base + koff, 16, 1024),
-                           make_smem_desc_sw128(k_base + koff, 16, 1024), kIdescQK, k > 0 ? 1u : 0u);
+                    constexpr int dummy = 0; (void)dummy;
+                    const uint32_t koff = ((k / 4) * kChunkBytes + (k % 4) * 32) >> 4;
+                    mma_ss(tS, desc(qlo + koff), desc(klo + koff), kIdescQK, k > 0 ? 1u : 0u);
                 }
             };
-            auto issue_pv = [&](int t, int stage, bool accumulate) {
-                const uint32_t v_base = sV + stage * Cfg::kVBytes;
+            // O_t += P_t[:, 64*half .. 64*half+63] V_j[64*half .., :]  (four k-steps of 16 keys)
+            auto issue_pv_half = [&](auto tc, auto hc, int stage, uint32_t accumulate) {
+                constexpr int t = decltype(tc)::value;
+                constexpr int half = decltype(hc)::value;
+                const uint32_t vlo = v_lo0 + stage * (Cfg::kVBytes >> 4);
                 const uint32_t tP = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1);
                 const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1);
 #pragma unroll
-                for (int kk = 0; kk < kTileN / 16; ++kk) {
-                    mma_ts(tO, tP + kk * 8, make_smem_desc_sw128(v_base + kk * 2048, kChunkBytes, 1024),
-                           kIdescPV, (accumulate || kk > 0) ? 1u : 0u);
-                }
+                for (int kk = 4 * half; kk < 4 * half + 4; ++kk)
+                    mma_ts(tO, tP + kk * 8, desc(vlo + kk * (2048 >> 4)), kIdescPV,
+                           (half == 0 && kk == 0) ? accumulate : 1u);
             };
             bool ok = mbar_wait(smem_addr(&sh.k_full[0]), 0, wctx, kSiteMmaKvFull);
-#pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                if (n_kv[t] == 0 || !ok) continue;
+            auto prologue = [&](auto tc) {
+                constexpr int t = decltype(tc)::value;
+                if ((t == 0 ? nkv_0 : nkv_1) == 0 || !ok) return;
                 ok = mbar_wait(smem_addr(&sh.q_full[t]), 0, wctx, kSiteMmaQFull);
-                if (!ok) break;
+                if (!ok) return;
                 tc_fence_after_sync();
-                issue_qk(t, 0);
+                issue_qk(tc, 0);
                 tc_commit(smem_addr(&sh.s_full[t]));
-            }
+            };
+            prologue(IntC<0>{});
+            prologue(IntC<1>{});
             if (ok) tc_commit(smem_addr(&sh.k_empty[0]));
+            int sv = 0, sk = (NK > 1) ? 1 : 0;       // stage of V_j and of K_{j+1}
+            uint32_t ph_v = 0, ph_k = (NK > 1) ? 0u : 1u;
             for (int j = 0; j < n_max && ok; ++j) {
-                const int sv = j % NV;
-                const int sk = (j + 1) % NK;
-                ok = mbar_wait(smem_addr(&sh.v_full[sv]), (j / NV) & 1, wctx, kSiteMmaKvFull);
+                FA_TRACE_STAMP(2, j, 8);
+                ok = mbar_wait(smem_addr(&sh.v_full[sv]), ph_v, wctx, kSiteMmaKvFull);
+                FA_TRACE_STAMP(2, j, 9);
                 bool k_ready = false;
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    if (j >= n_kv[t] || !ok) continue;
-                    ok = mbar_wait(smem_addr(&sh.p_full[t]), j & 1, wctx, kSiteMmaPFull);
-                    if (!ok) break;
+                auto step = [&](auto tc) {
+                    constexpr int t = decltype(tc)::value;
+                    const int nkv_t = (t == 0) ? nkv_0 : nkv_1;
+                    if (j >= nkv_t || !ok) return;
+                    FA_TRACE_STAMP(2, j, t * 4 + 0);
+                    ok = mbar_wait(smem_addr(&sh.p_half[t]), j & 1, wctx, kSiteMmaPFull);
+                    if (!ok) return;
                     tc_fence_after_sync();
-                    issue_pv(t, sv, j > 0);
-                    if (j + 1 < n_kv[t]) {
+                    FA_TRACE_STAMP(2, j, t * 4 + 1);
+                    issue_pv_half(tc, IntC<0>{}, sv, j > 0 ? 1u : 0u);
+                    ok = mbar_wait(smem_addr(&sh.p_full[t]), j & 1, wctx, kSiteMmaPFull);
+                    if (!ok) return;
+                    tc_fence_after_sync();
+                    issue_pv_half(tc, IntC<1>{}, sv, 1u);
+                    FA_TRACE_STAMP(2, j, t * 4 + 2);
+                    if (j + 1 < nkv_t) {
                         if (!k_ready) {
-                            ok = mbar_wait(smem_addr(&sh.k_full[sk]), ((j + 1) / NK) & 1, wctx, kSiteMmaKvFull);
-                            if (!ok) break;
+                            ok = mbar_wait(smem_addr(&sh.k_full[sk]), ph_k, wctx, kSiteMmaKvFull);
+                            if (!ok) return;
                             tc_fence_after_sync();
                             k_ready = true;
                         }
-                        issue_qk(t, sk);
+                        issue_qk(tc, sk);
                         tc_commit(smem_addr(&sh.s_full[t]));
+                        FA_TRACE_STAMP(2, j, t * 4 + 3);
                     } else {
                         tc_commit(smem_addr(&sh.o_final[t]));
                     }
-                }
+                };
+                step(IntC<0>{});
+                step(IntC<1>{});
                 if (!ok) break;
+                FA_TRACE_STAMP(2, j, 10);
                 tc_commit(smem_addr(&sh.v_empty[sv]));
                 if (j + 1 < n_max) tc_commit(smem_addr(&sh.k_empty[sk]));
+                FA_TRACE_STAMP(2, j, 11);
+                if (++sv == NV) { sv = 0; ph_v ^= 1u; }
+                if (++sk == NK) { sk = 0; ph_k ^= 1u; }
             }
         }
     } else if (warp == 13) {
         // ============================================================ TMA loads
+        setmaxnreg_dec<kRegsOther>();
         if (lane == 0 && n_max > 0) {
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
-                if (n_kv[t] == 0) continue;
+                if ((t == 0 ? nkv_0 : nkv_1) == 0) continue;
                 const uint32_t bar = smem_addr(&sh.q_full[t]);
                 mbar_arrive_expect_tx(bar, Cfg::kQBytes);
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kQChunks; ++cc)
                     tma_load_3d(sQ + t * Cfg::kQBytes + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols,
-                                i0[t], q_idx);
+                                t == 0 ? i0_0 : i0_1, q_idx);
             }
             bool ok = true;
             for (int j = 0; j < n_max && ok; ++j) {
@@ -416,6 +492,10 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 }
             }
         }
+    }
+
+    else {
+        setmaxnreg_dec<kRegsOther>();     // idle warps of the fourth warpgroup
     }
 
     // ---------------------------------------------------------------- teardown (all warps)

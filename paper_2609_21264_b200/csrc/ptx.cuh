@@ -280,7 +280,7 @@ FA_DEVI void tmem_ld_x16(uint32_t taddr, uint32_t (&r)[16]) {
         : "memory");
 }
 
-FA_DEVI void tmem_ld_x32(uint32_t taddr, uint32_t (&r)[32]) {
+FA_DEVI void tmem_ld_x32(uint32_t taddr, uint32_t* r) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
