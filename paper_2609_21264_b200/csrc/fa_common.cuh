@@ -17,7 +17,7 @@ enum WaitSite : uint32_t {
     kSiteSimpleQ = 0x0101, kSiteSimpleK = 0x0102, kSiteSimpleV = 0x0103, kSiteSimpleMma = 0x0104,
     kSiteLoadKvEmpty = 0x0201, kSiteLoadQEmpty = 0x0202,
     kSiteMmaQFull = 0x0301, kSiteMmaKvFull = 0x0302, kSiteMmaPFull = 0x0303,
-    kSiteMmaOReady = 0x0304, kSiteMmaSFree = 0x0305,
+    kSiteMmaOReady = 0x0304, kSiteMmaSFree = 0x0305, kSiteMmaTurn = 0x0306,
     kSiteSoftmaxSFull = 0x0401, kSiteSoftmaxPFree = 0x0402, kSiteSoftmaxCorrFree = 0x0403,
     kSiteCorrScale = 0x0501, kSiteCorrPvDone = 0x0502, kSiteCorrFinal = 0x0503,
     kSiteEpiOFull = 0x0601,
@@ -39,7 +39,7 @@ struct FwdParams {
 };
 
 #ifdef FA_TRACE
-constexpr int kTraceIters = 64, kTraceEvents = 16, kTraceRoles = 4;   // roles: softmax0, softmax1, mma, corr
+constexpr int kTraceIters = 64, kTraceEvents = 16, kTraceRoles = 6;   // roles: softmax0, softmax1, mma, corr
 #define FA_TRACE_STAMP(role, iter, ev)                                                          \
     do {                                                                                        \
         if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (iter) < kTraceIters) \

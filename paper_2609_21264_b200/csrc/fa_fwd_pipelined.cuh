@@ -6,9 +6,10 @@
 //               final normalisation and stores
 //   warps 4-7   softmax of query tile 1
 //   warps 8-11  correction: rescale of the O accumulators when a reference maximum moved
-//   warp  12    MMA issue (one thread): S_t = Q_t K_j^T and O_t += P_t V_j with tcgen05
-//   warp  13    TMA loads of Q_t, K_j, V_j into mbarrier-guarded shared-memory rings
-//   warps 14-15 idle (they keep the fourth warpgroup complete)
+//   warps 12,13 MMA issue (one thread each, one per query tile): S_t = Q_t K_j^T and
+//               O_t += P_t V_j with tcgen05
+//   warp  14    TMA loads of Q_t, K_j, V_j into mbarrier-guarded shared-memory rings
+//   warp  15    idle (it keeps the fourth warpgroup complete)
 // While one softmax warpgroup works on S_t(j), the tensor core runs the MMAs of
 // the other tile, so the exponentials overlap the contractions.
 //
@@ -52,6 +53,15 @@ template <int V>
 struct IntC { static constexpr int value = V; };
 
 constexpr float kRescaleThresholdLog2 = 8.0f;
+// Of every four pairs of exponentials, this many are evaluated by the polynomial on the FMA
+// pipe (on tiles without masked entries); the rest use MUFU ex2.  Measured on B200 with this
+// schedule, where one softmax warp per scheduler is active at a time, the offload does not pay
+// (a lone warp is issue-bound, and the polynomial costs more issue slots than it frees MUFU
+// cycles), so the default is 0; the option is kept for schedules with more warps in flight.
+#ifndef FA_POLY_PAIRS_PER_4
+#define FA_POLY_PAIRS_PER_4 0
+#endif
+constexpr int kPolyPairsPer4 = FA_POLY_PAIRS_PER_4;
 // Registers per thread after the per-role reallocation (512 threads start with 128 each):
 // 256 softmax threads x 192 + 128 correction threads x 64 + 128 other threads x 64 = 65536.
 constexpr int kRegsSoftmax = 192, kRegsCorrection = 64, kRegsOther = 64;
@@ -65,6 +75,7 @@ struct PipeShared {
     uint64_t p_full[2];      // softmax -> MMA: all of P_t(j) written
     uint64_t scale_full[2];  // softmax -> correction: alpha of iteration j published
     uint64_t o_final[2];     // MMA -> softmax: last PV of tile t done, O_t is final
+    uint64_t turn[2];        // MMA thread 1-t -> MMA thread t: your turn to issue
     float alpha[2][2][kTileM];   // [tile][j & 1][row]
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -130,17 +141,18 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         for (int t = 0; t < 2; ++t) {
             mbar_init(smem_addr(&sh.q_full[t]), 1);
             mbar_init(smem_addr(&sh.s_full[t]), 1);
-            mbar_init(smem_addr(&sh.p_half[t]), 8);       // 4 softmax warps + 4 correction warps
-            mbar_init(smem_addr(&sh.p_full[t]), 4);       // 4 softmax warps
+            mbar_init(smem_addr(&sh.p_half[t]), 8);       // unused in this schedule
+            mbar_init(smem_addr(&sh.p_full[t]), 8);       // 4 softmax warps + 4 correction warps
             mbar_init(smem_addr(&sh.scale_full[t]), 4);
             mbar_init(smem_addr(&sh.o_final[t]), 1);
+            mbar_init(smem_addr(&sh.turn[t]), 1);
         }
 #pragma unroll
         for (int s = 0; s < 4; ++s) {
             mbar_init(smem_addr(&sh.k_full[s]), 1);
-            mbar_init(smem_addr(&sh.k_empty[s]), 1);
+            mbar_init(smem_addr(&sh.k_empty[s]), 2);      // one arrival per MMA-issuing thread
             mbar_init(smem_addr(&sh.v_full[s]), 1);
-            mbar_init(smem_addr(&sh.v_empty[s]), 1);
+            mbar_init(smem_addr(&sh.v_empty[s]), 2);
         }
         fence_mbar_init();
     }
@@ -148,7 +160,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         tmem_alloc(smem_addr(&sh.tmem_base), Cfg::kTmemCols);
         tmem_relinquish_alloc_permit();
     }
-    if (warp == 13 && lane == 0) {
+    if (warp == 14 && lane == 0) {
         prefetch_tensormap(&tm_q);
         prefetch_tensormap(&tm_k);
         prefetch_tensormap(&tm_v);
@@ -186,64 +198,32 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             ok = __all_sync(0xffffffffu, mbar_wait(bar_s, j & 1, wctx, kSiteSoftmaxSFull));
             if (!ok) break;
             tc_fence_after_sync();
-            if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(t, j, 0);
+            if (lane == 0 && ((warp & 3) == 0 || (warp & 3) == 2)) FA_TRACE_STAMP(t + ((warp & 3) == 2 ? 4 : 0), j, 0);
             const int j0 = j * kTileN;
             const bool need_mask = (j0 + kTileN - 1 > kmax_row);
 
-            // the whole score row in registers: four loads in flight, one wait
-            uint32_t s[kTileN];
-            tmem_ld_x32(tS + 0, s + 0);
-            tmem_ld_x32(tS + 32, s + 32);
-            tmem_ld_x32(tS + 64, s + 64);
-            tmem_ld_x32(tS + 96, s + 96);
-            tc_wait_ld();
-            if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(t, j, 1);
-            if (need_mask) {
-#pragma unroll
-                for (int e = 0; e < kTileN; ++e)
-                    if (j0 + e > kmax_row) s[e] = 0xff800000u;   // -inf
-            }
-            float mx;
-            {
-                float a[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) a[q] = -INFINITY;
-#pragma unroll
-                for (int e = 0; e < kTileN; e += 16) {
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        a[q] = fmax3(a[q], __uint_as_float(s[e + 2 * q]), __uint_as_float(s[e + 2 * q + 1]));
-                }
-                mx = fmaxf(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]));
-                mx = fmax3(mx, a[6], a[7]);
-            }
-            // advance the reference maximum only when the row maximum grew by more than the threshold
-            float alpha = 1.f;
-            if (mx > m_ref + tau_raw) {
-                alpha = exp2_approx((m_ref - mx) * c);    // r = exp(u' - u); 0 on the first tile
-                m_ref = mx;
-            }
-            sh.alpha[t][j & 1][row] = alpha;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_scale);
-            if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(t, j, 2);
-
-            const float mc = (m_ref == -INFINITY) ? 0.f : m_ref * c;
-            // Exponentials in place (packed FMA for the argument), row sum, bf16 P back to TMEM
-            // over the first half of S.  The exponentials of chunk q+1 are issued before chunk q
-            // is summed, converted and stored, so the MUFU pipe does not drain between chunks.
             const float2 c2 = make_float2(c, c);
-            const float2 nmc2 = make_float2(-mc, -mc);
+            float2 nmc2;
             float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
+            float alpha = 1.f;
+            uint32_t s[kTileN];
+            // Exponentials in place against the reference maximum (packed FMA for the argument).
             auto exp_chunk = [&](int q) {
 #pragma unroll
                 for (int e = 0; e < 32; e += 2) {
                     const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[q * 32 + e]),
                                                             __uint_as_float(s[q * 32 + e + 1])), c2, nmc2);
-                    s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
-                    s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
+                    if (((e / 2) & 3) < kPolyPairsPer4 && !need_mask) {   // this pair on the FMA pipe
+                        const float2 y = exp2_poly2(x);
+                        s[q * 32 + e] = __float_as_uint(y.x);
+                        s[q * 32 + e + 1] = __float_as_uint(y.y);
+                    } else {                                   // this pair on the MUFU pipe
+                        s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
+                        s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
+                    }
                 }
             };
+            // Row sum, bf16 conversion and store of one chunk of P (over the first half of S).
             auto emit_chunk = [&](int q) {
                 uint32_t pk[16];
 #pragma unroll
@@ -257,26 +237,64 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 }
                 tmem_st_x16(tS + q * 16, pk);
             };
-            exp_chunk(0);
+            // The exponentials do not wait for the row maximum: they start against the reference
+            // maximum carried over from earlier tiles while the maximum of this tile is reduced on
+            // the ALU pipe.  Only if some row of the warp grew past the threshold (always on the
+            // first tile, rarely afterwards) is the reference advanced and the pass repeated; no
+            // P has been stored yet at that point, so S is still intact in TMEM.
+#pragma unroll 1
+            for (;;) {
+                tmem_ld_x32(tS + 0, s + 0);
+                tmem_ld_x32(tS + 32, s + 32);
+                tmem_ld_x32(tS + 64, s + 64);
+                tmem_ld_x32(tS + 96, s + 96);
+                tc_wait_ld();
+                if (lane == 0 && ((warp & 3) == 0 || (warp & 3) == 2)) FA_TRACE_STAMP(t + ((warp & 3) == 2 ? 4 : 0), j, 1);
+                if (need_mask) {
+#pragma unroll
+                    for (int e = 0; e < kTileN; ++e)
+                        if (j0 + e > kmax_row) s[e] = 0xff800000u;   // -inf
+                }
+                const float mc = (m_ref == -INFINITY) ? 0.f : m_ref * c;
+                nmc2 = make_float2(-mc, -mc);
+                float a[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) a[q] = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < kTileN; e += 16) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        a[q] = fmax3(a[q], __uint_as_float(s[e + 2 * q]), __uint_as_float(s[e + 2 * q + 1]));
+                }
+                exp_chunk(0);
+                float mx = fmaxf(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]));
+                mx = fmax3(mx, a[6], a[7]);
+                const bool grow = mx > m_ref + tau_raw;
+                if (!__any_sync(0xffffffffu, grow)) break;
+                if (grow) {
+                    alpha = exp2_approx((m_ref - mx) * c);    // r = exp(u' - u); 0 on the first tile
+                    m_ref = mx;
+                }
+            }
+            sh.alpha[t][j & 1][row] = alpha;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_scale);
+            if (lane == 0 && ((warp & 3) == 0 || (warp & 3) == 2)) FA_TRACE_STAMP(t + ((warp & 3) == 2 ? 4 : 0), j, 2);
+
             exp_chunk(1);
             emit_chunk(0);
             exp_chunk(2);
             emit_chunk(1);
-            // first half of P (keys 0..63) is in flight: let the MMA warp start O += P V early
-            tc_wait_st();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_ph);
             exp_chunk(3);
             emit_chunk(2);
             emit_chunk(3);
             l = l * alpha + ((sum_a.x + sum_a.y) + (sum_b.x + sum_b.y));
-            if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(t, j, 3);
+            if (lane == 0 && ((warp & 3) == 0 || (warp & 3) == 2)) FA_TRACE_STAMP(t + ((warp & 3) == 2 ? 4 : 0), j, 3);
             tc_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_p);
-            if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(t, j, 4);
+            if (lane == 0 && ((warp & 3) == 0 || (warp & 3) == 2)) FA_TRACE_STAMP(t + ((warp & 3) == 2 ? 4 : 0), j, 4);
         }
         // epilogue: O = G' / s (bf16), lse = u * scale + ln s
         if (ok && i0_t < p.Sq) {
@@ -347,111 +365,116 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                     tc_fence_before_sync();
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_addr(&sh.p_half[t]));
+                if (lane == 0) mbar_arrive(smem_addr(&sh.p_full[t]));
                 if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(3, j, t * 4 + 1);
             }
         }
-    } else if (warp == 12) {
-        // ============================================================ MMA issue
+    } else if (warp == 12 || warp == 13) {
+        // ============================================================ MMA issue for tile t = warp - 12
+        // One issuing thread per query tile: tcgen05.mma issue blocks while the tensor pipe is
+        // busy, so a single thread serving both tiles would serialise their waits behind each
+        // other's MMAs.  The two threads touch disjoint TMEM (S_t, O_t) and share the K/V stages,
+        // whose "empty" barriers therefore count two arrivals.
         setmaxnreg_dec<kRegsOther>();
         if (lane == 0 && n_max > 0) {
+            const int t = warp - 12;
+            const int nkv_t = (t == 0) ? nkv_0 : nkv_1;
             constexpr uint32_t kIdescQK = make_idesc_bf16_f32(kTileM, kTileN, false, false);
             constexpr uint32_t kIdescPV = make_idesc_bf16_f32(kTileM, DV, false, true);
             // Descriptor words are built once.  Per MMA only the 14-bit start-address field of the
             // low word moves (shared-memory addresses stay below 2^18, so no carry leaves it).
             constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // sbo, version, swizzle
-            const uint32_t q_lo0 = ((sQ & 0x3FFFFu) >> 4) | (1u << 16);
-            const uint32_t q_lo1 = q_lo0 + (Cfg::kQBytes >> 4);
+            const uint32_t q_lo = (((sQ + t * Cfg::kQBytes) & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((static_cast<uint32_t>(kChunkBytes) >> 4) << 16);
+            const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1);   // P_t overlays it
+            const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1);
+            const uint32_t bar_s = smem_addr(&sh.s_full[t]);
+            const uint32_t bar_ph = smem_addr(&sh.p_half[t]);
+            const uint32_t bar_p = smem_addr(&sh.p_full[t]);
             auto desc = [](uint32_t lo) -> uint64_t {
                 return (static_cast<uint64_t>(kDescHi) << 32) | lo;
             };
-            auto issue_qk = [&](auto tc, int stage) {
-                constexpr int t = decltype(tc)::value;
-                const uint32_t qlo = (t == 0) ? q_lo0 : q_lo1;
+            auto issue_qk = [&](int stage) {
                 const uint32_t klo = k_lo0 + stage * (Cfg::kKBytes >> 4);
-                const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1);
 #pragma unroll
                 for (int k = 0; k < DQK / 16; ++k) {
-                    constexpr int dummy = 0; (void)dummy;
                     const uint32_t koff = ((k / 4) * kChunkBytes + (k % 4) * 32) >> 4;
-                    mma_ss(tS, desc(qlo + koff), desc(klo + koff), kIdescQK, k > 0 ? 1u : 0u);
+                    mma_ss(tS, desc(q_lo + koff), desc(klo + koff), kIdescQK, k > 0 ? 1u : 0u);
                 }
             };
             // O_t += P_t[:, 64*half .. 64*half+63] V_j[64*half .., :]  (four k-steps of 16 keys)
-            auto issue_pv_half = [&](auto tc, auto hc, int stage, uint32_t accumulate) {
-                constexpr int t = decltype(tc)::value;
+            auto issue_pv_half = [&](auto hc, int stage, uint32_t accumulate) {
                 constexpr int half = decltype(hc)::value;
                 const uint32_t vlo = v_lo0 + stage * (Cfg::kVBytes >> 4);
-                const uint32_t tP = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1);
-                const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1);
 #pragma unroll
                 for (int kk = 4 * half; kk < 4 * half + 4; ++kk)
-                    mma_ts(tO, tP + kk * 8, desc(vlo + kk * (2048 >> 4)), kIdescPV,
+                    mma_ts(tO, tS + kk * 8, desc(vlo + kk * (2048 >> 4)), kIdescPV,
                            (half == 0 && kk == 0) ? accumulate : 1u);
             };
-            bool ok = mbar_wait(smem_addr(&sh.k_full[0]), 0, wctx, kSiteMmaKvFull);
-            auto prologue = [&](auto tc) {
-                constexpr int t = decltype(tc)::value;
-                if ((t == 0 ? nkv_0 : nkv_1) == 0 || !ok) return;
-                ok = mbar_wait(smem_addr(&sh.q_full[t]), 0, wctx, kSiteMmaQFull);
-                if (!ok) return;
-                tc_fence_after_sync();
-                issue_qk(tc, 0);
-                tc_commit(smem_addr(&sh.s_full[t]));
+            // The two issuing threads alternate strictly, one block of MMAs each (round r of thread
+            // 0, then round r of thread 1, then round r+1 of thread 0, ...), so that the tiles stay
+            // half a period apart: the softmax of one tile runs under the MMAs of the other.  All
+            // mbarrier waits of a round happen before the thread takes its turn.
+            const uint32_t bar_turn_mine = smem_addr(&sh.turn[t]);
+            const uint32_t bar_turn_other = smem_addr(&sh.turn[t ^ 1]);
+            int round = 0;
+            auto take_turn = [&]() -> bool {
+                if (t == 0 && round == 0) return true;
+                const uint32_t parity = (t == 0) ? ((round - 1) & 1) : (round & 1);
+                return mbar_wait(bar_turn_mine, parity, wctx, kSiteMmaTurn);
             };
-            prologue(IntC<0>{});
-            prologue(IntC<1>{});
-            if (ok) tc_commit(smem_addr(&sh.k_empty[0]));
+            auto pass_turn = [&]() { mbar_arrive(bar_turn_other); ++round; };
+
+            bool ok = mbar_wait(smem_addr(&sh.k_full[0]), 0, wctx, kSiteMmaKvFull);
+            if (ok && nkv_t > 0) ok = mbar_wait(smem_addr(&sh.q_full[t]), 0, wctx, kSiteMmaQFull);
+            ok = ok && take_turn();
+            if (ok) {
+                if (nkv_t > 0) {
+                    tc_fence_after_sync();
+                    issue_qk(0);
+                    tc_commit(bar_s);
+                }
+                tc_commit(smem_addr(&sh.k_empty[0]));   // arrives at once if nothing was issued
+                pass_turn();
+            }
             int sv = 0, sk = (NK > 1) ? 1 : 0;       // stage of V_j and of K_{j+1}
             uint32_t ph_v = 0, ph_k = (NK > 1) ? 0u : 1u;
             for (int j = 0; j < n_max && ok; ++j) {
-                FA_TRACE_STAMP(2, j, 8);
+                const uint32_t bar_ve = smem_addr(&sh.v_empty[sv]);
+                const uint32_t bar_ke = smem_addr(&sh.k_empty[sk]);
+                // Both threads wait for every stage, also on iterations without work for their
+                // tile, so that neither arrives twice in one phase of an "empty" barrier.
                 ok = mbar_wait(smem_addr(&sh.v_full[sv]), ph_v, wctx, kSiteMmaKvFull);
-                FA_TRACE_STAMP(2, j, 9);
-                bool k_ready = false;
-                auto step = [&](auto tc) {
-                    constexpr int t = decltype(tc)::value;
-                    const int nkv_t = (t == 0) ? nkv_0 : nkv_1;
-                    if (j >= nkv_t || !ok) return;
+                if (ok && j + 1 < n_max) ok = mbar_wait(smem_addr(&sh.k_full[sk]), ph_k, wctx, kSiteMmaKvFull);
+                if (ok && j < nkv_t) {
                     FA_TRACE_STAMP(2, j, t * 4 + 0);
-                    ok = mbar_wait(smem_addr(&sh.p_half[t]), j & 1, wctx, kSiteMmaPFull);
-                    if (!ok) return;
-                    tc_fence_after_sync();
+                    ok = mbar_wait(bar_p, j & 1, wctx, kSiteMmaPFull);
                     FA_TRACE_STAMP(2, j, t * 4 + 1);
-                    issue_pv_half(tc, IntC<0>{}, sv, j > 0 ? 1u : 0u);
-                    ok = mbar_wait(smem_addr(&sh.p_full[t]), j & 1, wctx, kSiteMmaPFull);
-                    if (!ok) return;
-                    tc_fence_after_sync();
-                    issue_pv_half(tc, IntC<1>{}, sv, 1u);
-                    FA_TRACE_STAMP(2, j, t * 4 + 2);
-                    if (j + 1 < nkv_t) {
-                        if (!k_ready) {
-                            ok = mbar_wait(smem_addr(&sh.k_full[sk]), ph_k, wctx, kSiteMmaKvFull);
-                            if (!ok) return;
-                            tc_fence_after_sync();
-                            k_ready = true;
-                        }
-                        issue_qk(tc, sk);
-                        tc_commit(smem_addr(&sh.s_full[t]));
-                        FA_TRACE_STAMP(2, j, t * 4 + 3);
-                    } else {
-                        tc_commit(smem_addr(&sh.o_final[t]));
-                    }
-                };
-                step(IntC<0>{});
-                step(IntC<1>{});
+                }
+                ok = ok && take_turn();
                 if (!ok) break;
-                FA_TRACE_STAMP(2, j, 10);
-                tc_commit(smem_addr(&sh.v_empty[sv]));
-                if (j + 1 < n_max) tc_commit(smem_addr(&sh.k_empty[sk]));
-                FA_TRACE_STAMP(2, j, 11);
+                tc_fence_after_sync();
+                if (j < nkv_t) {
+                    issue_pv_half(IntC<0>{}, sv, j > 0 ? 1u : 0u);
+                    issue_pv_half(IntC<1>{}, sv, 1u);
+                    FA_TRACE_STAMP(2, j, t * 4 + 2);
+                }
+                if (j + 1 < nkv_t) {
+                    issue_qk(sk);
+                    tc_commit(bar_s);
+                    FA_TRACE_STAMP(2, j, t * 4 + 3);
+                } else if (j + 1 == nkv_t) {
+                    tc_commit(smem_addr(&sh.o_final[t]));
+                }
+                tc_commit(bar_ve);
+                if (j + 1 < n_max) tc_commit(bar_ke);
+                pass_turn();
                 if (++sv == NV) { sv = 0; ph_v ^= 1u; }
                 if (++sk == NK) { sk = 0; ph_k ^= 1u; }
             }
         }
-    } else if (warp == 13) {
+    } else if (warp == 14) {
         // ============================================================ TMA loads
         setmaxnreg_dec<kRegsOther>();
         if (lane == 0 && n_max > 0) {
@@ -495,7 +518,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     }
 
     else {
-        setmaxnreg_dec<kRegsOther>();     // idle warps of the fourth warpgroup
+        setmaxnreg_dec<kRegsOther>();     // idle warp of the fourth warpgroup
     }
 
     // ---------------------------------------------------------------- teardown (all warps)
