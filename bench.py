@@ -297,12 +297,23 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--config", type=int, default=1, help="index into the five benchmark configurations")
+    ap.add_argument("--shape", default=None,
+                    help="time a custom shape instead of --config, e.g. "
+                         "B=1,Hq=16,Hkv=16,S=8192,dqk=128,dv=128,causal=1 (used for small ncu captures)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the short timing of the other configs")
     args = ap.parse_args()
     w = workloads.config(args.config)
+    if args.shape:
+        kv = dict(item.split("=") for item in args.shape.split(","))
+        S = int(kv.get("S", 2048))
+        dqk = int(kv.get("dqk", 128))
+        w = workloads.Workload("custom_" + args.shape.replace(",", "_").replace("=", ""), int(kv.get("B", 1)),
+                               int(kv.get("Hq", 16)), int(kv.get("Hkv", kv.get("Hq", 16))),
+                               int(kv.get("Sq", S)), int(kv.get("Sk", S)), dqk, int(kv.get("dv", dqk)),
+                               bool(int(kv.get("causal", 1))), dqk ** -0.5)
 
     if args.impl == "reference":
         rank, world, _ = launch.env_rank()

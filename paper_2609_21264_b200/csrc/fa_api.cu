@@ -143,7 +143,9 @@ fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const 
     auto kernel = fa::fa_fwd_pipelined_kernel<DQK, DV>;
     fa_status s = ensure_smem_attr(h, slot, kernel, smem);
     if (s != FA_OK) return s;
-    dim3 grid((p.n_q_tiles + 1) / 2, p.Hq, p.B);
+    const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq * p.B;
+    if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+    dim3 grid(static_cast<unsigned>(n_ctas), 1, 1);
     kernel<<<grid, fa::PipeCfg<DQK, DV>::kThreads, smem, st>>>(mq, mk, mv, p);
     if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
     h->launches += 1;
@@ -300,6 +302,18 @@ fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, 
     p.causal = causal ? 1 : 0;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
+    {
+        // Heads whose K and V (read again by every query tile of the head) fit in about a third of
+        // the 126 MB L2 together; at least one K/V head, i.e. one GQA group of query heads.
+        const long long kv_bytes = static_cast<long long>(Sk) * (dqk + dv) * 2;
+        const long long budget = 48ll << 20;
+        long long kv_heads = budget / kv_bytes;
+        if (kv_heads < 1) kv_heads = 1;
+        long long hpg = kv_heads * (Hq / Hkv);
+        const long long n_bh = static_cast<long long>(B) * Hq;
+        if (hpg > n_bh) hpg = n_bh;
+        p.heads_per_group = static_cast<int>(hpg);
+    }
     p.status = h->status_dev;
     p.wait_limit_ns = h->wait_limit_ns;
 #ifdef FA_TRACE

@@ -31,6 +31,7 @@ struct FwdParams {
     int causal;
     float scale_log2;         // scale * log2(e): scores are handled in log2 units
     int n_q_tiles;            // ceil(Sq / 128)
+    int heads_per_group;      // (batch, head) instances scheduled together (their K/V share L2)
     uint32_t* status;         // [0] = fa_status, [1] = wait site; mapped host memory
     unsigned long long wait_limit_ns;
 #ifdef FA_TRACE

@@ -120,9 +120,20 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     const uint32_t sK = sQ + 2 * Cfg::kQBytes;                   // NK stages
     const uint32_t sV = sK + NK * Cfg::kKBytes;                  // NV stages
 
-    const int pair = static_cast<int>(gridDim.x) - 1 - static_cast<int>(blockIdx.x);   // heavy first
-    const int hq = blockIdx.y;
-    const int b = blockIdx.z;
+    // 1-D grid.  The (batch, head) instances are cut into groups whose K/V fit in L2 together;
+    // groups run one after the other, and inside a group the CTAs are in longest-processing-time
+    // order: every head's last (with a causal mask: heaviest) pair of query tiles first, then the
+    // pair before it, and so on.  Consecutive CTAs are consecutive query heads (shared K/V heads).
+    const int n_pairs = (p.n_q_tiles + 1) / 2;
+    const int n_bh = p.B * p.Hq;
+    const int group = static_cast<int>(blockIdx.x) / (n_pairs * p.heads_per_group);
+    const int bh0 = group * p.heads_per_group;
+    const int group_size = (n_bh - bh0 < p.heads_per_group) ? (n_bh - bh0) : p.heads_per_group;
+    const int local = static_cast<int>(blockIdx.x) - group * n_pairs * p.heads_per_group;
+    const int pair = n_pairs - 1 - local / group_size;
+    const int bh = bh0 + local % group_size;
+    const int hq = bh % p.Hq;
+    const int b = bh / p.Hq;
     const int kvh = hq / (p.Hq / p.Hkv);
     const int q_idx = b * p.Hq + hq;
     const int kv_idx = b * p.Hkv + kvh;
