@@ -152,8 +152,8 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         for (int t = 0; t < 2; ++t) {
             mbar_init(smem_addr(&sh.q_full[t]), 1);
             mbar_init(smem_addr(&sh.s_full[t]), 1);
-            mbar_init(smem_addr(&sh.p_half[t]), 8);       // unused in this schedule
-            mbar_init(smem_addr(&sh.p_full[t]), 8);       // 4 softmax warps + 4 correction warps
+            mbar_init(smem_addr(&sh.p_half[t]), 8);       // 4 softmax warps + 4 correction warps
+            mbar_init(smem_addr(&sh.p_full[t]), 4);       // 4 softmax warps
             mbar_init(smem_addr(&sh.scale_full[t]), 4);
             mbar_init(smem_addr(&sh.o_final[t]), 1);
             mbar_init(smem_addr(&sh.turn[t]), 1);
@@ -297,6 +297,11 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             exp_chunk(2);
             emit_chunk(1);
             exp_chunk(3);
+            // first half of P (keys 0..63) is stored: the MMA thread may start O += P V on it
+            tc_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_ph);
             emit_chunk(2);
             emit_chunk(3);
             l = l * alpha + ((sum_a.x + sum_a.y) + (sum_b.x + sum_b.y));
@@ -376,7 +381,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                     tc_fence_before_sync();
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_addr(&sh.p_full[t]));
+                if (lane == 0) mbar_arrive(smem_addr(&sh.p_half[t]));
                 if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(3, j, t * 4 + 1);
             }
         }
@@ -460,7 +465,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 if (ok && j + 1 < n_max) ok = mbar_wait(smem_addr(&sh.k_full[sk]), ph_k, wctx, kSiteMmaKvFull);
                 if (ok && j < nkv_t) {
                     FA_TRACE_STAMP(2, j, t * 4 + 0);
-                    ok = mbar_wait(bar_p, j & 1, wctx, kSiteMmaPFull);
+                    ok = mbar_wait(bar_ph, j & 1, wctx, kSiteMmaPFull);
                     FA_TRACE_STAMP(2, j, t * 4 + 1);
                 }
                 ok = ok && take_turn();
@@ -468,6 +473,11 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 tc_fence_after_sync();
                 if (j < nkv_t) {
                     issue_pv_half(IntC<0>{}, sv, j > 0 ? 1u : 0u);
+                    // the other thread has nothing to issue while this tile's softmax is finishing,
+                    // so waiting here with the turn in hand costs nothing
+                    ok = mbar_wait(bar_p, j & 1, wctx, kSiteMmaPFull);
+                    if (!ok) break;
+                    tc_fence_after_sync();
                     issue_pv_half(IntC<1>{}, sv, 1u);
                     FA_TRACE_STAMP(2, j, t * 4 + 2);
                 }
