@@ -63,13 +63,29 @@ typedef struct fa_config {
     int32_t device;           /* CUDA device ordinal; -1 = the calling thread's current device */
     uint32_t flags;           /* bitwise OR of FA_FLAG_*; other bits must be 0                 */
     uint32_t wait_limit_ms;   /* limit of every device-side wait; 0 = default (2000 ms)        */
+    uint32_t kv_splits;       /* split-KV: 0 = library decides, 1 = never split, n > 1 = use n
+                                 splits whenever the scratch buffer can hold the partials      */
+    uint64_t scratch_bytes;   /* device scratch for split-KV partials, allocated by fa_create;
+                                 0 = default (32 MiB)                                          */
 } fa_config;
+
+/*
+ * Split-KV (the spatial decomposition of Algorithm 2: the key/value range of a query tile is
+ * partitioned over C CTAs, each running Algorithm 1 on its part, and the partial results are
+ * merged with the online-softmax reduction): used when a problem has too few query tiles to
+ * fill the GPU (short Sq with long Sk).  The partials (fp32 O_c and lse_c per query row) live
+ * in the handle's scratch buffer, and a second small kernel merges them.  The printed merge of
+ * Algorithm 2 rescales with the previous partial's maximum; the library uses the corrected
+ * form lse = ln sum_c exp(lse_c), O = sum_c exp(lse_c - lse) O_c.
+ */
 
 /*
  * Create a handle bound to one device.  `cfg` may be NULL (defaults, current
  * device).  The handle owns a small status word (pinned host memory mapped to
- * the device), a cache of TMA tensor maps keyed by (pointer, shape), and the
- * staging buffers of fa_forward_host.  Allocates; call outside stream capture.
+ * the device), a cache of TMA tensor maps keyed by (pointer, shape), the split-KV
+ * scratch buffer and the staging buffers of fa_forward_host.  Allocates; call
+ * outside stream capture.  A struct_size smaller than the current fa_config is accepted:
+ * missing trailing fields take their defaults.
  */
 fa_status fa_create(fa_handle** out, const fa_config* cfg);
 
@@ -90,7 +106,9 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg);
  * The call is asynchronous: it validates, enqueues the kernel on `stream` and
  * returns.  The caller owns all buffers and keeps them alive until the stream
  * has passed the kernel; O must not alias an input.  The library does not
- * synchronise and does not allocate device memory here.  Argument and launch
+ * synchronise and does not allocate device memory here (split-KV partials use the
+ * scratch buffer allocated by fa_create; launches through one handle must therefore not
+ * overlap on the device: use one handle per stream).  Argument and launch
  * errors are returned at once; a device-side timeout shows up in
  * fa_last_status after the caller has synchronised the stream.
  */
@@ -132,11 +150,13 @@ const char* fa_strerror(fa_status s);
 
 /*
  * Introspection used by tests and the benchmark: number of kernel launches
- * issued through the handle so far, and the name of the kernel variant the
- * last fa_forward selected (static string; "" before the first call).
+ * issued through the handle so far (a split-KV forward is two launches), the
+ * name of the kernel variant the last fa_forward selected (static string; ""
+ * before the first call), and the number of K/V splits it used.
  */
 uint64_t fa_launch_count(const fa_handle* h);
 const char* fa_last_kernel_name(const fa_handle* h);
+int fa_last_kv_splits(const fa_handle* h);   /* K/V splits the last fa_forward used (1 = none) */
 
 #ifdef __cplusplus
 }

@@ -23,7 +23,7 @@ FA_ERR_OOM = 6
 FA_FLAG_SERIAL_KERNEL = 1
 
 EXPORTS = ("fa_create", "fa_forward", "fa_forward_host", "fa_last_status", "fa_destroy",
-           "fa_strerror", "fa_launch_count", "fa_last_kernel_name")
+           "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits")
 
 
 class FaError(RuntimeError):
@@ -34,7 +34,8 @@ class FaError(RuntimeError):
 
 class fa_config(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32), ("device", ctypes.c_int32),
-                ("flags", ctypes.c_uint32), ("wait_limit_ms", ctypes.c_uint32)]
+                ("flags", ctypes.c_uint32), ("wait_limit_ms", ctypes.c_uint32),
+                ("kv_splits", ctypes.c_uint32), ("scratch_bytes", ctypes.c_uint64)]
 
 
 _lib = None
@@ -72,6 +73,8 @@ def load():
     lib.fa_launch_count.argtypes = [vp]
     lib.fa_last_kernel_name.restype = ctypes.c_char_p
     lib.fa_last_kernel_name.argtypes = [vp]
+    lib.fa_last_kv_splits.restype = i32
+    lib.fa_last_kv_splits.argtypes = [vp]
     _lib = lib
     return lib
 
@@ -80,9 +83,10 @@ def fa_strerror(status: int) -> str:
     return load().fa_strerror(int(status)).decode()
 
 
-def fa_create(device: int = -1, flags: int = 0, wait_limit_ms: int = 0) -> int:
+def fa_create(device: int = -1, flags: int = 0, wait_limit_ms: int = 0, kv_splits: int = 0,
+              scratch_bytes: int = 0) -> int:
     """Returns an opaque handle (integer address).  Raises FaError on failure."""
-    cfg = fa_config(ctypes.sizeof(fa_config), device, flags, wait_limit_ms)
+    cfg = fa_config(ctypes.sizeof(fa_config), device, flags, wait_limit_ms, kv_splits, scratch_bytes)
     out = ctypes.c_void_p()
     st = load().fa_create(ctypes.byref(out), ctypes.byref(cfg))
     if st != FA_OK:
@@ -115,6 +119,10 @@ def fa_destroy(h) -> int:
 
 def fa_launch_count(h) -> int:
     return int(load().fa_launch_count(h))
+
+
+def fa_last_kv_splits(h) -> int:
+    return int(load().fa_last_kv_splits(h))
 
 
 def fa_last_kernel_name(h) -> str:

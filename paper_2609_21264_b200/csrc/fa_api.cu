@@ -35,9 +35,14 @@ constexpr int kMapCacheSize = 16;
 
 struct fa_handle {
     int device = 0;
+    int num_sms = 1;
     uint32_t flags = 0;
     uint32_t* status_host = nullptr;   // pinned + mapped: [0] status, [1] wait site
     uint32_t* status_dev = nullptr;
+    uint32_t kv_splits_cfg = 0;              // 0 auto, 1 never, n force
+    void* scratch = nullptr;                 // split-KV partials
+    size_t scratch_bytes = 0;
+    int last_splits = 1;
     unsigned long long wait_limit_ns = 2000ull * 1000000ull;
     EncodeTiledFn encode = nullptr;
     std::vector<MapEntry> maps;
@@ -143,13 +148,44 @@ fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const 
     auto kernel = fa::fa_fwd_pipelined_kernel<DQK, DV>;
     fa_status s = ensure_smem_attr(h, slot, kernel, smem);
     if (s != FA_OK) return s;
-    const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq * p.B;
+    const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq * p.B * p.kv_splits;
     if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     dim3 grid(static_cast<unsigned>(n_ctas), 1, 1);
     kernel<<<grid, fa::PipeCfg<DQK, DV>::kThreads, smem, st>>>(mq, mk, mv, p);
     if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
     h->launches += 1;
+    if (p.kv_splits > 1) {
+        const long long n_rows = static_cast<long long>(p.B) * p.Hq * p.Sq;
+        const long long blocks = (n_rows + 3) / 4;
+        if (blocks > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+        fa::fa_combine_kernel<DV><<<static_cast<unsigned>(blocks), 128, 0, st>>>(
+            p.o_part, p.lse_part, p.O, p.lse, n_rows, p.kv_splits);
+        if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
+        h->launches += 1;
+    }
     return FA_OK;
+}
+
+// Number of K/V splits for a problem: 1 unless the query tiles alone leave most SMs idle and the
+// K/V range is long enough to cut; never more than the scratch buffer can hold partials for.
+int choose_kv_splits(const fa_handle* h, int B, int Hq, int Sq, int Sk, int dv, int causal, int n_q_tiles) {
+    const long long items = static_cast<long long>((n_q_tiles + 1) / 2) * B * Hq;
+    int max_tiles = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, causal);
+    if (!causal) max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
+    int splits = 1;
+    if (h->kv_splits_cfg == 1) return 1;
+    if (h->kv_splits_cfg > 1) {
+        splits = static_cast<int>(h->kv_splits_cfg);
+    } else if (items * 2 <= h->num_sms && max_tiles >= 8) {
+        splits = static_cast<int>(h->num_sms / items);
+        if (splits > max_tiles / 4) splits = max_tiles / 4;      // at least four tiles per split
+        if (splits > 32) splits = 32;
+    }
+    if (splits > max_tiles) splits = max_tiles;
+    if (splits < 1) splits = 1;
+    const long long rows = static_cast<long long>(B) * Hq * Sq;
+    while (splits > 1 && static_cast<unsigned long long>(splits) * rows * (dv + 1) * 4ull > h->scratch_bytes) --splits;
+    return splits;
 }
 
 bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
@@ -197,13 +233,20 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg) {
     *out = nullptr;
     int device = -1;
     uint32_t flags = 0, limit_ms = 0;
+    uint32_t kv_splits_cfg = 0;
+    uint64_t scratch_bytes = 0;
     if (cfg) {
-        if (cfg->struct_size < sizeof(fa_config)) return FA_ERR_INVALID_ARG;
+        // versioned by struct_size: the first four fields are mandatory, later ones optional
+        if (cfg->struct_size < 16 || cfg->struct_size > sizeof(fa_config)) return FA_ERR_INVALID_ARG;
         device = cfg->device;
         flags = cfg->flags;
         limit_ms = cfg->wait_limit_ms;
+        if (cfg->struct_size >= 20) kv_splits_cfg = cfg->kv_splits;
+        if (cfg->struct_size >= sizeof(fa_config)) scratch_bytes = cfg->scratch_bytes;
         if (flags & ~FA_FLAG_SERIAL_KERNEL) return FA_ERR_INVALID_ARG;
+        if (kv_splits_cfg > 64) return FA_ERR_INVALID_ARG;
     }
+    if (scratch_bytes == 0) scratch_bytes = 32ull << 20;
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || count <= 0) {
         cudaGetLastError();
@@ -217,11 +260,16 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg) {
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess)
         return FA_ERR_CUDA;
     if (major != 10) return FA_ERR_NO_DEVICE;
+    int num_sms = 0;
+    if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || num_sms <= 0)
+        return FA_ERR_CUDA;
 
     fa_handle* h = new (std::nothrow) fa_handle();
     if (!h) return FA_ERR_OOM;
     h->device = device;
+    h->num_sms = num_sms;
     h->flags = flags;
+    h->kv_splits_cfg = kv_splits_cfg;
     if (limit_ms) h->wait_limit_ns = static_cast<unsigned long long>(limit_ms) * 1000000ull;
     h->maps.reserve(kMapCacheSize);
 
@@ -248,6 +296,13 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg) {
         delete h;
         return FA_ERR_CUDA;
     }
+    if (cudaMalloc(&h->scratch, scratch_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFreeHost(h->status_host);
+        delete h;
+        return FA_ERR_OOM;
+    }
+    h->scratch_bytes = scratch_bytes;
     *out = h;
     return FA_OK;
 }
@@ -258,6 +313,7 @@ fa_status fa_destroy(fa_handle* h) {
     fa_status s = FA_OK;
     for (int i = 0; i < 5; ++i)
         if (h->stage[i] && cudaFree(h->stage[i]) != cudaSuccess) s = FA_ERR_CUDA;
+    if (h->scratch && cudaFree(h->scratch) != cudaSuccess) s = FA_ERR_CUDA;
     if (h->status_host && cudaFreeHost(h->status_host) != cudaSuccess) s = FA_ERR_CUDA;
     delete h;
     return s;
@@ -274,6 +330,7 @@ fa_status fa_last_status(fa_handle* h, uint32_t* detail) {
 }
 
 uint64_t fa_launch_count(const fa_handle* h) { return h ? h->launches : 0; }
+int fa_last_kv_splits(const fa_handle* h) { return h ? h->last_splits : 0; }
 const char* fa_last_kernel_name(const fa_handle* h) { return h ? h->last_kernel : ""; }
 
 fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, void* O, float* lse,
@@ -316,6 +373,25 @@ fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, 
     }
     p.status = h->status_dev;
     p.wait_limit_ns = h->wait_limit_ns;
+    p.kv_splits = 1;
+    p.tiles_per_split = 0x3fffffff;
+    p.o_part = nullptr;
+    p.lse_part = nullptr;
+    if (!(h->flags & FA_FLAG_SERIAL_KERNEL)) {
+        const int splits = choose_kv_splits(h, B, Hq, Sq, Sk, dv, p.causal, p.n_q_tiles);
+        if (splits > 1) {
+            int max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
+            if (p.causal) {
+                const int t = fa::kv_tiles_for_q_tile((p.n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, 1);
+                if (t < max_tiles) max_tiles = t;
+            }
+            p.kv_splits = splits;
+            p.tiles_per_split = (max_tiles + splits - 1) / splits;
+            p.o_part = static_cast<float*>(h->scratch);
+            p.lse_part = p.o_part + static_cast<size_t>(splits) * B * Hq * Sq * dv;
+        }
+    }
+    h->last_splits = p.kv_splits;
 #ifdef FA_TRACE
     p.trace = h->trace;
 #endif

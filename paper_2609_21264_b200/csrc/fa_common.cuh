@@ -32,6 +32,10 @@ struct FwdParams {
     float scale_log2;         // scale * log2(e): scores are handled in log2 units
     int n_q_tiles;            // ceil(Sq / 128)
     int heads_per_group;      // (batch, head) instances scheduled together (their K/V share L2)
+    int kv_splits;            // C >= 1: CTAs per item, each with its own range of K/V tiles
+    int tiles_per_split;      // K/V tiles per split (all of them when kv_splits == 1)
+    float* o_part;            // [C, B*Hq, Sq, dv] fp32 partial outputs (split-KV only)
+    float* lse_part;          // [C, B*Hq, Sq] fp32 partial log-sum-exps (split-KV only)
     uint32_t* status;         // [0] = fa_status, [1] = wait site; mapped host memory
     unsigned long long wait_limit_ns;
 #ifdef FA_TRACE

@@ -126,10 +126,14 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     // pair before it, and so on.  Consecutive CTAs are consecutive query heads (shared K/V heads).
     const int n_pairs = (p.n_q_tiles + 1) / 2;
     const int n_bh = p.B * p.Hq;
-    const int group = static_cast<int>(blockIdx.x) / (n_pairs * p.heads_per_group);
+    // With split-KV (the spatial decomposition of Algorithm 2) the C CTAs that share an item's
+    // query tiles and take disjoint ranges of its K/V tiles are adjacent in the grid.
+    const int item = static_cast<int>(blockIdx.x) / p.kv_splits;
+    const int split = static_cast<int>(blockIdx.x) - item * p.kv_splits;
+    const int group = item / (n_pairs * p.heads_per_group);
     const int bh0 = group * p.heads_per_group;
     const int group_size = (n_bh - bh0 < p.heads_per_group) ? (n_bh - bh0) : p.heads_per_group;
-    const int local = static_cast<int>(blockIdx.x) - group * n_pairs * p.heads_per_group;
+    const int local = item - group * n_pairs * p.heads_per_group;
     const int pair = n_pairs - 1 - local / group_size;
     const int bh = bh0 + local % group_size;
     const int hq = bh % p.Hq;
@@ -141,8 +145,16 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
 
     // per-tile scalars (no arrays: a runtime-indexed array would live in local memory)
     const int i0_0 = (2 * pair) * kTileM, i0_1 = i0_0 + kTileM;
-    const int nkv_0 = (i0_0 < p.Sq) ? kv_tiles_for_q_tile(i0_0, kTileM, p.Sq, p.Sk, p.causal) : 0;
-    const int nkv_1 = (i0_1 < p.Sq) ? kv_tiles_for_q_tile(i0_1, kTileM, p.Sq, p.Sk, p.causal) : 0;
+    // K/V tiles [j_base, j_base + nkv_t) of tile t belong to this CTA (all visible ones without split-KV)
+    const int j_base = split * p.tiles_per_split;
+    auto own_tiles = [&](int i0) -> int {
+        if (i0 >= p.Sq) return 0;
+        int n = kv_tiles_for_q_tile(i0, kTileM, p.Sq, p.Sk, p.causal) - j_base;
+        if (n > p.tiles_per_split) n = p.tiles_per_split;
+        return n > 0 ? n : 0;
+    };
+    const int nkv_0 = own_tiles(i0_0);
+    const int nkv_1 = own_tiles(i0_1);
     const int n_max = nkv_0 > nkv_1 ? nkv_0 : nkv_1;
 
     // ---------------------------------------------------------------- setup
@@ -210,7 +222,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             if (!ok) break;
             tc_fence_after_sync();
             if (lane == 0 && ((warp & 3) == 0 || (warp & 3) == 2)) FA_TRACE_STAMP(t + ((warp & 3) == 2 ? 4 : 0), j, 0);
-            const int j0 = j * kTileN;
+            const int j0 = (j_base + j) * kTileN;
             const bool need_mask = (j0 + kTileN - 1 > kmax_row);
 
             const float2 c2 = make_float2(c, c);
@@ -313,7 +325,40 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             if (lane == 0 && ((warp & 3) == 0 || (warp & 3) == 2)) FA_TRACE_STAMP(t + ((warp & 3) == 2 ? 4 : 0), j, 4);
         }
         // epilogue: O = G' / s (bf16), lse = u * scale + ln s
-        if (ok && i0_t < p.Sq) {
+        if (ok && i0_t < p.Sq && p.kv_splits > 1) {
+            // split-KV: this CTA's partial (G'_c / s_c in fp32, and u_c + ln s_c) goes to scratch;
+            // the combine kernel merges the C partials of a row (Algorithm 2's reduction).
+            const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
+            float* po_row = p.o_part + prow * DV;
+            bool have = nkv_t > 0;
+            if (have) have = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.o_final[t]), 0, wctx, kSiteEpiOFull));
+            if (nkv_t == 0 || have) {
+                tc_fence_after_sync();
+                const float inv_l = (nkv_t > 0 && l > 0.f) ? (1.f / l) : 0.f;
+                if (i_glob < p.Sq)
+                    p.lse_part[prow] = (nkv_t > 0 && l > 0.f) ? (m_ref * c * 0.6931471805599453f + logf(l)) : -INFINITY;
+                const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1) + lane_sel;
+#pragma unroll 1
+                for (int cc = 0; cc < DV / 32; ++cc) {
+                    uint32_t r[32];
+                    if (nkv_t > 0) {            // uniform over the CTA's tile: warp-collective load is safe
+                        tmem_ld_x32(tO + cc * 32, r);
+                        tc_wait_ld();
+                    }
+                    if (i_glob < p.Sq) {
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            float4 f;
+                            f.x = (nkv_t > 0) ? __uint_as_float(r[4 * v]) * inv_l : 0.f;
+                            f.y = (nkv_t > 0) ? __uint_as_float(r[4 * v + 1]) * inv_l : 0.f;
+                            f.z = (nkv_t > 0) ? __uint_as_float(r[4 * v + 2]) * inv_l : 0.f;
+                            f.w = (nkv_t > 0) ? __uint_as_float(r[4 * v + 3]) * inv_l : 0.f;
+                            reinterpret_cast<float4*>(po_row + cc * 32)[v] = f;
+                        }
+                    }
+                }
+            }
+        } else if (ok && i0_t < p.Sq) {
             __nv_bfloat16* o_row = p.O + (static_cast<size_t>(q_idx) * p.Sq + i_glob) * DV;
             if (nkv_t == 0) {         // no key visible to any row of this tile
                 if (i_glob < p.Sq) {
@@ -511,7 +556,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             }
             bool ok = true;
             for (int j = 0; j < n_max && ok; ++j) {
-                const int j0 = j * kTileN;
+                const int j0 = (j_base + j) * kTileN;
                 {
                     const int s = j % NK;
                     ok = mbar_wait(smem_addr(&sh.k_empty[s]), ((j / NK) & 1) ^ 1, wctx, kSiteLoadKvEmpty);
@@ -546,6 +591,46 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 12) tmem_dealloc(tmem_base, Cfg::kTmemCols);
+}
+
+
+// Merge of the split-KV partials (Algorithm 2's reduction over the C spatial partitions, in the
+// corrected form: every partial is rescaled to the common maximum).  With O_c = G'_c / s_c and
+// lse_c = u_c + ln s_c the merged result is lse = ln sum_c exp(lse_c), O = sum_c exp(lse_c - lse) O_c.
+// One warp per query row, each lane four output columns per 128-column pass; HBM-bound.
+template <int DV>
+__global__ void __launch_bounds__(128)
+fa_combine_kernel(const float* __restrict__ o_part, const float* __restrict__ lse_part,
+                  __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
+                  long long n_rows, int n_splits) {
+    const long long row = static_cast<long long>(blockIdx.x) * 4 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= n_rows) return;
+    float m = -INFINITY;
+    for (int cidx = 0; cidx < n_splits; ++cidx) m = fmaxf(m, lse_part[cidx * n_rows + row]);
+    float denom = 0.f;
+    if (m != -INFINITY)
+        for (int cidx = 0; cidx < n_splits; ++cidx) denom += expf(lse_part[cidx * n_rows + row] - m);
+    const float inv = denom > 0.f ? 1.f / denom : 0.f;
+#pragma unroll
+    for (int col = 0; col < DV; col += 128) {
+        if (col + lane * 4 >= DV) break;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int cidx = 0; cidx < n_splits; ++cidx) {
+            const float lc = lse_part[cidx * n_rows + row];
+            const float wgt = (lc == -INFINITY) ? 0.f : expf(lc - m) * inv;
+            const float4 v = *reinterpret_cast<const float4*>(o_part + (cidx * n_rows + row) * DV + col + lane * 4);
+            acc.x = fmaf(wgt, v.x, acc.x);
+            acc.y = fmaf(wgt, v.y, acc.y);
+            acc.z = fmaf(wgt, v.z, acc.z);
+            acc.w = fmaf(wgt, v.w, acc.w);
+        }
+        uint2 packed;
+        packed.x = ptx::pack_bf16x2(acc.x, acc.y);
+        packed.y = ptx::pack_bf16x2(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(O + row * DV + col + lane * 4) = packed;
+    }
+    if (lane == 0 && lse) lse[row] = (m == -INFINITY) ? -INFINITY : m + logf(denom);
 }
 
 }  // namespace fa
