@@ -158,6 +158,40 @@ uint64_t fa_launch_count(const fa_handle* h);
 const char* fa_last_kernel_name(const fa_handle* h);
 int fa_last_kv_splits(const fa_handle* h);   /* K/V splits the last fa_forward used (1 = none) */
 
+/*
+ * Allocation-free split-KV forward.  (The paper has no counterpart: this entry point exists for
+ * callers that cannot allocate, it is not a step of the paper's method.)
+ *
+ * Who needs it: code that must not call cudaMalloc or any allocating routine once it is running --
+ * a server that has handed all of HBM to its own pools, a real-time loop that cannot afford an
+ * allocation's latency and implicit synchronisation, a plug-in that only gets its host's buffers.
+ * fa_create allocates, so such callers cannot hold a handle; this function takes none.
+ *
+ * It computes exactly what fa_forward computes with kv_splits-way split-KV.  The fp32 partials that
+ * the combine kernel merges live in an array of FA_NOALLOC_SCRATCH_BYTES (8 MiB) in the library's
+ * device data segment: every GPU that loads the library carries that array until the process
+ * exits.  Consequences:
+ *   - the partials must fit: splits * B*Hq*Sq * (dv + 1) * 4 bytes <= FA_NOALLOC_SCRATCH_BYTES, where
+ *     splits = min(kv_splits, number of K/V tiles) (at least 2); larger problems are rejected with
+ *     FA_ERR_UNSUPPORTED and nothing is launched;
+ *   - all calls share the array and it keeps the previous call's contents.  Nothing needs clearing
+ *     (each call overwrites every slot it later reads), but two calls that overlap on the device --
+ *     different streams, or different host threads -- race on it: serialise them;
+ *   - the first call on a device performs a one-time set-up for that device (looks up the array's
+ *     device address, the driver's tensor-map encoder, raises the kernels' shared-memory limit).
+ *     Make that first call with the device current and before any stream capture begins.
+ * No call made here allocates host or device memory.  Arguments as for fa_forward; kv_splits in
+ * [2, 64]; device pointers; the work is enqueued on `stream` of the CURRENT device and the call
+ * returns without synchronising.  A device-side wait that runs out is not reported (there is no
+ * status word); results are then undefined, as with fa_forward.
+ */
+#define FA_NOALLOC_SCRATCH_BYTES (8u << 20)
+fa_status fa_forward_split_noalloc(const void* Q, const void* K, const void* V,
+                                   void* O, float* lse,
+                                   int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv,
+                                   int causal, float scale, int kv_splits, void* stream);
+size_t fa_noalloc_scratch_bytes(void);   /* FA_NOALLOC_SCRATCH_BYTES as built into the library */
+
 #ifdef __cplusplus
 }
 #endif

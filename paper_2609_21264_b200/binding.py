@@ -23,7 +23,8 @@ FA_ERR_OOM = 6
 FA_FLAG_SERIAL_KERNEL = 1
 
 EXPORTS = ("fa_create", "fa_forward", "fa_forward_host", "fa_last_status", "fa_destroy",
-           "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits")
+           "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits",
+           "fa_forward_split_noalloc", "fa_noalloc_scratch_bytes")
 
 
 class FaError(RuntimeError):
@@ -75,6 +76,10 @@ def load():
     lib.fa_last_kernel_name.argtypes = [vp]
     lib.fa_last_kv_splits.restype = i32
     lib.fa_last_kv_splits.argtypes = [vp]
+    lib.fa_forward_split_noalloc.restype = i32
+    lib.fa_forward_split_noalloc.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, f32, i32, vp]
+    lib.fa_noalloc_scratch_bytes.restype = ctypes.c_size_t
+    lib.fa_noalloc_scratch_bytes.argtypes = []
     _lib = lib
     return lib
 
@@ -119,6 +124,20 @@ def fa_destroy(h) -> int:
 
 def fa_launch_count(h) -> int:
     return int(load().fa_launch_count(h))
+
+
+def fa_forward_split_noalloc(Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, kv_splits, stream=0) -> int:
+    """Raw call of the allocation-free split-KV entry point (device pointers as integers, no handle).
+
+    For callers that may not allocate: the split-KV partials live in a fixed 8 MiB array inside
+    the library instead of a handle's scratch buffer.  Returns the status code.
+    """
+    return load().fa_forward_split_noalloc(Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv,
+                                           int(bool(causal)), float(scale), int(kv_splits), stream)
+
+
+def fa_noalloc_scratch_bytes() -> int:
+    return int(load().fa_noalloc_scratch_bytes())
 
 
 def fa_last_kv_splits(h) -> int:
