@@ -304,6 +304,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the short timing of the other configs")
+    ap.add_argument("--table6", action="store_true",
+                    help="also time the twelve attention shapes of the paper's Table 6 (key 'table6')")
     args = ap.parse_args()
     w = workloads.config(args.config)
     if args.shape:
@@ -406,6 +408,21 @@ def main():
             del ss
             torch.cuda.empty_cache()
         line["per_config"] = per
+
+    if args.table6 and world == 1:
+        rows = []
+        for wc, paper_us in workloads.TABLE6:
+            fa, fp, nb = workload_numbers(wc)
+            ss = make_device_sets(wc, n_sets_for(wc), device)
+            k = max(3, min(200, int(0.3 / max(fa / 1.0e15, 1e-5))))
+            sec, _ = run_device_timed(binding, h, wc, ss, k, 3, 1)
+            t = sec / k
+            rows.append({"workload": wc.name, "us": t * 1e6, "tflops_paper_convention": fp / t / 1e12,
+                         "tflops_algorithmic": fa / t / 1e12, "paper_xdna2_us": paper_us,
+                         "paper_xdna2_tflops": fp / (paper_us * 1e-6) / 1e12})
+            del ss
+            torch.cuda.empty_cache()
+        line["table6"] = rows
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = oracle_timed(w)

@@ -56,6 +56,12 @@ typedef enum fa_status {
  * between loads, MMAs and softmax) instead of the pipelined one.  Same results up to
  * rounding order; much slower.  Meant for tests. */
 #define FA_FLAG_SERIAL_KERNEL 1u
+/* fa_config.flags, test hook for the failure path: the load warp of the pipelined kernel leaves
+ * out the load of the first V tile, so the wait for it runs into the device-side limit
+ * (fa_config.wait_limit_ms).  The kernel then returns normally, results are invalid and
+ * fa_last_status reports FA_ERR_DEVICE_TIMEOUT; the context stays usable.  Nothing faults,
+ * traps or spins without bound.  Use with a short wait_limit_ms on a tiny problem. */
+#define FA_FLAG_DEBUG_DROP_V_LOAD 2u
 
 /* Optional creation parameters.  Zero-initialise, set struct_size = sizeof(fa_config). */
 typedef struct fa_config {

@@ -243,7 +243,7 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg) {
         limit_ms = cfg->wait_limit_ms;
         if (cfg->struct_size >= 20) kv_splits_cfg = cfg->kv_splits;
         if (cfg->struct_size >= sizeof(fa_config)) scratch_bytes = cfg->scratch_bytes;
-        if (flags & ~FA_FLAG_SERIAL_KERNEL) return FA_ERR_INVALID_ARG;
+        if (flags & ~(FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD)) return FA_ERR_INVALID_ARG;
         if (kv_splits_cfg > 64) return FA_ERR_INVALID_ARG;
     }
     if (scratch_bytes == 0) scratch_bytes = 32ull << 20;
@@ -373,6 +373,7 @@ fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, 
     }
     p.status = h->status_dev;
     p.wait_limit_ns = h->wait_limit_ns;
+    p.debug_drop_v_load = (h->flags & FA_FLAG_DEBUG_DROP_V_LOAD) ? 1 : 0;
     p.kv_splits = 1;
     p.tiles_per_split = 0x3fffffff;
     p.o_part = nullptr;

@@ -36,6 +36,7 @@ struct FwdParams {
     int tiles_per_split;      // K/V tiles per split (all of them when kv_splits == 1)
     float* o_part;            // [C, B*Hq, Sq, dv] fp32 partial outputs (split-KV only)
     float* lse_part;          // [C, B*Hq, Sq] fp32 partial log-sum-exps (split-KV only)
+    int debug_drop_v_load;    // test hook: the load warp skips the first V tile (exercises the wait limit)
     uint32_t* status;         // [0] = fa_status, [1] = wait site; mapped host memory
     unsigned long long wait_limit_ns;
 #ifdef FA_TRACE

@@ -568,7 +568,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                         tma_load_3d(sK + s * Cfg::kKBytes + cc * kChunkBytes, &tm_k, bar, cc * kChunkCols,
                                     j0, kv_idx);
                 }
-                {
+                if (!(p.debug_drop_v_load && j == 0)) {
                     const int s = j % NV;
                     ok = mbar_wait(smem_addr(&sh.v_empty[s]), ((j / NV) & 1) ^ 1, wctx, kSiteLoadKvEmpty);
                     if (!ok) break;

@@ -65,6 +65,25 @@ CONFIGS = (
 )
 
 
+# The twelve attention shapes of the paper's Table 6 (LLM configurations on XDNA 2, all B = 1,
+# dv = dk), with the latency the paper prints for its fused kernel in microseconds (context for
+# other hardware, never a target).
+TABLE6 = (
+    (_w("bert_base_s2048", 1, 12, 12, 2048, 64, 64, False, idx=10), 5775.0),
+    (_w("bert_large_s2048", 1, 16, 16, 2048, 64, 64, False, idx=11), 7526.0),
+    (_w("gpt2_small_s2048", 1, 12, 12, 2048, 64, 64, True, idx=12), 5810.0),
+    (_w("gpt2_medium_s2048", 1, 16, 16, 2048, 64, 64, True, idx=13), 7535.0),
+    (_w("gpt2_large_s2048", 1, 20, 20, 2048, 64, 64, True, idx=14), 9196.0),
+    (_w("llama2_7b_s2048", 1, 32, 32, 2048, 128, 128, True, idx=15), 34201.0),
+    (_w("llama3_8b_s2048", 1, 32, 8, 2048, 128, 128, True, idx=16), 34076.0),
+    (_w("qwen15_05b_s32768", 1, 16, 16, 32768, 64, 64, True, idx=17), 1214700.0),
+    (_w("qwen25_05b_gqa_s32768", 1, 14, 2, 32768, 64, 64, True, idx=18), 1062870.0),
+    (_w("qwen15_05b_s131072", 1, 16, 16, 131072, 64, 64, True, idx=19), 18996700.0),
+    (_w("deepseek_7b_s4096", 1, 32, 32, 4096, 128, 128, True, idx=20), 114443.0),
+    (_w("deepseek_67b_gqa_s4096", 1, 64, 8, 4096, 128, 128, True, idx=21), 227467.0),
+)
+
+
 def config(index_or_name) -> Workload:
     if isinstance(index_or_name, int):
         return CONFIGS[index_or_name]
