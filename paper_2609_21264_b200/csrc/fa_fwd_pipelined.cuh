@@ -53,15 +53,6 @@ template <int V>
 struct IntC { static constexpr int value = V; };
 
 constexpr float kRescaleThresholdLog2 = 8.0f;
-// Of every four pairs of exponentials, this many are evaluated by the polynomial on the FMA
-// pipe (on tiles without masked entries); the rest use MUFU ex2.  Measured on B200 with this
-// schedule, where one softmax warp per scheduler is active at a time, the offload does not pay
-// (a lone warp is issue-bound, and the polynomial costs more issue slots than it frees MUFU
-// cycles), so the default is 0; the option is kept for schedules with more warps in flight.
-#ifndef FA_POLY_PAIRS_PER_4
-#define FA_POLY_PAIRS_PER_4 0
-#endif
-constexpr int kPolyPairsPer4 = FA_POLY_PAIRS_PER_4;
 // Registers per thread after the per-role reallocation (512 threads start with 128 each):
 // 256 softmax threads x 192 + 128 correction threads x 64 + 128 other threads x 64 = 65536.
 constexpr int kRegsSoftmax = 192, kRegsCorrection = 64, kRegsOther = 64;
@@ -236,14 +227,8 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 for (int e = 0; e < 32; e += 2) {
                     const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[q * 32 + e]),
                                                             __uint_as_float(s[q * 32 + e + 1])), c2, nmc2);
-                    if (((e / 2) & 3) < kPolyPairsPer4 && !need_mask) {   // this pair on the FMA pipe
-                        const float2 y = exp2_poly2(x);
-                        s[q * 32 + e] = __float_as_uint(y.x);
-                        s[q * 32 + e + 1] = __float_as_uint(y.y);
-                    } else {                                   // this pair on the MUFU pipe
-                        s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
-                        s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
-                    }
+                    s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
+                    s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
                 }
             };
             // Row sum, bf16 conversion and store of one chunk of P (over the first half of S).
@@ -544,16 +529,18 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         // ============================================================ TMA loads
         setmaxnreg_dec<kRegsOther>();
         if (lane == 0 && n_max > 0) {
-#pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                if ((t == 0 ? nkv_0 : nkv_1) == 0) continue;
+            auto load_q = [&](int t) {
+                if ((t == 0 ? nkv_0 : nkv_1) == 0) return;
                 const uint32_t bar = smem_addr(&sh.q_full[t]);
                 mbar_arrive_expect_tx(bar, Cfg::kQBytes);
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kQChunks; ++cc)
                     tma_load_3d(sQ + t * Cfg::kQBytes + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols,
                                 t == 0 ? i0_0 : i0_1, q_idx);
-            }
+            };
+            // Order of the first requests: Q_0 and K_0 (all the first MMA needs), then Q_1, then V_0.
+            // When a whole wave of CTAs starts at once these first loads are HBM-bandwidth-bound.
+            load_q(0);
             bool ok = true;
             for (int j = 0; j < n_max && ok; ++j) {
                 const int j0 = (j_base + j) * kTileN;
@@ -567,6 +554,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                     for (int cc = 0; cc < Cfg::kQChunks; ++cc)
                         tma_load_3d(sK + s * Cfg::kKBytes + cc * kChunkBytes, &tm_k, bar, cc * kChunkCols,
                                     j0, kv_idx);
+                    if (j == 0) load_q(1);
                 }
                 if (!(p.debug_drop_v_load && j == 0)) {
                     const int s = j % NV;

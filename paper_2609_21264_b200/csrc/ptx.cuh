@@ -42,26 +42,6 @@ FA_DEVI float exp2_approx(float x) {
     return y;
 }
 
-// 2^x for two values on the FMA and ALU pipes (no MUFU).  x = n + f with n = round(x) taken
-// from the low mantissa bits of x + 1.5*2^23, f in [-0.5, 0.5]; 2^f by a cubic with maximum
-// relative error 7.5e-5 (well below bf16 rounding); 2^n by adding n to the exponent field.
-// Inputs below -125 (including -inf) return ~2^-125, i.e. zero for every purpose here.
-FA_DEVI float2 exp2_poly2(float2 x) {
-    x.x = fmaxf(x.x, -125.f);
-    x.y = fmaxf(x.y, -125.f);
-    const float2 t = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));
-    const float2 xr = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
-    const float2 f = __ffma2_rn(xr, make_float2(-1.f, -1.f), x);
-    float2 p = __ffma2_rn(make_float2(0.0551716685f, 0.0551716685f), f,
-                          make_float2(0.242611125f, 0.242611125f));
-    p = __ffma2_rn(p, f, make_float2(0.693260968f, 0.693260968f));
-    p = __ffma2_rn(p, f, make_float2(0.999928057f, 0.999928057f));
-    float2 r;
-    r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
-    r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
-    return r;
-}
-
 FA_DEVI float fmax3(float a, float b, float c) {
     float y;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
