@@ -125,6 +125,25 @@ fa_status fa_forward(fa_handle* h,
                      int causal, float scale, void* stream);
 
 /*
+ * fa_forward for tensors that are not contiguous [B, H, S, d] (Eq. 1 fixes no memory layout; a
+ * projection kernel usually leaves Q, K, V as [B, S, H, d]).  Each strides argument points to three
+ * int64 values {batch stride, head stride, row stride} in ELEMENTS; element (b, h, s, c) of a
+ * tensor sits at base + b*batch + h*head + s*row + c, the last dimension is contiguous.  Every
+ * stride must be positive and a multiple of 8 elements (16 bytes: the TMA unit and the 16-byte
+ * output stores require it), and a row stride must not be smaller than the head size.  lse stays
+ * contiguous [B, Hq, Sq].  Everything else is as for fa_forward; FA_ERR_INVALID_ARG if the strides
+ * cannot be expressed.
+ */
+fa_status fa_forward_strided(fa_handle* h,
+                             const void* Q, const void* K, const void* V,
+                             void* O, float* lse,
+                             int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv,
+                             int causal, float scale,
+                             const int64_t* q_strides, const int64_t* k_strides,
+                             const int64_t* v_strides, const int64_t* o_strides,
+                             void* stream);
+
+/*
  * The same operation with HOST buffers (same layouts and types): copies Q, K, V
  * to staging memory owned by the handle, runs fa_forward, copies O (and lse if
  * not NULL) back, all on `stream`, and synchronises `stream` before returning.

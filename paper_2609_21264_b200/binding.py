@@ -23,7 +23,7 @@ FA_ERR_OOM = 6
 FA_FLAG_SERIAL_KERNEL = 1
 FA_FLAG_DEBUG_DROP_V_LOAD = 2
 
-EXPORTS = ("fa_create", "fa_forward", "fa_forward_host", "fa_last_status", "fa_destroy",
+EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_host", "fa_last_status", "fa_destroy",
            "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits",
            "fa_forward_split_noalloc", "fa_noalloc_scratch_bytes")
 
@@ -65,6 +65,8 @@ def load():
     lib.fa_forward.argtypes = fwd_args
     lib.fa_forward_host.restype = i32
     lib.fa_forward_host.argtypes = fwd_args
+    lib.fa_forward_strided.restype = i32
+    lib.fa_forward_strided.argtypes = fwd_args[:-1] + [vp, vp, vp, vp, vp]
     lib.fa_last_status.restype = i32
     lib.fa_last_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.fa_destroy.restype = i32
@@ -104,6 +106,14 @@ def fa_forward(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, s
     """Raw call with device pointers as integers; returns the status code."""
     return load().fa_forward(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv,
                              int(bool(causal)), float(scale), stream)
+
+
+def fa_forward_strided(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale,
+                       q_strides, k_strides, v_strides, o_strides, stream=0) -> int:
+    """Raw call with device pointers and (batch, head, row) strides in elements; returns the status code."""
+    arr = [(ctypes.c_int64 * 3)(*[int(x) for x in st]) for st in (q_strides, k_strides, v_strides, o_strides)]
+    return load().fa_forward_strided(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, int(bool(causal)), float(scale),
+                                     arr[0], arr[1], arr[2], arr[3], stream)
 
 
 def fa_forward_host(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, stream=0) -> int:
@@ -150,21 +160,41 @@ def fa_last_kernel_name(h) -> str:
 
 
 def forward(h, q, k, v, *, causal: bool, scale: float = 0.0, out=None, lse=None, want_lse=True):
-    """Attention forward on torch CUDA tensors (bf16, contiguous, [B,H,S,d]); returns (O, lse)."""
+    """Attention forward on torch CUDA tensors (bf16, logical shape [B,H,S,d]); returns (O, lse).
+
+    Contiguous tensors go through fa_forward.  Views with other strides (say a [B,S,H,d] buffer
+    permuted to [B,H,S,d]) go through fa_forward_strided when their last dimension is contiguous;
+    `out`, when not given, then takes q's memory layout.
+    """
     import torch
     for t in (q, k, v):
-        if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or t.dim() != 4:
-            raise ValueError("q, k, v must be contiguous 4-D bf16 CUDA tensors")
+        if t.dtype != torch.bfloat16 or not t.is_cuda or t.dim() != 4:
+            raise ValueError("q, k, v must be 4-D bf16 CUDA tensors")
     B, Hq, Sq, dqk = q.shape
     _, Hkv, Sk, dv = v.shape
+    dense = all(t.is_contiguous() for t in (q, k, v)) and (out is None or out.is_contiguous())
     if out is None:
-        out = torch.empty((B, Hq, Sq, dv), dtype=torch.bfloat16, device=q.device)
+        if dense:
+            out = torch.empty((B, Hq, Sq, dv), dtype=torch.bfloat16, device=q.device)
+        else:   # same dimension order in memory as q
+            order = sorted(range(3), key=lambda i: -q.stride(i)) + [3]
+            shape = (B, Hq, Sq, dv)
+            buf = torch.empty([shape[i] for i in order], dtype=torch.bfloat16, device=q.device)
+            out = buf.permute([order.index(i) for i in range(4)])
     if lse is None and want_lse:
         lse = torch.empty((B, Hq, Sq), dtype=torch.float32, device=q.device)
     stream = torch.cuda.current_stream(q.device).cuda_stream
-    st = fa_forward(h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
-                    lse.data_ptr() if lse is not None else None,
-                    B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, stream)
+    lse_ptr = lse.data_ptr() if lse is not None else None
+    if dense:
+        st = fa_forward(h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse_ptr,
+                        B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, stream)
+    else:
+        for t in (q, k, v, out):
+            if t.stride(3) != 1:
+                raise ValueError("the last dimension must be contiguous")
+        st = fa_forward_strided(h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse_ptr,
+                                B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale,
+                                q.stride()[:3], k.stride()[:3], v.stride()[:3], out.stride()[:3], stream)
     if st != FA_OK:
         raise FaError(st, "fa_forward")
     return out, lse

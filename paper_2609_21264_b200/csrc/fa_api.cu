@@ -24,7 +24,8 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
 
 struct MapEntry {
     const void* ptr;
-    int d, S, BH, box_rows;
+    int d, S, H, B, box_rows;
+    long long sb, sh, ss;      // batch / head / row strides in elements
     uint64_t stamp;
     CUtensorMap map;
 };
@@ -73,12 +74,13 @@ class DeviceGuard {
     bool changed_ = false;
 };
 
-// bf16 tensor [BH, S, d] (row-major) seen as a 3-D TMA tensor (d, S, BH); box =
-// 64 columns x box_rows rows, 128-byte swizzle, out-of-range rows read as zero.
-fa_status get_map(fa_handle* h, const void* ptr, int d, int S, long long BH, int box_rows,
-                  const CUtensorMap** out) {
+// bf16 tensor with element (b, h, s, c) at ptr + b*sb + h*sh + s*ss + c, seen as a 4-D TMA
+// tensor (d, S, H, B); box = 64 columns x box_rows rows, 128-byte swizzle, rows past S read as zero.
+fa_status get_map(fa_handle* h, const void* ptr, int d, int S, int H, int B, long long sb, long long sh,
+                  long long ss, int box_rows, const CUtensorMap** out) {
     for (auto& e : h->maps) {
-        if (e.ptr == ptr && e.d == d && e.S == S && e.BH == BH && e.box_rows == box_rows) {
+        if (e.ptr == ptr && e.d == d && e.S == S && e.H == H && e.B == B && e.box_rows == box_rows &&
+            e.sb == sb && e.sh == sh && e.ss == ss) {
             e.stamp = ++h->stamp;
             *out = &e.map;
             return FA_OK;
@@ -86,19 +88,19 @@ fa_status get_map(fa_handle* h, const void* ptr, int d, int S, long long BH, int
     }
     MapEntry ne;
     memset(&ne, 0, sizeof ne);
-    ne.ptr = ptr; ne.d = d; ne.S = S; ne.BH = static_cast<int>(BH); ne.box_rows = box_rows;
-    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(S),
-                                static_cast<cuuint64_t>(BH)};
-    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2ull,
-                                   static_cast<cuuint64_t>(d) * 2ull * static_cast<cuuint64_t>(S)};
-    const cuuint32_t box[3] = {static_cast<cuuint32_t>(fa::kChunkCols),
-                               static_cast<cuuint32_t>(box_rows), 1u};
-    const cuuint32_t estr[3] = {1u, 1u, 1u};
-    const CUresult r = h->encode(&ne.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr),
+    ne.ptr = ptr; ne.d = d; ne.S = S; ne.H = H; ne.B = B; ne.box_rows = box_rows;
+    ne.sb = sb; ne.sh = sh; ne.ss = ss;
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(S),
+                                static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(B)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(ss) * 2ull, static_cast<cuuint64_t>(sh) * 2ull,
+                                   static_cast<cuuint64_t>(sb) * 2ull};
+    const cuuint32_t box[4] = {static_cast<cuuint32_t>(fa::kChunkCols), static_cast<cuuint32_t>(box_rows), 1u, 1u};
+    const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    const CUresult r = h->encode(&ne.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr),
                                  dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return FA_ERR_CUDA;
+    if (r != CUDA_SUCCESS) return FA_ERR_INVALID_ARG;     // strides or extents the TMA unit cannot express
     ne.stamp = ++h->stamp;
     if (static_cast<int>(h->maps.size()) < kMapCacheSize) {
         h->maps.push_back(ne);
@@ -159,7 +161,8 @@ fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const 
         const long long blocks = (n_rows + 3) / 4;
         if (blocks > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
         fa::fa_combine_kernel<DV><<<static_cast<unsigned>(blocks), 128, 0, st>>>(
-            p.o_part, p.lse_part, p.O, p.lse, n_rows, p.kv_splits);
+            p.o_part, p.lse_part, p.O, p.lse, n_rows, p.kv_splits, p.Hq, p.Sq,
+            p.o_stride_b, p.o_stride_h, p.o_stride_s);
         if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
         h->launches += 1;
     }
@@ -333,27 +336,38 @@ uint64_t fa_launch_count(const fa_handle* h) { return h ? h->launches : 0; }
 int fa_last_kv_splits(const fa_handle* h) { return h ? h->last_splits : 0; }
 const char* fa_last_kernel_name(const fa_handle* h) { return h ? h->last_kernel : ""; }
 
-fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, void* O, float* lse,
-                     int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal,
-                     float scale, void* stream) {
+fa_status fa_forward_strided(fa_handle* h, const void* Q, const void* K, const void* V, void* O, float* lse,
+                             int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal,
+                             float scale, const int64_t* q_strides, const int64_t* k_strides,
+                             const int64_t* v_strides, const int64_t* o_strides, void* stream) {
     if (!h) return FA_ERR_INVALID_ARG;
     fa_status s = check_args(Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, scale, true);
     if (s != FA_OK) return s;
+    if (!q_strides || !k_strides || !v_strides || !o_strides) return FA_ERR_INVALID_ARG;
+    for (int i = 0; i < 3; ++i) {
+        // TMA wants every stride to be a multiple of 16 bytes; 16-byte row stores want the same of O
+        if (q_strides[i] <= 0 || k_strides[i] <= 0 || v_strides[i] <= 0 || o_strides[i] <= 0) return FA_ERR_INVALID_ARG;
+        if ((q_strides[i] | k_strides[i] | v_strides[i] | o_strides[i]) & 7) return FA_ERR_INVALID_ARG;
+    }
+    if (q_strides[2] < dqk || k_strides[2] < dqk || v_strides[2] < dv || o_strides[2] < dv) return FA_ERR_INVALID_ARG;
     DeviceGuard guard(h->device);
     if (!guard.ok()) return FA_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (scale == 0.f) scale = 1.f / sqrtf(static_cast<float>(dqk));
 
     const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr;
-    if ((s = get_map(h, Q, dqk, Sq, static_cast<long long>(B) * Hq, fa::kTileM, &mq)) != FA_OK) return s;
+    if ((s = get_map(h, Q, dqk, Sq, Hq, B, q_strides[0], q_strides[1], q_strides[2], fa::kTileM, &mq)) != FA_OK) return s;
     CUtensorMap map_q = *mq;   // copies: a later insertion may evict or move cache entries
-    if ((s = get_map(h, K, dqk, Sk, static_cast<long long>(B) * Hkv, fa::kTileN, &mk)) != FA_OK) return s;
+    if ((s = get_map(h, K, dqk, Sk, Hkv, B, k_strides[0], k_strides[1], k_strides[2], fa::kTileN, &mk)) != FA_OK) return s;
     CUtensorMap map_k = *mk;
-    if ((s = get_map(h, V, dv, Sk, static_cast<long long>(B) * Hkv, fa::kTileN, &mv)) != FA_OK) return s;
+    if ((s = get_map(h, V, dv, Sk, Hkv, B, v_strides[0], v_strides[1], v_strides[2], fa::kTileN, &mv)) != FA_OK) return s;
     CUtensorMap map_v = *mv;
 
     fa::FwdParams p;
     p.O = static_cast<__nv_bfloat16*>(O);
+    p.o_stride_b = o_strides[0];
+    p.o_stride_h = o_strides[1];
+    p.o_stride_s = o_strides[2];
     p.lse = lse;
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Sk = Sk;
     p.causal = causal ? 1 : 0;
@@ -407,6 +421,17 @@ fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, 
     if (dqk == 64) return launch_simple<64, 64>(h, 0, map_q, map_k, map_v, p, st);
     if (dqk == 128) return launch_simple<128, 128>(h, 1, map_q, map_k, map_v, p, st);
     return launch_simple<192, 128>(h, 2, map_q, map_k, map_v, p, st);
+}
+
+fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, void* O, float* lse,
+                     int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal,
+                     float scale, void* stream) {
+    // contiguous [B, H, S, d]
+    const int64_t qs[3] = {static_cast<int64_t>(Hq) * Sq * dqk, static_cast<int64_t>(Sq) * dqk, dqk};
+    const int64_t ks[3] = {static_cast<int64_t>(Hkv) * Sk * dqk, static_cast<int64_t>(Sk) * dqk, dqk};
+    const int64_t vs[3] = {static_cast<int64_t>(Hkv) * Sk * dv, static_cast<int64_t>(Sk) * dv, dv};
+    const int64_t os[3] = {static_cast<int64_t>(Hq) * Sq * dv, static_cast<int64_t>(Sq) * dv, dv};
+    return fa_forward_strided(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, qs, ks, vs, os, stream);
 }
 
 fa_status fa_forward_host(fa_handle* h, const void* Qh, const void* Kh, const void* Vh, void* Oh,

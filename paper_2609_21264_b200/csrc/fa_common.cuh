@@ -25,7 +25,8 @@ enum WaitSite : uint32_t {
 };
 
 struct FwdParams {
-    __nv_bfloat16* O;         // [B, Hq, Sq, dv]
+    __nv_bfloat16* O;         // element (b, hq, i, c) at O + b*o_stride_b + hq*o_stride_h + i*o_stride_s + c
+    long long o_stride_b, o_stride_h, o_stride_s;   // in elements
     float* lse;               // [B, Hq, Sq] or nullptr
     int B, Hq, Hkv, Sq, Sk;
     int causal;

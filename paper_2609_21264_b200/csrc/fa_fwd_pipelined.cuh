@@ -131,7 +131,6 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int b = bh / p.Hq;
     const int kvh = hq / (p.Hq / p.Hkv);
     const int q_idx = b * p.Hq + hq;
-    const int kv_idx = b * p.Hkv + kvh;
     const int off = p.Sk - p.Sq;
 
     // per-tile scalars (no arrays: a runtime-indexed array would live in local memory)
@@ -344,7 +343,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 }
             }
         } else if (ok && i0_t < p.Sq) {
-            __nv_bfloat16* o_row = p.O + (static_cast<size_t>(q_idx) * p.Sq + i_glob) * DV;
+            __nv_bfloat16* o_row = p.O + (b * p.o_stride_b + hq * p.o_stride_h + static_cast<long long>(i_glob) * p.o_stride_s);
             if (nkv_t == 0) {         // no key visible to any row of this tile
                 if (i_glob < p.Sq) {
                     const uint4 z = make_uint4(0, 0, 0, 0);
@@ -535,8 +534,8 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 mbar_arrive_expect_tx(bar, Cfg::kQBytes);
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kQChunks; ++cc)
-                    tma_load_3d(sQ + t * Cfg::kQBytes + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols,
-                                t == 0 ? i0_0 : i0_1, q_idx);
+                    tma_load_4d(sQ + t * Cfg::kQBytes + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols,
+                                t == 0 ? i0_0 : i0_1, hq, b);
             };
             // Order of the first requests: Q_0 and K_0 (all the first MMA needs), then Q_1, then V_0.
             // When a whole wave of CTAs starts at once these first loads are HBM-bandwidth-bound.
@@ -552,8 +551,8 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                     mbar_arrive_expect_tx(bar, Cfg::kKBytes);
 #pragma unroll
                     for (int cc = 0; cc < Cfg::kQChunks; ++cc)
-                        tma_load_3d(sK + s * Cfg::kKBytes + cc * kChunkBytes, &tm_k, bar, cc * kChunkCols,
-                                    j0, kv_idx);
+                        tma_load_4d(sK + s * Cfg::kKBytes + cc * kChunkBytes, &tm_k, bar, cc * kChunkCols,
+                                    j0, kvh, b);
                     if (j == 0) load_q(1);
                 }
                 if (!(p.debug_drop_v_load && j == 0)) {
@@ -564,8 +563,8 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                     mbar_arrive_expect_tx(bar, Cfg::kVBytes);
 #pragma unroll
                     for (int cc = 0; cc < Cfg::kVChunks; ++cc)
-                        tma_load_3d(sV + s * Cfg::kVBytes + cc * kChunkBytes, &tm_v, bar, cc * kChunkCols,
-                                    j0, kv_idx);
+                        tma_load_4d(sV + s * Cfg::kVBytes + cc * kChunkBytes, &tm_v, bar, cc * kChunkCols,
+                                    j0, kvh, b);
                 }
             }
         }
@@ -590,7 +589,8 @@ template <int DV>
 __global__ void __launch_bounds__(128)
 fa_combine_kernel(const float* __restrict__ o_part, const float* __restrict__ lse_part,
                   __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
-                  long long n_rows, int n_splits) {
+                  long long n_rows, int n_splits, int Hq, int Sq,
+                  long long o_stride_b, long long o_stride_h, long long o_stride_s) {
     const long long row = static_cast<long long>(blockIdx.x) * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= n_rows) return;
@@ -600,6 +600,8 @@ fa_combine_kernel(const float* __restrict__ o_part, const float* __restrict__ ls
     if (m != -INFINITY)
         for (int cidx = 0; cidx < n_splits; ++cidx) denom += expf(lse_part[cidx * n_rows + row] - m);
     const float inv = denom > 0.f ? 1.f / denom : 0.f;
+    const long long bh = row / Sq;
+    __nv_bfloat16* o_row = O + (bh / Hq) * o_stride_b + (bh % Hq) * o_stride_h + (row - bh * Sq) * o_stride_s;
 #pragma unroll
     for (int col = 0; col < DV; col += 128) {
         if (col + lane * 4 >= DV) break;
@@ -616,7 +618,7 @@ fa_combine_kernel(const float* __restrict__ o_part, const float* __restrict__ ls
         uint2 packed;
         packed.x = ptx::pack_bf16x2(acc.x, acc.y);
         packed.y = ptx::pack_bf16x2(acc.z, acc.w);
-        *reinterpret_cast<uint2*>(O + row * DV + col + lane * 4) = packed;
+        *reinterpret_cast<uint2*>(o_row + col + lane * 4) = packed;
     }
     if (lane == 0 && lse) lse[row] = (m == -INFINITY) ? -INFINITY : m + logf(denom);
 }

@@ -68,7 +68,6 @@ fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int off = p.Sk - p.Sq;
     const int n_kv = kv_tiles_for_q_tile(i0, kTileM, p.Sq, p.Sk, p.causal);
     const int q_idx = b * p.Hq + hq;
-    const int kv_idx = b * p.Hkv + kvh;
 
     if (tid == 0) {
         abort_flag = 0;
@@ -113,7 +112,7 @@ fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q,
         mbar_arrive_expect_tx(bar_q, Cfg::kQBytes);
 #pragma unroll
         for (int c = 0; c < Cfg::kQChunks; ++c)
-            tma_load_3d(sQ + c * kChunkBytes, &tm_q, bar_q, c * kChunkCols, i0, q_idx);
+            tma_load_4d(sQ + c * kChunkBytes, &tm_q, bar_q, c * kChunkCols, i0, hq, b);
     }
 
     for (int j = 0; j < n_kv && ok; ++j) {
@@ -122,11 +121,11 @@ fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q,
             mbar_arrive_expect_tx(bar_k, Cfg::kKBytes);
 #pragma unroll
             for (int c = 0; c < Cfg::kQChunks; ++c)
-                tma_load_3d(sK + c * kChunkBytes, &tm_k, bar_k, c * kChunkCols, j0, kv_idx);
+                tma_load_4d(sK + c * kChunkBytes, &tm_k, bar_k, c * kChunkCols, j0, kvh, b);
             mbar_arrive_expect_tx(bar_v, Cfg::kVBytes);
 #pragma unroll
             for (int c = 0; c < Cfg::kVChunks; ++c)
-                tma_load_3d(sV + c * kChunkBytes, &tm_v, bar_v, c * kChunkCols, j0, kv_idx);
+                tma_load_4d(sV + c * kChunkBytes, &tm_v, bar_v, c * kChunkCols, j0, kvh, b);
 
             bool w = true;
             if (j == 0) w = mbar_wait(bar_q, 0, wctx, kSiteSimpleQ);
@@ -228,7 +227,7 @@ fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q,
 
     // ---- epilogue: O = G' / s (bf16), lse = ln2 * u + ln s
     if (ok && i_glob < p.Sq) {
-        __nv_bfloat16* o_row = p.O + (static_cast<size_t>(q_idx) * p.Sq + i_glob) * DV;
+        __nv_bfloat16* o_row = p.O + (b * p.o_stride_b + hq * p.o_stride_h + static_cast<long long>(i_glob) * p.o_stride_s);
         const bool empty = (n_kv == 0) || !(l_run > 0.f);
         if (p.lse && tid < kTileM) {
             p.lse[static_cast<size_t>(q_idx) * p.Sq + i_glob] =
@@ -248,7 +247,7 @@ fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q,
             tmem_ld_x32(tO + lane_sel + c * 32, r);   // warp-collective: all lanes take part
             tc_wait_ld();
             if (i_glob < p.Sq) {
-                __nv_bfloat16* o_row = p.O + (static_cast<size_t>(q_idx) * p.Sq + i_glob) * DV;
+                __nv_bfloat16* o_row = p.O + (b * p.o_stride_b + hq * p.o_stride_h + static_cast<long long>(i_glob) * p.o_stride_s);
                 uint32_t pk[16];
 #pragma unroll
                 for (int e = 0; e < 32; e += 2)

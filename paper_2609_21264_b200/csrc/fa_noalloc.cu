@@ -85,13 +85,16 @@ fa_status setup_current_device(int device) {
     return FA_OK;
 }
 
-bool encode_map(EncodeTiledFn encode, CUtensorMap* map, const void* ptr, int d, int S, long long BH) {
-    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(S), static_cast<cuuint64_t>(BH)};
-    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2ull,
-                                   static_cast<cuuint64_t>(d) * 2ull * static_cast<cuuint64_t>(S)};
-    const cuuint32_t box[3] = {static_cast<cuuint32_t>(fa::kChunkCols), static_cast<cuuint32_t>(fa::kTileM), 1u};
-    const cuuint32_t estr[3] = {1u, 1u, 1u};
-    return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+// contiguous [B, H, S, d] bf16 tensor as a 4-D TMA tensor (d, S, H, B)
+bool encode_map(EncodeTiledFn encode, CUtensorMap* map, const void* ptr, int d, int S, int H, int B) {
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(S),
+                                static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(B)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(d) * 2ull,
+                                   static_cast<cuuint64_t>(d) * 2ull * static_cast<cuuint64_t>(S),
+                                   static_cast<cuuint64_t>(d) * 2ull * static_cast<cuuint64_t>(S) * static_cast<cuuint64_t>(H)};
+    const cuuint32_t box[4] = {static_cast<cuuint32_t>(fa::kChunkCols), static_cast<cuuint32_t>(fa::kTileM), 1u, 1u};
+    const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -106,7 +109,8 @@ fa_status launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap
     if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
     const long long n_rows = static_cast<long long>(p.B) * p.Hq * p.Sq;
     fa::fa_combine_kernel<DV><<<static_cast<unsigned>((n_rows + 3) / 4), 128, 0, st>>>(
-        p.o_part, p.lse_part, p.O, p.lse, n_rows, p.kv_splits);
+        p.o_part, p.lse_part, p.O, p.lse, n_rows, p.kv_splits, p.Hq, p.Sq,
+            p.o_stride_b, p.o_stride_h, p.o_stride_s);
     if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
 }
@@ -153,14 +157,17 @@ fa_status fa_forward_split_noalloc(const void* Q, const void* K, const void* V, 
     if (need > kStaticScratchBytes) return FA_ERR_UNSUPPORTED;     // partials exceed the fixed scratch
 
     CUtensorMap mq, mk, mv;
-    if (!encode_map(dev.encode, &mq, Q, dqk, Sq, static_cast<long long>(B) * Hq) ||
-        !encode_map(dev.encode, &mk, K, dqk, Sk, static_cast<long long>(B) * Hkv) ||
-        !encode_map(dev.encode, &mv, V, dv, Sk, static_cast<long long>(B) * Hkv))
+    if (!encode_map(dev.encode, &mq, Q, dqk, Sq, Hq, B) ||
+        !encode_map(dev.encode, &mk, K, dqk, Sk, Hkv, B) ||
+        !encode_map(dev.encode, &mv, V, dv, Sk, Hkv, B))
         return FA_ERR_CUDA;
 
     fa::FwdParams p;
     memset(&p, 0, sizeof p);
     p.O = static_cast<__nv_bfloat16*>(O);
+    p.o_stride_b = static_cast<long long>(Hq) * Sq * dv;
+    p.o_stride_h = static_cast<long long>(Sq) * dv;
+    p.o_stride_s = dv;
     p.lse = lse;
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Sk = Sk;
     p.causal = causal ? 1 : 0;

@@ -153,6 +153,17 @@ FA_DEVI void tma_load_3d(uint32_t dst_smem, const CUtensorMap* map, uint32_t bar
         : "memory");
 }
 
+// 4-D tiled load global -> shared (coordinates: column, row, head, batch).
+FA_DEVI void tma_load_4d(uint32_t dst_smem, const CUtensorMap* map, uint32_t bar,
+                         int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar),
+          "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
 // 3-D tiled store shared -> global (bulk async group).
 FA_DEVI void tma_store_3d(const CUtensorMap* map, uint32_t src_smem, int c0, int c1, int c2) {
     asm volatile(

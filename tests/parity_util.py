@@ -18,7 +18,7 @@ def to_torch_bf16(bits: np.ndarray, device="cuda"):
 
 def bf16_tensor_to_f64(t) -> np.ndarray:
     import torch
-    return t.detach().to("cpu").view(torch.int16).numpy().view(np.uint16).astype(np.uint32).__lshift__(16) \
+    return t.detach().to("cpu").contiguous().view(torch.int16).numpy().view(np.uint16).astype(np.uint32).__lshift__(16) \
         .view(np.float32).astype(np.float64)
 
 
