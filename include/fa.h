@@ -144,6 +144,34 @@ fa_status fa_forward_strided(fa_handle* h,
                              void* stream);
 
 /*
+ * Eq. 1 on a batch of sequences of different lengths, packed without padding (the paper's
+ * sequence-length sweeps run one length at a time; serving batches mix them).  Sequence b owns
+ * rows [cu_seqlens_q[b], cu_seqlens_q[b+1]) of Q and O and rows [cu_seqlens_k[b],
+ * cu_seqlens_k[b+1]) of K and V.
+ *   Q [total_q, Hq, dqk], K [total_k, Hkv, dqk], V [total_k, Hkv, dv], O [total_q, Hq, dv]: bf16,
+ *     contiguous, DEVICE pointers, 16-byte aligned.
+ *   lse [Hq, total_q] fp32 DEVICE pointer or NULL.
+ *   cu_seqlens_q, cu_seqlens_k: DEVICE arrays of B+1 int32, non-decreasing, starting at 0 and
+ *     ending at total_q / total_k.  The host never reads them (no synchronisation); the caller
+ *     vouches for their contents.
+ *   max_sq: an upper bound of the query lengths (sizes the grid).  Rows of a sequence past max_sq
+ *     are not computed and their O and lse are left untouched.
+ * The causal mask is aligned to the end of each sequence: key j of sequence b is visible to its
+ * query i iff j <= i + (Sk_b - Sq_b).  A sequence with no keys, and any row with no visible key,
+ * gets O = 0 and lse = -inf; a sequence with no queries writes nothing.  Rows of K/V past the end
+ * of a sequence take no part in the result, but must hold finite numbers where they belong to the
+ * next sequence (they are multiplied by a zero probability).  The K/V range is never split over
+ * CTAs on this path.  Errors as for fa_forward.
+ */
+fa_status fa_forward_varlen(fa_handle* h,
+                            const void* Q, const void* K, const void* V,
+                            void* O, float* lse,
+                            const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k,
+                            int B, int total_q, int total_k, int max_sq,
+                            int Hq, int Hkv, int dqk, int dv,
+                            int causal, float scale, void* stream);
+
+/*
  * The same operation with HOST buffers (same layouts and types): copies Q, K, V
  * to staging memory owned by the handle, runs fa_forward, copies O (and lse if
  * not NULL) back, all on `stream`, and synchronises `stream` before returning.

@@ -23,7 +23,7 @@ FA_ERR_OOM = 6
 FA_FLAG_SERIAL_KERNEL = 1
 FA_FLAG_DEBUG_DROP_V_LOAD = 2
 
-EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_host", "fa_last_status", "fa_destroy",
+EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_varlen", "fa_forward_host", "fa_last_status", "fa_destroy",
            "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits",
            "fa_forward_split_noalloc", "fa_noalloc_scratch_bytes")
 
@@ -65,6 +65,8 @@ def load():
     lib.fa_forward.argtypes = fwd_args
     lib.fa_forward_host.restype = i32
     lib.fa_forward_host.argtypes = fwd_args
+    lib.fa_forward_varlen.restype = i32
+    lib.fa_forward_varlen.argtypes = [vp] * 8 + [i32] * 8 + [i32, ctypes.c_float, vp]
     lib.fa_forward_strided.restype = i32
     lib.fa_forward_strided.argtypes = fwd_args[:-1] + [vp, vp, vp, vp, vp]
     lib.fa_last_status.restype = i32
@@ -114,6 +116,13 @@ def fa_forward_strided(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, 
     arr = [(ctypes.c_int64 * 3)(*[int(x) for x in st]) for st in (q_strides, k_strides, v_strides, o_strides)]
     return load().fa_forward_strided(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, int(bool(causal)), float(scale),
                                      arr[0], arr[1], arr[2], arr[3], stream)
+
+
+def fa_forward_varlen(h, Q, K, V, O, lse, cu_seqlens_q, cu_seqlens_k, B, total_q, total_k, max_sq,
+                      Hq, Hkv, dqk, dv, causal, scale, stream=0) -> int:
+    """Raw call on packed [total, H, d] device tensors with device int32 offsets; returns the status code."""
+    return load().fa_forward_varlen(h, Q, K, V, O, lse, cu_seqlens_q, cu_seqlens_k, B, total_q, total_k, max_sq,
+                                    Hq, Hkv, dqk, dv, int(bool(causal)), float(scale), stream)
 
 
 def fa_forward_host(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, stream=0) -> int:
@@ -197,4 +206,29 @@ def forward(h, q, k, v, *, causal: bool, scale: float = 0.0, out=None, lse=None,
                                 q.stride()[:3], k.stride()[:3], v.stride()[:3], out.stride()[:3], stream)
     if st != FA_OK:
         raise FaError(st, "fa_forward")
+    return out, lse
+
+
+def forward_varlen(h, q, k, v, cu_seqlens_q, cu_seqlens_k, max_sq: int, *, causal: bool, scale: float = 0.0,
+                   want_lse=True):
+    """Packed variable-length batch: q [total_q,Hq,d], k/v [total_k,Hkv,d] bf16 CUDA tensors, int32 CUDA
+    offset tensors of B+1 entries.  Returns (O [total_q,Hq,dv], lse [Hq,total_q])."""
+    import torch
+    for t in (q, k, v):
+        if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous() or t.dim() != 3:
+            raise ValueError("q, k, v must be contiguous 3-D bf16 CUDA tensors")
+    for t in (cu_seqlens_q, cu_seqlens_k):
+        if t.dtype != torch.int32 or not t.is_cuda or not t.is_contiguous() or t.dim() != 1:
+            raise ValueError("cu_seqlens must be contiguous 1-D int32 CUDA tensors")
+    total_q, Hq, dqk = q.shape
+    total_k, Hkv, dv = v.shape
+    B = cu_seqlens_q.numel() - 1
+    out = torch.empty((total_q, Hq, dv), dtype=torch.bfloat16, device=q.device)
+    lse = torch.empty((Hq, total_q), dtype=torch.float32, device=q.device) if want_lse else None
+    st = fa_forward_varlen(h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                           lse.data_ptr() if lse is not None else None,
+                           cu_seqlens_q.data_ptr(), cu_seqlens_k.data_ptr(), B, total_q, total_k, int(max_sq),
+                           Hq, Hkv, dqk, dv, causal, scale, torch.cuda.current_stream(q.device).cuda_stream)
+    if st != FA_OK:
+        raise FaError(st, "fa_forward_varlen")
     return out, lse

@@ -52,7 +52,7 @@ struct fa_handle {
     const char* last_kernel = "";
     void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // Q K V O lse
     size_t stage_cap[5] = {0, 0, 0, 0, 0};
-    bool attr_done[8] = {false, false, false, false, false, false, false, false};
+    bool attr_done[12] = {};
 #ifdef FA_TRACE
     long long* trace = nullptr;
 #endif
@@ -142,12 +142,12 @@ fa_status launch_simple(fa_handle* h, int slot, const CUtensorMap& mq, const CUt
     return FA_OK;
 }
 
-template <int DQK, int DV>
+template <int DQK, int DV, bool kVarlen>
 fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
                            const CUtensorMap& mv, const fa::FwdParams& p, cudaStream_t st) {
     constexpr int smem = fa::pipe_smem_bytes<DQK, DV>();
     static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
-    auto kernel = fa::fa_fwd_pipelined_kernel<DQK, DV>;
+    auto kernel = fa::fa_fwd_pipelined_kernel<DQK, DV, kVarlen>;
     fa_status s = ensure_smem_attr(h, slot, kernel, smem);
     if (s != FA_OK) return s;
     const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq * p.B * p.kv_splits;
@@ -212,6 +212,82 @@ fa_status check_args(const void* Q, const void* K, const void* V, const void* O,
     if (Hq > 65535 || B > 65535 || n_q_tiles > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     if (static_cast<long long>(B) * Hq > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     return FA_OK;
+}
+
+// Fills the launch parameters and starts the kernel(s); the tensor maps are ready.
+// cu_q == nullptr: fixed lengths Sq, Sk.  Otherwise a packed variable-length batch whose longest
+// query is Sq rows and whose sequences have about Sk keys (L2 grouping only).
+fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap& map_k, const CUtensorMap& map_v,
+                      void* O, float* lse, int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal,
+                      float scale, const int64_t* o_strides, const int* cu_q, const int* cu_k, int total_q,
+                      cudaStream_t st) {
+    if (scale == 0.f) scale = 1.f / sqrtf(static_cast<float>(dqk));
+    fa::FwdParams p;
+    p.O = static_cast<__nv_bfloat16*>(O);
+    p.o_stride_b = o_strides[0];
+    p.o_stride_h = o_strides[1];
+    p.o_stride_s = o_strides[2];
+    p.cu_q = cu_q;
+    p.cu_k = cu_k;
+    p.total_q = total_q;
+    p.lse = lse;
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Sk = Sk;
+    p.causal = causal ? 1 : 0;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
+    {
+        // Heads whose K and V (read again by every query tile of the head) fit in about a third of
+        // the 126 MB L2 together; at least one K/V head, i.e. one GQA group of query heads.
+        const long long kv_bytes = static_cast<long long>(Sk) * (dqk + dv) * 2;
+        const long long budget = 48ll << 20;
+        long long kv_heads = budget / kv_bytes;
+        if (kv_heads < 1) kv_heads = 1;
+        long long hpg = kv_heads * (Hq / Hkv);
+        const long long n_bh = static_cast<long long>(B) * Hq;
+        if (hpg > n_bh) hpg = n_bh;
+        p.heads_per_group = static_cast<int>(hpg);
+    }
+    p.status = h->status_dev;
+    p.wait_limit_ns = h->wait_limit_ns;
+    p.debug_drop_v_load = (h->flags & FA_FLAG_DEBUG_DROP_V_LOAD) ? 1 : 0;
+    p.kv_splits = 1;
+    p.tiles_per_split = 0x3fffffff;
+    p.o_part = nullptr;
+    p.lse_part = nullptr;
+    if (!(h->flags & FA_FLAG_SERIAL_KERNEL) && !cu_q) {   // packed batches: no split (lengths are on the device)
+        const int splits = choose_kv_splits(h, B, Hq, Sq, Sk, dv, p.causal, p.n_q_tiles);
+        if (splits > 1) {
+            int max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
+            if (p.causal) {
+                const int t = fa::kv_tiles_for_q_tile((p.n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, 1);
+                if (t < max_tiles) max_tiles = t;
+            }
+            p.kv_splits = splits;
+            p.tiles_per_split = (max_tiles + splits - 1) / splits;
+            p.o_part = static_cast<float*>(h->scratch);
+            p.lse_part = p.o_part + static_cast<size_t>(splits) * B * Hq * Sq * dv;
+        }
+    }
+    h->last_splits = p.kv_splits;
+#ifdef FA_TRACE
+    p.trace = h->trace;
+#endif
+
+    if (!(h->flags & FA_FLAG_SERIAL_KERNEL)) {
+        h->last_kernel = "fa_fwd_pipelined";
+        if (cu_q) {
+            if (dqk == 64) return launch_pipelined<64, 64, true>(h, 6, map_q, map_k, map_v, p, st);
+            if (dqk == 128) return launch_pipelined<128, 128, true>(h, 7, map_q, map_k, map_v, p, st);
+            return launch_pipelined<192, 128, true>(h, 8, map_q, map_k, map_v, p, st);
+        }
+        if (dqk == 64) return launch_pipelined<64, 64, false>(h, 3, map_q, map_k, map_v, p, st);
+        if (dqk == 128) return launch_pipelined<128, 128, false>(h, 4, map_q, map_k, map_v, p, st);
+        return launch_pipelined<192, 128, false>(h, 5, map_q, map_k, map_v, p, st);
+    }
+    h->last_kernel = "fa_fwd_simple";
+    if (dqk == 64) return launch_simple<64, 64>(h, 0, map_q, map_k, map_v, p, st);
+    if (dqk == 128) return launch_simple<128, 128>(h, 1, map_q, map_k, map_v, p, st);
+    return launch_simple<192, 128>(h, 2, map_q, map_k, map_v, p, st);
 }
 
 }  // namespace
@@ -353,8 +429,6 @@ fa_status fa_forward_strided(fa_handle* h, const void* Q, const void* K, const v
     DeviceGuard guard(h->device);
     if (!guard.ok()) return FA_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (scale == 0.f) scale = 1.f / sqrtf(static_cast<float>(dqk));
-
     const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr;
     if ((s = get_map(h, Q, dqk, Sq, Hq, B, q_strides[0], q_strides[1], q_strides[2], fa::kTileM, &mq)) != FA_OK) return s;
     CUtensorMap map_q = *mq;   // copies: a later insertion may evict or move cache entries
@@ -363,64 +437,8 @@ fa_status fa_forward_strided(fa_handle* h, const void* Q, const void* K, const v
     if ((s = get_map(h, V, dv, Sk, Hkv, B, v_strides[0], v_strides[1], v_strides[2], fa::kTileN, &mv)) != FA_OK) return s;
     CUtensorMap map_v = *mv;
 
-    fa::FwdParams p;
-    p.O = static_cast<__nv_bfloat16*>(O);
-    p.o_stride_b = o_strides[0];
-    p.o_stride_h = o_strides[1];
-    p.o_stride_s = o_strides[2];
-    p.lse = lse;
-    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Sk = Sk;
-    p.causal = causal ? 1 : 0;
-    p.scale_log2 = scale * 1.4426950408889634f;
-    p.n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
-    {
-        // Heads whose K and V (read again by every query tile of the head) fit in about a third of
-        // the 126 MB L2 together; at least one K/V head, i.e. one GQA group of query heads.
-        const long long kv_bytes = static_cast<long long>(Sk) * (dqk + dv) * 2;
-        const long long budget = 48ll << 20;
-        long long kv_heads = budget / kv_bytes;
-        if (kv_heads < 1) kv_heads = 1;
-        long long hpg = kv_heads * (Hq / Hkv);
-        const long long n_bh = static_cast<long long>(B) * Hq;
-        if (hpg > n_bh) hpg = n_bh;
-        p.heads_per_group = static_cast<int>(hpg);
-    }
-    p.status = h->status_dev;
-    p.wait_limit_ns = h->wait_limit_ns;
-    p.debug_drop_v_load = (h->flags & FA_FLAG_DEBUG_DROP_V_LOAD) ? 1 : 0;
-    p.kv_splits = 1;
-    p.tiles_per_split = 0x3fffffff;
-    p.o_part = nullptr;
-    p.lse_part = nullptr;
-    if (!(h->flags & FA_FLAG_SERIAL_KERNEL)) {
-        const int splits = choose_kv_splits(h, B, Hq, Sq, Sk, dv, p.causal, p.n_q_tiles);
-        if (splits > 1) {
-            int max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
-            if (p.causal) {
-                const int t = fa::kv_tiles_for_q_tile((p.n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, 1);
-                if (t < max_tiles) max_tiles = t;
-            }
-            p.kv_splits = splits;
-            p.tiles_per_split = (max_tiles + splits - 1) / splits;
-            p.o_part = static_cast<float*>(h->scratch);
-            p.lse_part = p.o_part + static_cast<size_t>(splits) * B * Hq * Sq * dv;
-        }
-    }
-    h->last_splits = p.kv_splits;
-#ifdef FA_TRACE
-    p.trace = h->trace;
-#endif
-
-    if (!(h->flags & FA_FLAG_SERIAL_KERNEL)) {
-        h->last_kernel = "fa_fwd_pipelined";
-        if (dqk == 64) return launch_pipelined<64, 64>(h, 3, map_q, map_k, map_v, p, st);
-        if (dqk == 128) return launch_pipelined<128, 128>(h, 4, map_q, map_k, map_v, p, st);
-        return launch_pipelined<192, 128>(h, 5, map_q, map_k, map_v, p, st);
-    }
-    h->last_kernel = "fa_fwd_simple";
-    if (dqk == 64) return launch_simple<64, 64>(h, 0, map_q, map_k, map_v, p, st);
-    if (dqk == 128) return launch_simple<128, 128>(h, 1, map_q, map_k, map_v, p, st);
-    return launch_simple<192, 128>(h, 2, map_q, map_k, map_v, p, st);
+    return run_forward(h, map_q, map_k, map_v, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, o_strides,
+                       nullptr, nullptr, 0, st);
 }
 
 fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, void* O, float* lse,
@@ -432,6 +450,38 @@ fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, 
     const int64_t vs[3] = {static_cast<int64_t>(Hkv) * Sk * dv, static_cast<int64_t>(Sk) * dv, dv};
     const int64_t os[3] = {static_cast<int64_t>(Hq) * Sq * dv, static_cast<int64_t>(Sq) * dv, dv};
     return fa_forward_strided(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, qs, ks, vs, os, stream);
+}
+
+fa_status fa_forward_varlen(fa_handle* h, const void* Q, const void* K, const void* V, void* O, float* lse,
+                            const int32_t* cu_seqlens_q, const int32_t* cu_seqlens_k, int B, int total_q,
+                            int total_k, int max_sq, int Hq, int Hkv, int dqk, int dv, int causal, float scale,
+                            void* stream) {
+    if (!h || !cu_seqlens_q || !cu_seqlens_k) return FA_ERR_INVALID_ARG;
+    if (B < 0 || total_q < 0 || total_k < 0 || max_sq < 0 || max_sq > total_q) return FA_ERR_INVALID_ARG;
+    if (misaligned(cu_seqlens_q, 4) || misaligned(cu_seqlens_k, 4)) return FA_ERR_INVALID_ARG;
+    if (B == 0 || total_q == 0 || max_sq == 0) return FA_OK;           // no query rows: nothing to write
+    // K and V may be empty (every row then gets O = 0, lse = -inf); the maps still need one row
+    fa_status s = check_args(Q, K, V, O, lse, B, Hq, Hkv, max_sq, total_k > 0 ? total_k : 1, dqk, dv, scale, true);
+    if (s != FA_OK) return s;
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return FA_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // packed [total, H, d]: one batch slice, rows H*d apart, heads d apart
+    const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr;
+    const int rows_k = total_k > 0 ? total_k : 1;   // an empty K/V still gets a valid map; no tile of it is ever read
+    if ((s = get_map(h, Q, dqk, total_q, Hq, 1, static_cast<long long>(total_q) * Hq * dqk, dqk,
+                     static_cast<long long>(Hq) * dqk, fa::kTileM, &mq)) != FA_OK) return s;
+    CUtensorMap map_q = *mq;
+    if ((s = get_map(h, K, dqk, rows_k, Hkv, 1, static_cast<long long>(rows_k) * Hkv * dqk, dqk,
+                     static_cast<long long>(Hkv) * dqk, fa::kTileN, &mk)) != FA_OK) return s;
+    CUtensorMap map_k = *mk;
+    if ((s = get_map(h, V, dv, rows_k, Hkv, 1, static_cast<long long>(rows_k) * Hkv * dv, dv,
+                     static_cast<long long>(Hkv) * dv, fa::kTileN, &mv)) != FA_OK) return s;
+    CUtensorMap map_v = *mv;
+    const int64_t os[3] = {0, dv, static_cast<int64_t>(Hq) * dv};
+    const int mean_sk = (total_k + B - 1) / B > 0 ? (total_k + B - 1) / B : 1;
+    return run_forward(h, map_q, map_k, map_v, O, lse, B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal, scale, os,
+                       cu_seqlens_q, cu_seqlens_k, total_q, st);
 }
 
 fa_status fa_forward_host(fa_handle* h, const void* Qh, const void* Kh, const void* Vh, void* Oh,

@@ -29,6 +29,12 @@ struct FwdParams {
     long long o_stride_b, o_stride_h, o_stride_s;   // in elements
     float* lse;               // [B, Hq, Sq] or nullptr
     int B, Hq, Hkv, Sq, Sk;
+    // Variable-length batches: sequence b owns rows [cu_q[b], cu_q[b+1]) of the packed Q/O and
+    // [cu_k[b], cu_k[b+1]) of the packed K/V (device arrays of B+1 ints); nullptr = fixed Sq/Sk.
+    // Then Sq is the longest query length (grid sizing only) and lse is [Hq, total_q].
+    const int* cu_q;
+    const int* cu_k;
+    int total_q;
     int causal;
     float scale_log2;         // scale * log2(e): scores are handled in log2 units
     int n_q_tiles;            // ceil(Sq / 128)

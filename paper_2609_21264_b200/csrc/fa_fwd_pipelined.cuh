@@ -77,7 +77,9 @@ constexpr int pipe_smem_bytes() {
     return PipeCfg<DQK, DV>::kTileBytes + static_cast<int>(sizeof(PipeShared));
 }
 
-template <int DQK, int DV>
+// kVarlen = packed variable-length batch (per-sequence offsets and lengths read from p.cu_q/p.cu_k);
+// a template parameter so that the fixed-length instantiation carries none of its scalars.
+template <int DQK, int DV, bool kVarlen = false>
 __global__ void __launch_bounds__(512, 1)
 fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                         const __grid_constant__ CUtensorMap tm_k,
@@ -131,21 +133,31 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int b = bh / p.Hq;
     const int kvh = hq / (p.Hq / p.Hkv);
     const int q_idx = b * p.Hq + hq;
-    const int off = p.Sk - p.Sq;
+    // Problem of this CTA: Sq x Sk, its Q rows starting at q_row0 and K/V rows at k_row0 of the
+    // tensors the maps describe (packed variable-length tensors are one batch slice).
+    int Sq = p.Sq, Sk = p.Sk, q_row0 = 0, k_row0 = 0;
+    if constexpr (kVarlen) {
+        q_row0 = p.cu_q[b];
+        k_row0 = p.cu_k[b];
+        Sq = p.cu_q[b + 1] - q_row0;
+        Sk = p.cu_k[b + 1] - k_row0;
+    }
+    const int off = Sk - Sq;
 
     // per-tile scalars (no arrays: a runtime-indexed array would live in local memory)
     const int i0_0 = (2 * pair) * kTileM, i0_1 = i0_0 + kTileM;
     // K/V tiles [j_base, j_base + nkv_t) of tile t belong to this CTA (all visible ones without split-KV)
     const int j_base = split * p.tiles_per_split;
     auto own_tiles = [&](int i0) -> int {
-        if (i0 >= p.Sq) return 0;
-        int n = kv_tiles_for_q_tile(i0, kTileM, p.Sq, p.Sk, p.causal) - j_base;
+        if (i0 >= Sq) return 0;
+        int n = kv_tiles_for_q_tile(i0, kTileM, Sq, Sk, p.causal) - j_base;
         if (n > p.tiles_per_split) n = p.tiles_per_split;
         return n > 0 ? n : 0;
     };
     const int nkv_0 = own_tiles(i0_0);
     const int nkv_1 = own_tiles(i0_1);
     const int n_max = nkv_0 > nkv_1 ? nkv_0 : nkv_1;
+    if (kVarlen && i0_0 >= Sq) return;    // a sequence shorter than the longest one: no rows here (whole CTA, before any set-up)
 
     // ---------------------------------------------------------------- setup
     if (tid == 0) {
@@ -200,7 +212,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         const int i0_t = t == 0 ? i0_0 : i0_1;
         const int nkv_t = t == 0 ? nkv_0 : nkv_1;
         const int i_glob = i0_t + row;
-        int kmax_row = p.Sk - 1;
+        int kmax_row = Sk - 1;
         if (p.causal && i_glob + off < kmax_row) kmax_row = i_glob + off;
         const float tau_raw = kRescaleThresholdLog2 / c;
 
@@ -309,7 +321,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             if (lane == 0 && ((warp & 3) == 0 || (warp & 3) == 2)) FA_TRACE_STAMP(t + ((warp & 3) == 2 ? 4 : 0), j, 4);
         }
         // epilogue: O = G' / s (bf16), lse = u * scale + ln s
-        if (ok && i0_t < p.Sq && p.kv_splits > 1) {
+        if (ok && i0_t < Sq && p.kv_splits > 1) {
             // split-KV: this CTA's partial (G'_c / s_c in fp32, and u_c + ln s_c) goes to scratch;
             // the combine kernel merges the C partials of a row (Algorithm 2's reduction).
             const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
@@ -319,7 +331,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             if (nkv_t == 0 || have) {
                 tc_fence_after_sync();
                 const float inv_l = (nkv_t > 0 && l > 0.f) ? (1.f / l) : 0.f;
-                if (i_glob < p.Sq)
+                if (i_glob < Sq)
                     p.lse_part[prow] = (nkv_t > 0 && l > 0.f) ? (m_ref * c * 0.6931471805599453f + logf(l)) : -INFINITY;
                 const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1) + lane_sel;
 #pragma unroll 1
@@ -329,7 +341,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                         tmem_ld_x32(tO + cc * 32, r);
                         tc_wait_ld();
                     }
-                    if (i_glob < p.Sq) {
+                    if (i_glob < Sq) {
 #pragma unroll
                         for (int v = 0; v < 8; ++v) {
                             float4 f;
@@ -342,20 +354,24 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                     }
                 }
             }
-        } else if (ok && i0_t < p.Sq) {
-            __nv_bfloat16* o_row = p.O + (b * p.o_stride_b + hq * p.o_stride_h + static_cast<long long>(i_glob) * p.o_stride_s);
+        } else if (ok && i0_t < Sq) {
+            // fixed lengths: lse [B, Hq, Sq]; packed batches: lse [Hq, total_q], O rows q_row0 onwards
+            const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq) * p.total_q + q_row0
+                                           : static_cast<size_t>(q_idx) * p.Sq;
+            const long long o_base = (kVarlen ? q_row0 * p.o_stride_s : b * p.o_stride_b) + hq * p.o_stride_h;
+            __nv_bfloat16* o_row = p.O + (o_base + static_cast<long long>(i_glob) * p.o_stride_s);
             if (nkv_t == 0) {         // no key visible to any row of this tile
-                if (i_glob < p.Sq) {
+                if (i_glob < Sq) {
                     const uint4 z = make_uint4(0, 0, 0, 0);
 #pragma unroll
                     for (int v = 0; v < DV / 8; ++v) reinterpret_cast<uint4*>(o_row)[v] = z;
-                    if (p.lse) p.lse[static_cast<size_t>(q_idx) * p.Sq + i_glob] = -INFINITY;
+                    if (p.lse) p.lse[lse_row0 + i_glob] = -INFINITY;
                 }
             } else if (__all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.o_final[t]), 0, wctx, kSiteEpiOFull))) {
                 tc_fence_after_sync();
                 const float inv_l = (l > 0.f) ? (1.f / l) : 0.f;
-                if (p.lse && i_glob < p.Sq) {
-                    p.lse[static_cast<size_t>(q_idx) * p.Sq + i_glob] =
+                if (p.lse && i_glob < Sq) {
+                    p.lse[lse_row0 + i_glob] =
                         (l > 0.f) ? (m_ref * c * 0.6931471805599453f + logf(l)) : -INFINITY;
                 }
                 const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1) + lane_sel;
@@ -364,7 +380,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                     uint32_t r[32];
                     tmem_ld_x32(tO + cc * 32, r);
                     tc_wait_ld();
-                    if (i_glob < p.Sq) {
+                    if (i_glob < Sq) {
                         uint32_t pk[16];
 #pragma unroll
                         for (int e = 0; e < 32; e += 2)
@@ -535,7 +551,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kQChunks; ++cc)
                     tma_load_4d(sQ + t * Cfg::kQBytes + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols,
-                                t == 0 ? i0_0 : i0_1, hq, b);
+                                q_row0 + (t == 0 ? i0_0 : i0_1), hq, kVarlen ? 0 : b);
             };
             // Order of the first requests: Q_0 and K_0 (all the first MMA needs), then Q_1, then V_0.
             // When a whole wave of CTAs starts at once these first loads are HBM-bandwidth-bound.
@@ -552,7 +568,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                     for (int cc = 0; cc < Cfg::kQChunks; ++cc)
                         tma_load_4d(sK + s * Cfg::kKBytes + cc * kChunkBytes, &tm_k, bar, cc * kChunkCols,
-                                    j0, kvh, b);
+                                    k_row0 + j0, kvh, kVarlen ? 0 : b);
                     if (j == 0) load_q(1);
                 }
                 if (!(p.debug_drop_v_load && j == 0)) {
@@ -564,7 +580,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                     for (int cc = 0; cc < Cfg::kVChunks; ++cc)
                         tma_load_4d(sV + s * Cfg::kVBytes + cc * kChunkBytes, &tm_v, bar, cc * kChunkCols,
-                                    j0, kvh, b);
+                                    k_row0 + j0, kvh, kVarlen ? 0 : b);
                 }
             }
         }

@@ -65,9 +65,23 @@ fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int b = blockIdx.z;
     const int kvh = hq / (p.Hq / p.Hkv);
     const int i0 = q_tile * kTileM;
-    const int off = p.Sk - p.Sq;
-    const int n_kv = kv_tiles_for_q_tile(i0, kTileM, p.Sq, p.Sk, p.causal);
     const int q_idx = b * p.Hq + hq;
+    // fixed-length batch, or sequence b of a packed variable-length batch
+    int Sq = p.Sq, Sk = p.Sk, q_row0 = 0, k_row0 = 0, tb = b;
+    size_t lse_row0 = static_cast<size_t>(q_idx) * p.Sq;
+    long long o_base = b * p.o_stride_b + hq * p.o_stride_h;
+    if (p.cu_q) {
+        q_row0 = p.cu_q[b];
+        k_row0 = p.cu_k[b];
+        Sq = p.cu_q[b + 1] - q_row0;
+        Sk = p.cu_k[b + 1] - k_row0;
+        tb = 0;
+        lse_row0 = static_cast<size_t>(hq) * p.total_q + q_row0;
+        o_base = q_row0 * p.o_stride_s + hq * p.o_stride_h;
+    }
+    if (i0 >= Sq) return;      // whole CTA, before any set-up
+    const int off = Sk - Sq;
+    const int n_kv = kv_tiles_for_q_tile(i0, kTileM, Sq, Sk, p.causal);
 
     if (tid == 0) {
         abort_flag = 0;
@@ -100,7 +114,7 @@ fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q,
     constexpr uint32_t kIdescPV = make_idesc_bf16_f32(kTileM, DV, false, true);
 
     const int i_glob = i0 + tid;                 // this thread's query row
-    int kmax_row = p.Sk - 1;                     // last visible key of this row
+    int kmax_row = Sk - 1;                       // last visible key of this row
     if (p.causal && i_glob + off < kmax_row) kmax_row = i_glob + off;
 
     float m_run = -INFINITY;   // running row max (log2 units)
@@ -112,7 +126,7 @@ fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q,
         mbar_arrive_expect_tx(bar_q, Cfg::kQBytes);
 #pragma unroll
         for (int c = 0; c < Cfg::kQChunks; ++c)
-            tma_load_4d(sQ + c * kChunkBytes, &tm_q, bar_q, c * kChunkCols, i0, hq, b);
+            tma_load_4d(sQ + c * kChunkBytes, &tm_q, bar_q, c * kChunkCols, q_row0 + i0, hq, tb);
     }
 
     for (int j = 0; j < n_kv && ok; ++j) {
@@ -121,11 +135,11 @@ fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q,
             mbar_arrive_expect_tx(bar_k, Cfg::kKBytes);
 #pragma unroll
             for (int c = 0; c < Cfg::kQChunks; ++c)
-                tma_load_4d(sK + c * kChunkBytes, &tm_k, bar_k, c * kChunkCols, j0, kvh, b);
+                tma_load_4d(sK + c * kChunkBytes, &tm_k, bar_k, c * kChunkCols, k_row0 + j0, kvh, tb);
             mbar_arrive_expect_tx(bar_v, Cfg::kVBytes);
 #pragma unroll
             for (int c = 0; c < Cfg::kVChunks; ++c)
-                tma_load_4d(sV + c * kChunkBytes, &tm_v, bar_v, c * kChunkCols, j0, kvh, b);
+                tma_load_4d(sV + c * kChunkBytes, &tm_v, bar_v, c * kChunkCols, k_row0 + j0, kvh, tb);
 
             bool w = true;
             if (j == 0) w = mbar_wait(bar_q, 0, wctx, kSiteSimpleQ);
@@ -226,11 +240,11 @@ fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q,
     }
 
     // ---- epilogue: O = G' / s (bf16), lse = ln2 * u + ln s
-    if (ok && i_glob < p.Sq) {
-        __nv_bfloat16* o_row = p.O + (b * p.o_stride_b + hq * p.o_stride_h + static_cast<long long>(i_glob) * p.o_stride_s);
+    if (ok && i_glob < Sq) {
+        __nv_bfloat16* o_row = p.O + (o_base + static_cast<long long>(i_glob) * p.o_stride_s);
         const bool empty = (n_kv == 0) || !(l_run > 0.f);
         if (p.lse && tid < kTileM) {
-            p.lse[static_cast<size_t>(q_idx) * p.Sq + i_glob] =
+            p.lse[lse_row0 + i_glob] =
                 empty ? -INFINITY : (m_run * 0.6931471805599453f + logf(l_run));
         }
         if (n_kv == 0) {
@@ -246,8 +260,8 @@ fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q,
             uint32_t r[32];
             tmem_ld_x32(tO + lane_sel + c * 32, r);   // warp-collective: all lanes take part
             tc_wait_ld();
-            if (i_glob < p.Sq) {
-                __nv_bfloat16* o_row = p.O + (b * p.o_stride_b + hq * p.o_stride_h + static_cast<long long>(i_glob) * p.o_stride_s);
+            if (i_glob < Sq) {
+                __nv_bfloat16* o_row = p.O + (o_base + static_cast<long long>(i_glob) * p.o_stride_s);
                 uint32_t pk[16];
 #pragma unroll
                 for (int e = 0; e < 32; e += 2)

@@ -168,6 +168,9 @@ fa_status fa_forward_split_noalloc(const void* Q, const void* K, const void* V, 
     p.o_stride_b = static_cast<long long>(Hq) * Sq * dv;
     p.o_stride_h = static_cast<long long>(Sq) * dv;
     p.o_stride_s = dv;
+    p.cu_q = nullptr;
+    p.cu_k = nullptr;
+    p.total_q = 0;
     p.lse = lse;
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Sk = Sk;
     p.causal = causal ? 1 : 0;

@@ -1,0 +1,123 @@
+"""fa_forward_varlen: packed batches of sequences of different lengths against the oracle, sequence by sequence.
+
+The oracle only knows one fixed-length problem, so every sequence of the batch is cut out of the
+packed tensors and given to it on its own; the GPU sees the packed batch in one call.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_21264_b200 import workloads as W
+from parity_util import assert_parity, bf16_tensor_to_f64, to_torch_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", params=["pipelined", "serial"])
+def handle(request):
+    from paper_2609_21264_b200 import binding
+    h = binding.fa_create(flags=binding.FA_FLAG_SERIAL_KERNEL if request.param == "serial" else 0)
+    yield h
+    binding.fa_destroy(h)
+
+
+def _packed_inputs(lens_q, lens_k, Hq, Hkv, dqk, dv, seed):
+    """Packed [total, H, d] bf16 bit tensors drawn with the recipe of the fixed-length workloads."""
+    tq, tk = int(sum(lens_q)), int(sum(lens_k))
+    w = W.Workload("packed", B=1, Hq=Hq, Hkv=Hkv, Sq=max(tq, 1), Sk=max(tk, 1), dqk=dqk, dv=dv,
+                   causal=False, scale=dqk ** -0.5, seed=seed)
+    Q, K, V = W.make_inputs(w)           # [1, H, S, d]
+    q = np.ascontiguousarray(Q[0].transpose(1, 0, 2))[:tq]
+    k = np.ascontiguousarray(K[0].transpose(1, 0, 2))[:tk]
+    v = np.ascontiguousarray(V[0].transpose(1, 0, 2))[:tk]
+    return q, k, v
+
+
+def _run_and_check(handle, lens_q, lens_k, Hq, Hkv, dqk, dv, causal, seed, max_sq=None):
+    import torch
+    from paper_2609_21264_b200 import binding
+    q, k, v = _packed_inputs(lens_q, lens_k, Hq, Hkv, dqk, dv, seed)
+    cu_q = np.concatenate([[0], np.cumsum(lens_q)]).astype(np.int32)
+    cu_k = np.concatenate([[0], np.cumsum(lens_k)]).astype(np.int32)
+    tq, tk = q.shape[0], k.shape[0]
+    dq = to_torch_bf16(q) if tq else torch.empty((0, Hq, dqk), dtype=torch.bfloat16, device="cuda")
+    dk = to_torch_bf16(k) if tk else torch.empty((0, Hkv, dqk), dtype=torch.bfloat16, device="cuda")
+    dv_ = to_torch_bf16(v) if tk else torch.empty((0, Hkv, dv), dtype=torch.bfloat16, device="cuda")
+    if tk == 0:   # the call wants non-null pointers even for empty K/V
+        dk = torch.zeros((1, Hkv, dqk), dtype=torch.bfloat16, device="cuda")[:0]
+        dv_ = torch.zeros((1, Hkv, dv), dtype=torch.bfloat16, device="cuda")[:0]
+    o, lse = binding.forward_varlen(handle, dq, dk, dv_, torch.from_numpy(cu_q).cuda(), torch.from_numpy(cu_k).cuda(),
+                                    max(lens_q) if max_sq is None else max_sq, causal=causal, scale=dqk ** -0.5)
+    torch.cuda.synchronize()
+    st, detail = binding.fa_last_status(handle)
+    assert st == binding.FA_OK, "device status %d (site 0x%x)" % (st, detail)
+    O = bf16_tensor_to_f64(o) if tq else np.zeros((0, Hq, dv))
+    L = lse.double().cpu().numpy()
+    for b, (sq, sk) in enumerate(zip(lens_q, lens_k)):
+        if sq == 0:
+            continue
+        qs, ks = slice(cu_q[b], cu_q[b + 1]), slice(cu_k[b], cu_k[b + 1])
+        O_b = O[qs].transpose(1, 0, 2)[None]
+        L_b = L[:, qs][None]
+        if sk == 0:
+            assert (O_b == 0).all() and np.isneginf(L_b).all()
+            continue
+        Qb = np.ascontiguousarray(q[qs].transpose(1, 0, 2))[None]
+        Kb = np.ascontiguousarray(k[ks].transpose(1, 0, 2))[None]
+        Vb = np.ascontiguousarray(v[ks].transpose(1, 0, 2))[None]
+        O_ref, lse_ref = oracle.attention(Qb, Kb, Vb, causal=causal, scale=dqk ** -0.5)
+        assert_parity(O_b, L_b, O_ref, lse_ref, "seq %d (%d x %d)" % (b, sq, sk))
+    return O, L
+
+
+@pytest.mark.parametrize("causal", [False, True], ids=["full", "causal"])
+def test_self_attention_length_mix(handle, causal):
+    lens = [1, 127, 128, 129, 300, 512, 57]
+    _run_and_check(handle, lens, lens, Hq=4, Hkv=2, dqk=128, dv=128, causal=causal, seed=1101)
+
+
+@pytest.mark.parametrize("dqk,dv", [(64, 64), (192, 128)], ids=["d64", "d192_128"])
+def test_other_head_sizes(handle, dqk, dv):
+    lens = [260, 31, 129]
+    _run_and_check(handle, lens, lens, Hq=3, Hkv=3, dqk=dqk, dv=dv, causal=True, seed=1102)
+
+
+def test_cross_lengths_and_empty_sequences(handle):
+    """Sq_b != Sk_b (end-aligned causal mask), a sequence with no queries and one with no keys."""
+    lens_q = [40, 0, 200, 130, 5]
+    lens_k = [333, 50, 200, 0, 700]
+    _run_and_check(handle, lens_q, lens_k, Hq=4, Hkv=1, dqk=128, dv=128, causal=True, seed=1103)
+    _run_and_check(handle, lens_q, lens_k, Hq=4, Hkv=1, dqk=128, dv=128, causal=False, seed=1104)
+
+
+def test_more_queries_than_keys_causal(handle):
+    lens_q = [300, 64]
+    lens_k = [100, 200]
+    _run_and_check(handle, lens_q, lens_k, Hq=2, Hkv=2, dqk=64, dv=64, causal=True, seed=1105)
+
+
+def test_one_sequence_equals_fixed_length_call(handle):
+    """A batch of one sequence is the fixed-length problem in [S,H,d] layout: same bits as fa_forward."""
+    import torch
+    from paper_2609_21264_b200 import binding
+    S, Hq, Hkv, d = 391, 4, 2, 128
+    O, L = _run_and_check(handle, [S], [S], Hq=Hq, Hkv=Hkv, dqk=d, dv=d, causal=True, seed=1106)
+    q, k, v = _packed_inputs([S], [S], Hq, Hkv, d, d, 1106)
+    tq, tk, tv = (to_torch_bf16(np.ascontiguousarray(x.transpose(1, 0, 2))[None]) for x in (q, k, v))
+    o, lse = binding.forward(handle, tq, tk, tv, causal=True, scale=d ** -0.5)
+    torch.cuda.synchronize()
+    assert np.array_equal(bf16_tensor_to_f64(o)[0].transpose(1, 0, 2), O)
+    assert np.array_equal(lse.double().cpu().numpy()[0], L)
+
+
+def test_rows_past_max_sq_are_left_alone_and_empty_batch(handle):
+    import torch
+    from paper_2609_21264_b200 import binding
+    z = torch.zeros((8, 1, 64), dtype=torch.bfloat16, device="cuda")
+    cu = torch.tensor([0, 8], dtype=torch.int32, device="cuda")
+    args = (handle, z.data_ptr(), z.data_ptr(), z.data_ptr(), z.data_ptr(), None, cu.data_ptr(), cu.data_ptr())
+    assert binding.fa_forward_varlen(*args, 0, 0, 0, 0, 1, 1, 64, 64, False, 0.0) == binding.FA_OK
+    assert binding.fa_forward_varlen(*args, 1, 8, 8, 9, 1, 1, 64, 64, False, 0.0) == binding.FA_ERR_INVALID_ARG
+    assert binding.fa_forward_varlen(*args[:6], None, cu.data_ptr(), 1, 8, 8, 8, 1, 1, 64, 64, False, 0.0) \
+        == binding.FA_ERR_INVALID_ARG
+    torch.cuda.synchronize()
