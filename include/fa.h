@@ -62,6 +62,13 @@ typedef enum fa_status {
  * fa_last_status reports FA_ERR_DEVICE_TIMEOUT; the context stays usable.  Nothing faults,
  * traps or spins without bound.  Use with a short wait_limit_ms on a tiny problem. */
 #define FA_FLAG_DEBUG_DROP_V_LOAD 2u
+/* fa_config.flags: launch the kernels the ordinary way.  By default the pipelined kernel (and the
+ * split-KV combine kernel) are launched with programmatic stream serialisation: the GPU may
+ * schedule their CTAs while the kernel before them in the stream is still draining, and they
+ * wait on the device for that kernel's completion before they read or write global memory.
+ * Results and ordering guarantees are the same either way; the default saves the stream's
+ * completion-to-launch latency (a few microseconds per launch). */
+#define FA_FLAG_NO_DEPENDENT_LAUNCH 4u
 
 /* Optional creation parameters.  Zero-initialise, set struct_size = sizeof(fa_config). */
 typedef struct fa_config {

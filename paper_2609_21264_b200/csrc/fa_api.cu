@@ -144,7 +144,7 @@ fa_status launch_simple(fa_handle* h, int slot, const CUtensorMap& mq, const CUt
 
 template <int DQK, int DV, bool kVarlen>
 fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
-                           const CUtensorMap& mv, const fa::FwdParams& p, cudaStream_t st) {
+                           const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
     constexpr int smem = fa::pipe_smem_bytes<DQK, DV>();
     static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
     auto kernel = fa::fa_fwd_pipelined_kernel<DQK, DV, kVarlen>;
@@ -152,18 +152,31 @@ fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const 
     if (s != FA_OK) return s;
     const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq * p.B * p.kv_splits;
     if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
-    dim3 grid(static_cast<unsigned>(n_ctas), 1, 1);
-    kernel<<<grid, fa::PipeCfg<DQK, DV>::kThreads, smem, st>>>(mq, mk, mv, p);
-    if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
+    // Programmatic stream serialisation: the kernel may be scheduled while its predecessor in the
+    // stream drains (both kernels wait for that predecessor's completion before they touch global
+    // memory); without it every launch pays the full completion-to-launch latency of the stream.
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
+    cfg.blockDim = dim3(fa::PipeCfg<DQK, DV>::kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = (h->flags & FA_FLAG_NO_DEPENDENT_LAUNCH) ? 0 : 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mo, p) != cudaSuccess) return FA_ERR_CUDA;
     h->launches += 1;
     if (p.kv_splits > 1) {
         const long long n_rows = static_cast<long long>(p.B) * p.Hq * p.Sq;
         const long long blocks = (n_rows + 3) / 4;
         if (blocks > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
-        fa::fa_combine_kernel<DV><<<static_cast<unsigned>(blocks), 128, 0, st>>>(
-            p.o_part, p.lse_part, p.O, p.lse, n_rows, p.kv_splits, p.Hq, p.Sq,
-            p.o_stride_b, p.o_stride_h, p.o_stride_s);
-        if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
+        cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+        cfg.blockDim = dim3(128, 1, 1);
+        cfg.dynamicSmemBytes = 0;
+        if (cudaLaunchKernelEx(&cfg, fa::fa_combine_kernel<DV>, static_cast<const float*>(p.o_part),
+                               static_cast<const float*>(p.lse_part), p.O, p.lse, n_rows, p.kv_splits, p.Hq, p.Sq,
+                               p.o_stride_b, p.o_stride_h, p.o_stride_s) != cudaSuccess) return FA_ERR_CUDA;
         h->launches += 1;
     }
     return FA_OK;
@@ -218,7 +231,7 @@ fa_status check_args(const void* Q, const void* K, const void* V, const void* O,
 // cu_q == nullptr: fixed lengths Sq, Sk.  Otherwise a packed variable-length batch whose longest
 // query is Sq rows and whose sequences have about Sk keys (L2 grouping only).
 fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap& map_k, const CUtensorMap& map_v,
-                      void* O, float* lse, int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal,
+                      const CUtensorMap& map_o, void* O, float* lse, int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal,
                       float scale, const int64_t* o_strides, const int* cu_q, const int* cu_k, int total_q,
                       cudaStream_t st) {
     if (scale == 0.f) scale = 1.f / sqrtf(static_cast<float>(dqk));
@@ -276,13 +289,13 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
     if (!(h->flags & FA_FLAG_SERIAL_KERNEL)) {
         h->last_kernel = "fa_fwd_pipelined";
         if (cu_q) {
-            if (dqk == 64) return launch_pipelined<64, 64, true>(h, 6, map_q, map_k, map_v, p, st);
-            if (dqk == 128) return launch_pipelined<128, 128, true>(h, 7, map_q, map_k, map_v, p, st);
-            return launch_pipelined<192, 128, true>(h, 8, map_q, map_k, map_v, p, st);
+            if (dqk == 64) return launch_pipelined<64, 64, true>(h, 6, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_pipelined<128, 128, true>(h, 7, map_q, map_k, map_v, map_o, p, st);
+            return launch_pipelined<192, 128, true>(h, 8, map_q, map_k, map_v, map_o, p, st);
         }
-        if (dqk == 64) return launch_pipelined<64, 64, false>(h, 3, map_q, map_k, map_v, p, st);
-        if (dqk == 128) return launch_pipelined<128, 128, false>(h, 4, map_q, map_k, map_v, p, st);
-        return launch_pipelined<192, 128, false>(h, 5, map_q, map_k, map_v, p, st);
+        if (dqk == 64) return launch_pipelined<64, 64, false>(h, 3, map_q, map_k, map_v, map_o, p, st);
+        if (dqk == 128) return launch_pipelined<128, 128, false>(h, 4, map_q, map_k, map_v, map_o, p, st);
+        return launch_pipelined<192, 128, false>(h, 5, map_q, map_k, map_v, map_o, p, st);
     }
     h->last_kernel = "fa_fwd_simple";
     if (dqk == 64) return launch_simple<64, 64>(h, 0, map_q, map_k, map_v, p, st);
@@ -322,7 +335,7 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg) {
         limit_ms = cfg->wait_limit_ms;
         if (cfg->struct_size >= 20) kv_splits_cfg = cfg->kv_splits;
         if (cfg->struct_size >= sizeof(fa_config)) scratch_bytes = cfg->scratch_bytes;
-        if (flags & ~(FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD)) return FA_ERR_INVALID_ARG;
+        if (flags & ~(FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD | FA_FLAG_NO_DEPENDENT_LAUNCH)) return FA_ERR_INVALID_ARG;
         if (kv_splits_cfg > 64) return FA_ERR_INVALID_ARG;
     }
     if (scratch_bytes == 0) scratch_bytes = 32ull << 20;
@@ -429,15 +442,17 @@ fa_status fa_forward_strided(fa_handle* h, const void* Q, const void* K, const v
     DeviceGuard guard(h->device);
     if (!guard.ok()) return FA_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr;
+    const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;
     if ((s = get_map(h, Q, dqk, Sq, Hq, B, q_strides[0], q_strides[1], q_strides[2], fa::kTileM, &mq)) != FA_OK) return s;
     CUtensorMap map_q = *mq;   // copies: a later insertion may evict or move cache entries
     if ((s = get_map(h, K, dqk, Sk, Hkv, B, k_strides[0], k_strides[1], k_strides[2], fa::kTileN, &mk)) != FA_OK) return s;
     CUtensorMap map_k = *mk;
     if ((s = get_map(h, V, dv, Sk, Hkv, B, v_strides[0], v_strides[1], v_strides[2], fa::kTileN, &mv)) != FA_OK) return s;
     CUtensorMap map_v = *mv;
+    if ((s = get_map(h, O, dv, Sq, Hq, B, o_strides[0], o_strides[1], o_strides[2], fa::kTileM, &mo)) != FA_OK) return s;
+    CUtensorMap map_o = *mo;
 
-    return run_forward(h, map_q, map_k, map_v, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, o_strides,
+    return run_forward(h, map_q, map_k, map_v, map_o, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, o_strides,
                        nullptr, nullptr, 0, st);
 }
 
@@ -467,7 +482,7 @@ fa_status fa_forward_varlen(fa_handle* h, const void* Q, const void* K, const vo
     if (!guard.ok()) return FA_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // packed [total, H, d]: one batch slice, rows H*d apart, heads d apart
-    const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr;
+    const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;
     const int rows_k = total_k > 0 ? total_k : 1;   // an empty K/V still gets a valid map; no tile of it is ever read
     if ((s = get_map(h, Q, dqk, total_q, Hq, 1, static_cast<long long>(total_q) * Hq * dqk, dqk,
                      static_cast<long long>(Hq) * dqk, fa::kTileM, &mq)) != FA_OK) return s;
@@ -478,9 +493,12 @@ fa_status fa_forward_varlen(fa_handle* h, const void* Q, const void* K, const vo
     if ((s = get_map(h, V, dv, rows_k, Hkv, 1, static_cast<long long>(rows_k) * Hkv * dv, dv,
                      static_cast<long long>(Hkv) * dv, fa::kTileN, &mv)) != FA_OK) return s;
     CUtensorMap map_v = *mv;
+    if ((s = get_map(h, O, dv, total_q, Hq, 1, static_cast<long long>(total_q) * Hq * dv, dv,
+                     static_cast<long long>(Hq) * dv, fa::kTileM, &mo)) != FA_OK) return s;
+    CUtensorMap map_o = *mo;
     const int64_t os[3] = {0, dv, static_cast<int64_t>(Hq) * dv};
     const int mean_sk = (total_k + B - 1) / B > 0 ? (total_k + B - 1) / B : 1;
-    return run_forward(h, map_q, map_k, map_v, O, lse, B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal, scale, os,
+    return run_forward(h, map_q, map_k, map_v, map_o, O, lse, B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal, scale, os,
                        cu_seqlens_q, cu_seqlens_k, total_q, st);
 }
 

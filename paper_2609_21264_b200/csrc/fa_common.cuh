@@ -20,7 +20,7 @@ enum WaitSite : uint32_t {
     kSiteMmaOReady = 0x0304, kSiteMmaSFree = 0x0305, kSiteMmaTurn = 0x0306,
     kSiteSoftmaxSFull = 0x0401, kSiteSoftmaxPFree = 0x0402, kSiteSoftmaxCorrFree = 0x0403,
     kSiteCorrScale = 0x0501, kSiteCorrPvDone = 0x0502, kSiteCorrFinal = 0x0503,
-    kSiteEpiOFull = 0x0601,
+    kSiteEpiOFull = 0x0601, kSiteEpiStaged = 0x0602,
     kSiteSmemAlign = 0x0701,
 };
 
@@ -53,6 +53,8 @@ struct FwdParams {
 
 #ifdef FA_TRACE
 constexpr int kTraceIters = 64, kTraceEvents = 16, kTraceRoles = 6;   // roles: softmax0, softmax1, mma, corr
+#endif
+#if defined(FA_TRACE) && !defined(FA_TRACE_CTA_ONLY)
 #define FA_TRACE_STAMP(role, iter, ev)                                                          \
     do {                                                                                        \
         if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (iter) < kTraceIters) \

@@ -67,6 +67,7 @@ struct PipeShared {
     uint64_t scale_full[2];  // softmax -> correction: alpha of iteration j published
     uint64_t o_final[2];     // MMA -> softmax: last PV of tile t done, O_t is final
     uint64_t turn[2];        // MMA thread 1-t -> MMA thread t: your turn to issue
+    uint64_t o_staged[2];    // softmax warps -> storing thread: the bf16 O_t tile is in shared memory
     float alpha[2][2][kTileM];   // [tile][j & 1][row]
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -84,6 +85,7 @@ __global__ void __launch_bounds__(512, 1)
 fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                         const __grid_constant__ CUtensorMap tm_k,
                         const __grid_constant__ CUtensorMap tm_v,
+                        const __grid_constant__ CUtensorMap tm_o,
                         const FwdParams p) {
     using Cfg = PipeCfg<DQK, DV>;
     using namespace ptx;
@@ -99,8 +101,15 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int warp = tid >> 5;
     const int lane = tid & 31;
 
+    // The launch after this one may be scheduled while this grid drains; the inputs of this
+    // launch are not touched before the launch before it has completed.  Packed batches read their
+    // offsets right away, so they wait here; otherwise the wait comes after the CTA's set-up.
+    grid_launch_dependents();
+    if constexpr (kVarlen) grid_dependency_wait();
+
     const uint32_t smem_base = smem_addr(smem_raw);
     if ((smem_base & 1023u) != 0u) {          // uniform over the CTA; nothing has been set up yet
+        if constexpr (!kVarlen) grid_dependency_wait();
         if (tid == 0 && p.status) {
             volatile uint32_t* sw = p.status;
             sw[1] = kSiteSmemAlign;
@@ -171,6 +180,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             mbar_init(smem_addr(&sh.scale_full[t]), 4);
             mbar_init(smem_addr(&sh.o_final[t]), 1);
             mbar_init(smem_addr(&sh.turn[t]), 1);
+            mbar_init(smem_addr(&sh.o_staged[t]), 4);     // 4 softmax warps
         }
 #pragma unroll
         for (int s = 0; s < 4; ++s) {
@@ -189,10 +199,12 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         prefetch_tensormap(&tm_q);
         prefetch_tensormap(&tm_k);
         prefetch_tensormap(&tm_v);
+        prefetch_tensormap(&tm_o);
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    if constexpr (!kVarlen) grid_dependency_wait();
 
     const uint32_t tmem_base = sh.tmem_base;
     WaitCtx wctx{&sh.abort_flag, p.status, p.wait_limit_ns};
@@ -375,21 +387,60 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                         (l > 0.f) ? (m_ref * c * 0.6931471805599453f + logf(l)) : -INFINITY;
                 }
                 const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1) + lane_sel;
+                // A packed batch's last tile of a sequence is followed by the next sequence's rows,
+                // which a box store would overwrite: such tiles take the row-by-row path.
+                const bool box_store = !kVarlen || (i0_t + kTileM <= Sq);
+                if (box_store) {
+                    // The tile goes through shared memory (the Q tile's space: its last reader, the
+                    // final score MMA, is complete once o_final has fired) in the swizzled layout of
+                    // a TMA box, and one thread stores it; rows past Sq are clipped by the TMA unit.
+                    // Row-by-row global stores from 128 threads cost one LSU pass per 16 bytes.
+                    const uint32_t sO = sQ + t * Cfg::kQBytes + row * 128;
 #pragma unroll 1
-                for (int cc = 0; cc < DV / 32; ++cc) {
-                    uint32_t r[32];
-                    tmem_ld_x32(tO + cc * 32, r);
-                    tc_wait_ld();
-                    if (i_glob < Sq) {
-                        uint32_t pk[16];
+                    for (int cc = 0; cc < DV / 32; ++cc) {
+                        uint32_t r[32];
+                        tmem_ld_x32(tO + cc * 32, r);
+                        tc_wait_ld();
+                        const uint32_t chunk = sO + (cc >> 1) * kChunkBytes;
 #pragma unroll
-                        for (int e = 0; e < 32; e += 2)
-                            pk[e / 2] = pack_bf16x2(__uint_as_float(r[e]) * inv_l,
-                                                    __uint_as_float(r[e + 1]) * inv_l);
+                        for (int v = 0; v < 4; ++v) {
+                            const uint32_t piece = static_cast<uint32_t>(((cc & 1) * 4 + v) ^ (row & 7)) << 4;
+                            st_shared_v4(chunk + piece,
+                                         pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
+                                         pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
+                                         pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
+                                         pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_addr(&sh.o_staged[t]));
+                    if ((warp & 3) == 0 && lane == 0 &&
+                        mbar_wait(smem_addr(&sh.o_staged[t]), 0, wctx, kSiteEpiStaged)) {
 #pragma unroll
-                        for (int v = 0; v < 4; ++v)
-                            reinterpret_cast<uint4*>(o_row + cc * 32)[v] =
-                                make_uint4(pk[4 * v], pk[4 * v + 1], pk[4 * v + 2], pk[4 * v + 3]);
+                        for (int ch = 0; ch < DV / kChunkCols; ++ch)
+                            tma_store_4d(&tm_o, sQ + t * Cfg::kQBytes + ch * kChunkBytes, ch * kChunkCols,
+                                         q_row0 + i0_t, hq, kVarlen ? 0 : b);
+                        tma_store_commit();
+                        tma_store_wait_read_all();     // the CTA's shared memory outlives the reads
+                    }
+                } else {
+#pragma unroll 1
+                    for (int cc = 0; cc < DV / 32; ++cc) {
+                        uint32_t r[32];
+                        tmem_ld_x32(tO + cc * 32, r);
+                        tc_wait_ld();
+                        if (i_glob < Sq) {
+                            uint32_t pk[16];
+#pragma unroll
+                            for (int e = 0; e < 32; e += 2)
+                                pk[e / 2] = pack_bf16x2(__uint_as_float(r[e]) * inv_l,
+                                                        __uint_as_float(r[e + 1]) * inv_l);
+#pragma unroll
+                            for (int v = 0; v < 4; ++v)
+                                reinterpret_cast<uint4*>(o_row + cc * 32)[v] =
+                                    make_uint4(pk[4 * v], pk[4 * v + 1], pk[4 * v + 2], pk[4 * v + 3]);
+                        }
                     }
                 }
             }
@@ -607,6 +658,8 @@ fa_combine_kernel(const float* __restrict__ o_part, const float* __restrict__ ls
                   __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
                   long long n_rows, int n_splits, int Hq, int Sq,
                   long long o_stride_b, long long o_stride_h, long long o_stride_s) {
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();          // the partials come from the kernel before this one
     const long long row = static_cast<long long>(blockIdx.x) * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= n_rows) return;

@@ -100,12 +100,13 @@ bool encode_map(EncodeTiledFn encode, CUtensorMap* map, const void* ptr, int d, 
 }
 
 template <int DQK, int DV>
-fa_status launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const fa::FwdParams& p,
+fa_status launch(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mo,
+                 const fa::FwdParams& p,
                  cudaStream_t st) {
     const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq * p.B * p.kv_splits;
     if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     fa::fa_fwd_pipelined_kernel<DQK, DV><<<static_cast<unsigned>(n_ctas), fa::PipeCfg<DQK, DV>::kThreads,
-                                           fa::pipe_smem_bytes<DQK, DV>(), st>>>(mq, mk, mv, p);
+                                           fa::pipe_smem_bytes<DQK, DV>(), st>>>(mq, mk, mv, mo, p);
     if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
     const long long n_rows = static_cast<long long>(p.B) * p.Hq * p.Sq;
     fa::fa_combine_kernel<DV><<<static_cast<unsigned>((n_rows + 3) / 4), 128, 0, st>>>(
@@ -156,10 +157,11 @@ fa_status fa_forward_split_noalloc(const void* Q, const void* K, const void* V, 
     const unsigned long long need = static_cast<unsigned long long>(splits) * rows * (dv + 1) * 4ull;
     if (need > kStaticScratchBytes) return FA_ERR_UNSUPPORTED;     // partials exceed the fixed scratch
 
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq, mk, mv, mo;
     if (!encode_map(dev.encode, &mq, Q, dqk, Sq, Hq, B) ||
         !encode_map(dev.encode, &mk, K, dqk, Sk, Hkv, B) ||
-        !encode_map(dev.encode, &mv, V, dv, Sk, Hkv, B))
+        !encode_map(dev.encode, &mv, V, dv, Sk, Hkv, B) ||
+        !encode_map(dev.encode, &mo, O, dv, Sq, Hq, B))
         return FA_ERR_CUDA;
 
     fa::FwdParams p;
@@ -187,9 +189,9 @@ fa_status fa_forward_split_noalloc(const void* Q, const void* K, const void* V, 
     p.lse_part = p.o_part + static_cast<size_t>(splits) * rows * dv;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (dqk == 64) return launch<64, 64>(mq, mk, mv, p, st);
-    if (dqk == 128) return launch<128, 128>(mq, mk, mv, p, st);
-    return launch<192, 128>(mq, mk, mv, p, st);
+    if (dqk == 64) return launch<64, 64>(mq, mk, mv, mo, p, st);
+    if (dqk == 128) return launch<128, 128>(mq, mk, mv, mo, p, st);
+    return launch<192, 128>(mq, mk, mv, mo, p, st);
 }
 
 }  // extern "C"

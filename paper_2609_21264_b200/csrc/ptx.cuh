@@ -135,6 +135,18 @@ FA_DEVI bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& ctx, uint32
     }
 }
 
+// ------------------------------------------------------------------ programmatic dependent launch
+
+// Lets the next kernel of the stream (if it was launched with programmatic stream serialisation)
+// be scheduled as soon as every CTA of this grid has got here or has exited.
+FA_DEVI void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// Blocks until the preceding kernel of the stream has completed and its writes are visible.  A
+// no-op for a kernel that was launched the ordinary way.  Must come before the first access to
+// global memory that an earlier kernel may have written, and every CTA must pass it before it
+// exits (a grid whose CTAs skipped it could finish before its predecessor, and its own successor,
+// which waits for this grid only, would then overtake that predecessor).
+FA_DEVI void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ------------------------------------------------------------------ TMA
 
 FA_DEVI void prefetch_tensormap(const CUtensorMap* map) {
@@ -170,6 +182,17 @@ FA_DEVI void tma_store_3d(const CUtensorMap* map, uint32_t src_smem, int c0, int
         "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
         ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src_smem), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
+}
+// 4-D tiled store shared -> global (coordinates: column, row, head, batch); rows and columns of
+// the box that fall outside the tensor are not written.
+FA_DEVI void tma_store_4d(const CUtensorMap* map, uint32_t src_smem, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src_smem), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+FA_DEVI void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 FA_DEVI void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 FA_DEVI void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
