@@ -22,6 +22,7 @@ enum WaitSite : uint32_t {
     kSiteCorrScale = 0x0501, kSiteCorrPvDone = 0x0502, kSiteCorrFinal = 0x0503,
     kSiteEpiOFull = 0x0601, kSiteEpiStaged = 0x0602,
     kSiteSmemAlign = 0x0701,
+    kSiteItem = 0x0801,
 };
 
 struct FwdParams {
@@ -44,6 +45,7 @@ struct FwdParams {
     float* o_part;            // [C, B*Hq, Sq, dv] fp32 partial outputs (split-KV only)
     float* lse_part;          // [C, B*Hq, Sq] fp32 partial log-sum-exps (split-KV only)
     int debug_drop_v_load;    // test hook: the load warp skips the first V tile (exercises the wait limit)
+    unsigned int* sched_counter;   // persistent kernel: ticket counter of the work-item list (zero between launches)
     uint32_t* status;         // [0] = fa_status, [1] = wait site; mapped host memory
     unsigned long long wait_limit_ns;
 #ifdef FA_TRACE

@@ -171,6 +171,7 @@ fa_status fa_forward_split_noalloc(const void* Q, const void* K, const void* V, 
     p.o_stride_h = static_cast<long long>(Sq) * dv;
     p.o_stride_s = dv;
     p.cu_q = nullptr;
+    p.sched_counter = nullptr;
     p.cu_k = nullptr;
     p.total_q = 0;
     p.lse = lse;
