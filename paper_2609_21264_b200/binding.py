@@ -26,7 +26,7 @@ FA_FLAG_NO_DEPENDENT_LAUNCH = 4
 FA_FLAG_NO_PERSISTENT = 8
 FA_FLAG_FORCE_PERSISTENT = 16
 
-EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_varlen", "fa_forward_host", "fa_last_status", "fa_destroy",
+EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_varlen", "fa_forward_fp8", "fa_forward_host", "fa_last_status", "fa_destroy",
            "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits",
            "fa_forward_split_noalloc", "fa_noalloc_scratch_bytes")
 
@@ -70,6 +70,8 @@ def load():
     lib.fa_forward_host.argtypes = fwd_args
     lib.fa_forward_varlen.restype = i32
     lib.fa_forward_varlen.argtypes = [vp] * 8 + [i32] * 8 + [i32, ctypes.c_float, vp]
+    lib.fa_forward_fp8.restype = i32
+    lib.fa_forward_fp8.argtypes = [vp] * 9 + [i32] * 7 + [f32, vp]
     lib.fa_forward_strided.restype = i32
     lib.fa_forward_strided.argtypes = fwd_args[:-1] + [vp, vp, vp, vp, vp]
     lib.fa_last_status.restype = i32
@@ -126,6 +128,12 @@ def fa_forward_varlen(h, Q, K, V, O, lse, cu_seqlens_q, cu_seqlens_k, B, total_q
     """Raw call on packed [total, H, d] device tensors with device int32 offsets; returns the status code."""
     return load().fa_forward_varlen(h, Q, K, V, O, lse, cu_seqlens_q, cu_seqlens_k, B, total_q, total_k, max_sq,
                                     Hq, Hkv, dqk, dv, int(bool(causal)), float(scale), stream)
+
+
+def fa_forward_fp8(h, Q8, K8, V8, q_scale, k_scale, v_scale, O, lse, B, Hq, Hkv, Sq, Sk, d, causal, scale, stream=0) -> int:
+    """Raw call: e4m3 device tensors with block scales (device fp32 arrays or None); returns the status code."""
+    return load().fa_forward_fp8(h, Q8, K8, V8, q_scale, k_scale, v_scale, O, lse, B, Hq, Hkv, Sq, Sk, d,
+                                 int(bool(causal)), float(scale), stream)
 
 
 def fa_forward_host(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, stream=0) -> int:
@@ -234,4 +242,28 @@ def forward_varlen(h, q, k, v, cu_seqlens_q, cu_seqlens_k, max_sq: int, *, causa
                            Hq, Hkv, dqk, dv, causal, scale, torch.cuda.current_stream(q.device).cuda_stream)
     if st != FA_OK:
         raise FaError(st, "fa_forward_varlen")
+    return out, lse
+
+
+def forward_fp8(h, q8, k8, v8, q_scale, k_scale, v_scale, *, causal: bool, scale: float = 0.0, want_lse=True):
+    """Block-scaled e4m3 attention on torch CUDA tensors: q8/k8/v8 uint8 (or float8_e4m3fn) [B,H,S,128],
+    scales fp32 CUDA tensors or None.  Returns (O bf16 [B,Hq,Sq,128], lse fp32 [B,Hq,Sq])."""
+    import torch
+    for t in (q8, k8, v8):
+        if t.element_size() != 1 or not t.is_cuda or not t.is_contiguous() or t.dim() != 4:
+            raise ValueError("q8, k8, v8 must be contiguous 4-D one-byte CUDA tensors")
+    B, Hq, Sq, d = q8.shape
+    _, Hkv, Sk, _ = k8.shape
+    n_qt, n_kt = (Sq + 127) // 128, (Sk + 127) // 128
+    for t, shape in ((q_scale, (B, Hq, n_qt)), (k_scale, (B, Hkv, n_kt)), (v_scale, (B, Hkv))):
+        if t is not None and (t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != shape):
+            raise ValueError("scale tensors must be contiguous fp32 CUDA tensors of shape %s" % (shape,))
+    out = torch.empty((B, Hq, Sq, d), dtype=torch.bfloat16, device=q8.device)
+    lse = torch.empty((B, Hq, Sq), dtype=torch.float32, device=q8.device) if want_lse else None
+    ptr = lambda t: t.data_ptr() if t is not None else None
+    st = fa_forward_fp8(h, q8.data_ptr(), k8.data_ptr(), v8.data_ptr(), ptr(q_scale), ptr(k_scale), ptr(v_scale),
+                        out.data_ptr(), ptr(lse), B, Hq, Hkv, Sq, Sk, d, causal, scale,
+                        torch.cuda.current_stream(q8.device).cuda_stream)
+    if st != FA_OK:
+        raise FaError(st, "fa_forward_fp8")
     return out, lse

