@@ -55,8 +55,6 @@ struct FwdParams {
 
 #ifdef FA_TRACE
 constexpr int kTraceIters = 64, kTraceEvents = 16, kTraceRoles = 6;   // roles: softmax0, softmax1, mma, corr
-#endif
-#if defined(FA_TRACE) && !defined(FA_TRACE_CTA_ONLY)
 #define FA_TRACE_STAMP(role, iter, ev)                                                          \
     do {                                                                                        \
         if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (iter) < kTraceIters) \
