@@ -51,10 +51,11 @@ def load_peaks():
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.005):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.max_mhz = [], None          # (time, MHz, set of reasons)
+        self.window = [None, None]                     # timed region, marked by the caller
         self._halt = threading.Event()
         self.error = None
 
@@ -73,21 +74,35 @@ class ClockSampler(threading.Thread):
             get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
                 getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
             while not self._halt.is_set():
-                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                mhz = nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
                 mask = get_reasons(h)
-                for bit, name in names.items():
-                    if bit and (mask & bit):
-                        self.reasons.add(name)
+                self.samples.append((time.perf_counter(), mhz,
+                                     {name for bit, name in names.items() if bit and (mask & bit)}))
                 time.sleep(self.period)
         except Exception as ex:  # pragma: no cover
             self.error = repr(ex)
 
+    def wait_ready(self, timeout_s: float = 3.0):
+        t_end = time.perf_counter() + timeout_s
+        while not self.samples and self.error is None and time.perf_counter() < t_end:
+            time.sleep(0.002)
+
+    def mark(self, which: int):
+        self.window[which] = time.perf_counter()
+
     def stop(self):
         self._halt.set()
         self.join(timeout=2.0)
-        s = sorted(self.samples)
-        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(s),
+        t0, t1 = self.window
+        inside = [x for x in self.samples if t0 is not None and t1 is not None and t0 <= x[0] <= t1]
+        note = "samples taken inside the timed region"
+        if not inside:      # region shorter than one sampling period: the warm-up ran the same launches just before
+            inside = [x for x in self.samples if t1 is None or x[0] <= t1][-3:]
+            note = "timed region shorter than the sampling period: last samples of the warm-up (same launches)"
+        mhz = sorted(x[1] for x in inside)
+        reasons = set().union(*[x[2] for x in inside]) if inside else set()
+        return {"sm_mhz": (mhz[len(mhz) // 2] if mhz else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(reasons), "samples": len(mhz), "window": note,
                 **({"error": self.error} if self.error else {})}
 
 
@@ -132,7 +147,7 @@ def n_sets_for(w):
     return max(2, min(16, -(-2 * L2_BYTES // nbytes))) if nbytes < 2 * L2_BYTES else 1
 
 
-def run_device_timed(binding, h, w, sets, steps, warmup, world):
+def run_device_timed(binding, h, w, sets, steps, warmup, world, sampler=None):
     """Time `steps` launches (after `warmup`) with CUDA events on the launching stream; seconds."""
     import torch
     stream = torch.cuda.current_stream()
@@ -151,11 +166,15 @@ def run_device_timed(binding, h, w, sets, steps, warmup, world):
     launch.barrier(world)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     n0 = binding.fa_launch_count(h)
+    if sampler is not None:
+        sampler.mark(0)
     e0.record(stream)
     for i in range(steps):
         one(warmup + i)
     e1.record(stream)
     torch.cuda.synchronize()
+    if sampler is not None:
+        sampler.mark(1)
     launch.barrier(world)
     st, detail = binding.fa_last_status(h)
     if st != binding.FA_OK:
@@ -341,13 +360,13 @@ def main():
     warmup = args.warmup if args.warmup is not None else max(3, min(50, steps // 10))
     warmup = max(3, warmup)
 
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
     h = binding.fa_create(device=local)
     n_sets = n_sets_for(w)
     sets = make_device_sets(w, n_sets, device)
-
-    sampler = ClockSampler(physical_gpu_index(local))
-    sampler.start()
-    seconds, launches = run_device_timed(binding, h, w, sets, steps, warmup, world)
+    sampler.wait_ready()
+    seconds, launches = run_device_timed(binding, h, w, sets, steps, warmup, world, sampler)
     clocks = sampler.stop()
     seconds = launch.max_over_ranks(seconds, world, device)
     t_step = seconds / steps
@@ -381,6 +400,37 @@ def main():
             "value_paper_convention": world * fl_pap / t_step / 1e12,
             "paper_context": "3.62 TFLOP_GEMM/s on XDNA 2 (paper's headline, other hardware and shape)",
             "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches)}
+
+    if not args.no_sweep and world == 1 and w.dqk == 128 and w.dv == 128:
+        # the block-scaled e4m3 variant on the same shape (N(0, sigma^2) rounded to e4m3, unit scales), for context
+        gen = torch.Generator(device=device).manual_seed(w.seed)
+        q8, k8, v8 = (torch.randn(shape, generator=gen, device=device).mul_(w.sigma).to(torch.float8_e4m3fn).view(torch.uint8)
+                      for shape in w.shapes()[:3])
+        o8 = torch.empty((w.B, w.Hq, w.Sq, 128), dtype=torch.bfloat16, device=device)
+        l8 = torch.empty((w.B, w.Hq, w.Sq), dtype=torch.float32, device=device)
+        k = max(5, min(200, int(0.3 / max(fl_alg / 1.0e15, 1e-5))))
+        cs = torch.cuda.current_stream().cuda_stream
+
+        def one8():
+            st8 = binding.fa_forward_fp8(h, q8.data_ptr(), k8.data_ptr(), v8.data_ptr(), None, None, None, o8.data_ptr(),
+                                         l8.data_ptr(), w.B, w.Hq, w.Hkv, w.Sq, w.Sk, 128, w.causal, w.scale, cs)
+            if st8 != binding.FA_OK:
+                raise binding.FaError(st8, "fa_forward_fp8")
+
+        for _ in range(3):
+            one8()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(k):
+            one8()
+        e1.record()
+        torch.cuda.synchronize()
+        t8 = e0.elapsed_time(e1) * 1e-3 / k
+        line["block_scaled_e4m3"] = {"workload": w.name, "us": t8 * 1e6, "tflops_algorithmic": fl_alg / t8 / 1e12,
+                                     "speedup_over_bf16": t_step / t8, "steps": k,
+                                     "note": "fa_forward_fp8, N(0,sigma^2) rounded to e4m3, unit scales, one input set"}
+        del q8, k8, v8, o8, l8
 
     if not args.no_e2e:
         e2e_steps = max(3, min(steps, 50))

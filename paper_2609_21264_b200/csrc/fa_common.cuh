@@ -55,6 +55,10 @@ struct FwdParams {
 
 #ifdef FA_TRACE
 constexpr int kTraceIters = 64, kTraceEvents = 16, kTraceRoles = 6;   // roles: softmax0, softmax1, mma, corr
+#endif
+// -DFA_TRACE alone records one (SM, start, end, rounds) entry per CTA; -DFA_TRACE_STAMPS adds the
+// per-iteration clock stamps of CTA 0 (they cost a few hundred cycles each and slow the loop).
+#if defined(FA_TRACE) && defined(FA_TRACE_STAMPS)
 #define FA_TRACE_STAMP(role, iter, ev)                                                          \
     do {                                                                                        \
         if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (iter) < kTraceIters) \

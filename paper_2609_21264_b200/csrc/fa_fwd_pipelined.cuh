@@ -118,6 +118,14 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         }
         return;
     }
+#ifdef FA_TRACE
+    if (tid == 0 && p.trace) {      // per-CTA record: SM id, start, end, rounds (after the role stamps)
+        unsigned long long g; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g));
+        unsigned smid; asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+        long long* rec = p.trace + kTraceRoles * kTraceIters * kTraceEvents + 4ll * blockIdx.x;
+        rec[0] = smid; rec[1] = static_cast<long long>(g);
+    }
+#endif
     const uint32_t sQ = smem_base;                               // two tiles
     const uint32_t sK = sQ + 2 * Cfg::kQBytes;                   // NK stages
     const uint32_t sV = sK + NK * Cfg::kKBytes;                  // NV stages
@@ -645,6 +653,13 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 12) tmem_dealloc(tmem_base, Cfg::kTmemCols);
+#ifdef FA_TRACE
+    if (warp == 12 && lane == 0 && p.trace) {
+        unsigned long long g; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g));
+        long long* rec = p.trace + kTraceRoles * kTraceIters * kTraceEvents + 4ll * blockIdx.x;
+        rec[2] = static_cast<long long>(g); rec[3] = n_max;
+    }
+#endif
 }
 
 
