@@ -76,6 +76,14 @@ typedef enum fa_status {
  * sizes 64 and 128, no split-KV, not a packed batch); results agree to rounding order. */
 #define FA_FLAG_NO_PERSISTENT 8u
 #define FA_FLAG_FORCE_PERSISTENT 16u
+/* A third tiling: one query tile per CTA with its K/V tiles streamed through both softmax
+ * warpgroups (csrc/fa_fwd_stream.cuh).  It doubles the number of CTAs and shortens each one's
+ * dependency chain, which wins when the pair tiling leaves SMs idle or its longest CTA dominates
+ * (under about one wave of pairs: short sequences, few heads); the library estimates both and
+ * picks it with a 10 % margin, also instead of splitting the K/V range.  These flags force it on
+ * (fixed-length problems, head sizes 64 and 128) or off. */
+#define FA_FLAG_STREAM_KERNEL 32u
+#define FA_FLAG_NO_STREAM_KERNEL 64u
 
 /* Optional creation parameters.  Zero-initialise, set struct_size = sizeof(fa_config). */
 typedef struct fa_config {

@@ -25,6 +25,8 @@ FA_FLAG_DEBUG_DROP_V_LOAD = 2
 FA_FLAG_NO_DEPENDENT_LAUNCH = 4
 FA_FLAG_NO_PERSISTENT = 8
 FA_FLAG_FORCE_PERSISTENT = 16
+FA_FLAG_STREAM_KERNEL = 32
+FA_FLAG_NO_STREAM_KERNEL = 64
 
 EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_varlen", "fa_forward_fp8", "fa_forward_host", "fa_last_status", "fa_destroy",
            "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits",

@@ -14,6 +14,7 @@
 #include "fa_common.cuh"
 #include "fa_fwd_pipelined.cuh"
 #include "fa_fwd_persistent.cuh"
+#include "fa_fwd_stream.cuh"
 #include "fa_fwd_fp8.cuh"
 #include "fa_fwd_simple.cuh"
 
@@ -55,7 +56,7 @@ struct fa_handle {
     const char* last_kernel = "";
     void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // Q K V O lse
     size_t stage_cap[5] = {0, 0, 0, 0, 0};
-    bool attr_done[12] = {};
+    bool attr_done[24] = {};
 #ifdef FA_TRACE
     long long* trace = nullptr;
 #endif
@@ -276,6 +277,71 @@ fa_status launch_persistent(fa_handle* h, int slot, const CUtensorMap& mq, const
     return FA_OK;
 }
 
+// One query tile per CTA, K/V tiles streamed through two softmax warpgroups.
+template <int DQK, int DV>
+fa_status launch_stream(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
+                        const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
+    constexpr int smem = fa::stream_smem_bytes<DQK, DV>();
+    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+    auto kernel = fa::fa_fwd_stream_kernel<DQK, DV>;
+    fa_status s = ensure_smem_attr(h, slot, kernel, smem);
+    if (s != FA_OK) return s;
+    const long long n_ctas = static_cast<long long>(p.n_q_tiles) * p.Hq * p.B;
+    if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
+    cfg.blockDim = dim3(512, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = (h->flags & FA_FLAG_NO_DEPENDENT_LAUNCH) ? 0 : 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mo, p) != cudaSuccess) return FA_ERR_CUDA;
+    h->launches += 1;
+    return FA_OK;
+}
+
+// Estimated run times (microseconds) of a launch under the two tilings, from the measured cost of
+// a CTA: pair kernel a_p * rounds + f_p with rounds = K/V tiles of the pair's second query tile
+// (split-KV: rounds / C, plus the combine kernel); stream kernel a_s * (K/V tiles of the query tile)
+// + f_s.  Longest-first scheduling over the SMs is approximated by max(longest item, total / SMs),
+// and by whole waves when all items are equal.  Good to some 20 % on the shapes it was checked
+// on, which is enough to tell a grid of under one wave (the stream kernel's case) from the rest.
+struct TilingEstimate { double pair_us, stream_us; };
+TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int dqk, int causal, int n_q_tiles, int splits) {
+    const double a_p = dqk == 64 ? 1.36 : 2.0, f_p = dqk == 64 ? 6.0 : 6.7;
+    const double a_s = dqk == 64 ? 0.75 : 1.0, f_s = 5.0;
+    const double heads = static_cast<double>(B) * Hq;
+    double pair_total = 0, pair_max = 0, stream_total = 0, stream_max = 0;
+    for (int t = 0; t < n_q_tiles; ++t) {
+        const int r = fa::kv_tiles_for_q_tile(t * fa::kTileM, fa::kTileM, Sq, Sk, causal);
+        const double cs = a_s * r + f_s;
+        stream_total += cs;
+        if (cs > stream_max) stream_max = cs;
+        if ((t & 1) == 1 || t == n_q_tiles - 1) {        // second tile of a pair, or an unpaired last tile
+            const double rounds = (r + splits - 1) / splits;
+            const double cp = a_p * rounds + f_p;
+            pair_total += cp * splits;
+            if (cp > pair_max) pair_max = cp;
+        }
+    }
+    auto makespan = [&](double total_per_head, double longest, double n_items_per_head) {
+        const double n_items = n_items_per_head * heads;
+        if (!causal && Sq >= fa::kTileM) {                // equal items: whole waves
+            const double waves = static_cast<double>((static_cast<long long>(n_items) + num_sms - 1) / num_sms);
+            return waves * longest;
+        }
+        const double balanced = total_per_head * heads / num_sms;
+        return balanced > longest ? balanced : longest;
+    };
+    TilingEstimate e;
+    e.pair_us = makespan(pair_total, pair_max, static_cast<double>((n_q_tiles + 1) / 2) * splits) + (splits > 1 ? 6.0 : 0.0);
+    e.stream_us = makespan(stream_total, stream_max, n_q_tiles);
+    return e;
+}
+
 // Fills the launch parameters and starts the kernel(s); the tensor maps are ready.
 // cu_q == nullptr: fixed lengths Sq, Sk.  Otherwise a packed variable-length batch whose longest
 // query is Sq rows and whose sequences have about Sk keys (L2 grouping only).
@@ -338,6 +404,28 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
         if (h->flags & FA_FLAG_NO_PERSISTENT) persistent = false;
         if ((h->flags & FA_FLAG_FORCE_PERSISTENT) && !cu_q && p.kv_splits == 1 && dqk != 192 && !p.debug_drop_v_load)
             persistent = true;
+        // One query tile per CTA (twice the CTAs, each with a shorter chain) wins where the pair
+        // kernel's grid does not fill the GPU or its longest CTA dominates: decided from the two
+        // estimates, with a margin, before the K/V range is split.
+        bool stream = false;
+        if (!cu_q && dqk != 192 && !p.debug_drop_v_load && !(h->flags & FA_FLAG_NO_STREAM_KERNEL)) {
+            if (h->flags & FA_FLAG_STREAM_KERNEL) {
+                stream = true;
+            } else if (!persistent && h->kv_splits_cfg <= 1) {
+                const TilingEstimate e = estimate_tilings(h->num_sms, B, Hq, Sq, Sk, dqk, p.causal, p.n_q_tiles, p.kv_splits);
+                stream = e.stream_us < 0.9 * e.pair_us;
+            }
+        }
+        if (stream) {
+            p.kv_splits = 1;
+            p.tiles_per_split = 0x3fffffff;
+            p.o_part = nullptr;
+            p.lse_part = nullptr;
+            h->last_splits = 1;
+            h->last_kernel = "fa_fwd_stream";
+            if (dqk == 64) return launch_stream<64, 64>(h, 16, map_q, map_k, map_v, map_o, p, st);
+            return launch_stream<128, 128>(h, 17, map_q, map_k, map_v, map_o, p, st);
+        }
         if (persistent) {
             h->last_kernel = "fa_fwd_persistent";
             if (dqk == 64) return launch_persistent<64, 64>(h, 9, map_q, map_k, map_v, map_o, p, st);
@@ -392,7 +480,8 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg) {
         if (cfg->struct_size >= 20) kv_splits_cfg = cfg->kv_splits;
         if (cfg->struct_size >= sizeof(fa_config)) scratch_bytes = cfg->scratch_bytes;
         if (flags & ~(FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD | FA_FLAG_NO_DEPENDENT_LAUNCH |
-                      FA_FLAG_NO_PERSISTENT | FA_FLAG_FORCE_PERSISTENT)) return FA_ERR_INVALID_ARG;
+                      FA_FLAG_NO_PERSISTENT | FA_FLAG_FORCE_PERSISTENT | FA_FLAG_STREAM_KERNEL |
+                      FA_FLAG_NO_STREAM_KERNEL)) return FA_ERR_INVALID_ARG;
         if (kv_splits_cfg > 64) return FA_ERR_INVALID_ARG;
     }
     if (scratch_bytes == 0) scratch_bytes = 32ull << 20;

@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 def handles():
     from paper_2609_21264_b200 import binding
     hs = {"persistent": binding.fa_create(flags=binding.FA_FLAG_FORCE_PERSISTENT),
-          "per_item": binding.fa_create(flags=binding.FA_FLAG_NO_PERSISTENT)}
+          "per_item": binding.fa_create(flags=binding.FA_FLAG_NO_PERSISTENT | binding.FA_FLAG_NO_STREAM_KERNEL)}
     yield hs
     for h in hs.values():
         binding.fa_destroy(h)
@@ -87,7 +87,7 @@ def test_default_choice_by_shape():
     h = binding.fa_create()
     try:
         for (B, H, S, expect) in ((8, 32, 1024, "fa_fwd_persistent"), (1, 32, 2048, "fa_fwd_pipelined"),
-                                  (1, 12, 512, "fa_fwd_pipelined"), (1, 64, 16384, "fa_fwd_pipelined")):
+                                  (1, 12, 512, "fa_fwd_stream"), (1, 64, 16384, "fa_fwd_pipelined")):
             q = torch.zeros((B, H, S, 128), dtype=torch.bfloat16, device="cuda")
             binding.forward(h, q, q, q, causal=True)
             torch.cuda.synchronize()
