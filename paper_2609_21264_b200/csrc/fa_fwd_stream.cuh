@@ -54,7 +54,6 @@ struct StreamShared {
     uint64_t s_full[2];      // score MMA -> softmax b: S^b(j) is in TMEM
     uint64_t s_free[2];      // softmax b -> score MMA: S^b(j) is in registers
     uint64_t st_full[2];     // softmax b -> the other warpgroup and correction: u and r of tile j published
-    uint64_t st_seen[2];     // correction -> softmax b: r of tile j has been read (its slot may be rewritten)
     uint64_t p_ready[2];     // softmax b + correction -> PV MMA: P^b(j) written, O rescaled
     uint64_t p_free[2];      // PV MMA -> softmax b, correction: PV(j) complete
     uint64_t o_final;        // PV MMA -> epilogue
@@ -139,7 +138,6 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             mbar_init(smem_addr(&sh.s_full[i]), 1);
             mbar_init(smem_addr(&sh.s_free[i]), 4);       // the 4 warps of warpgroup i
             mbar_init(smem_addr(&sh.st_full[i]), 4);
-            mbar_init(smem_addr(&sh.st_seen[i]), 4);      // 4 correction warps
             mbar_init(smem_addr(&sh.p_ready[i]), 8);      // 4 softmax warps + 4 correction warps
             mbar_init(smem_addr(&sh.p_free[i]), 1);
         }
@@ -236,11 +234,13 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 m_ref = sh.mref[row];
                 r_prev = sh.alpha[(j - 1) & 1][row];
             }
-            // The slot of this tile's r is reused every second tile: the correction warps must have
-            // read r of tile j-2 (which also keeps the next phase of st_full from overtaking them;
-            // a parity wait cannot tell a phase from the one two phases later).
+            // P^g and the slot of this tile's r are reused every second tile: the PV MMA of tile j-2
+            // must be complete.  It was issued a whole tile ago, so this wait is normally over at
+            // once; it also means that the correction warps have consumed r of tile j-2, which
+            // keeps the next phase of st_full from overtaking them (a parity wait cannot tell a
+            // phase from the one two phases later).
             if (j >= 2) {
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.st_seen[g]), (use - 1u) & 1u, wctx, kSiteSoftmaxCorrFree));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_pf, (use - 1u) & 1u, wctx, kSiteSoftmaxPFree));
                 if (!ok) break;
             }
             float alpha = 1.f;
@@ -257,20 +257,16 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             const float2 c2 = make_float2(c, c);
             const float2 nmc2 = make_float2(-mc, -mc);
             float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
+            auto exp_chunk = [&](int q) {
 #pragma unroll
-            for (int e = 0; e < kTileN; e += 2) {
-                const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[e]), __uint_as_float(s[e + 1])), c2, nmc2);
-                s[e] = __float_as_uint(exp2_approx(x.x));
-                s[e + 1] = __float_as_uint(exp2_approx(x.y));
-            }
-            // P^g is reused every second tile: the PV MMA of tile j-2 must have read it.  The wait
-            // sits after the exponentials so that the MMA is not on this warpgroup's path.
-            if (j >= 2) {
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_pf, (use - 1u) & 1u, wctx, kSiteSoftmaxPFree));
-                if (!ok) break;
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
+                for (int e = 0; e < 32; e += 2) {
+                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[q * 32 + e]),
+                                                            __uint_as_float(s[q * 32 + e + 1])), c2, nmc2);
+                    s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
+                    s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
+                }
+            };
+            auto emit_chunk = [&](int q) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int e = 0; e < 32; e += 4) {
@@ -282,7 +278,16 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     pk[e / 2 + 1] = pack_bf16x2(v1.x, v1.y);
                 }
                 tmem_st_x16(tP + q * 16, pk);
-            }
+            };
+            // conversion and store of a chunk run under the exponentials of the next one
+            exp_chunk(0);
+            exp_chunk(1);
+            emit_chunk(0);
+            exp_chunk(2);
+            emit_chunk(1);
+            exp_chunk(3);
+            emit_chunk(2);
+            emit_chunk(3);
             l = l * (r_prev * alpha) + ((sum_a.x + sum_a.y) + (sum_b.x + sum_b.y));
             tc_wait_st();
             tc_fence_before_sync();
@@ -371,8 +376,6 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.st_full[j & 1]), use & 1u, wctx, kSiteCorrScale));
             if (!ok) break;
             const float alpha = sh.alpha[j & 1][row];
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_addr(&sh.st_seen[j & 1]));
             if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
                 // O must hold the complete sum up to tile j-1 before it is rescaled
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.p_free[(j - 1) & 1]),
