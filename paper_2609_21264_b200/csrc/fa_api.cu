@@ -311,8 +311,10 @@ fa_status launch_stream(fa_handle* h, int slot, const CUtensorMap& mq, const CUt
 // on, which is enough to tell a grid of under one wave (the stream kernel's case) from the rest.
 struct TilingEstimate { double pair_us, stream_us; };
 TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int dqk, int causal, int n_q_tiles, int splits) {
-    const double a_p = dqk == 64 ? 1.36 : 2.0, f_p = dqk == 64 ? 6.0 : 6.7;
-    const double a_s = dqk == 64 ? 0.75 : 1.0, f_s = 5.0;
+    // (at d_qk = 192 the pair kernel only has room for two K stages and one V stage and a longer MMA
+    // chain per round; the stream kernel is ahead there at every size measured)
+    const double a_p = dqk == 64 ? 1.36 : (dqk == 128 ? 2.0 : 2.9), f_p = dqk == 64 ? 6.0 : 6.7;
+    const double a_s = dqk == 64 ? 0.75 : (dqk == 128 ? 1.0 : 1.05), f_s = 5.0;
     const double heads = static_cast<double>(B) * Hq;
     double pair_total = 0, pair_max = 0, stream_total = 0, stream_max = 0;
     for (int t = 0; t < n_q_tiles; ++t) {
@@ -408,7 +410,7 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
         // kernel's grid does not fill the GPU or its longest CTA dominates: decided from the two
         // estimates, with a margin, before the K/V range is split.
         bool stream = false;
-        if (!cu_q && dqk != 192 && !p.debug_drop_v_load && !(h->flags & FA_FLAG_NO_STREAM_KERNEL)) {
+        if (!cu_q && !p.debug_drop_v_load && !(h->flags & FA_FLAG_NO_STREAM_KERNEL)) {
             if (h->flags & FA_FLAG_STREAM_KERNEL) {
                 stream = true;
             } else if (!persistent && h->kv_splits_cfg <= 1) {
@@ -424,7 +426,8 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
             h->last_splits = 1;
             h->last_kernel = "fa_fwd_stream";
             if (dqk == 64) return launch_stream<64, 64>(h, 16, map_q, map_k, map_v, map_o, p, st);
-            return launch_stream<128, 128>(h, 17, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_stream<128, 128>(h, 17, map_q, map_k, map_v, map_o, p, st);
+            return launch_stream<192, 128>(h, 18, map_q, map_k, map_v, map_o, p, st);
         }
         if (persistent) {
             h->last_kernel = "fa_fwd_persistent";

@@ -22,7 +22,7 @@
 //   warps 8-11      correction: O *= r when the reference maximum moved
 //   warp 12         score MMAs (one thread), warp 13: PV MMAs (one thread)
 //   warp 14         TMA loads of Q and K, warp 15: TMA loads of V
-// Fixed-length problems without split-KV; head sizes 64 and 128.
+// Fixed-length problems without split-KV.
 #pragma once
 
 #include "fa_fwd_pipelined.cuh"
@@ -37,8 +37,8 @@ struct StreamCfg {
     static constexpr int kQBytes = Base::kQBytes;
     static constexpr int kKBytes = Base::kKBytes;
     static constexpr int kVBytes = Base::kVBytes;
-    static constexpr int kKStages = 3;
-    static constexpr int kVStages = 3;
+    static constexpr int kKStages = (DQK == 192) ? 2 : 3;
+    static constexpr int kVStages = (DQK == 192) ? 2 : 3;
     static constexpr int kTileBytes = kQBytes + kKStages * kKBytes + kVStages * kVBytes;
     static constexpr int kTmemCols = 512;
     static constexpr int kColS = 0;        // S^b at kColS + 128 b

@@ -25,8 +25,8 @@ def handle():
 
 
 def _wl(name, B, Hq, Hkv, Sq, Sk, d, causal, seed, sigma=1.0, k_mult=1.0):
-    return W.Workload(name, B=B, Hq=Hq, Hkv=Hkv, Sq=Sq, Sk=Sk, dqk=d, dv=d, causal=causal, scale=d ** -0.5,
-                      sigma=sigma, k_mult=k_mult, seed=seed)
+    return W.Workload(name, B=B, Hq=Hq, Hkv=Hkv, Sq=Sq, Sk=Sk, dqk=d, dv=(128 if d == 192 else d), causal=causal,
+                      scale=d ** -0.5, sigma=sigma, k_mult=k_mult, seed=seed)
 
 
 CASES = [
@@ -40,6 +40,8 @@ CASES = [
     _wl("keys_times_eight", 1, 2, 2, 384, 900, 128, True, 1408, k_mult=8.0),
     _wl("sigma_three", 1, 2, 2, 300, 700, 64, True, 1409, sigma=3.0),
     _wl("tiny", 1, 1, 1, 5, 7, 128, False, 1410),
+    _wl("d192_128_causal", 1, 4, 4, 700, 700, 192, True, 1411),
+    _wl("d192_128_full_ragged", 2, 2, 1, 150, 930, 192, False, 1412),
 ]
 
 
