@@ -416,6 +416,9 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
             } else if (!persistent && h->kv_splits_cfg <= 1) {
                 const TilingEstimate e = estimate_tilings(h->num_sms, B, Hq, Sq, Sk, dqk, p.causal, p.n_q_tiles, p.kv_splits);
                 stream = e.stream_us < 0.9 * e.pair_us;
+                // at d = 64 the stream kernel is also 3-7 % ahead on long items (measured from 64
+                // K/V tiles per query tile on), closer than the estimate can tell
+                if (dqk == 64 && longest >= 32 && p.kv_splits == 1) stream = true;
             }
         }
         if (stream) {
