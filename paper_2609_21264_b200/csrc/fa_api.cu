@@ -278,12 +278,12 @@ fa_status launch_persistent(fa_handle* h, int slot, const CUtensorMap& mq, const
 }
 
 // One query tile per CTA, K/V tiles streamed through two softmax warpgroups.
-template <int DQK, int DV>
+template <int DQK, int DV, bool kVarlen = false>
 fa_status launch_stream(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
                         const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
     constexpr int smem = fa::stream_smem_bytes<DQK, DV>();
     static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
-    auto kernel = fa::fa_fwd_stream_kernel<DQK, DV>;
+    auto kernel = fa::fa_fwd_stream_kernel<DQK, DV, kVarlen>;
     fa_status s = ensure_smem_attr(h, slot, kernel, smem);
     if (s != FA_OK) return s;
     const long long n_ctas = static_cast<long long>(p.n_q_tiles) * p.Hq * p.B;
@@ -410,9 +410,11 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
         // kernel's grid does not fill the GPU or its longest CTA dominates: decided from the two
         // estimates, with a margin, before the K/V range is split.
         bool stream = false;
-        if (!cu_q && !p.debug_drop_v_load && !(h->flags & FA_FLAG_NO_STREAM_KERNEL)) {
+        if (!p.debug_drop_v_load && !(h->flags & FA_FLAG_NO_STREAM_KERNEL)) {
             if (h->flags & FA_FLAG_STREAM_KERNEL) {
                 stream = true;
+            } else if (cu_q) {
+                stream = (dqk == 192);       // lengths are on the device: no estimate; 192/128 is always ahead
             } else if (!persistent && h->kv_splits_cfg <= 1) {
                 const TilingEstimate e = estimate_tilings(h->num_sms, B, Hq, Sq, Sk, dqk, p.causal, p.n_q_tiles, p.kv_splits);
                 stream = e.stream_us < 0.9 * e.pair_us;
@@ -428,6 +430,11 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
             p.lse_part = nullptr;
             h->last_splits = 1;
             h->last_kernel = "fa_fwd_stream";
+            if (cu_q) {
+                if (dqk == 64) return launch_stream<64, 64, true>(h, 19, map_q, map_k, map_v, map_o, p, st);
+                if (dqk == 128) return launch_stream<128, 128, true>(h, 20, map_q, map_k, map_v, map_o, p, st);
+                return launch_stream<192, 128, true>(h, 21, map_q, map_k, map_v, map_o, p, st);
+            }
             if (dqk == 64) return launch_stream<64, 64>(h, 16, map_q, map_k, map_v, map_o, p, st);
             if (dqk == 128) return launch_stream<128, 128>(h, 17, map_q, map_k, map_v, map_o, p, st);
             return launch_stream<192, 128>(h, 18, map_q, map_k, map_v, map_o, p, st);

@@ -22,7 +22,7 @@
 //   warps 8-11      correction: O *= r when the reference maximum moved
 //   warp 12         score MMAs (one thread), warp 13: PV MMAs (one thread)
 //   warp 14         TMA loads of Q and K, warp 15: TMA loads of V
-// Fixed-length problems without split-KV.
+// No split-KV on this path.
 #pragma once
 
 #include "fa_fwd_pipelined.cuh"
@@ -71,7 +71,8 @@ constexpr int stream_smem_bytes() {
     return StreamCfg<DQK, DV>::kTileBytes + static_cast<int>(sizeof(StreamShared));
 }
 
-template <int DQK, int DV>
+// kVarlen = packed variable-length batch, as in the pair kernel.
+template <int DQK, int DV, bool kVarlen = false>
 __global__ void __launch_bounds__(512, 1)
 fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                      const __grid_constant__ CUtensorMap tm_k,
@@ -91,10 +92,11 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int lane = tid & 31;
 
     grid_launch_dependents();
+    if constexpr (kVarlen) grid_dependency_wait();    // the sequence offsets are read right away
 
     const uint32_t smem_base = smem_addr(smem_raw);
     if ((smem_base & 1023u) != 0u) {          // uniform over the CTA; nothing has been set up yet
-        grid_dependency_wait();
+        if constexpr (!kVarlen) grid_dependency_wait();
         if (tid == 0 && p.status) {
             volatile uint32_t* sw = p.status;
             sw[1] = kSiteSmemAlign;
@@ -122,9 +124,18 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int b = bh / p.Hq;
     const int kvh = hq / (p.Hq / p.Hkv);
     const int q_idx = b * p.Hq + hq;
-    const int off = p.Sk - p.Sq;
+    int Sq = p.Sq, Sk = p.Sk, q_row0 = 0, k_row0 = 0;
+    if constexpr (kVarlen) {
+        q_row0 = p.cu_q[b];
+        k_row0 = p.cu_k[b];
+        Sq = p.cu_q[b + 1] - q_row0;
+        Sk = p.cu_k[b + 1] - k_row0;
+    }
+    const int off = Sk - Sq;
     const int i0 = q_tile * kTileM;
-    const int n_kv = kv_tiles_for_q_tile(i0, kTileM, p.Sq, p.Sk, p.causal);
+    if (kVarlen && i0 >= Sq) return;      // a sequence shorter than the longest one (whole CTA, before any set-up)
+    const int n_kv = kv_tiles_for_q_tile(i0, kTileM, Sq, Sk, p.causal);
+    const int tb = kVarlen ? 0 : b;       // batch coordinate of the tensor maps (packed tensors have one slice)
 
     // ---------------------------------------------------------------- setup
     if (tid == 0) {
@@ -163,7 +174,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    grid_dependency_wait();
+    if constexpr (!kVarlen) grid_dependency_wait();
 
     const uint32_t tmem_base = sh.tmem_base;
     WaitCtx wctx{&sh.abort_flag, p.status, p.wait_limit_ns};
@@ -184,7 +195,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         const uint32_t bar_pr = smem_addr(&sh.p_ready[g]);
         const uint32_t bar_pf = smem_addr(&sh.p_free[g]);
         const int i_glob = i0 + row;
-        int kmax_row = p.Sk - 1;
+        int kmax_row = Sk - 1;
         if (p.causal && i_glob + off < kmax_row) kmax_row = i_glob + off;
         const float tau_raw = kRescaleThresholdLog2 / c;
 
@@ -296,12 +307,13 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         }
 
         // ---- epilogue: O = G' / s (bf16), lse = u * scale + ln s
-        if (ok && i0 < p.Sq) {
-            const size_t lse_row0 = static_cast<size_t>(q_idx) * p.Sq;
+        if (ok && i0 < Sq) {
+            // fixed lengths: lse [B, Hq, Sq]; packed batches: lse [Hq, total_q], O rows q_row0 onwards
+            const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq) * p.total_q + q_row0 : static_cast<size_t>(q_idx) * p.Sq;
+            const long long o_base = (kVarlen ? q_row0 * p.o_stride_s : b * p.o_stride_b) + hq * p.o_stride_h;
             if (n_kv == 0) {              // no key visible to any row of this tile
-                if (g == 0 && i_glob < p.Sq) {
-                    __nv_bfloat16* o_row = p.O + (b * p.o_stride_b + hq * p.o_stride_h +
-                                                  static_cast<long long>(i_glob) * p.o_stride_s);
+                if (g == 0 && i_glob < Sq) {
+                    __nv_bfloat16* o_row = p.O + (o_base + static_cast<long long>(i_glob) * p.o_stride_s);
                     const uint4 z = make_uint4(0, 0, 0, 0);
 #pragma unroll
                     for (int v = 0; v < DV / 8; ++v) reinterpret_cast<uint4*>(o_row)[v] = z;
@@ -328,38 +340,60 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     const float lt = sh.lsum[0][row] + sh.lsum[1][row];
                     const float m_fin = sh.mref[row];
                     const float inv_l = (lt > 0.f) ? (1.f / lt) : 0.f;
-                    if (g == 0 && p.lse && i_glob < p.Sq)
+                    if (g == 0 && p.lse && i_glob < Sq)
                         p.lse[lse_row0 + i_glob] = (lt > 0.f) ? (m_fin * c * 0.6931471805599453f + logf(lt)) : -INFINITY;
                     // warpgroup g converts columns [g*DV/2, (g+1)*DV/2) of O into the staging tile
                     // (the Q tile's space: the last score MMA is long complete), then one thread
                     // stores it with TMA; rows past Sq are clipped
                     const uint32_t tO = tmem_base + Cfg::kColO + lane_sel;
-                    const uint32_t sO = sQ + row * 128;
+                    // the last tile of a packed sequence is followed by the next sequence's rows, which a
+                    // box store would overwrite: it is stored row by row
+                    const bool box_store = !kVarlen || (i0 + kTileM <= Sq);
+                    if (box_store) {
+                        const uint32_t sO = sQ + row * 128;
 #pragma unroll 1
-                    for (int cc = g * (DV / 64); cc < (g + 1) * (DV / 64); ++cc) {
-                        uint32_t r[32];
-                        tmem_ld_x32(tO + cc * 32, r);
-                        tc_wait_ld();
-                        const uint32_t chunk = sO + (cc >> 1) * kChunkBytes;
+                        for (int cc = g * (DV / 64); cc < (g + 1) * (DV / 64); ++cc) {
+                            uint32_t r[32];
+                            tmem_ld_x32(tO + cc * 32, r);
+                            tc_wait_ld();
+                            const uint32_t chunk = sO + (cc >> 1) * kChunkBytes;
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            const uint32_t piece = static_cast<uint32_t>(((cc & 1) * 4 + v) ^ (row & 7)) << 4;
-                            st_shared_v4(chunk + piece,
-                                         pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
-                                         pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
-                                         pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
-                                         pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
+                            for (int v = 0; v < 4; ++v) {
+                                const uint32_t piece = static_cast<uint32_t>(((cc & 1) * 4 + v) ^ (row & 7)) << 4;
+                                st_shared_v4(chunk + piece,
+                                             pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
+                                             pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
+                                             pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
+                                             pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
+                            }
                         }
-                    }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_addr(&sh.o_staged));
-                    if (warp == 0 && lane == 0 && mbar_wait(smem_addr(&sh.o_staged), 0, wctx, kSiteEpiStaged)) {
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_addr(&sh.o_staged));
+                        if (warp == 0 && lane == 0 && mbar_wait(smem_addr(&sh.o_staged), 0, wctx, kSiteEpiStaged)) {
 #pragma unroll
-                        for (int ch = 0; ch < DV / kChunkCols; ++ch)
-                            tma_store_4d(&tm_o, sQ + ch * kChunkBytes, ch * kChunkCols, i0, hq, b);
-                        tma_store_commit();
-                        tma_store_wait_read_all();     // the CTA's shared memory outlives the reads
+                            for (int ch = 0; ch < DV / kChunkCols; ++ch)
+                                tma_store_4d(&tm_o, sQ + ch * kChunkBytes, ch * kChunkCols, q_row0 + i0, hq, tb);
+                            tma_store_commit();
+                            tma_store_wait_read_all();     // the CTA's shared memory outlives the reads
+                        }
+                    } else {
+                        __nv_bfloat16* o_row = p.O + (o_base + static_cast<long long>(i_glob) * p.o_stride_s);
+#pragma unroll 1
+                        for (int cc = g * (DV / 64); cc < (g + 1) * (DV / 64); ++cc) {
+                            uint32_t r[32];
+                            tmem_ld_x32(tO + cc * 32, r);
+                            tc_wait_ld();
+                            if (i_glob < Sq) {
+#pragma unroll
+                                for (int v = 0; v < 4; ++v)
+                                    reinterpret_cast<uint4*>(o_row + cc * 32)[v] = make_uint4(
+                                        pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
+                                        pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
+                                        pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
+                                        pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
+                            }
+                        }
                     }
                 }
             }
@@ -469,7 +503,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 mbar_arrive_expect_tx(bar, Cfg::kQBytes);
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kQChunks; ++cc)
-                    tma_load_4d(sQ + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols, i0, hq, b);
+                    tma_load_4d(sQ + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols, q_row0 + i0, hq, tb);
             }
             bool ok = true;
             for (int j = 0; j < n_kv && ok; ++j) {
@@ -480,7 +514,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 mbar_arrive_expect_tx(bar, Cfg::kKBytes);
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kQChunks; ++cc)
-                    tma_load_4d(sK + s * Cfg::kKBytes + cc * kChunkBytes, &tm_k, bar, cc * kChunkCols, j * kTileN, kvh, b);
+                    tma_load_4d(sK + s * Cfg::kKBytes + cc * kChunkBytes, &tm_k, bar, cc * kChunkCols, k_row0 + j * kTileN, kvh, tb);
             }
         }
     } else {
@@ -496,7 +530,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 mbar_arrive_expect_tx(bar, Cfg::kVBytes);
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kVChunks; ++cc)
-                    tma_load_4d(sV + s * Cfg::kVBytes + cc * kChunkBytes, &tm_v, bar, cc * kChunkCols, j * kTileN, kvh, b);
+                    tma_load_4d(sV + s * Cfg::kVBytes + cc * kChunkBytes, &tm_v, bar, cc * kChunkCols, k_row0 + j * kTileN, kvh, tb);
             }
         }
     }
