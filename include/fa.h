@@ -80,7 +80,7 @@ typedef enum fa_status {
  * warpgroups (csrc/fa_fwd_stream.cuh).  It doubles the number of CTAs and shortens each one's
  * dependency chain, which wins when the pair tiling leaves SMs idle or its longest CTA dominates
  * (under about one wave of pairs: short sequences, few heads); the library estimates both and
- * picks it with a 10 % margin, also instead of splitting the K/V range; at head sizes 192/128,
+ * picks it with a 10 % margin (each with its own split-KV count); at head sizes 192/128,
  * where the pair kernel is short of shared memory, it is ahead at every size.  These flags force
  * it on (fixed-length problems) or off. */
 #define FA_FLAG_STREAM_KERNEL 32u

@@ -191,8 +191,9 @@ fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const 
 
 // Number of K/V splits for a problem: 1 unless the query tiles alone leave most SMs idle and the
 // K/V range is long enough to cut; never more than the scratch buffer can hold partials for.
-int choose_kv_splits(const fa_handle* h, int B, int Hq, int Sq, int Sk, int dv, int causal, int n_q_tiles) {
-    const long long items = static_cast<long long>((n_q_tiles + 1) / 2) * B * Hq;
+int choose_kv_splits(const fa_handle* h, int B, int Hq, int Sq, int Sk, int dv, int causal, int n_q_tiles,
+                     bool one_tile_items = false) {
+    const long long items = static_cast<long long>(one_tile_items ? n_q_tiles : (n_q_tiles + 1) / 2) * B * Hq;
     int max_tiles = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, causal);
     if (!causal) max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
     int splits = 1;
@@ -286,7 +287,7 @@ fa_status launch_stream(fa_handle* h, int slot, const CUtensorMap& mq, const CUt
     auto kernel = fa::fa_fwd_stream_kernel<DQK, DV, kVarlen>;
     fa_status s = ensure_smem_attr(h, slot, kernel, smem);
     if (s != FA_OK) return s;
-    const long long n_ctas = static_cast<long long>(p.n_q_tiles) * p.Hq * p.B;
+    const long long n_ctas = static_cast<long long>(p.n_q_tiles) * p.Hq * p.B * p.kv_splits;
     if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -300,6 +301,18 @@ fa_status launch_stream(fa_handle* h, int slot, const CUtensorMap& mq, const CUt
     cfg.numAttrs = (h->flags & FA_FLAG_NO_DEPENDENT_LAUNCH) ? 0 : 1;
     if (cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mo, p) != cudaSuccess) return FA_ERR_CUDA;
     h->launches += 1;
+    if (p.kv_splits > 1) {
+        const long long n_rows = static_cast<long long>(p.B) * p.Hq * p.Sq;
+        const long long blocks = (n_rows + 3) / 4;
+        if (blocks > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+        cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+        cfg.blockDim = dim3(128, 1, 1);
+        cfg.dynamicSmemBytes = 0;
+        if (cudaLaunchKernelEx(&cfg, fa::fa_combine_kernel<DV>, static_cast<const float*>(p.o_part),
+                               static_cast<const float*>(p.lse_part), p.O, p.lse, n_rows, p.kv_splits, p.Hq, p.Sq,
+                               p.o_stride_b, p.o_stride_h, p.o_stride_s) != cudaSuccess) return FA_ERR_CUDA;
+        h->launches += 1;
+    }
     return FA_OK;
 }
 
@@ -310,7 +323,8 @@ fa_status launch_stream(fa_handle* h, int slot, const CUtensorMap& mq, const CUt
 // and by whole waves when all items are equal.  Good to some 20 % on the shapes it was checked
 // on, which is enough to tell a grid of under one wave (the stream kernel's case) from the rest.
 struct TilingEstimate { double pair_us, stream_us; };
-TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int dqk, int causal, int n_q_tiles, int splits) {
+TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int dqk, int causal, int n_q_tiles, int splits,
+                                int stream_splits) {
     // (at d_qk = 192 the pair kernel only has room for two K stages and one V stage and a longer MMA
     // chain per round; the stream kernel is ahead there at every size measured)
     const double a_p = dqk == 64 ? 1.36 : (dqk == 128 ? 2.0 : 2.9), f_p = dqk == 64 ? 6.0 : 6.7;
@@ -319,8 +333,8 @@ TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int 
     double pair_total = 0, pair_max = 0, stream_total = 0, stream_max = 0;
     for (int t = 0; t < n_q_tiles; ++t) {
         const int r = fa::kv_tiles_for_q_tile(t * fa::kTileM, fa::kTileM, Sq, Sk, causal);
-        const double cs = a_s * r + f_s;
-        stream_total += cs;
+        const double cs = a_s * ((r + stream_splits - 1) / stream_splits) + f_s;
+        stream_total += cs * stream_splits;
         if (cs > stream_max) stream_max = cs;
         if ((t & 1) == 1 || t == n_q_tiles - 1) {        // second tile of a pair, or an unpaired last tile
             const double rounds = (r + splits - 1) / splits;
@@ -340,7 +354,7 @@ TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int 
     };
     TilingEstimate e;
     e.pair_us = makespan(pair_total, pair_max, static_cast<double>((n_q_tiles + 1) / 2) * splits) + (splits > 1 ? 6.0 : 0.0);
-    e.stream_us = makespan(stream_total, stream_max, n_q_tiles);
+    e.stream_us = makespan(stream_total, stream_max, static_cast<double>(n_q_tiles) * stream_splits) + (stream_splits > 1 ? 6.0 : 0.0);
     return e;
 }
 
@@ -410,17 +424,20 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
         // kernel's grid does not fill the GPU or its longest CTA dominates: decided from the two
         // estimates, with a margin, before the K/V range is split.
         bool stream = false;
+        int stream_splits = 1;
         if (!p.debug_drop_v_load && !(h->flags & FA_FLAG_NO_STREAM_KERNEL)) {
+            if (!cu_q) stream_splits = choose_kv_splits(h, B, Hq, Sq, Sk, dv, p.causal, p.n_q_tiles, true);
             if (h->flags & FA_FLAG_STREAM_KERNEL) {
                 stream = true;
             } else if (cu_q) {
                 stream = (dqk == 192);       // lengths are on the device: no estimate; 192/128 is always ahead
-            } else if (!persistent && h->kv_splits_cfg <= 1) {
-                const TilingEstimate e = estimate_tilings(h->num_sms, B, Hq, Sq, Sk, dqk, p.causal, p.n_q_tiles, p.kv_splits);
+            } else if (!persistent) {
+                const TilingEstimate e = estimate_tilings(h->num_sms, B, Hq, Sq, Sk, dqk, p.causal, p.n_q_tiles, p.kv_splits,
+                                                          stream_splits);
                 stream = e.stream_us < 0.9 * e.pair_us;
                 // at d = 64 the stream kernel is also 3-7 % ahead on long items (measured from 64
                 // K/V tiles per query tile on), closer than the estimate can tell
-                if (dqk == 64 && longest >= 32 && p.kv_splits == 1) stream = true;
+                if (dqk == 64 && longest >= 32 && p.kv_splits == 1 && stream_splits == 1) stream = true;
             }
         }
         if (stream) {
@@ -428,7 +445,18 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
             p.tiles_per_split = 0x3fffffff;
             p.o_part = nullptr;
             p.lse_part = nullptr;
-            h->last_splits = 1;
+            if (stream_splits > 1) {
+                int max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
+                if (p.causal) {
+                    const int t = fa::kv_tiles_for_q_tile((p.n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, 1);
+                    if (t < max_tiles) max_tiles = t;
+                }
+                p.kv_splits = stream_splits;
+                p.tiles_per_split = (max_tiles + stream_splits - 1) / stream_splits;
+                p.o_part = static_cast<float*>(h->scratch);
+                p.lse_part = p.o_part + static_cast<size_t>(stream_splits) * B * Hq * Sq * dv;
+            }
+            h->last_splits = p.kv_splits;
             h->last_kernel = "fa_fwd_stream";
             if (cu_q) {
                 if (dqk == 64) return launch_stream<64, 64, true>(h, 19, map_q, map_k, map_v, map_o, p, st);

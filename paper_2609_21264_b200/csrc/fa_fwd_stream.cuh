@@ -22,7 +22,7 @@
 //   warps 8-11      correction: O *= r when the reference maximum moved
 //   warp 12         score MMAs (one thread), warp 13: PV MMAs (one thread)
 //   warp 14         TMA loads of Q and K, warp 15: TMA loads of V
-// No split-KV on this path.
+// Split-KV as in the pair kernel: partials to scratch, merged by fa_combine_kernel.
 #pragma once
 
 #include "fa_fwd_pipelined.cuh"
@@ -112,7 +112,10 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     // 1-D grid: L2-sized groups of (batch, head) instances one after the other; inside a group
     // every head's last (with a causal mask: heaviest) query tile first.
     const int n_bh = p.B * p.Hq;
-    const int item = static_cast<int>(blockIdx.x);
+    // With split-KV the C CTAs that share a query tile and take disjoint ranges of its K/V tiles are
+    // adjacent in the grid; each writes a normalised fp32 partial that the combine kernel merges.
+    const int item = static_cast<int>(blockIdx.x) / p.kv_splits;
+    const int split = static_cast<int>(blockIdx.x) - item * p.kv_splits;
     const int per_group = p.n_q_tiles * p.heads_per_group;
     const int group = item / per_group;
     const int bh0 = group * p.heads_per_group;
@@ -134,7 +137,11 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int off = Sk - Sq;
     const int i0 = q_tile * kTileM;
     if (kVarlen && i0 >= Sq) return;      // a sequence shorter than the longest one (whole CTA, before any set-up)
-    const int n_kv = kv_tiles_for_q_tile(i0, kTileM, Sq, Sk, p.causal);
+    // K/V tiles [j_base, j_base + n_kv) of the query tile belong to this CTA (all visible ones without split-KV)
+    const int j_base = split * p.tiles_per_split;
+    int n_kv = kv_tiles_for_q_tile(i0, kTileM, Sq, Sk, p.causal) - j_base;
+    if (n_kv > p.tiles_per_split) n_kv = p.tiles_per_split;
+    if (n_kv < 0) n_kv = 0;
     const int tb = kVarlen ? 0 : b;       // batch coordinate of the tensor maps (packed tensors have one slice)
 
     // ---------------------------------------------------------------- setup
@@ -206,7 +213,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             ok = __all_sync(0xffffffffu, mbar_wait(bar_s, use & 1u, wctx, kSiteSoftmaxSFull));
             if (!ok) break;
             tc_fence_after_sync();
-            const int j0 = j * kTileN;
+            const int j0 = (j_base + j) * kTileN;
             const bool need_mask = (j0 + kTileN - 1 > kmax_row);
 
             uint32_t s[kTileN];
@@ -311,7 +318,16 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             // fixed lengths: lse [B, Hq, Sq]; packed batches: lse [Hq, total_q], O rows q_row0 onwards
             const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq) * p.total_q + q_row0 : static_cast<size_t>(q_idx) * p.Sq;
             const long long o_base = (kVarlen ? q_row0 * p.o_stride_s : b * p.o_stride_b) + hq * p.o_stride_h;
-            if (n_kv == 0) {              // no key visible to any row of this tile
+            if (p.kv_splits > 1 && n_kv == 0) {      // an empty range: a neutral partial
+                if (i_glob < Sq) {
+                    const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
+                    float* po_row = p.o_part + prow * DV + g * (DV / 2);
+                    const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int v = 0; v < DV / 8; ++v) reinterpret_cast<float4*>(po_row)[v] = z;
+                    if (g == 0) p.lse_part[prow] = -INFINITY;
+                }
+            } else if (n_kv == 0) {       // no key visible to any row of this tile
                 if (g == 0 && i_glob < Sq) {
                     __nv_bfloat16* o_row = p.O + (o_base + static_cast<long long>(i_glob) * p.o_stride_s);
                     const uint4 z = make_uint4(0, 0, 0, 0);
@@ -340,7 +356,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     const float lt = sh.lsum[0][row] + sh.lsum[1][row];
                     const float m_fin = sh.mref[row];
                     const float inv_l = (lt > 0.f) ? (1.f / lt) : 0.f;
-                    if (g == 0 && p.lse && i_glob < Sq)
+                    if (g == 0 && p.lse && i_glob < Sq && p.kv_splits == 1)
                         p.lse[lse_row0 + i_glob] = (lt > 0.f) ? (m_fin * c * 0.6931471805599453f + logf(lt)) : -INFINITY;
                     // warpgroup g converts columns [g*DV/2, (g+1)*DV/2) of O into the staging tile
                     // (the Q tile's space: the last score MMA is long complete), then one thread
@@ -349,7 +365,26 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     // the last tile of a packed sequence is followed by the next sequence's rows, which a
                     // box store would overwrite: it is stored row by row
                     const bool box_store = !kVarlen || (i0 + kTileM <= Sq);
-                    if (box_store) {
+                    if (p.kv_splits > 1) {
+                        // split-KV: G'_c / s_c in fp32 and u_c + ln s_c go to scratch (Algorithm 2's partials)
+                        const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
+                        float* po_row = p.o_part + prow * DV;
+                        if (g == 0 && i_glob < Sq)
+                            p.lse_part[prow] = (lt > 0.f) ? (m_fin * c * 0.6931471805599453f + logf(lt)) : -INFINITY;
+#pragma unroll 1
+                        for (int cc = g * (DV / 64); cc < (g + 1) * (DV / 64); ++cc) {
+                            uint32_t r[32];
+                            tmem_ld_x32(tO + cc * 32, r);
+                            tc_wait_ld();
+                            if (i_glob < Sq) {
+#pragma unroll
+                                for (int v = 0; v < 8; ++v)
+                                    reinterpret_cast<float4*>(po_row + cc * 32)[v] = make_float4(
+                                        __uint_as_float(r[4 * v]) * inv_l, __uint_as_float(r[4 * v + 1]) * inv_l,
+                                        __uint_as_float(r[4 * v + 2]) * inv_l, __uint_as_float(r[4 * v + 3]) * inv_l);
+                            }
+                        }
+                    } else if (box_store) {
                         const uint32_t sO = sQ + row * 128;
 #pragma unroll 1
                         for (int cc = g * (DV / 64); cc < (g + 1) * (DV / 64); ++cc) {
@@ -514,7 +549,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 mbar_arrive_expect_tx(bar, Cfg::kKBytes);
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kQChunks; ++cc)
-                    tma_load_4d(sK + s * Cfg::kKBytes + cc * kChunkBytes, &tm_k, bar, cc * kChunkCols, k_row0 + j * kTileN, kvh, tb);
+                    tma_load_4d(sK + s * Cfg::kKBytes + cc * kChunkBytes, &tm_k, bar, cc * kChunkCols, k_row0 + (j_base + j) * kTileN, kvh, tb);
             }
         }
     } else {
@@ -530,7 +565,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 mbar_arrive_expect_tx(bar, Cfg::kVBytes);
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kVChunks; ++cc)
-                    tma_load_4d(sV + s * Cfg::kVBytes + cc * kChunkBytes, &tm_v, bar, cc * kChunkCols, k_row0 + j * kTileN, kvh, tb);
+                    tma_load_4d(sV + s * Cfg::kVBytes + cc * kChunkBytes, &tm_v, bar, cc * kChunkCols, k_row0 + (j_base + j) * kTileN, kvh, tb);
             }
         }
     }

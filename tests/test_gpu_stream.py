@@ -81,18 +81,47 @@ def test_repeated_launches_are_bit_stable(handle):
         assert torch.equal(o.view(torch.int16), first.view(torch.int16))
 
 
+SPLIT_CASES = [
+    _wl("split_decode_like", 1, 8, 2, 128, 4000, 128, False, 1421),
+    _wl("split_single_row_queries", 2, 4, 4, 1, 3000, 128, False, 1422),
+    _wl("split_causal_short_q", 1, 4, 4, 100, 2500, 64, True, 1423),
+    _wl("split_d192", 1, 2, 2, 130, 2100, 192, False, 1424),
+]
+
+
+@pytest.mark.parametrize("w", SPLIT_CASES, ids=[w.name for w in SPLIT_CASES])
+@pytest.mark.parametrize("splits", [0, 3, 7])
+def test_stream_kernel_split_kv(w, splits):
+    """K/V range cut over several CTAs of the stream kernel and merged by the combine kernel (0 = library's choice)."""
+    from paper_2609_21264_b200 import binding
+    h = binding.fa_create(flags=binding.FA_FLAG_STREAM_KERNEL, kv_splits=splits)
+    try:
+        Q, K, V = W.make_inputs(w)
+        O_ref, lse_ref = oracle.attention(Q, K, V, causal=w.causal, scale=w.scale)
+        O, lse = run_gpu(h, w, Q, K, V)
+        assert binding.fa_last_kernel_name(h) == "fa_fwd_stream"
+        assert binding.fa_last_kv_splits(h) > 1
+        assert_parity(O, lse, O_ref, lse_ref, w.name)
+    finally:
+        binding.fa_destroy(h)
+
+
 def test_choice_between_tilings():
-    """Small grids go to the stream kernel, decode-like shapes keep split-KV, full grids the pair kernel."""
+    """Small grids and decode-like shapes (with split-KV) go to the stream kernel, full grids to the pair kernel."""
     import torch
     from paper_2609_21264_b200 import binding
     h = binding.fa_create()
     try:
-        for (B, H, Sq, Sk, causal, expect) in ((1, 8, 1024, 1024, True, "fa_fwd_stream"), (1, 32, 128, 32768, False, "fa_fwd_pipelined"),
-                                                (1, 32, 2048, 2048, True, "fa_fwd_pipelined"), (1, 12, 2048, 2048, False, "fa_fwd_pipelined")):
+        for (B, H, Sq, Sk, causal, expect, split) in ((1, 8, 1024, 1024, True, "fa_fwd_stream", False),
+                                                       (1, 32, 128, 32768, False, "fa_fwd_stream", True),
+                                                       (1, 32, 2048, 2048, True, "fa_fwd_pipelined", False),
+                                                       (1, 12, 2048, 2048, False, "fa_fwd_pipelined", False)):
             q = torch.zeros((B, H, Sq, 128), dtype=torch.bfloat16, device="cuda")
             k = torch.zeros((B, H, Sk, 128), dtype=torch.bfloat16, device="cuda")
             binding.forward(h, q, k, k, causal=causal)
             torch.cuda.synchronize()
             assert binding.fa_last_kernel_name(h) == expect, (B, H, Sq, Sk)
+            if split:
+                assert binding.fa_last_kv_splits(h) > 1, (B, H, Sq, Sk)
     finally:
         binding.fa_destroy(h)
