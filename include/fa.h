@@ -216,6 +216,27 @@ fa_status fa_forward_fp8(fa_handle* h,
                          int causal, float scale, void* stream);
 
 /*
+ * What the library would launch for a problem: which kernel (tiling), how many K/V splits, how
+ * many CTAs, and the two run-time estimates behind the choice (0 when none was needed).  A pure
+ * host function: no handle, no device, no CUDA call; `num_sms` is the SM count to plan for (148 on
+ * B200) and `cfg` the creation parameters a handle would have (NULL = defaults; its device field is
+ * ignored).  `varlen` != 0 plans fa_forward_varlen with Sq = max_sq and Sk = the mean key length.
+ * The tile schedule is the first step of the path (one CTA per pair of query tiles in the paper's
+ * mapping, Section 4); here it is chosen per launch, and this call makes the choice inspectable.
+ * Returns FA_ERR_UNSUPPORTED for head sizes the kernels do not have, FA_ERR_INVALID_ARG otherwise.
+ */
+typedef struct fa_plan_info {
+    const char* kernel;          /* "fa_fwd_pipelined", "fa_fwd_stream", "fa_fwd_persistent", "fa_fwd_simple" */
+    int32_t kv_splits;           /* CTAs per work item along the K/V range (1 = no split)        */
+    int64_t ctas;                /* grid size of the attention kernel                            */
+    double estimate_pair_us;     /* estimated time with one CTA per pair of query tiles          */
+    double estimate_stream_us;   /* estimated time with one CTA per query tile                   */
+} fa_plan_info;
+fa_status fa_plan(int num_sms, const fa_config* cfg, int varlen,
+                  int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal,
+                  fa_plan_info* out);
+
+/*
  * The same operation with HOST buffers (same layouts and types): copies Q, K, V
  * to staging memory owned by the handle, runs fa_forward, copies O (and lse if
  * not NULL) back, all on `stream`, and synchronises `stream` before returning.

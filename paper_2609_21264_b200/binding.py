@@ -28,7 +28,7 @@ FA_FLAG_FORCE_PERSISTENT = 16
 FA_FLAG_STREAM_KERNEL = 32
 FA_FLAG_NO_STREAM_KERNEL = 64
 
-EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_varlen", "fa_forward_fp8", "fa_forward_host", "fa_last_status", "fa_destroy",
+EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_varlen", "fa_forward_fp8", "fa_plan", "fa_forward_host", "fa_last_status", "fa_destroy",
            "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits",
            "fa_forward_split_noalloc", "fa_noalloc_scratch_bytes")
 
@@ -52,6 +52,11 @@ def library_path() -> str:
     return _build.LIB_PATH
 
 
+class fa_plan_info(ctypes.Structure):
+    _fields_ = [("kernel", ctypes.c_char_p), ("kv_splits", ctypes.c_int32), ("ctas", ctypes.c_int64),
+                ("estimate_pair_us", ctypes.c_double), ("estimate_stream_us", ctypes.c_double)]
+
+
 def load():
     """Load libfa_b200.so (built in-tree by ``build.build()``); raises if it is missing."""
     global _lib
@@ -72,6 +77,8 @@ def load():
     lib.fa_forward_host.argtypes = fwd_args
     lib.fa_forward_varlen.restype = i32
     lib.fa_forward_varlen.argtypes = [vp] * 8 + [i32] * 8 + [i32, ctypes.c_float, vp]
+    lib.fa_plan.restype = i32
+    lib.fa_plan.argtypes = [i32, ctypes.POINTER(fa_config), i32] + [i32] * 8 + [ctypes.POINTER(fa_plan_info)]
     lib.fa_forward_fp8.restype = i32
     lib.fa_forward_fp8.argtypes = [vp] * 9 + [i32] * 7 + [f32, vp]
     lib.fa_forward_strided.restype = i32
@@ -136,6 +143,18 @@ def fa_forward_fp8(h, Q8, K8, V8, q_scale, k_scale, v_scale, O, lse, B, Hq, Hkv,
     """Raw call: e4m3 device tensors with block scales (device fp32 arrays or None); returns the status code."""
     return load().fa_forward_fp8(h, Q8, K8, V8, q_scale, k_scale, v_scale, O, lse, B, Hq, Hkv, Sq, Sk, d,
                                  int(bool(causal)), float(scale), stream)
+
+
+def fa_plan(num_sms, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, *, varlen=False, flags=0, kv_splits=0, scratch_bytes=0) -> dict:
+    """What the library would launch for this problem on a device with `num_sms` SMs (no GPU needed)."""
+    cfg = fa_config(ctypes.sizeof(fa_config), -1, flags, 0, kv_splits, scratch_bytes)
+    out = fa_plan_info()
+    st = load().fa_plan(num_sms, ctypes.byref(cfg), int(bool(varlen)), B, Hq, Hkv, Sq, Sk, dqk, dv, int(bool(causal)),
+                        ctypes.byref(out))
+    if st != FA_OK:
+        raise FaError(st, "fa_plan")
+    return {"kernel": out.kernel.decode(), "kv_splits": out.kv_splits, "ctas": out.ctas,
+            "estimate_pair_us": out.estimate_pair_us, "estimate_stream_us": out.estimate_stream_us}
 
 
 def fa_forward_host(h, Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, stream=0) -> int:

@@ -191,24 +191,24 @@ fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const 
 
 // Number of K/V splits for a problem: 1 unless the query tiles alone leave most SMs idle and the
 // K/V range is long enough to cut; never more than the scratch buffer can hold partials for.
-int choose_kv_splits(const fa_handle* h, int B, int Hq, int Sq, int Sk, int dv, int causal, int n_q_tiles,
-                     bool one_tile_items = false) {
+int choose_kv_splits(int num_sms, uint32_t kv_splits_cfg, size_t scratch_bytes, int B, int Hq, int Sq, int Sk, int dv,
+                     int causal, int n_q_tiles, bool one_tile_items = false) {
     const long long items = static_cast<long long>(one_tile_items ? n_q_tiles : (n_q_tiles + 1) / 2) * B * Hq;
     int max_tiles = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, causal);
     if (!causal) max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
     int splits = 1;
-    if (h->kv_splits_cfg == 1) return 1;
-    if (h->kv_splits_cfg > 1) {
-        splits = static_cast<int>(h->kv_splits_cfg);
-    } else if (items * 2 <= h->num_sms && max_tiles >= 8) {
-        splits = static_cast<int>(h->num_sms / items);
+    if (kv_splits_cfg == 1) return 1;
+    if (kv_splits_cfg > 1) {
+        splits = static_cast<int>(kv_splits_cfg);
+    } else if (items * 2 <= num_sms && max_tiles >= 8) {
+        splits = static_cast<int>(num_sms / items);
         if (splits > max_tiles / 4) splits = max_tiles / 4;      // at least four tiles per split
         if (splits > 32) splits = 32;
     }
     if (splits > max_tiles) splits = max_tiles;
     if (splits < 1) splits = 1;
     const long long rows = static_cast<long long>(B) * Hq * Sq;
-    while (splits > 1 && static_cast<unsigned long long>(splits) * rows * (dv + 1) * 4ull > h->scratch_bytes) --splits;
+    while (splits > 1 && static_cast<unsigned long long>(splits) * rows * (dv + 1) * 4ull > scratch_bytes) --splits;
     return splits;
 }
 
@@ -358,6 +358,82 @@ TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int 
     return e;
 }
 
+// Which kernel a launch uses and how its K/V range is split: a pure function of the problem, the
+// handle's configuration and the SM count (fa_plan exposes it).
+enum PlanKernel { kPlanSerial = 0, kPlanPair = 1, kPlanPersistent = 2, kPlanStream = 3 };
+struct LaunchPlan {
+    int kernel;
+    int kv_splits;
+    int tiles_per_split;
+    double pair_us, stream_us;     // the two estimates (0 when no estimate was needed)
+};
+LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size_t scratch_bytes, bool varlen,
+                       int B, int Hq, int Sq, int Sk, int dqk, int dv, int causal) {
+    LaunchPlan pl;
+    pl.kernel = kPlanPair;
+    pl.kv_splits = 1;
+    pl.tiles_per_split = 0x3fffffff;
+    pl.pair_us = pl.stream_us = 0.0;
+    const int n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
+    const bool drop = (flags & FA_FLAG_DEBUG_DROP_V_LOAD) != 0;
+    int max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;           // K/V tiles of the longest query tile
+    if (causal) {
+        const int t = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, 1);
+        if (t < max_tiles) max_tiles = t;
+    }
+    auto with_splits = [&](int splits) {
+        pl.kv_splits = splits;
+        pl.tiles_per_split = splits > 1 ? (max_tiles + splits - 1) / splits : 0x3fffffff;
+    };
+    if (flags & FA_FLAG_SERIAL_KERNEL) {
+        pl.kernel = kPlanSerial;
+        return pl;
+    }
+    // packed batches: no split (the lengths that decide it are on the device)
+    const int pair_splits = varlen ? 1 : choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles);
+    // The persistent kernel wins where a CTA's fixed cost is a visible share of an item's time and
+    // every SM gets several items: measured on B200 it is 5-20 % faster from about three items per
+    // SM on, level at 64-tile items and a few per cent slower below two items per SM (its one-time
+    // set-up and the coarser balance of a short list).  d = 192 has no room for its staging buffer.
+    const long long n_items = static_cast<long long>((n_q_tiles + 1) / 2) * Hq * B;
+    const int longest = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, causal);
+    const bool persistent_ok = !varlen && pair_splits == 1 && dqk != 192 && !drop;
+    bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= 32;
+    if (flags & FA_FLAG_NO_PERSISTENT) persistent = false;
+    if ((flags & FA_FLAG_FORCE_PERSISTENT) && persistent_ok) persistent = true;
+    // One query tile per CTA (twice the CTAs, each with a shorter chain) wins where the pair
+    // kernel's grid does not fill the GPU or its longest CTA dominates: decided from the two
+    // estimates, with a margin, each side with its own split count.
+    bool stream = false;
+    int stream_splits = 1;
+    if (!drop && !(flags & FA_FLAG_NO_STREAM_KERNEL)) {
+        if (!varlen) stream_splits = choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles, true);
+        if (flags & FA_FLAG_STREAM_KERNEL) {
+            stream = true;
+        } else if (varlen) {
+            stream = (dqk == 192);       // no estimate without the lengths; 192/128 is always ahead
+        } else if (!persistent) {
+            const TilingEstimate e = estimate_tilings(num_sms, B, Hq, Sq, Sk, dqk, causal, n_q_tiles, pair_splits, stream_splits);
+            pl.pair_us = e.pair_us;
+            pl.stream_us = e.stream_us;
+            stream = e.stream_us < 0.9 * e.pair_us;
+            // at d = 64 the stream kernel is also 3-7 % ahead on long items (measured from 64
+            // K/V tiles per query tile on), closer than the estimate can tell
+            if (dqk == 64 && longest >= 32 && pair_splits == 1 && stream_splits == 1) stream = true;
+        }
+    }
+    if (stream) {
+        pl.kernel = kPlanStream;
+        with_splits(stream_splits);
+    } else if (persistent) {
+        pl.kernel = kPlanPersistent;
+    } else {
+        pl.kernel = kPlanPair;
+        with_splits(pair_splits);
+    }
+    return pl;
+}
+
 // Fills the launch parameters and starts the kernel(s); the tensor maps are ready.
 // cu_q == nullptr: fixed lengths Sq, Sk.  Otherwise a packed variable-length batch whose longest
 // query is Sq rows and whose sequences have about Sk keys (L2 grouping only).
@@ -384,94 +460,38 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
     p.status = h->status_dev;
     p.wait_limit_ns = h->wait_limit_ns;
     p.debug_drop_v_load = (h->flags & FA_FLAG_DEBUG_DROP_V_LOAD) ? 1 : 0;
-    p.kv_splits = 1;
-    p.tiles_per_split = 0x3fffffff;
+    const LaunchPlan pl = plan_launch(h->num_sms, h->flags, h->kv_splits_cfg, h->scratch_bytes, cu_q != nullptr,
+                                      B, Hq, Sq, Sk, dqk, dv, p.causal);
+    p.kv_splits = pl.kv_splits;
+    p.tiles_per_split = pl.tiles_per_split;
     p.o_part = nullptr;
     p.lse_part = nullptr;
-    if (!(h->flags & FA_FLAG_SERIAL_KERNEL) && !cu_q) {   // packed batches: no split (lengths are on the device)
-        const int splits = choose_kv_splits(h, B, Hq, Sq, Sk, dv, p.causal, p.n_q_tiles);
-        if (splits > 1) {
-            int max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
-            if (p.causal) {
-                const int t = fa::kv_tiles_for_q_tile((p.n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, 1);
-                if (t < max_tiles) max_tiles = t;
-            }
-            p.kv_splits = splits;
-            p.tiles_per_split = (max_tiles + splits - 1) / splits;
-            p.o_part = static_cast<float*>(h->scratch);
-            p.lse_part = p.o_part + static_cast<size_t>(splits) * B * Hq * Sq * dv;
-        }
+    if (pl.kv_splits > 1) {
+        p.o_part = static_cast<float*>(h->scratch);
+        p.lse_part = p.o_part + static_cast<size_t>(pl.kv_splits) * B * Hq * Sq * dv;
     }
     h->last_splits = p.kv_splits;
 #ifdef FA_TRACE
     p.trace = h->trace;
 #endif
 
-    if (!(h->flags & FA_FLAG_SERIAL_KERNEL)) {
-        // The persistent kernel wins where a CTA's fixed cost is a visible share of an item's time
-        // and every SM gets several items: measured on B200 it is 5-20 % faster from about three
-        // items per SM on, level at 64-tile items and a few per cent slower below two items per SM
-        // (its one-time set-up and the coarser balance of a short list).  d = 192 has no room for
-        // its staging buffer.
-        const long long n_items = static_cast<long long>((p.n_q_tiles + 1) / 2) * Hq * B;
-        const int longest = fa::kv_tiles_for_q_tile((p.n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, p.causal);
-        bool persistent = !cu_q && p.kv_splits == 1 && dqk != 192 && !p.debug_drop_v_load &&
-                          n_items >= 3ll * h->num_sms && longest <= 32;
-        if (h->flags & FA_FLAG_NO_PERSISTENT) persistent = false;
-        if ((h->flags & FA_FLAG_FORCE_PERSISTENT) && !cu_q && p.kv_splits == 1 && dqk != 192 && !p.debug_drop_v_load)
-            persistent = true;
-        // One query tile per CTA (twice the CTAs, each with a shorter chain) wins where the pair
-        // kernel's grid does not fill the GPU or its longest CTA dominates: decided from the two
-        // estimates, with a margin, before the K/V range is split.
-        bool stream = false;
-        int stream_splits = 1;
-        if (!p.debug_drop_v_load && !(h->flags & FA_FLAG_NO_STREAM_KERNEL)) {
-            if (!cu_q) stream_splits = choose_kv_splits(h, B, Hq, Sq, Sk, dv, p.causal, p.n_q_tiles, true);
-            if (h->flags & FA_FLAG_STREAM_KERNEL) {
-                stream = true;
-            } else if (cu_q) {
-                stream = (dqk == 192);       // lengths are on the device: no estimate; 192/128 is always ahead
-            } else if (!persistent) {
-                const TilingEstimate e = estimate_tilings(h->num_sms, B, Hq, Sq, Sk, dqk, p.causal, p.n_q_tiles, p.kv_splits,
-                                                          stream_splits);
-                stream = e.stream_us < 0.9 * e.pair_us;
-                // at d = 64 the stream kernel is also 3-7 % ahead on long items (measured from 64
-                // K/V tiles per query tile on), closer than the estimate can tell
-                if (dqk == 64 && longest >= 32 && p.kv_splits == 1 && stream_splits == 1) stream = true;
-            }
+    if (pl.kernel == kPlanStream) {
+        h->last_kernel = "fa_fwd_stream";
+        if (cu_q) {
+            if (dqk == 64) return launch_stream<64, 64, true>(h, 19, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_stream<128, 128, true>(h, 20, map_q, map_k, map_v, map_o, p, st);
+            return launch_stream<192, 128, true>(h, 21, map_q, map_k, map_v, map_o, p, st);
         }
-        if (stream) {
-            p.kv_splits = 1;
-            p.tiles_per_split = 0x3fffffff;
-            p.o_part = nullptr;
-            p.lse_part = nullptr;
-            if (stream_splits > 1) {
-                int max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
-                if (p.causal) {
-                    const int t = fa::kv_tiles_for_q_tile((p.n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, 1);
-                    if (t < max_tiles) max_tiles = t;
-                }
-                p.kv_splits = stream_splits;
-                p.tiles_per_split = (max_tiles + stream_splits - 1) / stream_splits;
-                p.o_part = static_cast<float*>(h->scratch);
-                p.lse_part = p.o_part + static_cast<size_t>(stream_splits) * B * Hq * Sq * dv;
-            }
-            h->last_splits = p.kv_splits;
-            h->last_kernel = "fa_fwd_stream";
-            if (cu_q) {
-                if (dqk == 64) return launch_stream<64, 64, true>(h, 19, map_q, map_k, map_v, map_o, p, st);
-                if (dqk == 128) return launch_stream<128, 128, true>(h, 20, map_q, map_k, map_v, map_o, p, st);
-                return launch_stream<192, 128, true>(h, 21, map_q, map_k, map_v, map_o, p, st);
-            }
-            if (dqk == 64) return launch_stream<64, 64>(h, 16, map_q, map_k, map_v, map_o, p, st);
-            if (dqk == 128) return launch_stream<128, 128>(h, 17, map_q, map_k, map_v, map_o, p, st);
-            return launch_stream<192, 128>(h, 18, map_q, map_k, map_v, map_o, p, st);
-        }
-        if (persistent) {
-            h->last_kernel = "fa_fwd_persistent";
-            if (dqk == 64) return launch_persistent<64, 64>(h, 9, map_q, map_k, map_v, map_o, p, st);
-            return launch_persistent<128, 128>(h, 10, map_q, map_k, map_v, map_o, p, st);
-        }
+        if (dqk == 64) return launch_stream<64, 64>(h, 16, map_q, map_k, map_v, map_o, p, st);
+        if (dqk == 128) return launch_stream<128, 128>(h, 17, map_q, map_k, map_v, map_o, p, st);
+        return launch_stream<192, 128>(h, 18, map_q, map_k, map_v, map_o, p, st);
+    }
+    if (pl.kernel == kPlanPersistent) {
+        h->last_kernel = "fa_fwd_persistent";
+        if (dqk == 64) return launch_persistent<64, 64>(h, 9, map_q, map_k, map_v, map_o, p, st);
+        return launch_persistent<128, 128>(h, 10, map_q, map_k, map_v, map_o, p, st);
+    }
+    if (pl.kernel == kPlanPair) {
         h->last_kernel = "fa_fwd_pipelined";
         if (cu_q) {
             if (dqk == 64) return launch_pipelined<64, 64, true>(h, 6, map_q, map_k, map_v, map_o, p, st);
@@ -765,6 +785,38 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     cfg.numAttrs = (h->flags & FA_FLAG_NO_DEPENDENT_LAUNCH) ? 0 : 1;
     if (cudaLaunchKernelEx(&cfg, fa::fa_fwd_fp8_kernel, map_q, map_k, map_v, map_o, p, f) != cudaSuccess) return FA_ERR_CUDA;
     h->launches += 1;
+    return FA_OK;
+}
+
+fa_status fa_plan(int num_sms, const fa_config* cfg, int varlen, int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv,
+                  int causal, fa_plan_info* out) {
+    if (!out || num_sms <= 0 || B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || Hq % Hkv != 0) return FA_ERR_INVALID_ARG;
+    const bool dims_ok = (dqk == 64 && dv == 64) || (dqk == 128 && dv == 128) || (dqk == 192 && dv == 128);
+    if (!dims_ok) return FA_ERR_UNSUPPORTED;
+    uint32_t flags = 0, splits_cfg = 0;
+    uint64_t scratch = 32ull << 20;
+    if (cfg) {
+        if (cfg->struct_size < 16) return FA_ERR_INVALID_ARG;
+        flags = cfg->flags;
+        if (cfg->struct_size >= 20) splits_cfg = cfg->kv_splits;
+        if (cfg->struct_size >= sizeof(fa_config) && cfg->scratch_bytes) scratch = cfg->scratch_bytes;
+    }
+    const LaunchPlan pl = plan_launch(num_sms, flags, splits_cfg, static_cast<size_t>(scratch), varlen != 0,
+                                      B, Hq, Sq, Sk, dqk, dv, causal ? 1 : 0);
+    static const char* const names[4] = {"fa_fwd_simple", "fa_fwd_pipelined", "fa_fwd_persistent", "fa_fwd_stream"};
+    out->kernel = names[pl.kernel];
+    out->kv_splits = pl.kv_splits;
+    const long long n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
+    long long ctas = 0;
+    switch (pl.kernel) {
+        case kPlanSerial: ctas = n_q_tiles * Hq * B; break;
+        case kPlanPair: ctas = ((n_q_tiles + 1) / 2) * Hq * B * pl.kv_splits; break;
+        case kPlanPersistent: ctas = ((n_q_tiles + 1) / 2) * Hq * B; if (ctas > num_sms) ctas = num_sms; break;
+        default: ctas = n_q_tiles * Hq * B * pl.kv_splits; break;
+    }
+    out->ctas = ctas;
+    out->estimate_pair_us = pl.pair_us;
+    out->estimate_stream_us = pl.stream_us;
     return FA_OK;
 }
 

@@ -1,0 +1,71 @@
+"""fa_plan: the host-side choice of kernel, tiling and split count (no GPU needed).
+
+The expectations are the measured outcomes recorded for the B200 (148 SMs): the benchmark
+configurations, the paper's Table 6 rows and the decode-like shapes."""
+import pytest
+
+from paper_2609_21264_b200 import binding, workloads as W
+
+SMS = 148
+
+
+def plan(w, **kw):
+    return binding.fa_plan(SMS, w.B, w.Hq, w.Hkv, w.Sq, w.Sk, w.dqk, w.dv, w.causal, **kw)
+
+
+def test_benchmark_configurations():
+    expect = ["fa_fwd_stream", "fa_fwd_pipelined", "fa_fwd_pipelined", "fa_fwd_stream", "fa_fwd_pipelined"]
+    for w, kernel in zip(W.CONFIGS, expect):
+        p = plan(w)
+        assert p["kernel"] == kernel, (w.name, p)
+        assert p["kv_splits"] == 1
+    # grid sizes: one CTA per query tile or per pair of query tiles
+    assert plan(W.CONFIGS[0])["ctas"] == 12 * 4
+    assert plan(W.CONFIGS[1])["ctas"] == 32 * 8
+    assert plan(W.CONFIGS[3])["ctas"] == 128 * 32
+
+
+def test_table6_rows():
+    got = {w.name: plan(w)["kernel"] for w, _ in W.TABLE6}
+    assert got["gpt2_small_s2048"] == "fa_fwd_stream"          # 96 causal pairs: under a wave
+    assert got["bert_base_s2048"] == "fa_fwd_pipelined"        # 192 equal tiles would make two waves
+    assert got["llama3_8b_s2048"] == "fa_fwd_pipelined"
+    assert got["qwen15_05b_s32768"] == "fa_fwd_stream"         # d = 64 with long items
+    assert got["deepseek_67b_gqa_s4096"] == "fa_fwd_persistent"  # 1024 short items
+
+
+def test_decode_like_shapes_split_the_kv_range_on_the_stream_kernel():
+    p = binding.fa_plan(SMS, 1, 32, 8, 128, 32768, 128, 128, False)
+    assert p["kernel"] == "fa_fwd_stream" and p["kv_splits"] == 4 and p["ctas"] == 32 * 4
+    p = binding.fa_plan(SMS, 8, 32, 8, 1, 8192, 128, 128, False)
+    assert p["kernel"] == "fa_fwd_stream" and p["ctas"] == 256 * p["kv_splits"]
+    assert p["estimate_stream_us"] < p["estimate_pair_us"]
+
+
+def test_flags_and_configuration_override_the_choice():
+    w = W.CONFIGS[1]
+    assert plan(w, flags=binding.FA_FLAG_STREAM_KERNEL)["kernel"] == "fa_fwd_stream"
+    assert plan(w, flags=binding.FA_FLAG_FORCE_PERSISTENT | binding.FA_FLAG_NO_STREAM_KERNEL)["kernel"] == "fa_fwd_persistent"
+    assert plan(w, flags=binding.FA_FLAG_SERIAL_KERNEL)["kernel"] == "fa_fwd_simple"
+    assert plan(W.CONFIGS[0], flags=binding.FA_FLAG_NO_STREAM_KERNEL)["kernel"] == "fa_fwd_pipelined"
+    # a forced split count is honoured as far as the scratch buffer holds the partials
+    p = binding.fa_plan(SMS, 1, 32, 8, 128, 32768, 128, 128, False, kv_splits=7)
+    assert p["kv_splits"] == 7
+    p = binding.fa_plan(SMS, 1, 32, 8, 128, 32768, 128, 128, False, kv_splits=7, scratch_bytes=5 * 32 * 128 * 129 * 4)
+    assert p["kv_splits"] == 5
+    assert binding.fa_plan(SMS, 1, 32, 8, 128, 32768, 128, 128, False, kv_splits=1)["kv_splits"] == 1
+
+
+def test_packed_batches_and_head_size_192():
+    assert binding.fa_plan(SMS, 4, 16, 4, 2048, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_pipelined"
+    assert binding.fa_plan(SMS, 4, 16, 4, 2048, 1024, 192, 128, True, varlen=True)["kernel"] == "fa_fwd_stream"
+    assert binding.fa_plan(SMS, 1, 16, 16, 2048, 2048, 192, 128, True)["kernel"] == "fa_fwd_stream"
+
+
+def test_argument_errors():
+    with pytest.raises(binding.FaError):
+        binding.fa_plan(SMS, 1, 3, 2, 128, 128, 128, 128, False)        # Hq not a multiple of Hkv
+    with pytest.raises(binding.FaError):
+        binding.fa_plan(SMS, 1, 2, 2, 128, 128, 96, 96, False)          # no kernel for this head size
+    with pytest.raises(binding.FaError):
+        binding.fa_plan(0, 1, 2, 2, 128, 128, 128, 128, False)
