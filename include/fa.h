@@ -85,6 +85,13 @@ typedef enum fa_status {
  * it on (fixed-length problems) or off. */
 #define FA_FLAG_STREAM_KERNEL 32u
 #define FA_FLAG_NO_STREAM_KERNEL 64u
+/* With at most 64 queries per sequence and several query heads per K/V head (decoding with
+ * grouped-query attention), the stream kernel puts the rows of several heads of a group into one
+ * query tile, so every K/V tile is fetched and multiplied once for all of them: the largest
+ * divisor h of the group size with h * Sq <= 128 heads share a tile.  Results are those of the
+ * unpacked launch up to fp32 rounding order (a row's arithmetic does not depend on its
+ * neighbours).  This flag turns the packing off. */
+#define FA_FLAG_NO_HEAD_PACKING 128u
 
 /* Optional creation parameters.  Zero-initialise, set struct_size = sizeof(fa_config). */
 typedef struct fa_config {
@@ -229,6 +236,7 @@ typedef struct fa_plan_info {
     const char* kernel;          /* "fa_fwd_pipelined", "fa_fwd_stream", "fa_fwd_persistent", "fa_fwd_simple" */
     int32_t kv_splits;           /* CTAs per work item along the K/V range (1 = no split)        */
     int64_t ctas;                /* grid size of the attention kernel                            */
+    int32_t heads_per_tile;      /* query heads sharing a query tile (1 = none; see FA_FLAG_NO_HEAD_PACKING) */
     double estimate_pair_us;     /* estimated time with one CTA per pair of query tiles          */
     double estimate_stream_us;   /* estimated time with one CTA per query tile                   */
 } fa_plan_info;

@@ -27,6 +27,7 @@ FA_FLAG_NO_PERSISTENT = 8
 FA_FLAG_FORCE_PERSISTENT = 16
 FA_FLAG_STREAM_KERNEL = 32
 FA_FLAG_NO_STREAM_KERNEL = 64
+FA_FLAG_NO_HEAD_PACKING = 128
 
 EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_varlen", "fa_forward_fp8", "fa_plan", "fa_forward_host", "fa_last_status", "fa_destroy",
            "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits",
@@ -54,7 +55,7 @@ def library_path() -> str:
 
 class fa_plan_info(ctypes.Structure):
     _fields_ = [("kernel", ctypes.c_char_p), ("kv_splits", ctypes.c_int32), ("ctas", ctypes.c_int64),
-                ("estimate_pair_us", ctypes.c_double), ("estimate_stream_us", ctypes.c_double)]
+                ("heads_per_tile", ctypes.c_int32), ("estimate_pair_us", ctypes.c_double), ("estimate_stream_us", ctypes.c_double)]
 
 
 def load():
@@ -153,7 +154,7 @@ def fa_plan(num_sms, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, *, varlen=False, flags
                         ctypes.byref(out))
     if st != FA_OK:
         raise FaError(st, "fa_plan")
-    return {"kernel": out.kernel.decode(), "kv_splits": out.kv_splits, "ctas": out.ctas,
+    return {"kernel": out.kernel.decode(), "kv_splits": out.kv_splits, "ctas": out.ctas, "heads_per_tile": out.heads_per_tile,
             "estimate_pair_us": out.estimate_pair_us, "estimate_stream_us": out.estimate_stream_us}
 
 

@@ -16,6 +16,7 @@
 #include "fa_fwd_persistent.cuh"
 #include "fa_fwd_stream.cuh"
 #include "fa_fwd_fp8.cuh"
+#include "fa_fwd_fp8_stream.cuh"
 #include "fa_fwd_simple.cuh"
 
 namespace {
@@ -27,7 +28,7 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
 
 struct MapEntry {
     const void* ptr;
-    int d, S, H, B, box_rows, elem_bytes;
+    int d, S, H, B, box_rows, box_heads, elem_bytes;
     long long sb, sh, ss;      // batch / head / row strides in elements
     uint64_t stamp;
     CUtensorMap map;
@@ -56,7 +57,7 @@ struct fa_handle {
     const char* last_kernel = "";
     void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // Q K V O lse
     size_t stage_cap[5] = {0, 0, 0, 0, 0};
-    bool attr_done[24] = {};
+    bool attr_done[32] = {};
 #ifdef FA_TRACE
     long long* trace = nullptr;
 #endif
@@ -82,10 +83,10 @@ class DeviceGuard {
 // ptr + b*sb + h*sh + s*ss + c, seen as a 4-D TMA tensor (d, S, H, B); box = 128 bytes of columns
 // x box_rows rows, 128-byte swizzle, rows past S read as zero.
 fa_status get_map(fa_handle* h, const void* ptr, int d, int S, int H, int B, long long sb, long long sh,
-                  long long ss, int box_rows, const CUtensorMap** out, int elem_bytes = 2) {
+                  long long ss, int box_rows, const CUtensorMap** out, int elem_bytes = 2, int box_heads = 1) {
     for (auto& e : h->maps) {
         if (e.ptr == ptr && e.d == d && e.S == S && e.H == H && e.B == B && e.box_rows == box_rows &&
-            e.sb == sb && e.sh == sh && e.ss == ss && e.elem_bytes == elem_bytes) {
+            e.sb == sb && e.sh == sh && e.ss == ss && e.elem_bytes == elem_bytes && e.box_heads == box_heads) {
             e.stamp = ++h->stamp;
             *out = &e.map;
             return FA_OK;
@@ -94,13 +95,14 @@ fa_status get_map(fa_handle* h, const void* ptr, int d, int S, int H, int B, lon
     MapEntry ne;
     memset(&ne, 0, sizeof ne);
     ne.ptr = ptr; ne.d = d; ne.S = S; ne.H = H; ne.B = B; ne.box_rows = box_rows;
-    ne.sb = sb; ne.sh = sh; ne.ss = ss; ne.elem_bytes = elem_bytes;
+    ne.sb = sb; ne.sh = sh; ne.ss = ss; ne.elem_bytes = elem_bytes; ne.box_heads = box_heads;
     const cuuint64_t eb = static_cast<cuuint64_t>(elem_bytes);
     const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(S),
                                 static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(B)};
     const cuuint64_t strides[3] = {static_cast<cuuint64_t>(ss) * eb, static_cast<cuuint64_t>(sh) * eb,
                                    static_cast<cuuint64_t>(sb) * eb};
-    const cuuint32_t box[4] = {static_cast<cuuint32_t>(128 / elem_bytes), static_cast<cuuint32_t>(box_rows), 1u, 1u};
+    const cuuint32_t box[4] = {static_cast<cuuint32_t>(128 / elem_bytes), static_cast<cuuint32_t>(box_rows),
+                              static_cast<cuuint32_t>(box_heads), 1u};
     const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
     const CUresult r = h->encode(&ne.map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
                                  4, const_cast<void*>(ptr),
@@ -192,8 +194,8 @@ fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const 
 // Number of K/V splits for a problem: 1 unless the query tiles alone leave most SMs idle and the
 // K/V range is long enough to cut; never more than the scratch buffer can hold partials for.
 int choose_kv_splits(int num_sms, uint32_t kv_splits_cfg, size_t scratch_bytes, int B, int Hq, int Sq, int Sk, int dv,
-                     int causal, int n_q_tiles, bool one_tile_items = false) {
-    const long long items = static_cast<long long>(one_tile_items ? n_q_tiles : (n_q_tiles + 1) / 2) * B * Hq;
+                     int causal, int n_q_tiles, bool one_tile_items = false, int heads_per_item = 1) {
+    const long long items = static_cast<long long>(one_tile_items ? n_q_tiles : (n_q_tiles + 1) / 2) * B * (Hq / heads_per_item);
     int max_tiles = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, causal);
     if (!causal) max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
     int splits = 1;
@@ -279,15 +281,16 @@ fa_status launch_persistent(fa_handle* h, int slot, const CUtensorMap& mq, const
 }
 
 // One query tile per CTA, K/V tiles streamed through two softmax warpgroups.
-template <int DQK, int DV, bool kVarlen = false>
+template <int DQK, int DV, bool kVarlen = false, bool kPack = false>
 fa_status launch_stream(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
                         const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
     constexpr int smem = fa::stream_smem_bytes<DQK, DV>();
     static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
-    auto kernel = fa::fa_fwd_stream_kernel<DQK, DV, kVarlen>;
+    auto kernel = fa::fa_fwd_stream_kernel<DQK, DV, kVarlen, kPack>;
     fa_status s = ensure_smem_attr(h, slot, kernel, smem);
     if (s != FA_OK) return s;
-    const long long n_ctas = static_cast<long long>(p.n_q_tiles) * p.Hq * p.B * p.kv_splits;
+    // items: query tiles x heads, or packs of heads with their single query tile
+    const long long n_ctas = (kPack ? static_cast<long long>(p.Hq / p.pack_heads) : static_cast<long long>(p.n_q_tiles) * p.Hq) * p.B * p.kv_splits;
     if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -365,14 +368,16 @@ struct LaunchPlan {
     int kernel;
     int kv_splits;
     int tiles_per_split;
+    int pack_heads;                // > 1: stream kernel with that many query heads of a K/V head per query tile
     double pair_us, stream_us;     // the two estimates (0 when no estimate was needed)
 };
 LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size_t scratch_bytes, bool varlen,
-                       int B, int Hq, int Sq, int Sk, int dqk, int dv, int causal) {
+                       int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal) {
     LaunchPlan pl;
     pl.kernel = kPlanPair;
     pl.kv_splits = 1;
     pl.tiles_per_split = 0x3fffffff;
+    pl.pack_heads = 1;
     pl.pair_us = pl.stream_us = 0.0;
     const int n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
     const bool drop = (flags & FA_FLAG_DEBUG_DROP_V_LOAD) != 0;
@@ -388,6 +393,23 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     if (flags & FA_FLAG_SERIAL_KERNEL) {
         pl.kernel = kPlanSerial;
         return pl;
+    }
+    // Few queries per sequence and several query heads per K/V head (decoding with grouped-query
+    // attention): the heads of a group share the CTA's query tile, h heads of Sq rows each with
+    // h the largest divisor of the group size that fits, and every K/V tile is read and
+    // multiplied once for all of them.  Only the stream kernel has this mode.
+    if (!varlen && !drop && !(flags & (FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)) && Sq <= fa::kTileM / 2 &&
+        Hq / Hkv >= 2) {
+        const int group = Hq / Hkv;
+        int hp = 1;
+        for (int c = 2; c <= group && c * Sq <= fa::kTileM; ++c)
+            if (group % c == 0) hp = c;
+        if (hp > 1) {
+            pl.kernel = kPlanStream;
+            pl.pack_heads = hp;
+            with_splits(choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles, true, hp));
+            return pl;
+        }
     }
     // packed batches: no split (the lengths that decide it are on the device)
     const int pair_splits = varlen ? 1 : choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles);
@@ -440,7 +462,7 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
 fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap& map_k, const CUtensorMap& map_v,
                       const CUtensorMap& map_o, void* O, float* lse, int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal,
                       float scale, const int64_t* o_strides, const int* cu_q, const int* cu_k, int total_q,
-                      cudaStream_t st) {
+                      const LaunchPlan& pl, cudaStream_t st) {
     if (scale == 0.f) scale = 1.f / sqrtf(static_cast<float>(dqk));
     fa::FwdParams p;
     p.O = static_cast<__nv_bfloat16*>(O);
@@ -460,10 +482,9 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
     p.status = h->status_dev;
     p.wait_limit_ns = h->wait_limit_ns;
     p.debug_drop_v_load = (h->flags & FA_FLAG_DEBUG_DROP_V_LOAD) ? 1 : 0;
-    const LaunchPlan pl = plan_launch(h->num_sms, h->flags, h->kv_splits_cfg, h->scratch_bytes, cu_q != nullptr,
-                                      B, Hq, Sq, Sk, dqk, dv, p.causal);
     p.kv_splits = pl.kv_splits;
     p.tiles_per_split = pl.tiles_per_split;
+    p.pack_heads = pl.pack_heads;
     p.o_part = nullptr;
     p.lse_part = nullptr;
     if (pl.kv_splits > 1) {
@@ -477,6 +498,11 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
 
     if (pl.kernel == kPlanStream) {
         h->last_kernel = "fa_fwd_stream";
+        if (pl.pack_heads > 1) {
+            if (dqk == 64) return launch_stream<64, 64, false, true>(h, 23, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_stream<128, 128, false, true>(h, 24, map_q, map_k, map_v, map_o, p, st);
+            return launch_stream<192, 128, false, true>(h, 25, map_q, map_k, map_v, map_o, p, st);
+        }
         if (cu_q) {
             if (dqk == 64) return launch_stream<64, 64, true>(h, 19, map_q, map_k, map_v, map_o, p, st);
             if (dqk == 128) return launch_stream<128, 128, true>(h, 20, map_q, map_k, map_v, map_o, p, st);
@@ -542,7 +568,7 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg) {
         if (cfg->struct_size >= sizeof(fa_config)) scratch_bytes = cfg->scratch_bytes;
         if (flags & ~(FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD | FA_FLAG_NO_DEPENDENT_LAUNCH |
                       FA_FLAG_NO_PERSISTENT | FA_FLAG_FORCE_PERSISTENT | FA_FLAG_STREAM_KERNEL |
-                      FA_FLAG_NO_STREAM_KERNEL)) return FA_ERR_INVALID_ARG;
+                      FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)) return FA_ERR_INVALID_ARG;
         if (kv_splits_cfg > 64) return FA_ERR_INVALID_ARG;
     }
     if (scratch_bytes == 0) scratch_bytes = 32ull << 20;
@@ -660,17 +686,21 @@ fa_status fa_forward_strided(fa_handle* h, const void* Q, const void* K, const v
     if (!guard.ok()) return FA_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;
-    if ((s = get_map(h, Q, dqk, Sq, Hq, B, q_strides[0], q_strides[1], q_strides[2], fa::kTileM, &mq)) != FA_OK) return s;
+    const LaunchPlan pl = plan_launch(h->num_sms, h->flags, h->kv_splits_cfg, h->scratch_bytes, false,
+                                      B, Hq, Hkv, Sq, Sk, dqk, dv, causal ? 1 : 0);
+    // packed heads: the box of Q and O is the Sq rows of pack_heads heads
+    const int q_box_rows = pl.pack_heads > 1 ? Sq : fa::kTileM;
+    if ((s = get_map(h, Q, dqk, Sq, Hq, B, q_strides[0], q_strides[1], q_strides[2], q_box_rows, &mq, 2, pl.pack_heads)) != FA_OK) return s;
     CUtensorMap map_q = *mq;   // copies: a later insertion may evict or move cache entries
     if ((s = get_map(h, K, dqk, Sk, Hkv, B, k_strides[0], k_strides[1], k_strides[2], fa::kTileN, &mk)) != FA_OK) return s;
     CUtensorMap map_k = *mk;
     if ((s = get_map(h, V, dv, Sk, Hkv, B, v_strides[0], v_strides[1], v_strides[2], fa::kTileN, &mv)) != FA_OK) return s;
     CUtensorMap map_v = *mv;
-    if ((s = get_map(h, O, dv, Sq, Hq, B, o_strides[0], o_strides[1], o_strides[2], fa::kTileM, &mo)) != FA_OK) return s;
+    if ((s = get_map(h, O, dv, Sq, Hq, B, o_strides[0], o_strides[1], o_strides[2], q_box_rows, &mo, 2, pl.pack_heads)) != FA_OK) return s;
     CUtensorMap map_o = *mo;
 
     return run_forward(h, map_q, map_k, map_v, map_o, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, o_strides,
-                       nullptr, nullptr, 0, st);
+                       nullptr, nullptr, 0, pl, st);
 }
 
 fa_status fa_forward(fa_handle* h, const void* Q, const void* K, const void* V, void* O, float* lse,
@@ -715,8 +745,10 @@ fa_status fa_forward_varlen(fa_handle* h, const void* Q, const void* K, const vo
     CUtensorMap map_o = *mo;
     const int64_t os[3] = {0, dv, static_cast<int64_t>(Hq) * dv};
     const int mean_sk = (total_k + B - 1) / B > 0 ? (total_k + B - 1) / B : 1;
+    const LaunchPlan pl = plan_launch(h->num_sms, h->flags, h->kv_splits_cfg, h->scratch_bytes, true,
+                                      B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal ? 1 : 0);
     return run_forward(h, map_q, map_k, map_v, map_o, O, lse, B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal, scale, os,
-                       cu_seqlens_q, cu_seqlens_k, total_q, st);
+                       cu_seqlens_q, cu_seqlens_k, total_q, pl, st);
 }
 
 fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const void* V8,
@@ -735,15 +767,21 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (scale == 0.f) scale = 1.f / sqrtf(static_cast<float>(d));
 
+    // The tiling is planned as for 16-bit operands of the same shape (the 8-bit kernels' per-CTA
+    // costs are lower by a similar factor in both tilings).  Only the stream tiling splits K/V
+    // and packs heads.
+    const LaunchPlan pl = plan_launch(h->num_sms, h->flags, h->kv_splits_cfg, h->scratch_bytes, false,
+                                      B, Hq, Hkv, Sq, Sk, d, d, causal ? 1 : 0);
+    const int q_box_rows = pl.pack_heads > 1 ? Sq : fa::kTileM;
     const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;
     const long long hq_stride = static_cast<long long>(Sq) * d, hk_stride = static_cast<long long>(Sk) * d;
-    if ((s = get_map(h, Q8, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, fa::kTileM, &mq, 1)) != FA_OK) return s;
+    if ((s = get_map(h, Q8, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, q_box_rows, &mq, 1, pl.pack_heads)) != FA_OK) return s;
     CUtensorMap map_q = *mq;
     if ((s = get_map(h, K8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mk, 1)) != FA_OK) return s;
     CUtensorMap map_k = *mk;
     if ((s = get_map(h, V8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mv, 1)) != FA_OK) return s;
     CUtensorMap map_v = *mv;
-    if ((s = get_map(h, O, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, fa::kTileM, &mo, 2)) != FA_OK) return s;
+    if ((s = get_map(h, O, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, q_box_rows, &mo, 2, pl.pack_heads)) != FA_OK) return s;
     CUtensorMap map_o = *mo;
 
     fa::FwdParams p;
@@ -758,31 +796,64 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     p.scale_log2 = scale * 1.4426950408889634f;
     p.n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
     p.heads_per_group = heads_per_group(static_cast<long long>(Sk) * 2 * d, B, Hq, Hkv);      // one byte per element
-    p.kv_splits = 1;
-    p.tiles_per_split = 0x3fffffff;
     p.status = h->status_dev;
     p.wait_limit_ns = h->wait_limit_ns;
     fa::Fp8Params f;
     f.q_scale = q_scale; f.k_scale = k_scale; f.v_scale = v_scale;
     f.n_kv_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
-    h->last_splits = 1;
-    h->last_kernel = "fa_fwd_fp8";
+    const bool use_stream = pl.kernel == kPlanStream;
+    p.kv_splits = use_stream ? pl.kv_splits : 1;
+    p.tiles_per_split = use_stream ? pl.tiles_per_split : 0x3fffffff;
+    p.pack_heads = pl.pack_heads;
+    if (p.kv_splits > 1) {
+        p.o_part = static_cast<float*>(h->scratch);
+        p.lse_part = p.o_part + static_cast<size_t>(p.kv_splits) * B * Hq * Sq * d;
+    }
+    h->last_splits = p.kv_splits;
+    h->last_kernel = use_stream ? "fa_fwd_fp8_stream" : "fa_fwd_fp8";
 
-    constexpr int smem = fa::fp8_smem_bytes();
-    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
-    if ((s = ensure_smem_attr(h, 11, fa::fa_fwd_fp8_kernel, smem)) != FA_OK) return s;
-    const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * Hq * B;
-    if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
-    cfg.blockDim = dim3(fa::Fp8Cfg::kThreads, 1, 1);
-    cfg.dynamicSmemBytes = smem;
+    cfg.blockDim = dim3(512, 1, 1);
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = (h->flags & FA_FLAG_NO_DEPENDENT_LAUNCH) ? 0 : 1;
+    if (use_stream) {
+        constexpr int smem = fa::fp8_stream_smem_bytes();
+        static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+        const bool pack = pl.pack_heads > 1;
+        auto kernel = pack ? fa::fa_fwd_fp8_stream_kernel<true> : fa::fa_fwd_fp8_stream_kernel<false>;
+        if ((s = ensure_smem_attr(h, pack ? 26 : 22, kernel, smem)) != FA_OK) return s;
+        const long long n_ctas = (pack ? static_cast<long long>(Hq / pl.pack_heads) : static_cast<long long>(p.n_q_tiles) * Hq) * B * p.kv_splits;
+        if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+        cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
+        cfg.dynamicSmemBytes = smem;
+        if (cudaLaunchKernelEx(&cfg, kernel, map_q, map_k, map_v, map_o, p, f) != cudaSuccess) return FA_ERR_CUDA;
+        h->launches += 1;
+        if (p.kv_splits > 1) {
+            const long long n_rows = static_cast<long long>(B) * Hq * Sq;
+            const long long blocks = (n_rows + 3) / 4;
+            if (blocks > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+            cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+            cfg.blockDim = dim3(128, 1, 1);
+            cfg.dynamicSmemBytes = 0;
+            if (cudaLaunchKernelEx(&cfg, fa::fa_combine_kernel<128>, static_cast<const float*>(p.o_part),
+                                   static_cast<const float*>(p.lse_part), p.O, p.lse, n_rows, p.kv_splits, p.Hq, p.Sq,
+                                   p.o_stride_b, p.o_stride_h, p.o_stride_s) != cudaSuccess) return FA_ERR_CUDA;
+            h->launches += 1;
+        }
+        return FA_OK;
+    }
+    constexpr int smem = fa::fp8_smem_bytes();
+    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+    static_assert(fa::Fp8Cfg::kThreads == 512, "block size");
+    if ((s = ensure_smem_attr(h, 11, fa::fa_fwd_fp8_kernel, smem)) != FA_OK) return s;
+    const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * Hq * B;
+    if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+    cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
+    cfg.dynamicSmemBytes = smem;
     if (cudaLaunchKernelEx(&cfg, fa::fa_fwd_fp8_kernel, map_q, map_k, map_v, map_o, p, f) != cudaSuccess) return FA_ERR_CUDA;
     h->launches += 1;
     return FA_OK;
@@ -802,17 +873,18 @@ fa_status fa_plan(int num_sms, const fa_config* cfg, int varlen, int B, int Hq, 
         if (cfg->struct_size >= sizeof(fa_config) && cfg->scratch_bytes) scratch = cfg->scratch_bytes;
     }
     const LaunchPlan pl = plan_launch(num_sms, flags, splits_cfg, static_cast<size_t>(scratch), varlen != 0,
-                                      B, Hq, Sq, Sk, dqk, dv, causal ? 1 : 0);
+                                      B, Hq, Hkv, Sq, Sk, dqk, dv, causal ? 1 : 0);
     static const char* const names[4] = {"fa_fwd_simple", "fa_fwd_pipelined", "fa_fwd_persistent", "fa_fwd_stream"};
     out->kernel = names[pl.kernel];
     out->kv_splits = pl.kv_splits;
+    out->heads_per_tile = pl.pack_heads;
     const long long n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
     long long ctas = 0;
     switch (pl.kernel) {
         case kPlanSerial: ctas = n_q_tiles * Hq * B; break;
         case kPlanPair: ctas = ((n_q_tiles + 1) / 2) * Hq * B * pl.kv_splits; break;
         case kPlanPersistent: ctas = ((n_q_tiles + 1) / 2) * Hq * B; if (ctas > num_sms) ctas = num_sms; break;
-        default: ctas = n_q_tiles * Hq * B * pl.kv_splits; break;
+        default: ctas = n_q_tiles * (Hq / pl.pack_heads) * B * pl.kv_splits; break;
     }
     out->ctas = ctas;
     out->estimate_pair_us = pl.pair_us;

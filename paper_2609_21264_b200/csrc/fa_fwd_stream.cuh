@@ -72,7 +72,12 @@ constexpr int stream_smem_bytes() {
 }
 
 // kVarlen = packed variable-length batch, as in the pair kernel.
-template <int DQK, int DV, bool kVarlen = false>
+// kPack = the query tile holds the (at most 64) query rows of SEVERAL query heads that share one
+// K/V head (grouped-query attention with few queries per sequence, as when decoding): row
+// h * Sq + i of the tile is query i of the CTA's h-th head.  Every K/V tile is then read and
+// multiplied once for p.pack_heads heads instead of once per head.  The tensor maps of Q and
+// O have a box of Sq rows x pack_heads heads for it.
+template <int DQK, int DV, bool kVarlen = false, bool kPack = false>
 __global__ void __launch_bounds__(512, 1)
 fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                      const __grid_constant__ CUtensorMap tm_k,
@@ -116,17 +121,24 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     // adjacent in the grid; each writes a normalised fp32 partial that the combine kernel merges.
     const int item = static_cast<int>(blockIdx.x) / p.kv_splits;
     const int split = static_cast<int>(blockIdx.x) - item * p.kv_splits;
-    const int per_group = p.n_q_tiles * p.heads_per_group;
-    const int group = item / per_group;
-    const int bh0 = group * p.heads_per_group;
-    const int group_size = (n_bh - bh0 < p.heads_per_group) ? (n_bh - bh0) : p.heads_per_group;
-    const int local = item - group * per_group;
-    const int q_tile = p.n_q_tiles - 1 - local / group_size;
-    const int bh = bh0 + local % group_size;
-    const int hq = bh % p.Hq;
-    const int b = bh / p.Hq;
+    int q_tile = 0, hq, b;
+    if constexpr (kPack) {
+        // one item per pack of heads; all items are equally long
+        const int packs = p.Hq / p.pack_heads;
+        b = item / packs;
+        hq = (item - b * packs) * p.pack_heads;       // first head of the pack
+    } else {
+        const int per_group = p.n_q_tiles * p.heads_per_group;
+        const int group = item / per_group;
+        const int bh0 = group * p.heads_per_group;
+        const int group_size = (n_bh - bh0 < p.heads_per_group) ? (n_bh - bh0) : p.heads_per_group;
+        const int local = item - group * per_group;
+        q_tile = p.n_q_tiles - 1 - local / group_size;
+        const int bh = bh0 + local % group_size;
+        hq = bh % p.Hq;
+        b = bh / p.Hq;
+    }
     const int kvh = hq / (p.Hq / p.Hkv);
-    const int q_idx = b * p.Hq + hq;
     int Sq = p.Sq, Sk = p.Sk, q_row0 = 0, k_row0 = 0;
     if constexpr (kVarlen) {
         q_row0 = p.cu_q[b];
@@ -178,6 +190,11 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         prefetch_tensormap(&tm_v);
         prefetch_tensormap(&tm_o);
     }
+    if constexpr (kPack) {
+        // the rows of the query tile past the pack's last row are never loaded: zero scores there
+        for (int o = tid * 16; o < Cfg::kQBytes; o += 512 * 16) st_shared_v4(sQ + o, 0u, 0u, 0u, 0u);
+        fence_proxy_async_smem();
+    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -201,7 +218,12 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         const uint32_t bar_st_other = smem_addr(&sh.st_full[g ^ 1]);
         const uint32_t bar_pr = smem_addr(&sh.p_ready[g]);
         const uint32_t bar_pf = smem_addr(&sh.p_free[g]);
-        const int i_glob = i0 + row;
+        // the query this thread's row belongs to: index in its sequence, head, and whether it exists
+        const int h_local = kPack ? row / Sq : 0;
+        const int i_glob = kPack ? row - h_local * Sq : i0 + row;
+        const bool row_valid = kPack ? (h_local < p.pack_heads) : (i_glob < Sq);
+        const int hq_row = hq + h_local;
+        const int q_idx = b * p.Hq + hq_row;
         int kmax_row = Sk - 1;
         if (p.causal && i_glob + off < kmax_row) kmax_row = i_glob + off;
         const float tau_raw = kRescaleThresholdLog2 / c;
@@ -317,9 +339,9 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         if (ok && i0 < Sq) {
             // fixed lengths: lse [B, Hq, Sq]; packed batches: lse [Hq, total_q], O rows q_row0 onwards
             const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq) * p.total_q + q_row0 : static_cast<size_t>(q_idx) * p.Sq;
-            const long long o_base = (kVarlen ? q_row0 * p.o_stride_s : b * p.o_stride_b) + hq * p.o_stride_h;
+            const long long o_base = (kVarlen ? q_row0 * p.o_stride_s : b * p.o_stride_b) + hq_row * p.o_stride_h;
             if (p.kv_splits > 1 && n_kv == 0) {      // an empty range: a neutral partial
-                if (i_glob < Sq) {
+                if (row_valid) {
                     const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
                     float* po_row = p.o_part + prow * DV + g * (DV / 2);
                     const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -328,7 +350,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     if (g == 0) p.lse_part[prow] = -INFINITY;
                 }
             } else if (n_kv == 0) {       // no key visible to any row of this tile
-                if (g == 0 && i_glob < Sq) {
+                if (g == 0 && row_valid) {
                     __nv_bfloat16* o_row = p.O + (o_base + static_cast<long long>(i_glob) * p.o_stride_s);
                     const uint4 z = make_uint4(0, 0, 0, 0);
 #pragma unroll
@@ -356,7 +378,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     const float lt = sh.lsum[0][row] + sh.lsum[1][row];
                     const float m_fin = sh.mref[row];
                     const float inv_l = (lt > 0.f) ? (1.f / lt) : 0.f;
-                    if (g == 0 && p.lse && i_glob < Sq && p.kv_splits == 1)
+                    if (g == 0 && p.lse && row_valid && p.kv_splits == 1)
                         p.lse[lse_row0 + i_glob] = (lt > 0.f) ? (m_fin * c * 0.6931471805599453f + logf(lt)) : -INFINITY;
                     // warpgroup g converts columns [g*DV/2, (g+1)*DV/2) of O into the staging tile
                     // (the Q tile's space: the last score MMA is long complete), then one thread
@@ -369,14 +391,14 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                         // split-KV: G'_c / s_c in fp32 and u_c + ln s_c go to scratch (Algorithm 2's partials)
                         const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
                         float* po_row = p.o_part + prow * DV;
-                        if (g == 0 && i_glob < Sq)
+                        if (g == 0 && row_valid)
                             p.lse_part[prow] = (lt > 0.f) ? (m_fin * c * 0.6931471805599453f + logf(lt)) : -INFINITY;
 #pragma unroll 1
                         for (int cc = g * (DV / 64); cc < (g + 1) * (DV / 64); ++cc) {
                             uint32_t r[32];
                             tmem_ld_x32(tO + cc * 32, r);
                             tc_wait_ld();
-                            if (i_glob < Sq) {
+                            if (row_valid) {
 #pragma unroll
                                 for (int v = 0; v < 8; ++v)
                                     reinterpret_cast<float4*>(po_row + cc * 32)[v] = make_float4(
@@ -419,7 +441,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                             uint32_t r[32];
                             tmem_ld_x32(tO + cc * 32, r);
                             tc_wait_ld();
-                            if (i_glob < Sq) {
+                            if (row_valid) {
 #pragma unroll
                                 for (int v = 0; v < 4; ++v)
                                     reinterpret_cast<uint4*>(o_row + cc * 32)[v] = make_uint4(
@@ -535,7 +557,9 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         if (lane == 0 && n_kv > 0) {
             {
                 const uint32_t bar = smem_addr(&sh.q_full);
-                mbar_arrive_expect_tx(bar, Cfg::kQBytes);
+                // with packed heads the box is Sq rows x pack_heads heads (row h * Sq + i of the tile)
+                mbar_arrive_expect_tx(bar, kPack ? static_cast<uint32_t>(Cfg::kQChunks * p.pack_heads * Sq * 128)
+                                                 : static_cast<uint32_t>(Cfg::kQBytes));
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kQChunks; ++cc)
                     tma_load_4d(sQ + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols, q_row0 + i0, hq, tb);

@@ -19,10 +19,13 @@ from parity_util import bf16_tensor_to_f64, LSE_MAX_ABS
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module")
-def handle():
+# both tilings of the 8-bit path: two query tiles per CTA, and one query tile per CTA with the
+# K/V tiles streamed through both softmax warpgroups
+@pytest.fixture(scope="module", params=["pair", "stream"])
+def handle(request):
     from paper_2609_21264_b200 import binding
-    h = binding.fa_create()
+    flags = binding.FA_FLAG_NO_STREAM_KERNEL if request.param == "pair" else binding.FA_FLAG_STREAM_KERNEL
+    h = binding.fa_create(flags=flags)
     yield h
     binding.fa_destroy(h)
 
@@ -35,7 +38,7 @@ def _run(handle, w, q8, k8, v8, sq, sk, sv):
     torch.cuda.synchronize()
     st, detail = binding.fa_last_status(handle)
     assert st == binding.FA_OK, "device status %d (site 0x%x)" % (st, detail)
-    assert binding.fa_last_kernel_name(handle) == "fa_fwd_fp8"
+    assert binding.fa_last_kernel_name(handle) in ("fa_fwd_fp8", "fa_fwd_fp8_stream")
     return bf16_tensor_to_f64(o), lse.double().cpu().numpy()
 
 
@@ -50,6 +53,11 @@ CASES = [
     _wl("fp8_causal_more_q_than_k", 1, 3, 3, 400, 140, True, 1303),
     _wl("fp8_llama_like_s1024", 1, 8, 2, 1024, 1024, True, 1304),
     _wl("fp8_sigma2", 1, 4, 1, 512, 512, True, 1305, sigma=2.0),
+    _wl("fp8_one_tile_many_keys", 1, 2, 1, 100, 2100, False, 1308),      # the stream tiling splits K/V here
+    _wl("fp8_short_q_causal_long_k", 2, 4, 2, 130, 1500, True, 1309),
+    _wl("fp8_group4_sq16_heads_share_a_tile", 2, 8, 2, 16, 900, False, 1340),
+    _wl("fp8_group8_sq9_causal", 1, 8, 1, 9, 1300, True, 1341),
+    _wl("fp8_group6_single_query", 1, 12, 2, 1, 2500, False, 1342),
 ]
 
 
@@ -114,6 +122,62 @@ def test_fp8_scales_are_applied_per_block(handle):
     O2, lse2 = _run(handle, w, q8b, k8b, v8, sqb, skb, sv)
     assert np.abs(lse1 - lse2).max() <= 1e-5
     assert np.abs(O1 - O2).max() <= 2.0 ** -7 * np.abs(O1).max()
+
+
+def _check(w, O, lse, O_ref, lse_ref, Vd):
+    fin = np.isfinite(lse_ref)
+    assert np.array_equal(np.isneginf(lse), np.isneginf(lse_ref))
+    assert np.abs(lse[fin] - lse_ref[fin]).max() <= LSE_MAX_ABS
+    err = np.abs(O - O_ref)
+    vmax = np.abs(Vd).max(axis=(2, 3))
+    bound = 2.0 ** -4 * np.repeat(vmax, w.Hq // w.Hkv, axis=1)[:, :, None, None] + 2.0 ** -8 * np.abs(O_ref) + 1e-3
+    assert (err <= bound).all(), (w.name, float(err.max()), float((err / bound).max()))
+    assert err.mean() <= 1e-2 * w.sigma, (w.name, float(err.mean()))
+
+
+@pytest.mark.parametrize("splits", [2, 3, 7])
+def test_fp8_split_kv_with_fixed_split_counts(splits):
+    """Attention of few queries over a long 8-bit K/V sequence, the K/V range divided among CTAs
+    (uneven and, with a causal mask, partly empty ranges included), merged by the combine kernel."""
+    import torch
+    from paper_2609_21264_b200 import binding
+    h = binding.fa_create(flags=binding.FA_FLAG_STREAM_KERNEL, kv_splits=splits)
+    try:
+        for w in (_wl("fp8_split_full", 1, 4, 2, 70, 1700, False, 1310 + splits),
+                  _wl("fp8_split_causal", 1, 2, 1, 300, 900, True, 1320 + splits)):
+            Q, K, V = (W.bf16_bits_to_f64(x) for x in W.make_inputs(w))
+            q8, sq, Qd = W.quantize_e4m3_blocks(Q, 128)
+            k8, sk, Kd = W.quantize_e4m3_blocks(K, 128)
+            v8, sv, Vd = W.quantize_e4m3_blocks(V, None)
+            O_ref, lse_ref = oracle.attention(Qd, Kd, Vd, causal=w.causal, scale=w.scale)
+            O, lse = _run(h, w, q8, k8, v8, sq, sk, sv)
+            assert binding.fa_last_kernel_name(h) == "fa_fwd_fp8_stream"
+            assert binding.fa_last_kv_splits(h) == splits
+            _check(w, O, lse, O_ref, lse_ref, Vd)
+    finally:
+        binding.fa_destroy(h)
+
+
+def test_fp8_default_handle_plans_both_tilings():
+    from paper_2609_21264_b200 import binding
+    import torch
+    h = binding.fa_create()
+    try:
+        seen = {}
+        for w in (_wl("fp8_plan_decode", 1, 8, 2, 128, 8192, False, 1330),      # one query tile, long K/V: stream + split
+                  _wl("fp8_plan_large", 2, 32, 8, 1024, 1024, True, 1331)):    # several waves of pairs
+            q8 = torch.randint(0, 120, (w.B, w.Hq, w.Sq, 128), dtype=torch.uint8, device="cuda")
+            k8 = torch.randint(0, 120, (w.B, w.Hkv, w.Sk, 128), dtype=torch.uint8, device="cuda")
+            v8 = torch.randint(0, 120, (w.B, w.Hkv, w.Sk, 128), dtype=torch.uint8, device="cuda")
+            o, lse = binding.forward_fp8(h, q8, k8, v8, None, None, None, causal=w.causal, scale=w.scale)
+            torch.cuda.synchronize()
+            assert binding.fa_last_status(h)[0] == binding.FA_OK
+            assert torch.isfinite(o.float()).all()
+            seen[w.name] = (binding.fa_last_kernel_name(h), binding.fa_last_kv_splits(h))
+        assert seen["fp8_plan_decode"][0] == "fa_fwd_fp8_stream" and seen["fp8_plan_decode"][1] > 1, seen
+        assert seen["fp8_plan_large"] == ("fa_fwd_fp8", 1), seen
+    finally:
+        binding.fa_destroy(h)
 
 
 def test_fp8_unsupported_head_size(handle):

@@ -37,9 +37,27 @@ def test_table6_rows():
 def test_decode_like_shapes_split_the_kv_range_on_the_stream_kernel():
     p = binding.fa_plan(SMS, 1, 32, 8, 128, 32768, 128, 128, False)
     assert p["kernel"] == "fa_fwd_stream" and p["kv_splits"] == 4 and p["ctas"] == 32 * 4
-    p = binding.fa_plan(SMS, 8, 32, 8, 1, 8192, 128, 128, False)
-    assert p["kernel"] == "fa_fwd_stream" and p["ctas"] == 256 * p["kv_splits"]
+    p = binding.fa_plan(SMS, 8, 32, 32, 1, 8192, 128, 128, False)
+    assert p["kernel"] == "fa_fwd_stream" and p["ctas"] == 256 * p["kv_splits"] and p["heads_per_tile"] == 1
     assert p["estimate_stream_us"] < p["estimate_pair_us"]
+
+
+def test_few_queries_with_grouped_heads_share_a_query_tile():
+    # 4 query heads per K/V head, one query each: all four in one tile, a quarter of the CTAs
+    p = binding.fa_plan(SMS, 8, 32, 8, 1, 8192, 128, 128, False)
+    assert p["kernel"] == "fa_fwd_stream" and p["heads_per_tile"] == 4 and p["ctas"] == 64 * p["kv_splits"]
+    assert p["kv_splits"] == 2                                   # 64 items on 148 SMs
+    # the largest divisor of the group size whose rows fit 128
+    assert binding.fa_plan(SMS, 1, 16, 2, 16, 4096, 128, 128, True)["heads_per_tile"] == 8
+    assert binding.fa_plan(SMS, 1, 16, 2, 20, 4096, 128, 128, True)["heads_per_tile"] == 4
+    assert binding.fa_plan(SMS, 1, 12, 2, 33, 4096, 64, 64, True)["heads_per_tile"] == 3
+    assert binding.fa_plan(SMS, 1, 12, 2, 64, 4096, 64, 64, True)["heads_per_tile"] == 2
+    # not with more than 64 queries, one head per K/V head, packed batches, or when switched off
+    assert binding.fa_plan(SMS, 1, 12, 2, 65, 4096, 64, 64, True)["heads_per_tile"] == 1
+    assert binding.fa_plan(SMS, 1, 12, 12, 16, 4096, 64, 64, True)["heads_per_tile"] == 1
+    assert binding.fa_plan(SMS, 4, 16, 4, 16, 1024, 128, 128, True, varlen=True)["heads_per_tile"] == 1
+    for flag in (binding.FA_FLAG_NO_HEAD_PACKING, binding.FA_FLAG_NO_STREAM_KERNEL, binding.FA_FLAG_SERIAL_KERNEL):
+        assert binding.fa_plan(SMS, 8, 32, 8, 1, 8192, 128, 128, False, flags=flag)["heads_per_tile"] == 1
 
 
 def test_flags_and_configuration_override_the_choice():
