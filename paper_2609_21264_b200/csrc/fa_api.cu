@@ -805,9 +805,19 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     p.kv_splits = use_stream ? pl.kv_splits : 1;
     p.tiles_per_split = use_stream ? pl.tiles_per_split : 0x3fffffff;
     p.pack_heads = pl.pack_heads;
-    if (p.kv_splits > 1) {
+    // A pack of at most 32 (64) rows is loaded four times (twice) and every copy takes a quarter
+    // (half) of each K/V tile's keys: the partials per query row multiply accordingly.
+    int copies = 1;
+    if (use_stream && pl.pack_heads > 1) {
+        const int rows = pl.pack_heads * Sq;
+        copies = rows <= 32 ? 4 : (rows <= 64 ? 2 : 1);
+        const unsigned long long per_partial = static_cast<unsigned long long>(B) * Hq * Sq * (d + 1) * 4ull;
+        while (copies > 1 && per_partial * p.kv_splits * copies > h->scratch_bytes) copies /= 2;
+    }
+    const int n_partials = p.kv_splits * copies;
+    if (n_partials > 1) {
         p.o_part = static_cast<float*>(h->scratch);
-        p.lse_part = p.o_part + static_cast<size_t>(p.kv_splits) * B * Hq * Sq * d;
+        p.lse_part = p.o_part + static_cast<size_t>(n_partials) * B * Hq * Sq * d;
     }
     h->last_splits = p.kv_splits;
     h->last_kernel = use_stream ? "fa_fwd_fp8_stream" : "fa_fwd_fp8";
@@ -824,15 +834,17 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
         constexpr int smem = fa::fp8_stream_smem_bytes();
         static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
         const bool pack = pl.pack_heads > 1;
-        auto kernel = pack ? fa::fa_fwd_fp8_stream_kernel<true> : fa::fa_fwd_fp8_stream_kernel<false>;
-        if ((s = ensure_smem_attr(h, pack ? 26 : 22, kernel, smem)) != FA_OK) return s;
+        auto kernel = !pack ? fa::fa_fwd_fp8_stream_kernel<false, 1>
+                             : (copies == 4 ? fa::fa_fwd_fp8_stream_kernel<true, 4>
+                                            : (copies == 2 ? fa::fa_fwd_fp8_stream_kernel<true, 2> : fa::fa_fwd_fp8_stream_kernel<true, 1>));
+        if ((s = ensure_smem_attr(h, !pack ? 22 : (copies == 4 ? 28 : (copies == 2 ? 27 : 26)), kernel, smem)) != FA_OK) return s;
         const long long n_ctas = (pack ? static_cast<long long>(Hq / pl.pack_heads) : static_cast<long long>(p.n_q_tiles) * Hq) * B * p.kv_splits;
         if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
         cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
         cfg.dynamicSmemBytes = smem;
         if (cudaLaunchKernelEx(&cfg, kernel, map_q, map_k, map_v, map_o, p, f) != cudaSuccess) return FA_ERR_CUDA;
         h->launches += 1;
-        if (p.kv_splits > 1) {
+        if (n_partials > 1) {
             const long long n_rows = static_cast<long long>(B) * Hq * Sq;
             const long long blocks = (n_rows + 3) / 4;
             if (blocks > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
@@ -840,7 +852,7 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
             cfg.blockDim = dim3(128, 1, 1);
             cfg.dynamicSmemBytes = 0;
             if (cudaLaunchKernelEx(&cfg, fa::fa_combine_kernel<128>, static_cast<const float*>(p.o_part),
-                                   static_cast<const float*>(p.lse_part), p.O, p.lse, n_rows, p.kv_splits, p.Hq, p.Sq,
+                                   static_cast<const float*>(p.lse_part), p.O, p.lse, n_rows, n_partials, p.Hq, p.Sq,
                                    p.o_stride_b, p.o_stride_h, p.o_stride_s) != cudaSuccess) return FA_ERR_CUDA;
             h->launches += 1;
         }

@@ -29,7 +29,16 @@ struct Fp8StreamCfg {
 constexpr int fp8_stream_smem_bytes() { return Fp8StreamCfg::kTileBytes + static_cast<int>(sizeof(StreamShared)); }
 
 // kPack: several query heads of one K/V head share the query tile, as in fa_fwd_stream_kernel.
-template <bool kPack = false>
+// kRep (with kPack, 2 or 4): the pack has at most 128 / kRep rows and is loaded kRep times, copy
+// r into rows [r * 128 / kRep, (r + 1) * 128 / kRep) of the query tile.  Copy r only takes the
+// keys [r * 128 / kRep, ...) of every K/V tile: its threads read that slice of the score tile,
+// exponentiate it and write that slice of P, whose other columns stay zero.  The copies are thus
+// kRep independent attention problems over disjoint keys, each with its own row state, and they
+// leave the kernel as kRep partials per split, merged by fa_combine_kernel like split-KV
+// partials.  A softmax warp then issues 1 / kRep of the exponentials per K/V tile (an
+// instruction costs the same for one live row as for 32), which takes a few-row problem from the
+// MUFU bound to the bound of the K/V stream.
+template <bool kPack = false, int kRep = 1>
 __global__ void __launch_bounds__(512, 1)
 fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                      const __grid_constant__ CUtensorMap tm_k,
@@ -40,6 +49,10 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     constexpr bool kVarlen = false;
     constexpr int DV = Cfg::kD;
     constexpr int kTile8 = Cfg::kTile8;
+    static_assert(kRep == 1 || (kPack && (kRep == 2 || kRep == 4)), "copies of the query rows need packed heads");
+    constexpr int kRepRows = kTileM / kRep;      // rows of one copy of the pack
+    constexpr int kCols = kTileN / kRep;         // keys of a K/V tile that one copy takes
+    constexpr int kChunks = kCols / 32;
     using namespace ptx;
     constexpr int NK = Cfg::kKStages;
     constexpr int NV = Cfg::kVStages;
@@ -175,8 +188,13 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         const uint32_t bar_pr = smem_addr(&sh.p_ready[g]);
         const uint32_t bar_pf = smem_addr(&sh.p_free[g]);
         // the query this thread's row belongs to: index in its sequence, head, and whether it exists
-        const int h_local = kPack ? row / Sq : 0;
-        const int i_glob = kPack ? row - h_local * Sq : i0 + row;
+        const int copy = row / kRepRows;              // which copy of the pack (0 without copies)
+        const int row_in_copy = row - copy * kRepRows;
+        const int h_local = kPack ? row_in_copy / Sq : 0;
+        const int i_glob = kPack ? row_in_copy - h_local * Sq : i0 + row;
+        const int col0 = copy * kCols;                // first key of a tile that this row takes
+        const bool partial_out = p.kv_splits > 1 || kRep > 1;
+        const int part = split * kRep + copy;         // index of this row's partial
         const bool row_valid = kPack ? (h_local < p.pack_heads) : (i_glob < Sq);
         const int hq_row = hq + h_local;
         const int q_idx = b * p.Hq + hq_row;
@@ -186,6 +204,14 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         const float cq = p.scale_log2 * ((f.q_scale && row_valid) ? __ldg(f.q_scale + static_cast<size_t>(q_idx) * p.n_q_tiles + q_tile) : 1.f);
         const float* k_scale = f.k_scale ? f.k_scale + static_cast<size_t>(kv_idx) * f.n_kv_tiles + j_base : nullptr;
 
+        if constexpr (kRep > 1) {
+            // the columns of P^g that belong to the other copies' keys are never written: zero once
+            uint32_t z[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) z[e] = 0u;
+            tmem_st_x32(tP, z);
+            tc_wait_st();
+        }
         float l = 0.f;             // this warpgroup's partial row sum, relative to the current u
         bool ok = true;
         for (int j = g; j < n_kv; j += 2) {
@@ -197,11 +223,9 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             const int j0 = (j_base + j) * kTileN;
             const bool need_mask = (j0 + kTileN - 1 > kmax_row);
 
-            uint32_t s[kTileN];
-            tmem_ld_x32(tS + 0, s + 0);
-            tmem_ld_x32(tS + 32, s + 32);
-            tmem_ld_x32(tS + 64, s + 64);
-            tmem_ld_x32(tS + 96, s + 96);
+            uint32_t s[kCols];
+#pragma unroll
+            for (int q = 0; q < kChunks; ++q) tmem_ld_x32(tS + col0 + q * 32, s + q * 32);
             tc_wait_ld();
             // S^g is in registers: the score MMA of tile j+2 may overwrite it
             tc_fence_before_sync();
@@ -209,14 +233,14 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             if (lane == 0) mbar_arrive(bar_sf);
             if (need_mask) {
 #pragma unroll
-                for (int e = 0; e < kTileN; ++e)
-                    if (j0 + e > kmax_row) s[e] = 0xff800000u;   // -inf
+                for (int e = 0; e < kCols; ++e)
+                    if (j0 + col0 + e > kmax_row) s[e] = 0xff800000u;   // -inf
             }
             float a[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q) a[q] = -INFINITY;
 #pragma unroll
-            for (int e = 0; e < kTileN; e += 16) {
+            for (int e = 0; e < kCols; e += 16) {
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
                     a[q] = fmax3(a[q], __uint_as_float(s[e + 2 * q]), __uint_as_float(s[e + 2 * q + 1]));
@@ -275,17 +299,16 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     sum_b = __fadd2_rn(sum_b, v1);
                     pk[e / 4] = pack_e4m3x4(v0.x, v0.y, v1.x, v1.y);
                 }
-                tmem_st_x8(tP + q * 8, pk);
+                tmem_st_x8(tP + col0 / 4 + q * 8, pk);
             };
             // conversion and store of a chunk run under the exponentials of the next one
             exp_chunk(0);
-            exp_chunk(1);
-            emit_chunk(0);
-            exp_chunk(2);
-            emit_chunk(1);
-            exp_chunk(3);
-            emit_chunk(2);
-            emit_chunk(3);
+#pragma unroll
+            for (int q = 1; q < kChunks; ++q) {
+                exp_chunk(q);
+                emit_chunk(q - 1);
+            }
+            emit_chunk(kChunks - 1);
             l = l * (r_prev * alpha) + ((sum_a.x + sum_a.y) + (sum_b.x + sum_b.y));
             tc_wait_st();
             tc_fence_before_sync();
@@ -298,9 +321,9 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             // fixed lengths: lse [B, Hq, Sq]; packed batches: lse [Hq, total_q], O rows q_row0 onwards
             const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq) * p.total_q + q_row0 : static_cast<size_t>(q_idx) * p.Sq;
             const long long o_base = (kVarlen ? q_row0 * p.o_stride_s : b * p.o_stride_b) + hq_row * p.o_stride_h;
-            if (p.kv_splits > 1 && n_kv == 0) {      // an empty range: a neutral partial
+            if (partial_out && n_kv == 0) {      // an empty range: a neutral partial
                 if (row_valid) {
-                    const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
+                    const size_t prow = (static_cast<size_t>(part) * n_bh + q_idx) * p.Sq + i_glob;
                     float* po_row = p.o_part + prow * DV + g * (DV / 2);
                     const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
@@ -337,7 +360,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     const float m_fin = sh.mref[row];
                     const float sv = f.v_scale ? __ldg(f.v_scale + kv_idx) : 1.f;
                     const float inv_l = (lt > 0.f) ? (sv / lt) : 0.f;
-                    if (g == 0 && p.lse && row_valid && p.kv_splits == 1)
+                    if (g == 0 && p.lse && row_valid && !partial_out)
                         p.lse[lse_row0 + i_glob] = (lt > 0.f) ? (m_fin * 0.6931471805599453f + logf(lt)) : -INFINITY;
                     // warpgroup g converts columns [g*DV/2, (g+1)*DV/2) of O into the staging tile
                     // (the Q tile's space: the last score MMA is long complete), then one thread
@@ -346,9 +369,9 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     // the last tile of a packed sequence is followed by the next sequence's rows, which a
                     // box store would overwrite: it is stored row by row
                     const bool box_store = !kVarlen || (i0 + kTileM <= Sq);
-                    if (p.kv_splits > 1) {
+                    if (partial_out) {
                         // split-KV: G'_c / s_c in fp32 and u_c + ln s_c go to scratch (Algorithm 2's partials)
-                        const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
+                        const size_t prow = (static_cast<size_t>(part) * n_bh + q_idx) * p.Sq + i_glob;
                         float* po_row = p.o_part + prow * DV;
                         if (g == 0 && row_valid)
                             p.lse_part[prow] = (lt > 0.f) ? (m_fin * 0.6931471805599453f + logf(lt)) : -INFINITY;
@@ -515,8 +538,9 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             {
                 const uint32_t bar = smem_addr(&sh.q_full);
                 // with packed heads the box is Sq rows x pack_heads heads (row h * Sq + i of the tile)
-                mbar_arrive_expect_tx(bar, kPack ? static_cast<uint32_t>(p.pack_heads * Sq * 128) : static_cast<uint32_t>(kTile8));
-                tma_load_4d(sQ, &tm_q, bar, 0, q_row0 + i0, hq, tb);
+                mbar_arrive_expect_tx(bar, kPack ? static_cast<uint32_t>(kRep * p.pack_heads * Sq * 128) : static_cast<uint32_t>(kTile8));
+#pragma unroll
+                for (int r = 0; r < kRep; ++r) tma_load_4d(sQ + r * kRepRows * 128, &tm_q, bar, 0, q_row0 + i0, hq, tb);
             }
             bool ok = true;
             for (int j = 0; j < n_kv && ok; ++j) {

@@ -58,6 +58,9 @@ CASES = [
     _wl("fp8_group4_sq16_heads_share_a_tile", 2, 8, 2, 16, 900, False, 1340),
     _wl("fp8_group8_sq9_causal", 1, 8, 1, 9, 1300, True, 1341),
     _wl("fp8_group6_single_query", 1, 12, 2, 1, 2500, False, 1342),
+    _wl("fp8_group4_sq4_causal_four_copies", 2, 8, 2, 4, 1111, True, 1343),
+    _wl("fp8_group4_sq13_causal_two_copies", 1, 8, 2, 13, 777, True, 1344),
+    _wl("fp8_group2_sq3_more_queries_than_keys", 1, 4, 2, 3, 2, True, 1345),
 ]
 
 
