@@ -254,6 +254,76 @@ def oracle_timed(w, budget_s=20.0):
             "sample": sample, "seconds": dt}
 
 
+# Few queries over a long K/V sequence with grouped heads (B, Hq, Hkv, Sq, Sk, d): decoding.
+DECODE_SHAPES = ((8, 32, 8, 1, 8192, 128), (64, 32, 8, 1, 4096, 128), (1, 32, 8, 16, 131072, 128), (4, 32, 8, 128, 8192, 128))
+
+
+def time_libraries(binding, h, device):
+    """Library attention kernels on the same GPU and shapes, for context: PyTorch's
+    scaled_dot_product_attention with each of its fused back ends, and flash_attn where it is
+    installed.  One input set per shape (the library kernels and ours see the same L2 state);
+    a back end that refuses a shape is recorded with its message."""
+    import torch
+    import torch.nn.functional as F
+    from torch.nn.attention import SDPBackend, sdpa_kernel
+    try:
+        from flash_attn import flash_attn_func
+    except Exception:                                   # not installed, or no kernels for this GPU
+        flash_attn_func = None
+
+    def timed(f, k):
+        for _ in range(3):
+            f()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(k):
+            f()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3 / k
+
+    def one_shape(name, B, Hq, Hkv, Sq, Sk, dqk, dv, causal, scale, flops, kv_bytes):
+        gen = torch.Generator(device=device).manual_seed(7)
+        q = torch.randn((B, Hq, Sq, dqk), generator=gen, device=device).to(torch.bfloat16)
+        k = torch.randn((B, Hkv, Sk, dqk), generator=gen, device=device).to(torch.bfloat16)
+        v = torch.randn((B, Hkv, Sk, dv), generator=gen, device=device).to(torch.bfloat16)
+        n = max(3, min(100, int(0.2 / max(flops / 0.5e15, kv_bytes / 3e12, 1e-5))))
+        row = {"workload": name, "steps": n}
+
+        def record(key, f):
+            try:
+                t = timed(f, n)
+                row[key] = {"us": t * 1e6, "tflops_algorithmic": flops / t / 1e12, "kv_read_gbs": kv_bytes / t / 1e9}
+            except Exception as e:                      # this back end has no kernel for the shape
+                torch.cuda.synchronize()
+                row[key] = {"error": str(e).splitlines()[0][:160]}
+
+        record("ours", lambda: binding.forward(h, q, k, v, causal=causal, scale=scale))
+        for key, be in (("torch_sdpa_cudnn", SDPBackend.CUDNN_ATTENTION), ("torch_sdpa_flash", SDPBackend.FLASH_ATTENTION),
+                        ("torch_sdpa_efficient", SDPBackend.EFFICIENT_ATTENTION)):
+            def f(be=be):
+                with sdpa_kernel([be]):
+                    return F.scaled_dot_product_attention(q, k, v, is_causal=causal, scale=scale, enable_gqa=(Hq != Hkv))
+            record(key, f)
+        if flash_attn_func is not None:
+            qt, kt, vt = (x.transpose(1, 2).contiguous() for x in (q, k, v))      # [B, S, H, d]
+            record("flash_attn", lambda: flash_attn_func(qt, kt, vt, softmax_scale=scale, causal=causal))
+        return row
+
+    rows = []
+    for wc in workloads.CONFIGS:
+        fa, _, _ = workload_numbers(wc)
+        rows.append(one_shape(wc.name, wc.B, wc.Hq, wc.Hkv, wc.Sq, wc.Sk, wc.dqk, wc.dv, wc.causal, wc.scale, fa,
+                              2 * wc.B * wc.Hkv * wc.Sk * (wc.dqk + wc.dv)))
+        torch.cuda.empty_cache()
+    for (B, Hq, Hkv, Sq, Sk, d) in DECODE_SHAPES:
+        rows.append(one_shape("decode_b%d_h%d_%d_q%d_k%d_d%d" % (B, Hq, Hkv, Sq, Sk, d), B, Hq, Hkv, Sq, Sk, d, d, False,
+                              d ** -0.5, 4.0 * B * Hq * Sq * Sk * d, 2 * B * Hkv * Sk * 2 * d))
+        torch.cuda.empty_cache()
+    return rows
+
+
 def config_dict(w, extra=None):
     d = {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "Sq": w.Sq, "Sk": w.Sk, "dqk": w.dqk,
          "dv": w.dv, "causal": w.causal, "scale": w.scale, "inputs": "bf16 N(0,1), seeded",
@@ -325,6 +395,9 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the short timing of the other configs")
     ap.add_argument("--table6", action="store_true",
                     help="also time the twelve attention shapes of the paper's Table 6 (key 'table6')")
+    ap.add_argument("--libraries", action="store_true",
+                    help="also time the attention kernels of the libraries in the image (torch SDPA back ends, flash_attn) "
+                         "on the five configurations and a few decode shapes, for context (key 'libraries')")
     args = ap.parse_args()
     w = workloads.config(args.config)
     if args.shape:
@@ -432,6 +505,59 @@ def main():
                                      "note": "fa_forward_fp8, N(0,sigma^2) rounded to e4m3, unit scales, one input set"}
         del q8, k8, v8, o8, l8
 
+    if not args.no_sweep and world == 1:
+        # Decoding with grouped heads (few queries over a long K/V sequence): bound by the K/V read, so the
+        # figure of merit is bytes per second against the measured copy bandwidth.  bf16 and e4m3 K/V.
+        dB, dHq, dHkv, dSq, dSk = 64, 32, 8, 1, 4096
+        gen = torch.Generator(device=device).manual_seed(11)
+        qd = torch.randn((dB, dHq, dSq, 128), generator=gen, device=device).to(torch.bfloat16)
+        kd = torch.randn((dB, dHkv, dSk, 128), generator=gen, device=device).to(torch.bfloat16)
+        vd = torch.randn((dB, dHkv, dSk, 128), generator=gen, device=device).to(torch.bfloat16)
+        od = torch.empty_like(qd)
+        ld = torch.empty((dB, dHq, dSq), dtype=torch.float32, device=device)
+        cs = torch.cuda.current_stream().cuda_stream
+
+        def timed_launches(f, k=20):
+            for _ in range(3):
+                f()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(k):
+                f()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e-3 / k
+
+        def dec16():
+            st = binding.fa_forward(h, qd.data_ptr(), kd.data_ptr(), vd.data_ptr(), od.data_ptr(), ld.data_ptr(),
+                                    dB, dHq, dHkv, dSq, dSk, 128, 128, False, 0.0, cs)
+            if st != binding.FA_OK:
+                raise binding.FaError(st, "fa_forward")
+
+        t16 = timed_launches(dec16)
+        plan = binding.fa_plan(torch.cuda.get_device_properties(device).multi_processor_count, dB, dHq, dHkv, dSq, dSk, 128, 128, False)
+        bytes16 = 2 * (2 * dB * dHkv * dSk * 128 + 2 * dB * dHq * dSq * 128) + 4 * dB * dHq * dSq
+        q8, k8, v8 = (x.to(torch.float8_e4m3fn).view(torch.uint8) for x in (qd, kd, vd))
+
+        def dec8():
+            st = binding.fa_forward_fp8(h, q8.data_ptr(), k8.data_ptr(), v8.data_ptr(), None, None, None, od.data_ptr(),
+                                        ld.data_ptr(), dB, dHq, dHkv, dSq, dSk, 128, False, 0.0, cs)
+            if st != binding.FA_OK:
+                raise binding.FaError(st, "fa_forward_fp8")
+
+        t8 = timed_launches(dec8)
+        bytes8 = 2 * dB * dHkv * dSk * 128 + dB * dHq * dSq * 128 * 3 + 4 * dB * dHq * dSq
+        line["decode"] = {"workload": "B=%d Hq=%d Hkv=%d Sq=%d Sk=%d d=128 non-causal" % (dB, dHq, dHkv, dSq, dSk),
+                          "heads_per_tile": plan["heads_per_tile"], "kv_splits": plan["kv_splits"],
+                          "bf16": {"us": t16 * 1e6, "compulsory_bytes": bytes16, "gbs": bytes16 / t16 / 1e9,
+                                   "frac_of_measured_hbm": bytes16 / t16 / 1e9 / peaks["hbm_gbs"]},
+                          "e4m3": {"us": t8 * 1e6, "compulsory_bytes": bytes8, "gbs": bytes8 / t8 / 1e9,
+                                   "frac_of_measured_hbm": bytes8 / t8 / 1e9 / peaks["hbm_gbs"]},
+                          "note": "inputs larger than L2 (1.07 GB / 0.54 GB of K and V); 20 launches each after 3 warm-up launches"}
+        del qd, kd, vd, od, ld, q8, k8, v8
+        torch.cuda.empty_cache()
+
     if not args.no_e2e:
         e2e_steps = max(3, min(steps, 50))
         dt, h2d, d2h, _ = run_e2e_timed(binding, h, w, e2e_steps, 3, world)
@@ -473,6 +599,9 @@ def main():
             del ss
             torch.cuda.empty_cache()
         line["table6"] = rows
+
+    if args.libraries and world == 1:
+        line["libraries"] = time_libraries(binding, h, device)
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = oracle_timed(w)
