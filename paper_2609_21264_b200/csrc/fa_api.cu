@@ -398,7 +398,8 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     // attention): the heads of a group share the CTA's query tile, h heads of Sq rows each with
     // h the largest divisor of the group size that fits, and every K/V tile is read and
     // multiplied once for all of them.  Only the stream kernel has this mode.
-    if (!varlen && !drop && !(flags & (FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)) && Sq <= fa::kTileM / 2 &&
+    // (Packed batches: Sq is the longest query of the batch and there is no split.)
+    if (!drop && !(flags & (FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)) && Sq <= fa::kTileM / 2 &&
         Hq / Hkv >= 2) {
         const int group = Hq / Hkv;
         int hp = 1;
@@ -407,7 +408,7 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
         if (hp > 1) {
             pl.kernel = kPlanStream;
             pl.pack_heads = hp;
-            with_splits(choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles, true, hp));
+            with_splits(varlen ? 1 : choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles, true, hp));
             return pl;
         }
     }
@@ -433,7 +434,9 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
         if (flags & FA_FLAG_STREAM_KERNEL) {
             stream = true;
         } else if (varlen) {
-            stream = (dqk == 192);       // no estimate without the lengths; 192/128 is always ahead
+            // no estimate without the lengths: 192/128 is always ahead, and with a single query tile
+            // per sequence the pair kernel's second tile would be empty
+            stream = (dqk == 192) || n_q_tiles == 1;
         } else if (!persistent) {
             const TilingEstimate e = estimate_tilings(num_sms, B, Hq, Sq, Sk, dqk, causal, n_q_tiles, pair_splits, stream_splits);
             pl.pair_us = e.pair_us;
@@ -498,6 +501,11 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
 
     if (pl.kernel == kPlanStream) {
         h->last_kernel = "fa_fwd_stream";
+        if (pl.pack_heads > 1 && cu_q) {
+            if (dqk == 64) return launch_stream<64, 64, true, true>(h, 29, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_stream<128, 128, true, true>(h, 30, map_q, map_k, map_v, map_o, p, st);
+            return launch_stream<192, 128, true, true>(h, 31, map_q, map_k, map_v, map_o, p, st);
+        }
         if (pl.pack_heads > 1) {
             if (dqk == 64) return launch_stream<64, 64, false, true>(h, 23, map_q, map_k, map_v, map_o, p, st);
             if (dqk == 128) return launch_stream<128, 128, false, true>(h, 24, map_q, map_k, map_v, map_o, p, st);
@@ -729,10 +737,15 @@ fa_status fa_forward_varlen(fa_handle* h, const void* Q, const void* K, const vo
     if (!guard.ok()) return FA_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // packed [total, H, d]: one batch slice, rows H*d apart, heads d apart
+    const int mean_sk = (total_k + B - 1) / B > 0 ? (total_k + B - 1) / B : 1;
+    const LaunchPlan pl = plan_launch(h->num_sms, h->flags, h->kv_splits_cfg, h->scratch_bytes, true,
+                                      B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal ? 1 : 0);
+    // packed heads: the box of Q is the max_sq rows (from the sequence's first row) of pack_heads heads
+    const int q_box_rows = pl.pack_heads > 1 ? max_sq : fa::kTileM;
     const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;
     const int rows_k = total_k > 0 ? total_k : 1;   // an empty K/V still gets a valid map; no tile of it is ever read
     if ((s = get_map(h, Q, dqk, total_q, Hq, 1, static_cast<long long>(total_q) * Hq * dqk, dqk,
-                     static_cast<long long>(Hq) * dqk, fa::kTileM, &mq)) != FA_OK) return s;
+                     static_cast<long long>(Hq) * dqk, q_box_rows, &mq, 2, pl.pack_heads)) != FA_OK) return s;
     CUtensorMap map_q = *mq;
     if ((s = get_map(h, K, dqk, rows_k, Hkv, 1, static_cast<long long>(rows_k) * Hkv * dqk, dqk,
                      static_cast<long long>(Hkv) * dqk, fa::kTileN, &mk)) != FA_OK) return s;
@@ -744,9 +757,6 @@ fa_status fa_forward_varlen(fa_handle* h, const void* Q, const void* K, const vo
                      static_cast<long long>(Hq) * dv, fa::kTileM, &mo)) != FA_OK) return s;
     CUtensorMap map_o = *mo;
     const int64_t os[3] = {0, dv, static_cast<int64_t>(Hq) * dv};
-    const int mean_sk = (total_k + B - 1) / B > 0 ? (total_k + B - 1) / B : 1;
-    const LaunchPlan pl = plan_launch(h->num_sms, h->flags, h->kv_splits_cfg, h->scratch_bytes, true,
-                                      B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal ? 1 : 0);
     return run_forward(h, map_q, map_k, map_v, map_o, O, lse, B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal, scale, os,
                        cu_seqlens_q, cu_seqlens_k, total_q, pl, st);
 }

@@ -219,9 +219,12 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         const uint32_t bar_pr = smem_addr(&sh.p_ready[g]);
         const uint32_t bar_pf = smem_addr(&sh.p_free[g]);
         // the query this thread's row belongs to: index in its sequence, head, and whether it exists
-        const int h_local = kPack ? row / Sq : 0;
-        const int i_glob = kPack ? row - h_local * Sq : i0 + row;
-        const bool row_valid = kPack ? (h_local < p.pack_heads) : (i_glob < Sq);
+        // (packed batches: every head's rows are p.Sq apart in the tile, the longest query of the
+        // batch, and a shorter sequence leaves the rest of its head's rows unused)
+        const int pack_rows = kVarlen ? p.Sq : Sq;
+        const int h_local = kPack ? row / pack_rows : 0;
+        const int i_glob = kPack ? row - h_local * pack_rows : i0 + row;
+        const bool row_valid = kPack ? (h_local < p.pack_heads && i_glob < Sq) : (i_glob < Sq);
         const int hq_row = hq + h_local;
         const int q_idx = b * p.Hq + hq_row;
         int kmax_row = Sk - 1;
@@ -338,7 +341,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         // ---- epilogue: O = G' / s (bf16), lse = u * scale + ln s
         if (ok && i0 < Sq) {
             // fixed lengths: lse [B, Hq, Sq]; packed batches: lse [Hq, total_q], O rows q_row0 onwards
-            const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq) * p.total_q + q_row0 : static_cast<size_t>(q_idx) * p.Sq;
+            const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq_row) * p.total_q + q_row0 : static_cast<size_t>(q_idx) * p.Sq;
             const long long o_base = (kVarlen ? q_row0 * p.o_stride_s : b * p.o_stride_b) + hq_row * p.o_stride_h;
             if (p.kv_splits > 1 && n_kv == 0) {      // an empty range: a neutral partial
                 if (row_valid) {
@@ -558,7 +561,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             {
                 const uint32_t bar = smem_addr(&sh.q_full);
                 // with packed heads the box is Sq rows x pack_heads heads (row h * Sq + i of the tile)
-                mbar_arrive_expect_tx(bar, kPack ? static_cast<uint32_t>(Cfg::kQChunks * p.pack_heads * Sq * 128)
+                mbar_arrive_expect_tx(bar, kPack ? static_cast<uint32_t>(Cfg::kQChunks * p.pack_heads * (kVarlen ? p.Sq : Sq) * 128)
                                                  : static_cast<uint32_t>(Cfg::kQBytes));
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kQChunks; ++cc)

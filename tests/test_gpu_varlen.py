@@ -124,3 +124,27 @@ def test_rows_past_max_sq_are_left_alone_and_empty_batch(handle):
     assert binding.fa_forward_varlen(*args[:6], None, cu.data_ptr(), 1, 8, 8, 8, 1, 1, 64, 64, False, 0.0) \
         == binding.FA_ERR_INVALID_ARG
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("dqk,dv,Hq,Hkv", [(128, 128, 8, 2), (64, 64, 6, 2), (192, 128, 16, 1)], ids=["d128_g4", "d64_g3", "d192_g16"])
+@pytest.mark.parametrize("causal", [False, True], ids=["full", "causal"])
+def test_decode_batches_with_grouped_heads(handle, dqk, dv, Hq, Hkv, causal):
+    """Few queries per sequence (here at most 40, lengths differing per sequence) against K/V of very
+    different lengths, several query heads per K/V head: on the stream tiling the heads of a group
+    share a query tile, each head's rows max_sq apart, and a sequence with fewer queries leaves
+    the rest of its rows unused.  Includes a sequence without queries and one without keys."""
+    from paper_2609_21264_b200 import binding
+    lens_q = [1, 40, 7, 0, 16, 3, 1]
+    lens_k = [900, 333, 1500, 64, 20, 0, 129]
+    _run_and_check(handle, lens_q, lens_k, Hq=Hq, Hkv=Hkv, dqk=dqk, dv=dv, causal=causal, seed=1110 + dqk)
+    # single-token decode for every sequence
+    _run_and_check(handle, [1] * 9, [50, 700, 128, 129, 1, 2048, 300, 64, 1000], Hq=Hq, Hkv=Hkv, dqk=dqk, dv=dv,
+                   causal=causal, seed=1120 + dqk)
+
+
+def test_decode_batches_plan_shared_query_tiles():
+    from paper_2609_21264_b200 import binding
+    p = binding.fa_plan(148, 32, 32, 8, 1, 4096, 128, 128, True, varlen=True)
+    assert p["kernel"] == "fa_fwd_stream" and p["heads_per_tile"] == 4 and p["kv_splits"] == 1 and p["ctas"] == 32 * 8
+    assert binding.fa_plan(148, 32, 32, 8, 1, 4096, 128, 128, True, varlen=True,
+                           flags=binding.FA_FLAG_NO_HEAD_PACKING)["heads_per_tile"] == 1

@@ -52,10 +52,12 @@ def test_few_queries_with_grouped_heads_share_a_query_tile():
     assert binding.fa_plan(SMS, 1, 16, 2, 20, 4096, 128, 128, True)["heads_per_tile"] == 4
     assert binding.fa_plan(SMS, 1, 12, 2, 33, 4096, 64, 64, True)["heads_per_tile"] == 3
     assert binding.fa_plan(SMS, 1, 12, 2, 64, 4096, 64, 64, True)["heads_per_tile"] == 2
-    # not with more than 64 queries, one head per K/V head, packed batches, or when switched off
+    # not with more than 64 queries, one head per K/V head, or when switched off
     assert binding.fa_plan(SMS, 1, 12, 2, 65, 4096, 64, 64, True)["heads_per_tile"] == 1
     assert binding.fa_plan(SMS, 1, 12, 12, 16, 4096, 64, 64, True)["heads_per_tile"] == 1
-    assert binding.fa_plan(SMS, 4, 16, 4, 16, 1024, 128, 128, True, varlen=True)["heads_per_tile"] == 1
+    # packed batches of sequences (lengths on the device): packed heads, no split
+    p = binding.fa_plan(SMS, 4, 16, 4, 16, 1024, 128, 128, True, varlen=True)
+    assert p["kernel"] == "fa_fwd_stream" and p["heads_per_tile"] == 4 and p["kv_splits"] == 1 and p["ctas"] == 4 * 4
     for flag in (binding.FA_FLAG_NO_HEAD_PACKING, binding.FA_FLAG_NO_STREAM_KERNEL, binding.FA_FLAG_SERIAL_KERNEL):
         assert binding.fa_plan(SMS, 8, 32, 8, 1, 8192, 128, 128, False, flags=flag)["heads_per_tile"] == 1
 
