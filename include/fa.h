@@ -191,7 +191,9 @@ fa_status fa_forward_strided(fa_handle* h,
  * gets O = 0 and lse = -inf; a sequence with no queries writes nothing.  Rows of K/V past the end
  * of a sequence take no part in the result, but must hold finite numbers where they belong to the
  * next sequence (they are multiplied by a zero probability).  The K/V range is never split over
- * CTAs on this path.  Errors as for fa_forward.
+ * CTAs on this path.  With max_sq <= 64 and several query heads per K/V head the heads of a group
+ * share a query tile (see FA_FLAG_NO_HEAD_PACKING): a decode step over sequences of different
+ * lengths then reads every K/V head once.  Errors as for fa_forward.
  */
 fa_status fa_forward_varlen(fa_handle* h,
                             const void* Q, const void* K, const void* V,
@@ -213,7 +215,11 @@ fa_status fa_forward_varlen(fa_handle* h,
  * before the second one (the row sums use the unrounded values).  O is bf16 [B, Hq, Sq, 128], lse
  * fp32 [B, Hq, Sq] or NULL, both of Eq. 1 applied to the represented Q, K, V.  Only head size 128;
  * other sizes, and handles created with FA_FLAG_SERIAL_KERNEL, return FA_ERR_UNSUPPORTED.  The
- * K/V range is never split on this path.  Other arguments and errors as for fa_forward.
+ * tiling is planned as for fa_forward (pair or stream tiling, split-KV and shared query tiles for
+ * grouped heads on the stream tiling; the partials use the handle's scratch buffer); with shared
+ * query tiles of at most 64 rows the rows are additionally processed as two or four copies that
+ * each take a slice of every K/V tile's keys and are merged like split-KV partials.  Other
+ * arguments and errors as for fa_forward.
  */
 fa_status fa_forward_fp8(fa_handle* h,
                          const void* Q8, const void* K8, const void* V8,
