@@ -666,7 +666,10 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
 // Merge of the split-KV partials (Algorithm 2's reduction over the C spatial partitions, in the
 // corrected form: every partial is rescaled to the common maximum).  With O_c = G'_c / s_c and
 // lse_c = u_c + ln s_c the merged result is lse = ln sum_c exp(lse_c), O = sum_c exp(lse_c - lse) O_c.
-// One warp per query row, each lane four output columns per 128-column pass; HBM-bound.
+// One warp per query row.  The kernel runs behind the attention kernel of a latency-bound launch, so
+// it is written for few dependent round trips to memory: the lanes take the C log-sum-exps side by
+// side (two passes, reduced with shuffles), then every lane accumulates its four output columns
+// with the loads of four partials in flight at a time.
 template <int DV>
 __global__ void __launch_bounds__(128)
 fa_combine_kernel(const float* __restrict__ o_part, const float* __restrict__ lse_part,
@@ -678,22 +681,47 @@ fa_combine_kernel(const float* __restrict__ o_part, const float* __restrict__ ls
     const long long row = static_cast<long long>(blockIdx.x) * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= n_rows) return;
+    const float* lrow = lse_part + row;                 // partial c at lrow[c * n_rows]
     float m = -INFINITY;
-    for (int cidx = 0; cidx < n_splits; ++cidx) m = fmaxf(m, lse_part[cidx * n_rows + row]);
+    for (int cidx = lane; cidx < n_splits; cidx += 32) m = fmaxf(m, lrow[cidx * n_rows]);
+#pragma unroll
+    for (int sh = 16; sh > 0; sh >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, sh));
     float denom = 0.f;
     if (m != -INFINITY)
-        for (int cidx = 0; cidx < n_splits; ++cidx) denom += expf(lse_part[cidx * n_rows + row] - m);
+        for (int cidx = lane; cidx < n_splits; cidx += 32) denom += expf(lrow[cidx * n_rows] - m);
+#pragma unroll
+    for (int sh = 16; sh > 0; sh >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, sh);
     const float inv = denom > 0.f ? 1.f / denom : 0.f;
     const long long bh = row / Sq;
     __nv_bfloat16* o_row = O + (bh / Hq) * o_stride_b + (bh % Hq) * o_stride_h + (row - bh * Sq) * o_stride_s;
+    auto weight = [&](float lc) { return (lc == -INFINITY || m == -INFINITY) ? 0.f : expf(lc - m) * inv; };
 #pragma unroll
     for (int col = 0; col < DV; col += 128) {
         if (col + lane * 4 >= DV) break;
+        const float* orow = o_part + row * DV + col + lane * 4;     // partial c at orow[c * n_rows * DV]
+        const long long step = n_rows * DV;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int cidx = 0; cidx < n_splits; ++cidx) {
-            const float lc = lse_part[cidx * n_rows + row];
-            const float wgt = (lc == -INFINITY) ? 0.f : expf(lc - m) * inv;
-            const float4 v = *reinterpret_cast<const float4*>(o_part + (cidx * n_rows + row) * DV + col + lane * 4);
+        int cidx = 0;
+        for (; cidx + 4 <= n_splits; cidx += 4) {
+            float lc[4];
+            float4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                lc[u] = lrow[(cidx + u) * n_rows];
+                v[u] = *reinterpret_cast<const float4*>(orow + (cidx + u) * step);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float wgt = weight(lc[u]);
+                acc.x = fmaf(wgt, v[u].x, acc.x);
+                acc.y = fmaf(wgt, v[u].y, acc.y);
+                acc.z = fmaf(wgt, v[u].z, acc.z);
+                acc.w = fmaf(wgt, v[u].w, acc.w);
+            }
+        }
+        for (; cidx < n_splits; ++cidx) {
+            const float wgt = weight(lrow[cidx * n_rows]);
+            const float4 v = *reinterpret_cast<const float4*>(orow + cidx * step);
             acc.x = fmaf(wgt, v.x, acc.x);
             acc.y = fmaf(wgt, v.y, acc.y);
             acc.z = fmaf(wgt, v.z, acc.z);
