@@ -206,15 +206,15 @@ fa_status fa_forward_varlen(fa_handle* h,
 /*
  * Block-scaled 8-bit variant (the counterpart of the paper's block floating-point data path,
  * Section 3): Q8, K8, V8 hold e4m3 values (one byte each, the "fn" encoding without infinities),
- * contiguous [B, H, S, 128] DEVICE tensors, 16-byte aligned.  The represented tensors are
+ * contiguous [B, H, S, d] DEVICE tensors with d = 64 or 128, 16-byte aligned.  The represented tensors are
  *   Q[b,h,i,:] = q_scale[b,h,i/128] * Q8[b,h,i,:]     q_scale [B, Hq,  ceil(Sq/128)]
  *   K[b,h,j,:] = k_scale[b,h,j/128] * K8[b,h,j,:]     k_scale [B, Hkv, ceil(Sk/128)]
  *   V[b,h,j,:] = v_scale[b,h]       * V8[b,h,j,:]     v_scale [B, Hkv]
  * with positive fp32 scales in DEVICE memory (a NULL scale pointer means 1).  Both contractions
  * run on the 8-bit tensor-core path with fp32 accumulation; the probabilities are rounded to e4m3
- * before the second one (the row sums use the unrounded values).  O is bf16 [B, Hq, Sq, 128], lse
- * fp32 [B, Hq, Sq] or NULL, both of Eq. 1 applied to the represented Q, K, V.  Only head size 128;
- * other sizes, and handles created with FA_FLAG_SERIAL_KERNEL, return FA_ERR_UNSUPPORTED.  The
+ * before the second one (the row sums use the unrounded values).  O is bf16 [B, Hq, Sq, d], lse
+ * fp32 [B, Hq, Sq] or NULL, both of Eq. 1 applied to the represented Q, K, V.  Head sizes 64 and
+ * 128; other sizes, and handles created with FA_FLAG_SERIAL_KERNEL, return FA_ERR_UNSUPPORTED.  The
  * tiling is planned as for fa_forward (pair or stream tiling, split-KV and shared query tiles for
  * grouped heads on the stream tiling; the partials use the handle's scratch buffer); with shared
  * query tiles of at most 64 rows the rows are additionally processed as two or four copies that

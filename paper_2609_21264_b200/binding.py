@@ -268,8 +268,8 @@ def forward_varlen(h, q, k, v, cu_seqlens_q, cu_seqlens_k, max_sq: int, *, causa
 
 
 def forward_fp8(h, q8, k8, v8, q_scale, k_scale, v_scale, *, causal: bool, scale: float = 0.0, want_lse=True):
-    """Block-scaled e4m3 attention on torch CUDA tensors: q8/k8/v8 uint8 (or float8_e4m3fn) [B,H,S,128],
-    scales fp32 CUDA tensors or None.  Returns (O bf16 [B,Hq,Sq,128], lse fp32 [B,Hq,Sq])."""
+    """Block-scaled e4m3 attention on torch CUDA tensors: q8/k8/v8 uint8 (or float8_e4m3fn) [B,H,S,d]
+    with d = 64 or 128, scales fp32 CUDA tensors or None.  Returns (O bf16 [B,Hq,Sq,d], lse fp32 [B,Hq,Sq])."""
     import torch
     for t in (q8, k8, v8):
         if t.element_size() != 1 or not t.is_cuda or not t.is_contiguous() or t.dim() != 4:

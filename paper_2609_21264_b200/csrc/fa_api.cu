@@ -28,7 +28,7 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
 
 struct MapEntry {
     const void* ptr;
-    int d, S, H, B, box_rows, box_heads, elem_bytes;
+    int d, S, H, B, box_rows, box_heads, elem_bytes, swizzle_bytes;
     long long sb, sh, ss;      // batch / head / row strides in elements
     uint64_t stamp;
     CUtensorMap map;
@@ -57,7 +57,7 @@ struct fa_handle {
     const char* last_kernel = "";
     void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // Q K V O lse
     size_t stage_cap[5] = {0, 0, 0, 0, 0};
-    bool attr_done[32] = {};
+    bool attr_done[40] = {};
 #ifdef FA_TRACE
     long long* trace = nullptr;
 #endif
@@ -83,10 +83,11 @@ class DeviceGuard {
 // ptr + b*sb + h*sh + s*ss + c, seen as a 4-D TMA tensor (d, S, H, B); box = 128 bytes of columns
 // x box_rows rows, 128-byte swizzle, rows past S read as zero.
 fa_status get_map(fa_handle* h, const void* ptr, int d, int S, int H, int B, long long sb, long long sh,
-                  long long ss, int box_rows, const CUtensorMap** out, int elem_bytes = 2, int box_heads = 1) {
+                  long long ss, int box_rows, const CUtensorMap** out, int elem_bytes = 2, int box_heads = 1,
+                  int swizzle_bytes = 128) {
     for (auto& e : h->maps) {
         if (e.ptr == ptr && e.d == d && e.S == S && e.H == H && e.B == B && e.box_rows == box_rows &&
-            e.sb == sb && e.sh == sh && e.ss == ss && e.elem_bytes == elem_bytes && e.box_heads == box_heads) {
+            e.sb == sb && e.sh == sh && e.ss == ss && e.elem_bytes == elem_bytes && e.box_heads == box_heads && e.swizzle_bytes == swizzle_bytes) {
             e.stamp = ++h->stamp;
             *out = &e.map;
             return FA_OK;
@@ -95,19 +96,20 @@ fa_status get_map(fa_handle* h, const void* ptr, int d, int S, int H, int B, lon
     MapEntry ne;
     memset(&ne, 0, sizeof ne);
     ne.ptr = ptr; ne.d = d; ne.S = S; ne.H = H; ne.B = B; ne.box_rows = box_rows;
-    ne.sb = sb; ne.sh = sh; ne.ss = ss; ne.elem_bytes = elem_bytes; ne.box_heads = box_heads;
+    ne.sb = sb; ne.sh = sh; ne.ss = ss; ne.elem_bytes = elem_bytes; ne.box_heads = box_heads; ne.swizzle_bytes = swizzle_bytes;
     const cuuint64_t eb = static_cast<cuuint64_t>(elem_bytes);
     const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(S),
                                 static_cast<cuuint64_t>(H), static_cast<cuuint64_t>(B)};
     const cuuint64_t strides[3] = {static_cast<cuuint64_t>(ss) * eb, static_cast<cuuint64_t>(sh) * eb,
                                    static_cast<cuuint64_t>(sb) * eb};
-    const cuuint32_t box[4] = {static_cast<cuuint32_t>(128 / elem_bytes), static_cast<cuuint32_t>(box_rows),
+    const cuuint32_t box[4] = {static_cast<cuuint32_t>(swizzle_bytes / elem_bytes), static_cast<cuuint32_t>(box_rows),
                               static_cast<cuuint32_t>(box_heads), 1u};
     const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
     const CUresult r = h->encode(&ne.map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
                                  4, const_cast<void*>(ptr),
                                  dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return FA_ERR_INVALID_ARG;     // strides or extents the TMA unit cannot express
     ne.stamp = ++h->stamp;
@@ -774,9 +776,9 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
                          void* O, float* lse, int B, int Hq, int Hkv, int Sq, int Sk, int d, int causal,
                          float scale, void* stream) {
     if (!h) return FA_ERR_INVALID_ARG;
-    fa_status s = check_args(Q8, K8, V8, O, lse, B, Hq, Hkv, Sq, Sk, 128, 128, scale, true);
+    if (d != 64 && d != 128) return (d > 0) ? FA_ERR_UNSUPPORTED : FA_ERR_INVALID_ARG;
+    fa_status s = check_args(Q8, K8, V8, O, lse, B, Hq, Hkv, Sq, Sk, d, d, scale, true);
     if (s != FA_OK) return s;
-    if (d != 128) return FA_ERR_UNSUPPORTED;
     if ((q_scale && misaligned(q_scale, 4)) || (k_scale && misaligned(k_scale, 4)) || (v_scale && misaligned(v_scale, 4)))
         return FA_ERR_INVALID_ARG;
     if (h->flags & (FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD)) return FA_ERR_UNSUPPORTED;
@@ -791,13 +793,14 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     const LaunchPlan pl = plan_launch(h->num_sms, h->flags, h->kv_splits_cfg, h->scratch_bytes, false,
                                       B, Hq, Hkv, Sq, Sk, d, d, causal ? 1 : 0);
     const int q_box_rows = pl.pack_heads > 1 ? Sq : fa::kTileM;
+    // an e4m3 row is d bytes: one box column of d bytes, swizzled over d bytes
     const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;
     const long long hq_stride = static_cast<long long>(Sq) * d, hk_stride = static_cast<long long>(Sk) * d;
-    if ((s = get_map(h, Q8, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, q_box_rows, &mq, 1, pl.pack_heads)) != FA_OK) return s;
+    if ((s = get_map(h, Q8, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, q_box_rows, &mq, 1, pl.pack_heads, d)) != FA_OK) return s;
     CUtensorMap map_q = *mq;
-    if ((s = get_map(h, K8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mk, 1)) != FA_OK) return s;
+    if ((s = get_map(h, K8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mk, 1, 1, d)) != FA_OK) return s;
     CUtensorMap map_k = *mk;
-    if ((s = get_map(h, V8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mv, 1)) != FA_OK) return s;
+    if ((s = get_map(h, V8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mv, 1, 1, d)) != FA_OK) return s;
     CUtensorMap map_v = *mv;
     if ((s = get_map(h, O, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, q_box_rows, &mo, 2, pl.pack_heads)) != FA_OK) return s;
     CUtensorMap map_o = *mo;
@@ -829,6 +832,9 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     if (use_stream && pl.pack_heads > 1) {
         const int rows = pl.pack_heads * Sq;
         copies = rows <= 32 ? 4 : (rows <= 64 ? 2 : 1);
+        // every copy is one more partial per split for the merge kernel to read: with many splits
+        // (short CTAs, where the exponentials saved are few) the merge would cost more than it saves
+        while (copies > 1 && copies * p.kv_splits > 32) copies /= 2;
         const unsigned long long per_partial = static_cast<unsigned long long>(B) * Hq * Sq * (d + 1) * 4ull;
         while (copies > 1 && per_partial * p.kv_splits * copies > h->scratch_bytes) copies /= 2;
     }
@@ -848,14 +854,22 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = (h->flags & FA_FLAG_NO_DEPENDENT_LAUNCH) ? 0 : 1;
+    const bool d128 = (d == 128);
     if (use_stream) {
-        constexpr int smem = fa::fp8_stream_smem_bytes();
-        static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+        const int smem = d128 ? fa::fp8_stream_smem_bytes<128>() : fa::fp8_stream_smem_bytes<64>();
+        static_assert(fa::fp8_stream_smem_bytes<128>() <= 227 * 1024, "shared memory budget exceeded");
         const bool pack = pl.pack_heads > 1;
-        auto kernel = !pack ? fa::fa_fwd_fp8_stream_kernel<false, 1>
-                             : (copies == 4 ? fa::fa_fwd_fp8_stream_kernel<true, 4>
-                                            : (copies == 2 ? fa::fa_fwd_fp8_stream_kernel<true, 2> : fa::fa_fwd_fp8_stream_kernel<true, 1>));
-        if ((s = ensure_smem_attr(h, !pack ? 22 : (copies == 4 ? 28 : (copies == 2 ? 27 : 26)), kernel, smem)) != FA_OK) return s;
+        using Kernel = void (*)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, fa::FwdParams, fa::Fp8Params);
+        // variant: 0 = one head per tile, 1..3 = packed heads with 1, 2, 4 copies of the rows
+        const int variant = !pack ? 0 : (copies == 4 ? 3 : (copies == 2 ? 2 : 1));
+        static const Kernel kernels[2][4] = {
+            {fa::fa_fwd_fp8_stream_kernel<64, false, 1>, fa::fa_fwd_fp8_stream_kernel<64, true, 1>,
+             fa::fa_fwd_fp8_stream_kernel<64, true, 2>, fa::fa_fwd_fp8_stream_kernel<64, true, 4>},
+            {fa::fa_fwd_fp8_stream_kernel<128, false, 1>, fa::fa_fwd_fp8_stream_kernel<128, true, 1>,
+             fa::fa_fwd_fp8_stream_kernel<128, true, 2>, fa::fa_fwd_fp8_stream_kernel<128, true, 4>}};
+        static const int slots[2][4] = {{32, 33, 34, 35}, {22, 26, 27, 28}};
+        Kernel kernel = kernels[d128 ? 1 : 0][variant];
+        if ((s = ensure_smem_attr(h, slots[d128 ? 1 : 0][variant], kernel, smem)) != FA_OK) return s;
         const long long n_ctas = (pack ? static_cast<long long>(Hq / pl.pack_heads) : static_cast<long long>(p.n_q_tiles) * Hq) * B * p.kv_splits;
         if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
         cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
@@ -869,22 +883,23 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
             cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
             cfg.blockDim = dim3(128, 1, 1);
             cfg.dynamicSmemBytes = 0;
-            if (cudaLaunchKernelEx(&cfg, fa::fa_combine_kernel<128>, static_cast<const float*>(p.o_part),
+            auto combine = d128 ? fa::fa_combine_kernel<128> : fa::fa_combine_kernel<64>;
+            if (cudaLaunchKernelEx(&cfg, combine, static_cast<const float*>(p.o_part),
                                    static_cast<const float*>(p.lse_part), p.O, p.lse, n_rows, n_partials, p.Hq, p.Sq,
                                    p.o_stride_b, p.o_stride_h, p.o_stride_s) != cudaSuccess) return FA_ERR_CUDA;
             h->launches += 1;
         }
         return FA_OK;
     }
-    constexpr int smem = fa::fp8_smem_bytes();
-    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
-    static_assert(fa::Fp8Cfg::kThreads == 512, "block size");
-    if ((s = ensure_smem_attr(h, 11, fa::fa_fwd_fp8_kernel, smem)) != FA_OK) return s;
+    const int smem = d128 ? fa::fp8_smem_bytes<128>() : fa::fp8_smem_bytes<64>();
+    static_assert(fa::fp8_smem_bytes<128>() <= 227 * 1024, "shared memory budget exceeded");
+    auto kernel = d128 ? fa::fa_fwd_fp8_kernel<128> : fa::fa_fwd_fp8_kernel<64>;
+    if ((s = ensure_smem_attr(h, d128 ? 11 : 36, kernel, smem)) != FA_OK) return s;
     const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * Hq * B;
     if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
     cfg.dynamicSmemBytes = smem;
-    if (cudaLaunchKernelEx(&cfg, fa::fa_fwd_fp8_kernel, map_q, map_k, map_v, map_o, p, f) != cudaSuccess) return FA_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kernel, map_q, map_k, map_v, map_o, p, f) != cudaSuccess) return FA_ERR_CUDA;
     h->launches += 1;
     return FA_OK;
 }

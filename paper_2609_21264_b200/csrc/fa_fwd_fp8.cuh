@@ -16,7 +16,7 @@
 //     the row sums use the unrounded fp32 values, as in the bf16 kernel.
 // Everything else (roles, barriers, the two-tile schedule, lazy reference maximum kept in scaled
 // log2 units, bounded waits, TMA-store epilogue, dependent launch) is the bf16 kernel's; read
-// fa_fwd_pipelined.cuh first.  Head size 128, fixed-length contiguous [B,H,S,d] tensors, no
+// fa_fwd_pipelined.cuh first.  Head sizes 64 and 128, fixed-length contiguous [B,H,S,d] tensors, no
 // split-KV.  O is bf16, lse fp32.
 // TMEM: S_0 [0,128) S_1 [128,256) O_0 [256,384) O_1 [384,512); e4m3 P_t overlays S_t[0,32).
 #pragma once
@@ -29,12 +29,19 @@
 
 namespace fa {
 
+// D = head size of Q/K and of V: 128 (rows of 128 bytes, 128-byte swizzle) or 64 (rows of 64 bytes,
+// 64-byte swizzle: 8-row groups 512 bytes apart, a 32-key step of V 2048 bytes).
+template <int D>
 struct Fp8Cfg {
-    static constexpr int kD = 128;                       // head size of Q/K and of V
-    static constexpr int kTileBytes8 = kTileM * kD;      // one 128 x 128 e4m3 tile = 16 KB, one swizzled chunk
-    static constexpr int kOBytes = 2 * kChunkBytes;      // bf16 output tile (two 64-column chunks)
-    static constexpr int kKStages = 3;
-    static constexpr int kVStages = 3;
+    static_assert(D == 64 || D == 128, "head sizes of the 8-bit kernels");
+    static constexpr int kD = D;
+    static constexpr int kTileBytes8 = kTileM * kD;      // one 128 x D e4m3 tile (16 or 8 KB), one swizzled chunk
+    static constexpr int kOBytes = (D / kChunkCols) * kChunkBytes;      // bf16 output tile (64-column chunks)
+    static constexpr int kKStages = (D == 128) ? 3 : 4;
+    static constexpr int kVStages = (D == 128) ? 3 : 4;
+    // descriptor high word: stride between 8-row groups, version, swizzle mode
+    static constexpr uint32_t kDescHi = ((D == 128 ? 1024u : 512u) >> 4) | (1u << 14) | ((D == 128 ? 2u : 4u) << 29);
+    static constexpr uint32_t kVStep = (32u * D) >> 4;   // 32 keys of V, in descriptor address units
     // Q_0, Q_1, the K and V rings, and one staging buffer per query tile for the bf16 output
     static constexpr int kSmemTiles = (2 + kKStages + kVStages) * kTileBytes8 + 2 * kOBytes;
     static constexpr int kTmemCols = 512;
@@ -49,15 +56,17 @@ struct Fp8Params {
     int n_kv_tiles;          // ceil(Sk / 128)
 };
 
-constexpr int fp8_smem_bytes() { return Fp8Cfg::kSmemTiles + static_cast<int>(sizeof(PipeShared)); }
+template <int D>
+constexpr int fp8_smem_bytes() { return Fp8Cfg<D>::kSmemTiles + static_cast<int>(sizeof(PipeShared)); }
 
+template <int D>
 __global__ void __launch_bounds__(512, 1)
 fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
                   const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v,
                   const __grid_constant__ CUtensorMap tm_o,
                   const FwdParams p, const Fp8Params f) {
-    using Cfg = Fp8Cfg;
+    using Cfg = Fp8Cfg<D>;
     using namespace ptx;
     constexpr int NK = Cfg::kKStages;
     constexpr int NV = Cfg::kVStages;
@@ -363,11 +372,11 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
             const int nkv_t = (t == 0) ? nkv_0 : nkv_1;
             constexpr uint32_t kIdescQK = make_idesc_e4m3_f32(kTileM, kTileN, false, false);
             constexpr uint32_t kIdescPV = make_idesc_e4m3_f32(kTileM, DV, false, true);
-            constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // sbo, version, swizzle
-            // e4m3 rows of 128 elements are exactly one 128-byte swizzled row: a tile is one chunk
+            constexpr uint32_t kDescHi = Cfg::kDescHi;
+            // an e4m3 row of D elements is exactly one swizzled row of D bytes: a tile is one chunk
             const uint32_t q_lo = (((sQ + t * kTile8) & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
-            const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((16384u >> 4) << 16);   // one 128-byte chunk spans dv: the chunk stride is not used
+            const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((16384u >> 4) << 16);   // one swizzled row spans dv: the chunk stride is not used
             const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1);   // P_t overlays it
             const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1);
             const uint32_t bar_s = smem_addr(&sh.s_full[t]);
@@ -376,7 +385,7 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
             auto desc = [](uint32_t lo) -> uint64_t {
                 return (static_cast<uint64_t>(kDescHi) << 32) | lo;
             };
-            // S_t = Q_t K_j^T: four k-steps of 32 elements (32 bytes along the swizzled row)
+            // S_t = Q_t K_j^T: D / 32 k-steps of 32 elements (32 bytes along the swizzled row)
             auto issue_qk = [&](int stage) {
                 const uint32_t klo = k_lo0 + stage * (kTile8 >> 4);
 #pragma unroll
@@ -384,13 +393,13 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
                     mma_ss_f8(tS, desc(q_lo + k * 2), desc(klo + k * 2), kIdescQK, k > 0 ? 1u : 0u);
             };
             // O_t += P_t[:, 64*half .. 64*half+63] V_j[64*half .., :]: two k-steps of 32 keys
-            // (8 TMEM columns of P, 32 rows of 128 bytes of V)
+            // (8 TMEM columns of P, 32 rows of D bytes of V)
             auto issue_pv_half = [&](auto hc, int stage, uint32_t accumulate) {
                 constexpr int half = decltype(hc)::value;
                 const uint32_t vlo = v_lo0 + stage * (kTile8 >> 4);
 #pragma unroll
                 for (int kk = 2 * half; kk < 2 * half + 2; ++kk)
-                    mma_ts_f8(tO, tS + kk * 8, desc(vlo + kk * (4096 >> 4)), kIdescPV,
+                    mma_ts_f8(tO, tS + kk * 8, desc(vlo + kk * Cfg::kVStep), kIdescPV,
                               (half == 0 && kk == 0) ? accumulate : 1u);
             };
             const uint32_t bar_turn_mine = smem_addr(&sh.turn[t]);

@@ -6,7 +6,7 @@
 // tile and are folded into the exp2 constant of that tile, so the reference maximum that the
 // two warpgroups hand to each other is kept in scaled log2 units.  Used by fa_forward_fp8 where
 // the stream tiling is planned: grids under a wave and decode-like shapes with split-KV
-// (attention over an 8-bit K/V cache).  Head size 128, fixed-length contiguous tensors.
+// (attention over an 8-bit K/V cache).  Head sizes 64 and 128, fixed-length contiguous tensors.
 //   TMEM  S^0 [0,128)  S^1 [128,256)  O [256,384)  P^0 [384,416)  P^1 [448,480)
 #pragma once
 
@@ -15,10 +15,11 @@
 
 namespace fa {
 
+template <int D>
 struct Fp8StreamCfg {
-    static constexpr int kD = 128;
-    static constexpr int kTile8 = kTileM * kD;           // one 128 x 128 e4m3 tile = 16 KB, one swizzled chunk
-    static constexpr int kOBytes = 2 * kChunkBytes;      // bf16 output tile
+    static constexpr int kD = D;
+    static constexpr int kTile8 = kTileM * kD;           // one 128 x D e4m3 tile (16 or 8 KB), one swizzled chunk
+    static constexpr int kOBytes = (D / kChunkCols) * kChunkBytes;      // bf16 output tile
     static constexpr int kKStages = 4;
     static constexpr int kVStages = 4;
     static constexpr int kTileBytes = (1 + kKStages + kVStages) * kTile8 + kOBytes;
@@ -26,7 +27,8 @@ struct Fp8StreamCfg {
     static constexpr int kColS = 0, kColO = 256, kColP = 384;   // P^b at kColP + 64 b (32 columns used)
 };
 
-constexpr int fp8_stream_smem_bytes() { return Fp8StreamCfg::kTileBytes + static_cast<int>(sizeof(StreamShared)); }
+template <int D>
+constexpr int fp8_stream_smem_bytes() { return Fp8StreamCfg<D>::kTileBytes + static_cast<int>(sizeof(StreamShared)); }
 
 // kPack: several query heads of one K/V head share the query tile, as in fa_fwd_stream_kernel.
 // kRep (with kPack, 2 or 4): the pack has at most 128 / kRep rows and is loaded kRep times, copy
@@ -38,14 +40,14 @@ constexpr int fp8_stream_smem_bytes() { return Fp8StreamCfg::kTileBytes + static
 // partials.  A softmax warp then issues 1 / kRep of the exponentials per K/V tile (an
 // instruction costs the same for one live row as for 32), which takes a few-row problem from the
 // MUFU bound to the bound of the K/V stream.
-template <bool kPack = false, int kRep = 1>
+template <int D, bool kPack = false, int kRep = 1>
 __global__ void __launch_bounds__(512, 1)
 fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                      const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v,
                      const __grid_constant__ CUtensorMap tm_o,
                      const FwdParams p, const Fp8Params f) {
-    using Cfg = Fp8StreamCfg;
+    using Cfg = Fp8StreamCfg<D>;
     constexpr bool kVarlen = false;
     constexpr int DV = Cfg::kD;
     constexpr int kTile8 = Cfg::kTile8;
@@ -476,7 +478,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         setmaxnreg_dec<kRegsOther>();
         if (lane == 0 && n_kv > 0) {
             constexpr uint32_t kIdescQK = make_idesc_e4m3_f32(kTileM, kTileN, false, false);
-            constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // sbo, version, swizzle
+            constexpr uint32_t kDescHi = Fp8Cfg<D>::kDescHi;
             const uint32_t q_lo = ((sQ & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
             auto desc = [](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(kDescHi) << 32) | lo; };
@@ -492,7 +494,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 const uint32_t tS = tmem_base + Cfg::kColS + (j & 1) * 128;
                 const uint32_t klo = k_lo0 + sk * (kTile8 >> 4);
 #pragma unroll
-                for (int kk = 0; kk < Cfg::kD / 32; ++kk)      // four k-steps of 32 elements = 32 bytes
+                for (int kk = 0; kk < Cfg::kD / 32; ++kk)      // k-steps of 32 elements = 32 bytes
                     mma_ss_f8(tS, desc(q_lo + kk * 2), desc(klo + kk * 2), kIdescQK, kk > 0 ? 1u : 0u);
                 tc_commit(smem_addr(&sh.s_full[j & 1]));
                 tc_commit(smem_addr(&sh.k_empty[sk]));
@@ -504,8 +506,8 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         setmaxnreg_dec<kRegsOther>();
         if (lane == 0 && n_kv > 0) {
             constexpr uint32_t kIdescPV = make_idesc_e4m3_f32(kTileM, DV, false, true);
-            constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-            const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((16384u >> 4) << 16);   // one 128-byte chunk spans dv: the chunk stride is not used
+            constexpr uint32_t kDescHi = Fp8Cfg<D>::kDescHi;
+            const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((16384u >> 4) << 16);   // one swizzled row spans dv: the chunk stride is not used
             const uint32_t tO = tmem_base + Cfg::kColO;
             auto desc = [](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(kDescHi) << 32) | lo; };
             int sv = 0;
@@ -520,8 +522,8 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 const uint32_t tP = tmem_base + Cfg::kColP + (j & 1) * 64;
                 const uint32_t vlo = v_lo0 + sv * (kTile8 >> 4);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)                  // four k-steps of 32 keys: 8 P columns, 32 V rows of 128 bytes
-                    mma_ts_f8(tO, tP + kk * 8, desc(vlo + kk * (4096 >> 4)), kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+                for (int kk = 0; kk < 4; ++kk)                  // four k-steps of 32 keys: 8 P columns, 32 V rows of D bytes
+                    mma_ts_f8(tO, tP + kk * 8, desc(vlo + kk * Fp8Cfg<D>::kVStep), kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
                 tc_commit(smem_addr(&sh.p_free[j & 1]));
                 tc_commit(smem_addr(&sh.v_empty[sv]));
                 if (j + 1 == n_kv) tc_commit(smem_addr(&sh.o_final));
@@ -538,9 +540,9 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             {
                 const uint32_t bar = smem_addr(&sh.q_full);
                 // with packed heads the box is Sq rows x pack_heads heads (row h * Sq + i of the tile)
-                mbar_arrive_expect_tx(bar, kPack ? static_cast<uint32_t>(kRep * p.pack_heads * Sq * 128) : static_cast<uint32_t>(kTile8));
+                mbar_arrive_expect_tx(bar, kPack ? static_cast<uint32_t>(kRep * p.pack_heads * Sq * D) : static_cast<uint32_t>(kTile8));
 #pragma unroll
-                for (int r = 0; r < kRep; ++r) tma_load_4d(sQ + r * kRepRows * 128, &tm_q, bar, 0, q_row0 + i0, hq, tb);
+                for (int r = 0; r < kRep; ++r) tma_load_4d(sQ + r * kRepRows * D, &tm_q, bar, 0, q_row0 + i0, hq, tb);
             }
             bool ok = true;
             for (int j = 0; j < n_kv && ok; ++j) {

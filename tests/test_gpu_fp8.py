@@ -42,8 +42,8 @@ def _run(handle, w, q8, k8, v8, sq, sk, sv):
     return bf16_tensor_to_f64(o), lse.double().cpu().numpy()
 
 
-def _wl(name, B, Hq, Hkv, Sq, Sk, causal, seed, sigma=1.0):
-    return W.Workload(name, B=B, Hq=Hq, Hkv=Hkv, Sq=Sq, Sk=Sk, dqk=128, dv=128, causal=causal, scale=128 ** -0.5,
+def _wl(name, B, Hq, Hkv, Sq, Sk, causal, seed, sigma=1.0, d=128):
+    return W.Workload(name, B=B, Hq=Hq, Hkv=Hkv, Sq=Sq, Sk=Sk, dqk=d, dv=d, causal=causal, scale=d ** -0.5,
                       sigma=sigma, seed=seed)
 
 
@@ -61,6 +61,14 @@ CASES = [
     _wl("fp8_group4_sq4_causal_four_copies", 2, 8, 2, 4, 1111, True, 1343),
     _wl("fp8_group4_sq13_causal_two_copies", 1, 8, 2, 13, 777, True, 1344),
     _wl("fp8_group2_sq3_more_queries_than_keys", 1, 4, 2, 3, 2, True, 1345),
+    # head size 64: rows of 64 bytes, 64-byte swizzle
+    _wl("fp8_d64_gqa_causal_ragged", 2, 8, 2, 333, 333, True, 1350, d=64),
+    _wl("fp8_d64_mha_full_sq_ne_sk", 1, 4, 4, 200, 457, False, 1351, d=64),
+    _wl("fp8_d64_gpt2_like_s1024", 1, 12, 12, 1024, 1024, True, 1352, d=64),
+    _wl("fp8_d64_one_tile_many_keys", 1, 2, 1, 100, 2100, False, 1353, d=64),
+    _wl("fp8_d64_group7_single_query", 2, 14, 2, 1, 3000, False, 1354, d=64),
+    _wl("fp8_d64_group4_sq10_causal", 1, 8, 2, 10, 900, True, 1355, d=64),
+    _wl("fp8_d64_group2_sq50", 1, 4, 2, 50, 640, True, 1356, d=64),
 ]
 
 
@@ -186,8 +194,8 @@ def test_fp8_default_handle_plans_both_tilings():
 def test_fp8_unsupported_head_size(handle):
     import torch
     from paper_2609_21264_b200 import binding
-    z = torch.zeros((1, 1, 128, 64), dtype=torch.uint8, device="cuda")
-    o = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device="cuda")
+    z = torch.zeros((1, 1, 128, 192), dtype=torch.uint8, device="cuda")
+    o = torch.zeros((1, 1, 128, 192), dtype=torch.bfloat16, device="cuda")
     st = binding.fa_forward_fp8(handle, z.data_ptr(), z.data_ptr(), z.data_ptr(), None, None, None, o.data_ptr(), None,
-                                1, 1, 1, 128, 128, 64, False, 0.0)
+                                1, 1, 1, 128, 128, 192, False, 0.0)
     assert st == binding.FA_ERR_UNSUPPORTED

@@ -96,7 +96,8 @@ def test_random_decode_shape_matches_oracle(handle, w):
     assert_parity(O, lse, O_ref, lse_ref, w.name)
 
 
-@pytest.mark.parametrize("w", [w for w in DECODE_CASES if w.dqk == 128], ids=[w.name for w in DECODE_CASES if w.dqk == 128])
+@pytest.mark.parametrize("w", [w for w in DECODE_CASES if w.dqk in (64, 128)],
+                         ids=[w.name for w in DECODE_CASES if w.dqk in (64, 128)])
 def test_random_decode_shape_e4m3_matches_oracle_on_represented_tensors(handle, w):
     import torch
     from paper_2609_21264_b200 import binding

@@ -50,7 +50,8 @@ def test_sigma_sweep_stays_below_the_papers_error_curve(handle, causal):
         print("sigma %.2f  MAE %.2e (paper %.2e)  min Pearson %.6f (paper %.4f)" % row)
 
 
-def test_sigma_sweep_of_the_block_scaled_e4m3_path():
+@pytest.mark.parametrize("d", [64, 128], ids=["d64_the_papers_shape", "d128"])
+def test_sigma_sweep_of_the_block_scaled_e4m3_path(d):
     """The same protocol for the 8-bit variant: Q, K (one scale per 128-row block) and V (one per
     head) quantised to e4m3 from the same N(0, sigma^2) inputs.
 
@@ -65,7 +66,7 @@ def test_sigma_sweep_of_the_block_scaled_e4m3_path():
     import torch
     from paper_2609_21264_b200 import binding
     g = json.load(open(GOLDEN))
-    H, d, S = g["shape"]["H"], 128, g["shape"]["S"]          # the 8-bit kernels have head size 128
+    H, S = g["shape"]["H"], g["shape"]["S"]
     h = binding.fa_create()
     report = []
     try:
