@@ -76,3 +76,33 @@ def test_kv_tile_count_matches_visibility_rule():
                        if (not causal) or j <= i + Sk - Sq]
                 want = 0 if not vis else max(vis) // 128 + 1
                 assert kv_tiles(i0, 128, Sq, Sk, causal) == want
+
+
+def test_flag_and_status_constants_match_the_header():
+    """The binding's FA_FLAG_* / FA_* constants are the header's, name for name and value for value."""
+    from paper_2609_21264_b200 import binding
+    text = open(os.path.join(ROOT, "include", "fa.h")).read()
+    flags = dict(re.findall(r"#define\s+(FA_FLAG_[A-Z_]+)\s+(\d+)u", text))
+    assert len(flags) >= 8
+    for name, value in flags.items():
+        assert getattr(binding, name) == int(value), name
+    values = [int(v) for v in flags.values()]
+    assert len(set(values)) == len(values) and all(v & (v - 1) == 0 for v in values)     # distinct single bits
+    for name in dir(binding):
+        if name.startswith("FA_FLAG_"):
+            assert name in flags, name
+
+
+def test_plan_info_struct_matches_the_header():
+    """fa_plan_info is read through ctypes: field order and types must follow the header's struct."""
+    from paper_2609_21264_b200 import binding
+    text = open(os.path.join(ROOT, "include", "fa.h")).read()
+    body = re.search(r"typedef struct fa_plan_info \{(.*?)\} fa_plan_info;", text, flags=re.S).group(1)
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    fields = re.findall(r"(const char\*|int32_t|int64_t|double)\s+([a-z_]+(?:\s*,\s*[a-z_]+)*)\s*;", body)
+    header = []
+    for ctype, names in fields:
+        for n in names.split(","):
+            header.append((n.strip(), ctype))
+    ctypes_of = {"const char*": ctypes.c_char_p, "int32_t": ctypes.c_int32, "int64_t": ctypes.c_int64, "double": ctypes.c_double}
+    assert [(n, ctypes_of[t]) for n, t in header] == list(binding.fa_plan_info._fields_)
