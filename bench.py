@@ -395,6 +395,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the short timing of the other configs")
     ap.add_argument("--table6", action="store_true",
                     help="also time the twelve attention shapes of the paper's Table 6 (key 'table6')")
+    ap.add_argument("--no-decode", action="store_true", help="skip the grouped-head decode step (key 'decode')")
     ap.add_argument("--libraries", action="store_true",
                     help="also time the attention kernels of the libraries in the image (torch SDPA back ends, flash_attn) "
                          "on the five configurations and a few decode shapes, for context (key 'libraries')")
@@ -505,7 +506,7 @@ def main():
                                      "note": "fa_forward_fp8, N(0,sigma^2) rounded to e4m3, unit scales, one input set"}
         del q8, k8, v8, o8, l8
 
-    if not args.no_sweep and world == 1:
+    if not args.no_decode and world == 1:
         # Decoding with grouped heads (few queries over a long K/V sequence): bound by the K/V read, so the
         # figure of merit is bytes per second against the measured copy bandwidth.  bf16 and e4m3 K/V.
         dB, dHq, dHkv, dSq, dSk = 64, 32, 8, 1, 4096
