@@ -190,8 +190,9 @@ fa_status fa_forward_strided(fa_handle* h,
  * query i iff j <= i + (Sk_b - Sq_b).  A sequence with no keys, and any row with no visible key,
  * gets O = 0 and lse = -inf; a sequence with no queries writes nothing.  Rows of K/V past the end
  * of a sequence take no part in the result, but must hold finite numbers where they belong to the
- * next sequence (they are multiplied by a zero probability).  The K/V range is never split over
- * CTAs on this path.  With max_sq <= 64 and several query heads per K/V head the heads of a group
+ * next sequence (they are multiplied by a zero probability).  The K/V range is split over CTAs
+ * only for batches with a single 128-row query tile per sequence (max_sq <= 128) that would
+ * leave most SMs idle; every CTA then cuts its own sequence into the equal shares.  With max_sq <= 64 and several query heads per K/V head the heads of a group
  * share a query tile (see FA_FLAG_NO_HEAD_PACKING): a decode step over sequences of different
  * lengths then reads every K/V head once.  Errors as for fa_forward.
  */

@@ -315,14 +315,16 @@ fa_status launch_stream(fa_handle* h, int slot, const CUtensorMap& mq, const CUt
     if (cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mo, p) != cudaSuccess) return FA_ERR_CUDA;
     h->launches += 1;
     if (p.kv_splits > 1) {
-        const long long n_rows = static_cast<long long>(p.B) * p.Hq * p.Sq;
+        // packed batches are one batch slice of total_q rows per head ([Hq, total_q] partials and lse)
+        const int rows_per_head = kVarlen ? p.total_q : p.Sq;
+        const long long n_rows = static_cast<long long>(kVarlen ? 1 : p.B) * p.Hq * rows_per_head;
         const long long blocks = (n_rows + 3) / 4;
         if (blocks > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
         cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
         cfg.blockDim = dim3(128, 1, 1);
         cfg.dynamicSmemBytes = 0;
         if (cudaLaunchKernelEx(&cfg, fa::fa_combine_kernel<DV>, static_cast<const float*>(p.o_part),
-                               static_cast<const float*>(p.lse_part), p.O, p.lse, n_rows, p.kv_splits, p.Hq, p.Sq,
+                               static_cast<const float*>(p.lse_part), p.O, p.lse, n_rows, p.kv_splits, p.Hq, rows_per_head,
                                p.o_stride_b, p.o_stride_h, p.o_stride_s) != cudaSuccess) return FA_ERR_CUDA;
         h->launches += 1;
     }
@@ -418,7 +420,8 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
         if (hp > 1) {
             pl.kernel = kPlanStream;
             pl.pack_heads = hp;
-            with_splits(varlen ? 1 : choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles, true, hp));
+            // (packed batches: Sk is the mean K/V length; every CTA cuts its own sequence into the C shares)
+            with_splits(choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles, true, hp));
             return pl;
         }
     }
@@ -440,7 +443,8 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     bool stream = false;
     int stream_splits = 1;
     if (!drop && !(flags & FA_FLAG_NO_STREAM_KERNEL)) {
-        if (!varlen) stream_splits = choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles, true);
+        // packed batches split only with a single query tile per sequence (decode-like), by the mean K/V length
+        if (!varlen || n_q_tiles == 1) stream_splits = choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles, true);
         if (flags & FA_FLAG_STREAM_KERNEL) {
             stream = true;
         } else if (varlen) {
@@ -501,8 +505,10 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
     p.o_part = nullptr;
     p.lse_part = nullptr;
     if (pl.kv_splits > 1) {
+        // partials [C, B*Hq, Sq, dv] and [C, B*Hq, Sq]; packed batches: [C, Hq, total_q, dv] and [C, Hq, total_q]
+        const size_t rows = cu_q ? static_cast<size_t>(Hq) * total_q : static_cast<size_t>(B) * Hq * Sq;
         p.o_part = static_cast<float*>(h->scratch);
-        p.lse_part = p.o_part + static_cast<size_t>(pl.kv_splits) * B * Hq * Sq * dv;
+        p.lse_part = p.o_part + static_cast<size_t>(pl.kv_splits) * rows * dv;
     }
     h->last_splits = p.kv_splits;
 #ifdef FA_TRACE

@@ -150,9 +150,12 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int i0 = q_tile * kTileM;
     if (kVarlen && i0 >= Sq) return;      // a sequence shorter than the longest one (whole CTA, before any set-up)
     // K/V tiles [j_base, j_base + n_kv) of the query tile belong to this CTA (all visible ones without split-KV)
-    const int j_base = split * p.tiles_per_split;
-    int n_kv = kv_tiles_for_q_tile(i0, kTileM, Sq, Sk, p.causal) - j_base;
-    if (n_kv > p.tiles_per_split) n_kv = p.tiles_per_split;
+    // (packed batches: the host does not know the lengths, so the C equal shares are cut here)
+    const int n_kv_all = kv_tiles_for_q_tile(i0, kTileM, Sq, Sk, p.causal);
+    const int tiles_per_split = (kVarlen && p.kv_splits > 1) ? (n_kv_all + p.kv_splits - 1) / p.kv_splits : p.tiles_per_split;
+    const int j_base = split * tiles_per_split;
+    int n_kv = n_kv_all - j_base;
+    if (n_kv > tiles_per_split) n_kv = tiles_per_split;
     if (n_kv < 0) n_kv = 0;
     const int tb = kVarlen ? 0 : b;       // batch coordinate of the tensor maps (packed tensors have one slice)
 
@@ -345,7 +348,8 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             const long long o_base = (kVarlen ? q_row0 * p.o_stride_s : b * p.o_stride_b) + hq_row * p.o_stride_h;
             if (p.kv_splits > 1 && n_kv == 0) {      // an empty range: a neutral partial
                 if (row_valid) {
-                    const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
+                    const size_t prow = kVarlen ? (static_cast<size_t>(split) * p.Hq + hq_row) * p.total_q + q_row0 + i_glob
+                                                : (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
                     float* po_row = p.o_part + prow * DV + g * (DV / 2);
                     const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
@@ -392,7 +396,9 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     const bool box_store = !kVarlen || (i0 + kTileM <= Sq);
                     if (p.kv_splits > 1) {
                         // split-KV: G'_c / s_c in fp32 and u_c + ln s_c go to scratch (Algorithm 2's partials)
-                        const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
+                        // fixed lengths: partials [C, B*Hq, Sq]; packed batches: [C, Hq, total_q]
+                        const size_t prow = kVarlen ? (static_cast<size_t>(split) * p.Hq + hq_row) * p.total_q + q_row0 + i_glob
+                                                    : (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
                         float* po_row = p.o_part + prow * DV;
                         if (g == 0 && row_valid)
                             p.lse_part[prow] = (lt > 0.f) ? (m_fin * c * 0.6931471805599453f + logf(lt)) : -INFINITY;

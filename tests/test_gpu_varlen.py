@@ -148,3 +148,26 @@ def test_decode_batches_plan_shared_query_tiles():
     assert p["kernel"] == "fa_fwd_stream" and p["heads_per_tile"] == 4 and p["kv_splits"] == 1 and p["ctas"] == 32 * 8
     assert binding.fa_plan(148, 32, 32, 8, 1, 4096, 128, 128, True, varlen=True,
                            flags=binding.FA_FLAG_NO_HEAD_PACKING)["heads_per_tile"] == 1
+
+
+@pytest.mark.parametrize("splits", [0, 3, 5], ids=["auto", "3_splits", "5_splits"])
+@pytest.mark.parametrize("grouped", [True, False], ids=["grouped_heads", "one_head_per_kv_head"])
+def test_small_decode_batches_split_the_kv_range(splits, grouped):
+    """A few sequences with one query tile each leave most SMs without work: the K/V range of every
+    sequence is cut into C shares by its own CTAs (the lengths are only known on the device),
+    the partials are merged by the combine kernel.  Includes an empty K/V sequence, a sequence
+    with fewer tiles than shares, and a causal mask."""
+    from paper_2609_21264_b200 import binding
+    h = binding.fa_create(flags=binding.FA_FLAG_STREAM_KERNEL, kv_splits=splits)
+    try:
+        Hq, Hkv = (8, 2) if grouped else (4, 4)
+        for causal in (False, True):
+            _run_and_check(h, [1, 5, 1, 30], [4000, 130, 0, 2500], Hq=Hq, Hkv=Hkv, dqk=128, dv=128, causal=causal, seed=1130 + splits)
+            assert binding.fa_last_kernel_name(h) == "fa_fwd_stream"
+            if splits:
+                assert binding.fa_last_kv_splits(h) == splits
+            else:
+                assert binding.fa_last_kv_splits(h) > 1
+        _run_and_check(h, [100, 128, 7], [3000, 1500, 700], Hq=Hq, Hkv=Hkv, dqk=64, dv=64, causal=True, seed=1140 + splits)
+    finally:
+        binding.fa_destroy(h)

@@ -55,9 +55,12 @@ def test_few_queries_with_grouped_heads_share_a_query_tile():
     # not with more than 64 queries, one head per K/V head, or when switched off
     assert binding.fa_plan(SMS, 1, 12, 2, 65, 4096, 64, 64, True)["heads_per_tile"] == 1
     assert binding.fa_plan(SMS, 1, 12, 12, 16, 4096, 64, 64, True)["heads_per_tile"] == 1
-    # packed batches of sequences (lengths on the device): packed heads, no split
+    # packed batches of sequences (lengths on the device): packed heads; a small batch also splits the
+    # K/V range (every CTA cuts its own sequence), a large one does not
     p = binding.fa_plan(SMS, 4, 16, 4, 16, 1024, 128, 128, True, varlen=True)
-    assert p["kernel"] == "fa_fwd_stream" and p["heads_per_tile"] == 4 and p["kv_splits"] == 1 and p["ctas"] == 4 * 4
+    assert p["kernel"] == "fa_fwd_stream" and p["heads_per_tile"] == 4 and p["kv_splits"] == 4 and p["ctas"] == 4 * 4 * 4
+    p = binding.fa_plan(SMS, 64, 16, 4, 16, 1024, 128, 128, True, varlen=True)
+    assert p["heads_per_tile"] == 4 and p["kv_splits"] == 1 and p["ctas"] == 64 * 4
     for flag in (binding.FA_FLAG_NO_HEAD_PACKING, binding.FA_FLAG_NO_STREAM_KERNEL, binding.FA_FLAG_SERIAL_KERNEL):
         assert binding.fa_plan(SMS, 8, 32, 8, 1, 8192, 128, 128, False, flags=flag)["heads_per_tile"] == 1
 
