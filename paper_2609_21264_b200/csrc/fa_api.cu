@@ -153,15 +153,17 @@ fa_status launch_simple(fa_handle* h, int slot, const CUtensorMap& mq, const CUt
     return FA_OK;
 }
 
-template <int DQK, int DV, bool kVarlen>
+template <int DQK, int DV, bool kVarlen, bool kHeadPair = false>
 fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
                            const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
     constexpr int smem = fa::pipe_smem_bytes<DQK, DV>();
     static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
-    auto kernel = fa::fa_fwd_pipelined_kernel<DQK, DV, kVarlen>;
+    auto kernel = fa::fa_fwd_pipelined_kernel<DQK, DV, kVarlen, kHeadPair>;
     fa_status s = ensure_smem_attr(h, slot, kernel, smem);
     if (s != FA_OK) return s;
-    const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq * p.B * p.kv_splits;
+    // items: pairs of adjacent query tiles of a head, or one query tile of a pair of adjacent heads
+    const long long n_ctas = (kHeadPair ? static_cast<long long>(p.n_q_tiles) * (p.Hq / 2)
+                                        : static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq) * p.B * p.kv_splits;
     if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     // Programmatic stream serialisation: the kernel may be scheduled while its predecessor in the
     // stream drains (both kernels wait for that predecessor's completion before they touch global
@@ -273,7 +275,8 @@ fa_status launch_persistent(fa_handle* h, int slot, const CUtensorMap& mq, const
     auto kernel = fa::fa_fwd_persistent_kernel<DQK, DV>;
     fa_status s = ensure_smem_attr(h, slot, kernel, smem);
     if (s != FA_OK) return s;
-    const long long n_items = static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq * p.B;
+    const long long n_items = p.head_pair ? static_cast<long long>(p.n_q_tiles) * (p.Hq / 2) * p.B
+                                          : static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq * p.B;
     if (n_items > 0x3fffffffLL) return FA_ERR_UNSUPPORTED;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -339,7 +342,7 @@ fa_status launch_stream(fa_handle* h, int slot, const CUtensorMap& mq, const CUt
 // on, which is enough to tell a grid of under one wave (the stream kernel's case) from the rest.
 struct TilingEstimate { double pair_us, stream_us; };
 TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int dqk, int causal, int n_q_tiles, int splits,
-                                int stream_splits) {
+                                int stream_splits, bool head_pair) {
     // (at d_qk = 192 the pair kernel only has room for two K stages and one V stage and a longer MMA
     // chain per round; the stream kernel is ahead there at every size measured)
     const double a_p = dqk == 64 ? 1.36 : (dqk == 128 ? 2.0 : 2.9), f_p = dqk == 64 ? 6.0 : 6.7;
@@ -351,7 +354,11 @@ TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int 
         const double cs = a_s * ((r + stream_splits - 1) / stream_splits) + f_s;
         stream_total += cs * stream_splits;
         if (cs > stream_max) stream_max = cs;
-        if ((t & 1) == 1 || t == n_q_tiles - 1) {        // second tile of a pair, or an unpaired last tile
+        if (head_pair) {                                  // every query tile is an item of two heads
+            const double cp = a_p * r + f_p;
+            pair_total += 0.5 * cp;
+            if (cp > pair_max) pair_max = cp;
+        } else if ((t & 1) == 1 || t == n_q_tiles - 1) {  // second tile of a pair, or an unpaired last tile
             const double rounds = (r + splits - 1) / splits;
             const double cp = a_p * rounds + f_p;
             pair_total += cp * splits;
@@ -368,7 +375,8 @@ TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int 
         return balanced > longest ? balanced : longest;
     };
     TilingEstimate e;
-    e.pair_us = makespan(pair_total, pair_max, static_cast<double>((n_q_tiles + 1) / 2) * splits) + (splits > 1 ? 6.0 : 0.0);
+    e.pair_us = makespan(pair_total, pair_max, head_pair ? 0.5 * n_q_tiles : static_cast<double>((n_q_tiles + 1) / 2) * splits) +
+                (splits > 1 ? 6.0 : 0.0);
     e.stream_us = makespan(stream_total, stream_max, static_cast<double>(n_q_tiles) * stream_splits) + (stream_splits > 1 ? 6.0 : 0.0);
     return e;
 }
@@ -381,6 +389,7 @@ struct LaunchPlan {
     int kv_splits;
     int tiles_per_split;
     int pack_heads;                // > 1: stream kernel with that many query heads of a K/V head per query tile
+    bool head_pair;                // pair kernel: the CTA's two tiles are one query tile of two adjacent heads of a group
     double pair_us, stream_us;     // the two estimates (0 when no estimate was needed)
 };
 LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size_t scratch_bytes, bool varlen,
@@ -390,6 +399,7 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     pl.kv_splits = 1;
     pl.tiles_per_split = 0x3fffffff;
     pl.pack_heads = 1;
+    pl.head_pair = false;
     pl.pair_us = pl.stream_us = 0.0;
     const int n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
     const bool drop = (flags & FA_FLAG_DEBUG_DROP_V_LOAD) != 0;
@@ -440,6 +450,10 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     // One query tile per CTA (twice the CTAs, each with a shorter chain) wins where the pair
     // kernel's grid does not fill the GPU or its longest CTA dominates: decided from the two
     // estimates, with a margin, each side with its own split count.
+    // Causal grouped-query attention: pairing the same query tile of two heads of a group gives both
+    // tiles of a pair-kernel CTA the same number of K/V tiles (no round that one of them runs alone).
+    const bool head_pair_ok = !varlen && !drop && causal && pair_splits == 1 && (Hq / Hkv) % 2 == 0 &&
+                              !(flags & FA_FLAG_NO_HEAD_PACKING);
     bool stream = false;
     int stream_splits = 1;
     if (!drop && !(flags & FA_FLAG_NO_STREAM_KERNEL)) {
@@ -452,7 +466,7 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
             // per sequence the pair kernel's second tile would be empty
             stream = (dqk == 192) || n_q_tiles == 1;
         } else if (!persistent) {
-            const TilingEstimate e = estimate_tilings(num_sms, B, Hq, Sq, Sk, dqk, causal, n_q_tiles, pair_splits, stream_splits);
+            const TilingEstimate e = estimate_tilings(num_sms, B, Hq, Sq, Sk, dqk, causal, n_q_tiles, pair_splits, stream_splits, head_pair_ok);
             pl.pair_us = e.pair_us;
             pl.stream_us = e.stream_us;
             stream = e.stream_us < 0.9 * e.pair_us;
@@ -466,9 +480,11 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
         with_splits(stream_splits);
     } else if (persistent) {
         pl.kernel = kPlanPersistent;
+        pl.head_pair = head_pair_ok;
     } else {
         pl.kernel = kPlanPair;
         with_splits(pair_splits);
+        pl.head_pair = head_pair_ok;
     }
     return pl;
 }
@@ -502,6 +518,7 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
     p.kv_splits = pl.kv_splits;
     p.tiles_per_split = pl.tiles_per_split;
     p.pack_heads = pl.pack_heads;
+    p.head_pair = pl.head_pair ? 1 : 0;
     p.o_part = nullptr;
     p.lse_part = nullptr;
     if (pl.kv_splits > 1) {
@@ -547,6 +564,11 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
             if (dqk == 64) return launch_pipelined<64, 64, true>(h, 6, map_q, map_k, map_v, map_o, p, st);
             if (dqk == 128) return launch_pipelined<128, 128, true>(h, 7, map_q, map_k, map_v, map_o, p, st);
             return launch_pipelined<192, 128, true>(h, 8, map_q, map_k, map_v, map_o, p, st);
+        }
+        if (pl.head_pair) {
+            if (dqk == 64) return launch_pipelined<64, 64, false, true>(h, 37, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_pipelined<128, 128, false, true>(h, 38, map_q, map_k, map_v, map_o, p, st);
+            return launch_pipelined<192, 128, false, true>(h, 39, map_q, map_k, map_v, map_o, p, st);
         }
         if (dqk == 64) return launch_pipelined<64, 64, false>(h, 3, map_q, map_k, map_v, map_o, p, st);
         if (dqk == 128) return launch_pipelined<128, 128, false>(h, 4, map_q, map_k, map_v, map_o, p, st);
@@ -899,9 +921,12 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     }
     const int smem = d128 ? fa::fp8_smem_bytes<128>() : fa::fp8_smem_bytes<64>();
     static_assert(fa::fp8_smem_bytes<128>() <= 227 * 1024, "shared memory budget exceeded");
-    auto kernel = d128 ? fa::fa_fwd_fp8_kernel<128> : fa::fa_fwd_fp8_kernel<64>;
-    if ((s = ensure_smem_attr(h, d128 ? 11 : 36, kernel, smem)) != FA_OK) return s;
-    const long long n_ctas = static_cast<long long>((p.n_q_tiles + 1) / 2) * Hq * B;
+    // causal grouped heads: the CTA's two tiles are one query tile of two adjacent heads (see plan_launch)
+    const bool hp = pl.head_pair && (pl.kernel == kPlanPair || pl.kernel == kPlanPersistent);
+    auto kernel = hp ? (d128 ? fa::fa_fwd_fp8_kernel<128, true> : fa::fa_fwd_fp8_kernel<64, true>)
+                     : (d128 ? fa::fa_fwd_fp8_kernel<128, false> : fa::fa_fwd_fp8_kernel<64, false>);
+    if ((s = ensure_smem_attr(h, hp ? (d128 ? 14 : 15) : (d128 ? 11 : 36), kernel, smem)) != FA_OK) return s;
+    const long long n_ctas = (hp ? static_cast<long long>(p.n_q_tiles) * (Hq / 2) : static_cast<long long>((p.n_q_tiles + 1) / 2) * Hq) * B;
     if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
     cfg.dynamicSmemBytes = smem;
@@ -933,8 +958,11 @@ fa_status fa_plan(int num_sms, const fa_config* cfg, int varlen, int B, int Hq, 
     long long ctas = 0;
     switch (pl.kernel) {
         case kPlanSerial: ctas = n_q_tiles * Hq * B; break;
-        case kPlanPair: ctas = ((n_q_tiles + 1) / 2) * Hq * B * pl.kv_splits; break;
-        case kPlanPersistent: ctas = ((n_q_tiles + 1) / 2) * Hq * B; if (ctas > num_sms) ctas = num_sms; break;
+        case kPlanPair: ctas = (pl.head_pair ? n_q_tiles * (Hq / 2) : ((n_q_tiles + 1) / 2) * Hq) * B * pl.kv_splits; break;
+        case kPlanPersistent:
+            ctas = (pl.head_pair ? n_q_tiles * (Hq / 2) : ((n_q_tiles + 1) / 2) * Hq) * B;
+            if (ctas > num_sms) ctas = num_sms;
+            break;
         default: ctas = n_q_tiles * (Hq / pl.pack_heads) * B * pl.kv_splits; break;
     }
     out->ctas = ctas;

@@ -43,6 +43,7 @@ struct FwdParams {
     int kv_splits;            // C >= 1: CTAs per item, each with its own range of K/V tiles
     int tiles_per_split;      // K/V tiles per split (all of them when kv_splits == 1)
     int pack_heads;           // query heads of one K/V head sharing a query tile (stream kernels with kPack; else unused)
+    int head_pair;            // persistent kernel: 1 = an item is one query tile of two adjacent heads of a group
     float* o_part;            // [C, B*Hq, Sq, dv] fp32 partial outputs (split-KV only)
     float* lse_part;          // [C, B*Hq, Sq] fp32 partial log-sum-exps (split-KV only)
     int debug_drop_v_load;    // test hook: the load warp skips the first V tile (exercises the wait limit)

@@ -59,7 +59,9 @@ struct Fp8Params {
 template <int D>
 constexpr int fp8_smem_bytes() { return Fp8Cfg<D>::kSmemTiles + static_cast<int>(sizeof(PipeShared)); }
 
-template <int D>
+// kHeadPair: the two query tiles are the same query tile of two adjacent heads of a K/V group, as in
+// fa_fwd_pipelined_kernel.
+template <int D, bool kHeadPair = false>
 __global__ void __launch_bounds__(512, 1)
 fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
                   const __grid_constant__ CUtensorMap tm_k,
@@ -99,15 +101,17 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
     const uint32_t sStage = sV + NV * kTile8;                    // bf16 output tiles pass through here (one buffer per tile)
 
     // grid order: see the bf16 kernel (L2-sized head groups, longest-first inside a group)
-    const int n_pairs = (p.n_q_tiles + 1) / 2;
+    const int n_pairs = kHeadPair ? p.n_q_tiles : (p.n_q_tiles + 1) / 2;
     const int n_bh = p.B * p.Hq;
     const int item = static_cast<int>(blockIdx.x);
-    const int group = item / (n_pairs * p.heads_per_group);
-    const int bh0 = group * p.heads_per_group;
-    const int group_size = (n_bh - bh0 < p.heads_per_group) ? (n_bh - bh0) : p.heads_per_group;
-    const int local = item - group * n_pairs * p.heads_per_group;
+    const int hpg = kHeadPair ? p.heads_per_group / 2 : p.heads_per_group;     // (pairs of) heads per group
+    const int n_units = kHeadPair ? n_bh / 2 : n_bh;
+    const int group = item / (n_pairs * hpg);
+    const int bh0 = group * hpg;
+    const int group_size = (n_units - bh0 < hpg) ? (n_units - bh0) : hpg;
+    const int local = item - group * n_pairs * hpg;
     const int pair = n_pairs - 1 - local / group_size;
-    const int bh = bh0 + local % group_size;
+    const int bh = kHeadPair ? 2 * (bh0 + local % group_size) : bh0 + local % group_size;   // first head of the item
     const int hq = bh % p.Hq;
     const int b = bh / p.Hq;
     const int kvh = hq / (p.Hq / p.Hkv);
@@ -115,7 +119,7 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int kv_idx = b * p.Hkv + kvh;
     const int off = p.Sk - p.Sq;
 
-    const int i0_0 = (2 * pair) * kTileM, i0_1 = i0_0 + kTileM;
+    const int i0_0 = (kHeadPair ? pair : 2 * pair) * kTileM, i0_1 = kHeadPair ? i0_0 : i0_0 + kTileM;
     auto own_tiles = [&](int i0) -> int {
         if (i0 >= p.Sq) return 0;
         return kv_tiles_for_q_tile(i0, kTileM, p.Sq, p.Sk, p.causal);
@@ -177,13 +181,15 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
         const uint32_t bar_ph = smem_addr(&sh.p_half[t]);
         const uint32_t bar_scale = smem_addr(&sh.scale_full[t]);
         const int i0_t = t == 0 ? i0_0 : i0_1;
+        const int hq_t = kHeadPair ? hq + t : hq;          // query head of this tile
+        const int q_idx_t = kHeadPair ? q_idx + t : q_idx;
         const int nkv_t = t == 0 ? nkv_0 : nkv_1;
         const int i_glob = i0_t + row;
         int kmax_row = p.Sk - 1;
         if (p.causal && i_glob + off < kmax_row) kmax_row = i_glob + off;
         // scale * log2 e * (scale of this query tile); the key tile's scale joins per iteration
         const float cq = p.scale_log2 *
-                         ((f.q_scale && i0_t < p.Sq) ? __ldg(f.q_scale + static_cast<size_t>(q_idx) * p.n_q_tiles + (i0_t / kTileM)) : 1.f);
+                         ((f.q_scale && i0_t < p.Sq) ? __ldg(f.q_scale + static_cast<size_t>(q_idx_t) * p.n_q_tiles + (i0_t / kTileM)) : 1.f);
         const float* k_scale = f.k_scale ? f.k_scale + static_cast<size_t>(kv_idx) * f.n_kv_tiles : nullptr;
         float sk_next = (k_scale && nkv_t > 0) ? __ldg(k_scale) : 1.f;
 
@@ -283,10 +289,10 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
         }
         // epilogue: O = sv * G' / s (bf16), lse = u + ln s
         if (ok && i0_t < p.Sq) {
-            const size_t lse_row0 = static_cast<size_t>(q_idx) * p.Sq;
+            const size_t lse_row0 = static_cast<size_t>(q_idx_t) * p.Sq;
             if (nkv_t == 0) {         // no key visible to any row of this tile
                 if (i_glob < p.Sq) {
-                    __nv_bfloat16* o_row = p.O + (b * p.o_stride_b + hq * p.o_stride_h +
+                    __nv_bfloat16* o_row = p.O + (b * p.o_stride_b + hq_t * p.o_stride_h +
                                                   static_cast<long long>(i_glob) * p.o_stride_s);
                     const uint4 z = make_uint4(0, 0, 0, 0);
 #pragma unroll
@@ -324,7 +330,7 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
                     mbar_wait(smem_addr(&sh.o_staged[t]), 0, wctx, kSiteEpiStaged)) {
 #pragma unroll
                     for (int ch = 0; ch < DV / kChunkCols; ++ch)
-                        tma_store_4d(&tm_o, sStage + t * Cfg::kOBytes + ch * kChunkBytes, ch * kChunkCols, i0_t, hq, b);
+                        tma_store_4d(&tm_o, sStage + t * Cfg::kOBytes + ch * kChunkBytes, ch * kChunkCols, i0_t, hq_t, b);
                     tma_store_commit();
                     tma_store_wait_read_all();     // the CTA's shared memory outlives the reads
                 }
@@ -463,7 +469,7 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
                 if ((t == 0 ? nkv_0 : nkv_1) == 0) return;
                 const uint32_t bar = smem_addr(&sh.q_full[t]);
                 mbar_arrive_expect_tx(bar, kTile8);
-                tma_load_4d(sQ + t * kTile8, &tm_q, bar, 0, t == 0 ? i0_0 : i0_1, hq, b);
+                tma_load_4d(sQ + t * kTile8, &tm_q, bar, 0, t == 0 ? i0_0 : i0_1, kHeadPair ? hq + t : hq, b);
             };
             load_q(0);
             bool ok = true;

@@ -73,29 +73,36 @@ constexpr int persist_smem_bytes() {
 // One work item, decoded from its place in the longest-first order.
 struct PersistItem {
     int b, hq, kvh;
-    int i0_0;                // first row of query tile 0 (tile 1 starts 128 rows further)
+    int hq1;                 // query head of tile 1 (the same head, or the next one when heads are paired)
+    int i0_0, i0_1;          // first rows of the two query tiles (128 rows apart, or equal when heads are paired)
     int nkv_0, nkv_1, n_max; // K/V tiles of tile 0, tile 1, and the larger of the two
 };
 
 __device__ __forceinline__ PersistItem persist_decode(const FwdParams& p, int idx) {
     // Groups of (batch, head) instances whose K/V fit in L2 together follow one another; inside a
     // group every head's last (with a causal mask: heaviest) pair comes first.
-    const int n_pairs = (p.n_q_tiles + 1) / 2;
-    const int n_bh = p.B * p.Hq;
-    const int per_group = n_pairs * p.heads_per_group;
+    // With paired heads (p.head_pair) an item is ONE query tile of two adjacent query heads of a
+    // K/V group, as in the pair kernel's kHeadPair mode, and the units below are pairs of heads.
+    const int hp = p.head_pair;
+    const int n_pairs = hp ? p.n_q_tiles : (p.n_q_tiles + 1) / 2;
+    const int n_units = hp ? p.B * p.Hq / 2 : p.B * p.Hq;
+    const int hpg = hp ? p.heads_per_group / 2 : p.heads_per_group;
+    const int per_group = n_pairs * hpg;
     const int group = idx / per_group;
-    const int bh0 = group * p.heads_per_group;
-    const int group_size = (n_bh - bh0 < p.heads_per_group) ? (n_bh - bh0) : p.heads_per_group;
+    const int bh0 = group * hpg;
+    const int group_size = (n_units - bh0 < hpg) ? (n_units - bh0) : hpg;
     const int local = idx - group * per_group;
     const int pair = n_pairs - 1 - local / group_size;
-    const int bh = bh0 + local % group_size;
+    const int bh = hp ? 2 * (bh0 + local % group_size) : bh0 + local % group_size;
     PersistItem it;
     it.hq = bh % p.Hq;
+    it.hq1 = it.hq + hp;
     it.b = bh / p.Hq;
     it.kvh = it.hq / (p.Hq / p.Hkv);
-    it.i0_0 = 2 * pair * kTileM;
+    it.i0_0 = (hp ? pair : 2 * pair) * kTileM;
+    it.i0_1 = hp ? it.i0_0 : it.i0_0 + kTileM;
     it.nkv_0 = kv_tiles_for_q_tile(it.i0_0, kTileM, p.Sq, p.Sk, p.causal);
-    it.nkv_1 = (it.i0_0 + kTileM < p.Sq) ? kv_tiles_for_q_tile(it.i0_0 + kTileM, kTileM, p.Sq, p.Sk, p.causal) : 0;
+    it.nkv_1 = (it.i0_1 < p.Sq) ? kv_tiles_for_q_tile(it.i0_1, kTileM, p.Sq, p.Sk, p.causal) : 0;
     it.n_max = it.nkv_0 > it.nkv_1 ? it.nkv_0 : it.nkv_1;
     return it;
 }
@@ -138,7 +145,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
     const uint32_t sV = sK + NK * Cfg::kKBytes;                  // NV stages
     const uint32_t sStage = sV + NV * Cfg::kVBytes;              // one bf16 output tile
 
-    const int n_items = ((p.n_q_tiles + 1) / 2) * p.B * p.Hq;
+    const int n_items = p.head_pair ? p.n_q_tiles * p.B * (p.Hq / 2) : ((p.n_q_tiles + 1) / 2) * p.B * p.Hq;
     const int G = static_cast<int>(gridDim.x);
     const int cta = static_cast<int>(blockIdx.x);
 
@@ -235,7 +242,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             {
                 const PersistItem item = persist_decode(p, idx);
                 nkv_t = t == 0 ? item.nkv_0 : item.nkv_1;
-                i0_t = item.i0_0 + t * kTileM;
+                i0_t = t == 0 ? item.i0_0 : item.i0_1;
                 my_use = uc + ((t == 1 && item.nkv_0 > 0) ? 1u : 0u);
                 uc += (item.nkv_0 > 0 ? 1u : 0u) + (item.nkv_1 > 0 ? 1u : 0u);
             }
@@ -342,10 +349,11 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             // ---- epilogue of the item: O = G' / s (bf16), lse = u * scale + ln s
             if (i0_t >= p.Sq) continue;
             const PersistItem item = persist_decode(p, idx);     // again: nothing of it was kept live
-            const size_t lse_row0 = (static_cast<size_t>(item.b) * p.Hq + item.hq) * p.Sq;
+            const int hq_t = t == 0 ? item.hq : item.hq1;
+            const size_t lse_row0 = (static_cast<size_t>(item.b) * p.Hq + hq_t) * p.Sq;
             if (nkv_t == 0) {             // no key visible to any row of this tile
                 if (i_glob < p.Sq) {
-                    __nv_bfloat16* o_row = p.O + (item.b * p.o_stride_b + item.hq * p.o_stride_h +
+                    __nv_bfloat16* o_row = p.O + (item.b * p.o_stride_b + hq_t * p.o_stride_h +
                                                   static_cast<long long>(i_glob) * p.o_stride_s);
                     const uint4 z = make_uint4(0, 0, 0, 0);
 #pragma unroll
@@ -391,7 +399,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 if (ok) {
 #pragma unroll
                     for (int ch = 0; ch < DV / kChunkCols; ++ch)
-                        tma_store_4d(&tm_o, sStage + ch * kChunkBytes, ch * kChunkCols, i0_t, item.hq, item.b);
+                        tma_store_4d(&tm_o, sStage + ch * kChunkBytes, ch * kChunkCols, i0_t, hq_t, item.b);
                     tma_store_commit();
                     tma_store_wait_read_all();
                     mbar_arrive(smem_addr(&sh.stage_empty));
@@ -633,7 +641,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                     for (int cc = 0; cc < Base::kQChunks; ++cc)
                         tma_load_4d(sQ + t * Cfg::kQBytes + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols,
-                                    item.i0_0 + t * kTileM, item.hq, item.b);
+                                    t == 0 ? item.i0_0 : item.i0_1, t == 0 ? item.hq : item.hq1, item.b);
                     if (t == 0) ++qc0; else ++qc1;
                 }
             }

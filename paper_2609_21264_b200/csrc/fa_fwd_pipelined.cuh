@@ -80,7 +80,11 @@ constexpr int pipe_smem_bytes() {
 
 // kVarlen = packed variable-length batch (per-sequence offsets and lengths read from p.cu_q/p.cu_k);
 // a template parameter so that the fixed-length instantiation carries none of its scalars.
-template <int DQK, int DV, bool kVarlen = false>
+// kHeadPair = the CTA's two query tiles are the SAME query tile of two adjacent query heads that share
+// a K/V head (grouped-query attention with an even group size) instead of two adjacent query tiles
+// of one head.  With a causal mask both tiles then see the same number of K/V tiles, so neither
+// runs a last round alone, and the items come in lengths 1, 2, 3, ... instead of 2, 4, 6, ...
+template <int DQK, int DV, bool kVarlen = false, bool kHeadPair = false>
 __global__ void __launch_bounds__(512, 1)
 fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                         const __grid_constant__ CUtensorMap tm_k,
@@ -134,18 +138,21 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     // groups run one after the other, and inside a group the CTAs are in longest-processing-time
     // order: every head's last (with a causal mask: heaviest) pair of query tiles first, then the
     // pair before it, and so on.  Consecutive CTAs are consecutive query heads (shared K/V heads).
-    const int n_pairs = (p.n_q_tiles + 1) / 2;
+    // (kHeadPair: an item is one query tile of a pair of heads; bh then counts pairs of heads)
+    const int n_pairs = kHeadPair ? p.n_q_tiles : (p.n_q_tiles + 1) / 2;
     const int n_bh = p.B * p.Hq;
     // With split-KV (the spatial decomposition of Algorithm 2) the C CTAs that share an item's
     // query tiles and take disjoint ranges of its K/V tiles are adjacent in the grid.
     const int item = static_cast<int>(blockIdx.x) / p.kv_splits;
     const int split = static_cast<int>(blockIdx.x) - item * p.kv_splits;
-    const int group = item / (n_pairs * p.heads_per_group);
-    const int bh0 = group * p.heads_per_group;
-    const int group_size = (n_bh - bh0 < p.heads_per_group) ? (n_bh - bh0) : p.heads_per_group;
-    const int local = item - group * n_pairs * p.heads_per_group;
+    const int hpg = kHeadPair ? p.heads_per_group / 2 : p.heads_per_group;     // (pairs of) heads per group
+    const int n_units = kHeadPair ? n_bh / 2 : n_bh;
+    const int group = item / (n_pairs * hpg);
+    const int bh0 = group * hpg;
+    const int group_size = (n_units - bh0 < hpg) ? (n_units - bh0) : hpg;
+    const int local = item - group * n_pairs * hpg;
     const int pair = n_pairs - 1 - local / group_size;
-    const int bh = bh0 + local % group_size;
+    const int bh = kHeadPair ? 2 * (bh0 + local % group_size) : bh0 + local % group_size;   // first head of the item
     const int hq = bh % p.Hq;
     const int b = bh / p.Hq;
     const int kvh = hq / (p.Hq / p.Hkv);
@@ -162,7 +169,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int off = Sk - Sq;
 
     // per-tile scalars (no arrays: a runtime-indexed array would live in local memory)
-    const int i0_0 = (2 * pair) * kTileM, i0_1 = i0_0 + kTileM;
+    const int i0_0 = (kHeadPair ? pair : 2 * pair) * kTileM, i0_1 = kHeadPair ? i0_0 : i0_0 + kTileM;
     // K/V tiles [j_base, j_base + nkv_t) of tile t belong to this CTA (all visible ones without split-KV)
     const int j_base = split * p.tiles_per_split;
     auto own_tiles = [&](int i0) -> int {
@@ -230,6 +237,8 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         const uint32_t bar_ph = smem_addr(&sh.p_half[t]);
         const uint32_t bar_scale = smem_addr(&sh.scale_full[t]);
         const int i0_t = t == 0 ? i0_0 : i0_1;
+        const int hq_t = kHeadPair ? hq + t : hq;          // query head of this tile
+        const int q_idx_t = kHeadPair ? q_idx + t : q_idx;
         const int nkv_t = t == 0 ? nkv_0 : nkv_1;
         const int i_glob = i0_t + row;
         int kmax_row = Sk - 1;
@@ -344,7 +353,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         if (ok && i0_t < Sq && p.kv_splits > 1) {
             // split-KV: this CTA's partial (G'_c / s_c in fp32, and u_c + ln s_c) goes to scratch;
             // the combine kernel merges the C partials of a row (Algorithm 2's reduction).
-            const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx) * p.Sq + i_glob;
+            const size_t prow = (static_cast<size_t>(split) * n_bh + q_idx_t) * p.Sq + i_glob;
             float* po_row = p.o_part + prow * DV;
             bool have = nkv_t > 0;
             if (have) have = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.o_final[t]), 0, wctx, kSiteEpiOFull));
@@ -376,9 +385,9 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             }
         } else if (ok && i0_t < Sq) {
             // fixed lengths: lse [B, Hq, Sq]; packed batches: lse [Hq, total_q], O rows q_row0 onwards
-            const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq) * p.total_q + q_row0
-                                           : static_cast<size_t>(q_idx) * p.Sq;
-            const long long o_base = (kVarlen ? q_row0 * p.o_stride_s : b * p.o_stride_b) + hq * p.o_stride_h;
+            const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq_t) * p.total_q + q_row0
+                                           : static_cast<size_t>(q_idx_t) * p.Sq;
+            const long long o_base = (kVarlen ? q_row0 * p.o_stride_s : b * p.o_stride_b) + hq_t * p.o_stride_h;
             __nv_bfloat16* o_row = p.O + (o_base + static_cast<long long>(i_glob) * p.o_stride_s);
             if (nkv_t == 0) {         // no key visible to any row of this tile
                 if (i_glob < Sq) {
@@ -428,7 +437,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                         for (int ch = 0; ch < DV / kChunkCols; ++ch)
                             tma_store_4d(&tm_o, sQ + t * Cfg::kQBytes + ch * kChunkBytes, ch * kChunkCols,
-                                         q_row0 + i0_t, hq, kVarlen ? 0 : b);
+                                         q_row0 + i0_t, hq_t, kVarlen ? 0 : b);
                         tma_store_commit();
                         tma_store_wait_read_all();     // the CTA's shared memory outlives the reads
                     }
@@ -610,7 +619,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                 for (int cc = 0; cc < Cfg::kQChunks; ++cc)
                     tma_load_4d(sQ + t * Cfg::kQBytes + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols,
-                                q_row0 + (t == 0 ? i0_0 : i0_1), hq, kVarlen ? 0 : b);
+                                q_row0 + (t == 0 ? i0_0 : i0_1), kHeadPair ? hq + t : hq, kVarlen ? 0 : b);
             };
             // Order of the first requests: Q_0 and K_0 (all the first MMA needs), then Q_1, then V_0.
             // When a whole wave of CTAs starts at once these first loads are HBM-bandwidth-bound.
