@@ -99,7 +99,7 @@ typedef struct fa_config {
     int32_t device;           /* CUDA device ordinal; -1 = the calling thread's current device */
     uint32_t flags;           /* bitwise OR of FA_FLAG_*; other bits must be 0                 */
     uint32_t wait_limit_ms;   /* limit of every device-side wait; 0 = default (2000 ms)        */
-    uint32_t kv_splits;       /* split-KV: 0 = library decides, 1 = never split, n > 1 = use n
+    uint32_t kv_splits;       /* split-KV: 0 = library decides, 1 = never split, 2..256 = use n
                                  splits whenever the scratch buffer can hold the partials      */
     uint64_t scratch_bytes;   /* device scratch for split-KV partials, allocated by fa_create;
                                  0 = default (32 MiB)                                          */

@@ -215,7 +215,7 @@ int choose_kv_splits(int num_sms, uint32_t kv_splits_cfg, size_t scratch_bytes, 
         const int wave = static_cast<int>(num_sms / items);
         const double ideal = sqrt(3.3 * max_tiles);
         splits = 1;
-        while (splits * 2 <= wave && splits * 2 <= 32 && splits * 1.41 < ideal) splits *= 2;
+        while (splits * 2 <= wave && splits * 2 <= 128 && splits * 1.41 < ideal) splits *= 2;
         const int per_split = (max_tiles + splits - 1) / splits;
         splits = (max_tiles + per_split - 1) / per_split;
     }
@@ -615,7 +615,7 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg) {
         if (flags & ~(FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD | FA_FLAG_NO_DEPENDENT_LAUNCH |
                       FA_FLAG_NO_PERSISTENT | FA_FLAG_FORCE_PERSISTENT | FA_FLAG_STREAM_KERNEL |
                       FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)) return FA_ERR_INVALID_ARG;
-        if (kv_splits_cfg > 64) return FA_ERR_INVALID_ARG;
+        if (kv_splits_cfg > 256) return FA_ERR_INVALID_ARG;
     }
     if (scratch_bytes == 0) scratch_bytes = 32ull << 20;
     int count = 0;
