@@ -452,7 +452,8 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     // estimates, with a margin, each side with its own split count.
     // Causal grouped-query attention: pairing the same query tile of two heads of a group gives both
     // tiles of a pair-kernel CTA the same number of K/V tiles (no round that one of them runs alone).
-    const bool head_pair_ok = !varlen && !drop && causal && pair_splits == 1 && (Hq / Hkv) % 2 == 0 &&
+    // (Without a mask it only matters for an odd number of query tiles, whose last tile would be alone.)
+    const bool head_pair_ok = !varlen && !drop && (causal || (n_q_tiles & 1)) && pair_splits == 1 && (Hq / Hkv) % 2 == 0 &&
                               !(flags & FA_FLAG_NO_HEAD_PACKING);
     bool stream = false;
     int stream_splits = 1;

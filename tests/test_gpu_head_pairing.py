@@ -17,8 +17,8 @@ from parity_util import assert_parity, to_torch_bf16, bf16_tensor_to_f64
 pytestmark = pytest.mark.gpu
 
 
-def _wl(name, B, Hq, Hkv, Sq, Sk, d, seed):
-    return W.Workload(name, B=B, Hq=Hq, Hkv=Hkv, Sq=Sq, Sk=Sk, dqk=d, dv=(128 if d == 192 else d), causal=True,
+def _wl(name, B, Hq, Hkv, Sq, Sk, d, seed, causal=True):
+    return W.Workload(name, B=B, Hq=Hq, Hkv=Hkv, Sq=Sq, Sk=Sk, dqk=d, dv=(128 if d == 192 else d), causal=causal,
                       scale=d ** -0.5, seed=seed)
 
 
@@ -30,6 +30,9 @@ CASES = [
     _wl("g2_d192", 1, 4, 2, 300, 300, 192, 1605),
     _wl("g4_fewer_queries_than_keys", 3, 16, 4, 260, 900, 128, 1606),
     _wl("g4_llama_like_s1024", 2, 16, 4, 1024, 1024, 128, 1607),
+    # no mask: paired for an odd number of query tiles (the last tile of a head would be alone in its CTA)
+    _wl("g4_no_mask_three_tiles", 4, 16, 4, 333, 500, 128, 1608, causal=False),
+    _wl("g2_no_mask_five_tiles_d64", 3, 12, 6, 600, 600, 64, 1609, causal=False),
 ]
 
 
@@ -38,7 +41,7 @@ def _run(flags, w, Q, K, V):
     from paper_2609_21264_b200 import binding
     h = binding.fa_create(flags=flags)
     try:
-        o, lse = binding.forward(h, to_torch_bf16(Q), to_torch_bf16(K), to_torch_bf16(V), causal=True, scale=w.scale)
+        o, lse = binding.forward(h, to_torch_bf16(Q), to_torch_bf16(K), to_torch_bf16(V), causal=w.causal, scale=w.scale)
         torch.cuda.synchronize()
         st, detail = binding.fa_last_status(h)
         assert st == binding.FA_OK, "device status %d (site 0x%x)" % (st, detail)
@@ -61,12 +64,12 @@ def test_paired_heads_equal_the_unpaired_launch_and_the_oracle(w, persistent):
     assert k1 == k2 == ("fa_fwd_persistent" if persistent else "fa_fwd_pipelined")
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     n_q_tiles = (w.Sq + 127) // 128
-    plan = binding.fa_plan(sms, w.B, w.Hq, w.Hkv, w.Sq, w.Sk, w.dqk, w.dv, True, flags=base)
+    plan = binding.fa_plan(sms, w.B, w.Hq, w.Hkv, w.Sq, w.Sk, w.dqk, w.dv, w.causal, flags=base)
     if plan["kv_splits"] == 1:      # (a split K/V range keeps the pairs of adjacent query tiles)
         assert plan["ctas"] == min(n_q_tiles * (w.Hq // 2) * w.B, sms if persistent else 1 << 30), plan     # one item per tile and pair of heads
     assert torch.equal(o1.view(torch.int16), o2.view(torch.int16))
     assert torch.equal(l1, l2)
-    O_ref, lse_ref = oracle.attention(Q, K, V, causal=True, scale=w.scale)
+    O_ref, lse_ref = oracle.attention(Q, K, V, causal=w.causal, scale=w.scale)
     assert_parity(bf16_tensor_to_f64(o1), l1.double().cpu().numpy(), O_ref, lse_ref, w.name)
 
 
