@@ -48,7 +48,6 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                      const __grid_constant__ CUtensorMap tm_o,
                      const FwdParams p, const Fp8Params f) {
     using Cfg = Fp8StreamCfg<D>;
-    constexpr bool kVarlen = false;
     constexpr int DV = Cfg::kD;
     constexpr int kTile8 = Cfg::kTile8;
     static_assert(kRep == 1 || (kPack && (kRep == 2 || kRep == 4)), "copies of the query rows need packed heads");
@@ -67,11 +66,10 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     const int lane = tid & 31;
 
     grid_launch_dependents();
-    if constexpr (kVarlen) grid_dependency_wait();    // the sequence offsets are read right away
 
     const uint32_t smem_base = smem_addr(smem_raw);
     if ((smem_base & 1023u) != 0u) {          // uniform over the CTA; nothing has been set up yet
-        if constexpr (!kVarlen) grid_dependency_wait();
+        grid_dependency_wait();
         if (tid == 0 && p.status) {
             volatile uint32_t* sw = p.status;
             sw[1] = kSiteSmemAlign;
@@ -111,22 +109,14 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     }
     const int kvh = hq / (p.Hq / p.Hkv);
     const int kv_idx = b * p.Hkv + kvh;
-    int Sq = p.Sq, Sk = p.Sk, q_row0 = 0, k_row0 = 0;
-    if constexpr (kVarlen) {
-        q_row0 = p.cu_q[b];
-        k_row0 = p.cu_k[b];
-        Sq = p.cu_q[b + 1] - q_row0;
-        Sk = p.cu_k[b + 1] - k_row0;
-    }
+    const int Sq = p.Sq, Sk = p.Sk;
     const int off = Sk - Sq;
     const int i0 = q_tile * kTileM;
-    if (kVarlen && i0 >= Sq) return;      // a sequence shorter than the longest one (whole CTA, before any set-up)
     // K/V tiles [j_base, j_base + n_kv) of the query tile belong to this CTA (all visible ones without split-KV)
     const int j_base = split * p.tiles_per_split;
     int n_kv = kv_tiles_for_q_tile(i0, kTileM, Sq, Sk, p.causal) - j_base;
     if (n_kv > p.tiles_per_split) n_kv = p.tiles_per_split;
     if (n_kv < 0) n_kv = 0;
-    const int tb = kVarlen ? 0 : b;       // batch coordinate of the tensor maps (packed tensors have one slice)
 
     // ---------------------------------------------------------------- setup
     if (tid == 0) {
@@ -170,7 +160,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if constexpr (!kVarlen) grid_dependency_wait();
+    grid_dependency_wait();
 
     const uint32_t tmem_base = sh.tmem_base;
     WaitCtx wctx{&sh.abort_flag, p.status, p.wait_limit_ns};
@@ -320,9 +310,8 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
 
         // ---- epilogue: O = G' / s (bf16), lse = u * scale + ln s
         if (ok && i0 < Sq) {
-            // fixed lengths: lse [B, Hq, Sq]; packed batches: lse [Hq, total_q], O rows q_row0 onwards
-            const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq) * p.total_q + q_row0 : static_cast<size_t>(q_idx) * p.Sq;
-            const long long o_base = (kVarlen ? q_row0 * p.o_stride_s : b * p.o_stride_b) + hq_row * p.o_stride_h;
+            const size_t lse_row0 = static_cast<size_t>(q_idx) * p.Sq;
+            const long long o_base = b * p.o_stride_b + hq_row * p.o_stride_h;
             if (partial_out && n_kv == 0) {      // an empty range: a neutral partial
                 if (row_valid) {
                     const size_t prow = (static_cast<size_t>(part) * n_bh + q_idx) * p.Sq + i_glob;
@@ -368,9 +357,6 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     // (the Q tile's space: the last score MMA is long complete), then one thread
                     // stores it with TMA; rows past Sq are clipped
                     const uint32_t tO = tmem_base + Cfg::kColO + lane_sel;
-                    // the last tile of a packed sequence is followed by the next sequence's rows, which a
-                    // box store would overwrite: it is stored row by row
-                    const bool box_store = !kVarlen || (i0 + kTileM <= Sq);
                     if (partial_out) {
                         // split-KV: G'_c / s_c in fp32 and u_c + ln s_c go to scratch (Algorithm 2's partials)
                         const size_t prow = (static_cast<size_t>(part) * n_bh + q_idx) * p.Sq + i_glob;
@@ -390,7 +376,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                                         __uint_as_float(r[4 * v + 2]) * inv_l, __uint_as_float(r[4 * v + 3]) * inv_l);
                             }
                         }
-                    } else if (box_store) {
+                    } else {
                         const uint32_t sO = sStage + row * 128;
 #pragma unroll 1
                         for (int cc = g * (DV / 64); cc < (g + 1) * (DV / 64); ++cc) {
@@ -414,26 +400,9 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                         if (warp == 0 && lane == 0 && mbar_wait(smem_addr(&sh.o_staged), 0, wctx, kSiteEpiStaged)) {
 #pragma unroll
                             for (int ch = 0; ch < DV / kChunkCols; ++ch)
-                                tma_store_4d(&tm_o, sStage + ch * kChunkBytes, ch * kChunkCols, q_row0 + i0, hq, tb);
+                                tma_store_4d(&tm_o, sStage + ch * kChunkBytes, ch * kChunkCols, i0, hq, b);
                             tma_store_commit();
                             tma_store_wait_read_all();     // the CTA's shared memory outlives the reads
-                        }
-                    } else {
-                        __nv_bfloat16* o_row = p.O + (o_base + static_cast<long long>(i_glob) * p.o_stride_s);
-#pragma unroll 1
-                        for (int cc = g * (DV / 64); cc < (g + 1) * (DV / 64); ++cc) {
-                            uint32_t r[32];
-                            tmem_ld_x32(tO + cc * 32, r);
-                            tc_wait_ld();
-                            if (row_valid) {
-#pragma unroll
-                                for (int v = 0; v < 4; ++v)
-                                    reinterpret_cast<uint4*>(o_row + cc * 32)[v] = make_uint4(
-                                        pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
-                                        pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
-                                        pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
-                                        pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
-                            }
                         }
                     }
                 }
@@ -542,7 +511,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 // with packed heads the box is Sq rows x pack_heads heads (row h * Sq + i of the tile)
                 mbar_arrive_expect_tx(bar, kPack ? static_cast<uint32_t>(kRep * p.pack_heads * Sq * D) : static_cast<uint32_t>(kTile8));
 #pragma unroll
-                for (int r = 0; r < kRep; ++r) tma_load_4d(sQ + r * kRepRows * D, &tm_q, bar, 0, q_row0 + i0, hq, tb);
+                for (int r = 0; r < kRep; ++r) tma_load_4d(sQ + r * kRepRows * D, &tm_q, bar, 0, i0, hq, b);
             }
             bool ok = true;
             for (int j = 0; j < n_kv && ok; ++j) {
@@ -551,7 +520,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 if (!ok) break;
                 const uint32_t bar = smem_addr(&sh.k_full[s]);
                 mbar_arrive_expect_tx(bar, kTile8);
-                tma_load_4d(sK + s * kTile8, &tm_k, bar, 0, k_row0 + (j_base + j) * kTileN, kvh, tb);
+                tma_load_4d(sK + s * kTile8, &tm_k, bar, 0, (j_base + j) * kTileN, kvh, b);
             }
         }
     } else {
@@ -565,7 +534,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 if (!ok) break;
                 const uint32_t bar = smem_addr(&sh.v_full[s]);
                 mbar_arrive_expect_tx(bar, kTile8);
-                tma_load_4d(sV + s * kTile8, &tm_v, bar, 0, k_row0 + (j_base + j) * kTileN, kvh, tb);
+                tma_load_4d(sV + s * kTile8, &tm_v, bar, 0, (j_base + j) * kTileN, kvh, b);
             }
         }
     }
