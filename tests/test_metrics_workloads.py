@@ -75,3 +75,40 @@ def test_sample_rows_are_in_range():
     rows = W.sample_rows(w, 32, seed=1, heads=[0, 31])
     assert rows.shape[1] == 3 and (rows[:, 2] < w.Sq).all() and (rows[:, 1] < w.Hq).all()
     assert {0, 127, 128, w.Sq - 1} <= set(rows[:, 2].tolist())
+
+
+def _decode_e4m3(codes):
+    """e4m3 ("fn": no infinities, 0x7f/0xff are NaN) written out: 1 sign, 4 exponent (bias 7), 3 mantissa bits."""
+    c = codes.astype(np.int64)
+    s, e, m = c >> 7, (c >> 3) & 15, c & 7
+    mag = np.where(e == 0, m * 2.0 ** -9, (1.0 + m / 8.0) * 2.0 ** (e - 7.0))
+    return np.where(s == 1, -mag, mag)
+
+
+def test_block_quantiser_of_the_8_bit_path():
+    """What the 8-bit tests hand to the oracle (codes x scales) is what the codes mean under the
+    format's definition, the scales are amax / 448 per block, and every value is rounded to a
+    nearest representable one."""
+    from paper_2609_21264_b200 import workloads as W
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((2, 3, 300, 64)) * rng.uniform(0.01, 30.0, size=(2, 3, 300, 1))
+    x[0, 0, :128] = 0.0                                         # an all-zero block keeps scale 1
+    for block_rows in (128, None):
+        codes, scales, deq = W.quantize_e4m3_blocks(x, block_rows)
+        assert codes.dtype == np.uint8 and codes.shape == x.shape and scales.dtype == np.float32
+        assert not np.isin(codes, (0x7f, 0xff)).any()           # no NaN codes
+        if block_rows:
+            per_row = np.repeat(scales.astype(np.float64), block_rows, axis=2)[:, :, :300, None]
+            amax = np.stack([np.abs(x[:, :, i:i + block_rows]).max(axis=(2, 3)) for i in range(0, 300, block_rows)], axis=2)
+        else:
+            per_row = scales.astype(np.float64)[:, :, None, None]
+            amax = np.abs(x).max(axis=(2, 3))
+        assert np.array_equal(deq, _decode_e4m3(codes) * per_row)
+        want = np.where(amax > 0, amax / 448.0, 1.0).astype(np.float32)
+        assert np.array_equal(scales, want)
+        # nearest: the error is at most half a step of the format at that magnitude (3 mantissa bits; the
+        # fp32 scale and quotient add a few parts in 1e7)
+        y = x / per_row
+        step = np.where(np.abs(y) < 2.0 ** -6, 2.0 ** -9, 2.0 ** (np.floor(np.log2(np.maximum(np.abs(y), 2.0 ** -6))) - 3))
+        assert (np.abs(_decode_e4m3(codes) - y) <= 0.5 * step * (1 + 1e-6) + 1e-9).all()
+        assert (np.abs(_decode_e4m3(codes)) <= 448.0).all()
