@@ -57,7 +57,7 @@ struct fa_handle {
     const char* last_kernel = "";
     void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // Q K V O lse
     size_t stage_cap[5] = {0, 0, 0, 0, 0};
-    bool attr_done[40] = {};
+    std::vector<const void*> attr_done;     // kernels whose shared-memory limit has been raised
 #ifdef FA_TRACE
     long long* trace = nullptr;
 #endif
@@ -126,25 +126,29 @@ fa_status get_map(fa_handle* h, const void* ptr, int d, int S, int H, int B, lon
     return FA_OK;
 }
 
+// Raises a kernel's dynamic shared-memory limit once per handle (the attribute is per device and
+// function; the handle remembers which kernels it has prepared, by their address).
 template <typename Kernel>
-fa_status ensure_smem_attr(fa_handle* h, int slot, Kernel kernel, int bytes) {
-    if (h->attr_done[slot]) return FA_OK;
+fa_status ensure_smem_attr(fa_handle* h, Kernel kernel, int bytes) {
+    const void* key = reinterpret_cast<const void*>(kernel);
+    for (const void* k : h->attr_done)
+        if (k == key) return FA_OK;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
         cudaGetLastError();
         return FA_ERR_CUDA;
     }
-    h->attr_done[slot] = true;
+    h->attr_done.push_back(key);
     return FA_OK;
 }
 
 template <int DQK, int DV>
-fa_status launch_simple(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
+fa_status launch_simple(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& mk,
                         const CUtensorMap& mv, const fa::FwdParams& p, cudaStream_t st) {
     using Cfg = fa::SimpleCfg<DQK, DV>;
     // ask for more than half of the SM's shared memory so that one CTA owns the SM's TMEM
     const int smem = Cfg::kSmemBytes > 120 * 1024 ? Cfg::kSmemBytes : 120 * 1024;
     auto kernel = fa::fa_fwd_simple_kernel<DQK, DV>;
-    fa_status s = ensure_smem_attr(h, slot, kernel, smem);
+    fa_status s = ensure_smem_attr(h, kernel, smem);
     if (s != FA_OK) return s;
     dim3 grid(p.n_q_tiles, p.Hq, p.B);
     kernel<<<grid, 128, smem, st>>>(mq, mk, mv, p);
@@ -154,12 +158,12 @@ fa_status launch_simple(fa_handle* h, int slot, const CUtensorMap& mq, const CUt
 }
 
 template <int DQK, int DV, bool kVarlen, bool kHeadPair = false>
-fa_status launch_pipelined(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
+fa_status launch_pipelined(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& mk,
                            const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
     constexpr int smem = fa::pipe_smem_bytes<DQK, DV>();
     static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
     auto kernel = fa::fa_fwd_pipelined_kernel<DQK, DV, kVarlen, kHeadPair>;
-    fa_status s = ensure_smem_attr(h, slot, kernel, smem);
+    fa_status s = ensure_smem_attr(h, kernel, smem);
     if (s != FA_OK) return s;
     // items: pairs of adjacent query tiles of a head, or one query tile of a pair of adjacent heads
     const long long n_ctas = (kHeadPair ? static_cast<long long>(p.n_q_tiles) * (p.Hq / 2)
@@ -268,12 +272,12 @@ int heads_per_group(long long kv_bytes_per_head, int B, int Hq, int Hkv) {
 // Persistent kernel: one CTA per SM (fewer when there are fewer items), every CTA walks its share
 // of the items.  Fixed-length problems without split-KV only.
 template <int DQK, int DV>
-fa_status launch_persistent(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
+fa_status launch_persistent(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& mk,
                             const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
     constexpr int smem = fa::persist_smem_bytes<DQK, DV>();
     static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
     auto kernel = fa::fa_fwd_persistent_kernel<DQK, DV>;
-    fa_status s = ensure_smem_attr(h, slot, kernel, smem);
+    fa_status s = ensure_smem_attr(h, kernel, smem);
     if (s != FA_OK) return s;
     const long long n_items = p.head_pair ? static_cast<long long>(p.n_q_tiles) * (p.Hq / 2) * p.B
                                           : static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq * p.B;
@@ -295,12 +299,12 @@ fa_status launch_persistent(fa_handle* h, int slot, const CUtensorMap& mq, const
 
 // One query tile per CTA, K/V tiles streamed through two softmax warpgroups.
 template <int DQK, int DV, bool kVarlen = false, bool kPack = false>
-fa_status launch_stream(fa_handle* h, int slot, const CUtensorMap& mq, const CUtensorMap& mk,
+fa_status launch_stream(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& mk,
                         const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
     constexpr int smem = fa::stream_smem_bytes<DQK, DV>();
     static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
     auto kernel = fa::fa_fwd_stream_kernel<DQK, DV, kVarlen, kPack>;
-    fa_status s = ensure_smem_attr(h, slot, kernel, smem);
+    fa_status s = ensure_smem_attr(h, kernel, smem);
     if (s != FA_OK) return s;
     // items: query tiles x heads, or packs of heads with their single query tile
     const long long n_ctas = (kPack ? static_cast<long long>(p.Hq / p.pack_heads) : static_cast<long long>(p.n_q_tiles) * p.Hq) * p.B * p.kv_splits;
@@ -536,49 +540,49 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
     if (pl.kernel == kPlanStream) {
         h->last_kernel = "fa_fwd_stream";
         if (pl.pack_heads > 1 && cu_q) {
-            if (dqk == 64) return launch_stream<64, 64, true, true>(h, 29, map_q, map_k, map_v, map_o, p, st);
-            if (dqk == 128) return launch_stream<128, 128, true, true>(h, 30, map_q, map_k, map_v, map_o, p, st);
-            return launch_stream<192, 128, true, true>(h, 31, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 64) return launch_stream<64, 64, true, true>(h, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_stream<128, 128, true, true>(h, map_q, map_k, map_v, map_o, p, st);
+            return launch_stream<192, 128, true, true>(h, map_q, map_k, map_v, map_o, p, st);
         }
         if (pl.pack_heads > 1) {
-            if (dqk == 64) return launch_stream<64, 64, false, true>(h, 23, map_q, map_k, map_v, map_o, p, st);
-            if (dqk == 128) return launch_stream<128, 128, false, true>(h, 24, map_q, map_k, map_v, map_o, p, st);
-            return launch_stream<192, 128, false, true>(h, 25, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 64) return launch_stream<64, 64, false, true>(h, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_stream<128, 128, false, true>(h, map_q, map_k, map_v, map_o, p, st);
+            return launch_stream<192, 128, false, true>(h, map_q, map_k, map_v, map_o, p, st);
         }
         if (cu_q) {
-            if (dqk == 64) return launch_stream<64, 64, true>(h, 19, map_q, map_k, map_v, map_o, p, st);
-            if (dqk == 128) return launch_stream<128, 128, true>(h, 20, map_q, map_k, map_v, map_o, p, st);
-            return launch_stream<192, 128, true>(h, 21, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 64) return launch_stream<64, 64, true>(h, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_stream<128, 128, true>(h, map_q, map_k, map_v, map_o, p, st);
+            return launch_stream<192, 128, true>(h, map_q, map_k, map_v, map_o, p, st);
         }
-        if (dqk == 64) return launch_stream<64, 64>(h, 16, map_q, map_k, map_v, map_o, p, st);
-        if (dqk == 128) return launch_stream<128, 128>(h, 17, map_q, map_k, map_v, map_o, p, st);
-        return launch_stream<192, 128>(h, 18, map_q, map_k, map_v, map_o, p, st);
+        if (dqk == 64) return launch_stream<64, 64>(h, map_q, map_k, map_v, map_o, p, st);
+        if (dqk == 128) return launch_stream<128, 128>(h, map_q, map_k, map_v, map_o, p, st);
+        return launch_stream<192, 128>(h, map_q, map_k, map_v, map_o, p, st);
     }
     if (pl.kernel == kPlanPersistent) {
         h->last_kernel = "fa_fwd_persistent";
-        if (dqk == 64) return launch_persistent<64, 64>(h, 9, map_q, map_k, map_v, map_o, p, st);
-        return launch_persistent<128, 128>(h, 10, map_q, map_k, map_v, map_o, p, st);
+        if (dqk == 64) return launch_persistent<64, 64>(h, map_q, map_k, map_v, map_o, p, st);
+        return launch_persistent<128, 128>(h, map_q, map_k, map_v, map_o, p, st);
     }
     if (pl.kernel == kPlanPair) {
         h->last_kernel = "fa_fwd_pipelined";
         if (cu_q) {
-            if (dqk == 64) return launch_pipelined<64, 64, true>(h, 6, map_q, map_k, map_v, map_o, p, st);
-            if (dqk == 128) return launch_pipelined<128, 128, true>(h, 7, map_q, map_k, map_v, map_o, p, st);
-            return launch_pipelined<192, 128, true>(h, 8, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 64) return launch_pipelined<64, 64, true>(h, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_pipelined<128, 128, true>(h, map_q, map_k, map_v, map_o, p, st);
+            return launch_pipelined<192, 128, true>(h, map_q, map_k, map_v, map_o, p, st);
         }
         if (pl.head_pair) {
-            if (dqk == 64) return launch_pipelined<64, 64, false, true>(h, 37, map_q, map_k, map_v, map_o, p, st);
-            if (dqk == 128) return launch_pipelined<128, 128, false, true>(h, 38, map_q, map_k, map_v, map_o, p, st);
-            return launch_pipelined<192, 128, false, true>(h, 39, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 64) return launch_pipelined<64, 64, false, true>(h, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_pipelined<128, 128, false, true>(h, map_q, map_k, map_v, map_o, p, st);
+            return launch_pipelined<192, 128, false, true>(h, map_q, map_k, map_v, map_o, p, st);
         }
-        if (dqk == 64) return launch_pipelined<64, 64, false>(h, 3, map_q, map_k, map_v, map_o, p, st);
-        if (dqk == 128) return launch_pipelined<128, 128, false>(h, 4, map_q, map_k, map_v, map_o, p, st);
-        return launch_pipelined<192, 128, false>(h, 5, map_q, map_k, map_v, map_o, p, st);
+        if (dqk == 64) return launch_pipelined<64, 64, false>(h, map_q, map_k, map_v, map_o, p, st);
+        if (dqk == 128) return launch_pipelined<128, 128, false>(h, map_q, map_k, map_v, map_o, p, st);
+        return launch_pipelined<192, 128, false>(h, map_q, map_k, map_v, map_o, p, st);
     }
     h->last_kernel = "fa_fwd_simple";
-    if (dqk == 64) return launch_simple<64, 64>(h, 0, map_q, map_k, map_v, p, st);
-    if (dqk == 128) return launch_simple<128, 128>(h, 1, map_q, map_k, map_v, p, st);
-    return launch_simple<192, 128>(h, 2, map_q, map_k, map_v, p, st);
+    if (dqk == 64) return launch_simple<64, 64>(h, map_q, map_k, map_v, p, st);
+    if (dqk == 128) return launch_simple<128, 128>(h, map_q, map_k, map_v, p, st);
+    return launch_simple<192, 128>(h, map_q, map_k, map_v, p, st);
 }
 
 }  // namespace
@@ -896,9 +900,8 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
              fa::fa_fwd_fp8_stream_kernel<64, true, 2>, fa::fa_fwd_fp8_stream_kernel<64, true, 4>},
             {fa::fa_fwd_fp8_stream_kernel<128, false, 1>, fa::fa_fwd_fp8_stream_kernel<128, true, 1>,
              fa::fa_fwd_fp8_stream_kernel<128, true, 2>, fa::fa_fwd_fp8_stream_kernel<128, true, 4>}};
-        static const int slots[2][4] = {{32, 33, 34, 35}, {22, 26, 27, 28}};
         Kernel kernel = kernels[d128 ? 1 : 0][variant];
-        if ((s = ensure_smem_attr(h, slots[d128 ? 1 : 0][variant], kernel, smem)) != FA_OK) return s;
+        if ((s = ensure_smem_attr(h, kernel, smem)) != FA_OK) return s;
         const long long n_ctas = (pack ? static_cast<long long>(Hq / pl.pack_heads) : static_cast<long long>(p.n_q_tiles) * Hq) * B * p.kv_splits;
         if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
         cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
@@ -926,7 +929,7 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     const bool hp = pl.head_pair && (pl.kernel == kPlanPair || pl.kernel == kPlanPersistent);
     auto kernel = hp ? (d128 ? fa::fa_fwd_fp8_kernel<128, true> : fa::fa_fwd_fp8_kernel<64, true>)
                      : (d128 ? fa::fa_fwd_fp8_kernel<128, false> : fa::fa_fwd_fp8_kernel<64, false>);
-    if ((s = ensure_smem_attr(h, hp ? (d128 ? 14 : 15) : (d128 ? 11 : 36), kernel, smem)) != FA_OK) return s;
+    if ((s = ensure_smem_attr(h, kernel, smem)) != FA_OK) return s;
     const long long n_ctas = (hp ? static_cast<long long>(p.n_q_tiles) * (Hq / 2) : static_cast<long long>((p.n_q_tiles + 1) / 2) * Hq) * B;
     if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
