@@ -445,10 +445,14 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     // every SM gets several items: measured on B200 it is 5-20 % faster from about three items per
     // SM on, level at 64-tile items and a few per cent slower below two items per SM (its one-time
     // set-up and the coarser balance of a short list).  d = 192 has no room for its staging buffer.
+    // Under a causal mask the items differ in length and the list balances worse the longer its
+    // longest item is: measured, lists of 3.5 items per SM are 4-6 % ahead with items of up to
+    // 4 K/V tiles and 1-4 % behind with longer ones, and ahead again from 4.3 items per SM on.
     const long long n_items = static_cast<long long>((n_q_tiles + 1) / 2) * Hq * B;
     const int longest = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, causal);
     const bool persistent_ok = !varlen && pair_splits == 1 && dqk != 192 && !drop;
-    bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= 32;
+    const long long min_items_per_sm = (!causal || longest <= 4) ? 3 : 4;
+    bool persistent = persistent_ok && n_items >= min_items_per_sm * num_sms && longest <= 32;
     if (flags & FA_FLAG_NO_PERSISTENT) persistent = false;
     if ((flags & FA_FLAG_FORCE_PERSISTENT) && persistent_ok) persistent = true;
     // One query tile per CTA (twice the CTAs, each with a shorter chain) wins where the pair

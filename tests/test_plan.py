@@ -34,6 +34,15 @@ def test_table6_rows():
     assert got["deepseek_67b_gqa_s4096"] == "fa_fwd_persistent"  # 1024 short items
 
 
+def test_persistent_kernel_needs_more_items_per_sm_under_a_causal_mask_with_long_items():
+    kernel = lambda B, Hq, Hkv, S, causal: binding.fa_plan(SMS, B, Hq, Hkv, S, S, 128, 128, causal)["kernel"]
+    assert kernel(2, 32, 8, 2048, True) == "fa_fwd_pipelined"       # 512 items of up to 16 K/V tiles: 3.5 per SM
+    assert kernel(2, 32, 32, 2048, True) == "fa_fwd_pipelined"
+    assert kernel(3, 32, 8, 2048, True) == "fa_fwd_persistent"      # 768 items: 5.2 per SM
+    assert kernel(8, 32, 8, 512, True) == "fa_fwd_persistent"       # 512 items of up to 4 tiles
+    assert kernel(2, 32, 8, 2048, False) == "fa_fwd_persistent"     # equal items: three per SM are enough
+
+
 def test_decode_like_shapes_split_the_kv_range_on_the_stream_kernel():
     p = binding.fa_plan(SMS, 1, 32, 8, 128, 32768, 128, 128, False)
     assert p["kernel"] == "fa_fwd_stream" and p["kv_splits"] == 4 and p["ctas"] == 32 * 4
