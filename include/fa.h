@@ -90,7 +90,10 @@ typedef enum fa_status {
  * query tile, so every K/V tile is fetched and multiplied once for all of them: the largest
  * divisor h of the group size with h * Sq <= 128 heads share a tile.  Results are those of the
  * unpacked launch up to fp32 rounding order (a row's arithmetic does not depend on its
- * neighbours).  This flag turns the packing off. */
+ * neighbours).  This flag turns the packing off.  It also turns off the pairing of heads on the
+ * tilings with two query tiles per CTA (an even group size under a causal mask or with an odd
+ * number of query tiles: the CTA's tiles are the same query tile of two adjacent heads of a
+ * group instead of two adjacent query tiles of one head; results bit-identical either way). */
 #define FA_FLAG_NO_HEAD_PACKING 128u
 
 /* Optional creation parameters.  Zero-initialise, set struct_size = sizeof(fa_config). */

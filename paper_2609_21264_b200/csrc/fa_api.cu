@@ -461,7 +461,8 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     // Causal grouped-query attention: pairing the same query tile of two heads of a group gives both
     // tiles of a pair-kernel CTA the same number of K/V tiles (no round that one of them runs alone).
     // (Without a mask it only matters for an odd number of query tiles, whose last tile would be alone.)
-    const bool head_pair_ok = !varlen && !drop && (causal || (n_q_tiles & 1)) && pair_splits == 1 && (Hq / Hkv) % 2 == 0 &&
+    // (Packed batches: every sequence's tiles pair up the same way; n_q_tiles is the longest one's.)
+    const bool head_pair_ok = !drop && (causal || (n_q_tiles & 1)) && pair_splits == 1 && (Hq / Hkv) % 2 == 0 &&
                               !(flags & FA_FLAG_NO_HEAD_PACKING);
     bool stream = false;
     int stream_splits = 1;
@@ -472,8 +473,12 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
             stream = true;
         } else if (varlen) {
             // no estimate without the lengths: 192/128 is always ahead, and with a single query tile
-            // per sequence the pair kernel's second tile would be empty
-            stream = (dqk == 192) || n_q_tiles == 1;
+            // per sequence the pair kernel's second tile would be empty, unless it is the same tile
+            // of the next head of the group: with more items than SMs that halves the number of
+            // CTAs and their fixed cost (B64 x 128 tokens, Hq 32 / Hkv 8: 57 vs 114 us)
+            const bool paired_single_tiles = n_q_tiles == 1 && head_pair_ok && dqk != 192 && stream_splits == 1 &&
+                                             static_cast<long long>(B) * Hq > num_sms;
+            stream = (dqk == 192) || (n_q_tiles == 1 && !paired_single_tiles);
         } else if (!persistent) {
             const TilingEstimate e = estimate_tilings(num_sms, B, Hq, Sq, Sk, dqk, causal, n_q_tiles, pair_splits, stream_splits, head_pair_ok);
             pl.pair_us = e.pair_us;
@@ -569,6 +574,11 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
     }
     if (pl.kernel == kPlanPair) {
         h->last_kernel = "fa_fwd_pipelined";
+        if (cu_q && pl.head_pair) {
+            if (dqk == 64) return launch_pipelined<64, 64, true, true>(h, map_q, map_k, map_v, map_o, p, st);
+            if (dqk == 128) return launch_pipelined<128, 128, true, true>(h, map_q, map_k, map_v, map_o, p, st);
+            return launch_pipelined<192, 128, true, true>(h, map_q, map_k, map_v, map_o, p, st);
+        }
         if (cu_q) {
             if (dqk == 64) return launch_pipelined<64, 64, true>(h, map_q, map_k, map_v, map_o, p, st);
             if (dqk == 128) return launch_pipelined<128, 128, true>(h, map_q, map_k, map_v, map_o, p, st);

@@ -95,3 +95,62 @@ def test_paired_heads_on_the_8_bit_path():
                 binding.fa_destroy(h)
         assert torch.equal(outs[0][0].view(torch.int16), outs[1][0].view(torch.int16))
         assert torch.equal(outs[0][1], outs[1][1])
+
+
+# (lens_q, lens_k, Hq, Hkv, d, causal): packed batches; the last two are many single-tile sequences, which the
+# plan gives to the pair kernel with paired heads instead of one CTA per head
+PACKED = [
+    ("mix_g4", [1, 127, 128, 129, 300, 512, 57], None, 8, 2, 128, True),
+    ("cross_lengths_empty_g2_d64", [40, 0, 200, 130, 5], [333, 50, 200, 0, 700], 4, 2, 64, True),
+    ("no_mask_three_tiles_g2", [300, 20, 333], None, 4, 2, 128, False),
+    ("d192_g2", [260, 31, 129], None, 4, 2, 192, True),
+    ("single_tiles_g4", [128, 100, 1, 77, 128, 64] * 4, None, 8, 2, 128, True),
+    ("single_tiles_long_keys_g2_d64", [16, 128, 90] * 14, [700, 128, 300] * 14, 4, 2, 64, True),
+]
+
+
+@pytest.mark.parametrize("name,lens_q,lens_k,Hq,Hkv,d,causal", PACKED, ids=[c[0] for c in PACKED])
+def test_paired_heads_in_packed_batches(name, lens_q, lens_k, Hq, Hkv, d, causal):
+    import torch
+    from paper_2609_21264_b200 import binding
+    lens_k = lens_q if lens_k is None else lens_k
+    dv = 128 if d == 192 else d
+    tq, tk = sum(lens_q), sum(lens_k)
+    w = W.Workload("packed", B=1, Hq=Hq, Hkv=Hkv, Sq=tq, Sk=tk, dqk=d, dv=dv, causal=False, scale=d ** -0.5, seed=1650 + len(lens_q))
+    Q, K, V = W.make_inputs(w)                                    # [1, H, total, d] -> [total, H, d]
+    q, k, v = (np.ascontiguousarray(x[0].transpose(1, 0, 2)) for x in (Q, K, V))
+    cu_q = np.concatenate([[0], np.cumsum(lens_q)]).astype(np.int32)
+    cu_k = np.concatenate([[0], np.cumsum(lens_k)]).astype(np.int32)
+    base = binding.FA_FLAG_NO_STREAM_KERNEL
+    outs = []
+    for flags in (base, base | binding.FA_FLAG_NO_HEAD_PACKING):
+        h = binding.fa_create(flags=flags)
+        try:
+            o, lse = binding.forward_varlen(h, to_torch_bf16(q), to_torch_bf16(k), to_torch_bf16(v), torch.from_numpy(cu_q).cuda(),
+                                            torch.from_numpy(cu_k).cuda(), max(lens_q), causal=causal, scale=w.scale)
+            torch.cuda.synchronize()
+            st, detail = binding.fa_last_status(h)
+            assert st == binding.FA_OK, "device status %d (site 0x%x)" % (st, detail)
+            assert binding.fa_last_kernel_name(h) == "fa_fwd_pipelined"
+            outs.append((o, lse))
+        finally:
+            binding.fa_destroy(h)
+    n_q_tiles = (max(lens_q) + 127) // 128
+    plan = binding.fa_plan(148, len(lens_q), Hq, Hkv, max(lens_q), max(1, tk // len(lens_k)), d, dv, causal, flags=base, varlen=True)
+    paired = causal or n_q_tiles % 2 == 1
+    assert plan["ctas"] == (n_q_tiles * (Hq // 2) if paired else (n_q_tiles + 1) // 2 * Hq) * len(lens_q), plan
+    assert torch.equal(outs[0][0].view(torch.int16), outs[1][0].view(torch.int16))
+    assert torch.equal(outs[0][1], outs[1][1])
+    O, L = bf16_tensor_to_f64(outs[0][0]), outs[0][1].double().cpu().numpy()
+    for b, (sq, sk) in enumerate(zip(lens_q, lens_k)):
+        if sq == 0:
+            continue
+        qs, ks = slice(cu_q[b], cu_q[b + 1]), slice(cu_k[b], cu_k[b + 1])
+        O_b, L_b = O[qs].transpose(1, 0, 2)[None], L[:, qs][None]
+        if sk == 0:
+            assert (O_b == 0).all() and np.isneginf(L_b).all()
+            continue
+        sl = lambda x, s: np.ascontiguousarray(x[s].transpose(1, 0, 2))[None]
+        O_ref, lse_ref = oracle.attention(sl(q, qs), sl(k, ks), sl(v, ks), causal=causal, scale=w.scale)
+        assert_parity(O_b, L_b, O_ref, lse_ref, "%s seq %d (%d x %d)" % (name, b, sq, sk))
+

@@ -101,3 +101,13 @@ def test_argument_errors():
         binding.fa_plan(SMS, 1, 2, 2, 128, 128, 96, 96, False)          # no kernel for this head size
     with pytest.raises(binding.FaError):
         binding.fa_plan(0, 1, 2, 2, 128, 128, 128, 128, False)
+
+
+def test_many_single_tile_sequences_take_the_pair_kernel_with_paired_heads():
+    plan = lambda B, Hq, Hkv, d, **kw: binding.fa_plan(SMS, B, Hq, Hkv, 128, 128, d, 128 if d == 192 else d, True, varlen=True, **kw)
+    p = plan(64, 32, 8, 128)
+    assert p["kernel"] == "fa_fwd_pipelined" and p["ctas"] == 64 * 16 and p["kv_splits"] == 1, p
+    assert plan(4, 32, 8, 128)["kernel"] == "fa_fwd_stream"              # 128 items: under a wave of single tiles
+    assert plan(64, 32, 32, 128)["kernel"] == "fa_fwd_stream"            # one head per K/V head: nothing to pair
+    assert plan(64, 32, 8, 192)["kernel"] == "fa_fwd_stream"             # 192/128 stays on the stream kernel
+    assert plan(64, 32, 8, 128, flags=binding.FA_FLAG_NO_HEAD_PACKING)["kernel"] == "fa_fwd_stream"
