@@ -69,11 +69,12 @@ typedef enum fa_status {
  * Results and ordering guarantees are the same either way; the default saves the stream's
  * completion-to-launch latency (a few microseconds per launch). */
 #define FA_FLAG_NO_DEPENDENT_LAUNCH 4u
-/* fa_config.flags: kernel choice.  The library runs fixed-length problems with many short work
- * items (at least three pairs of query tiles per SM, at most 32 K/V tiles each) on a persistent variant
- * of the pipelined kernel (one CTA per SM walking a list of items) and everything else on the
- * one-item-per-CTA kernel.  These two flags override the choice where both kernels apply (head
- * sizes 64 and 128, no split-KV, not a packed batch); results agree to rounding order. */
+/* fa_config.flags: kernel choice.  The library runs problems with many short work items (at
+ * least three pairs of query tiles per SM, four under a causal mask with more than 4 K/V tiles
+ * each, at most 32 K/V tiles each; packed batches counted by their longest sequence) on a
+ * persistent variant of the pipelined kernel (one CTA per SM walking a list of items) and
+ * everything else on the one-item-per-CTA kernel.  These two flags override the choice where
+ * both kernels apply (head sizes 64 and 128, no split-KV); results are bit-identical. */
 #define FA_FLAG_NO_PERSISTENT 8u
 #define FA_FLAG_FORCE_PERSISTENT 16u
 /* A third tiling: one query tile per CTA with its K/V tiles streamed through both softmax

@@ -270,13 +270,13 @@ int heads_per_group(long long kv_bytes_per_head, int B, int Hq, int Hkv) {
 }
 
 // Persistent kernel: one CTA per SM (fewer when there are fewer items), every CTA walks its share
-// of the items.  Fixed-length problems without split-KV only.
-template <int DQK, int DV>
+// of the items.  No split-KV.
+template <int DQK, int DV, bool kVarlen = false>
 fa_status launch_persistent(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& mk,
                             const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
     constexpr int smem = fa::persist_smem_bytes<DQK, DV>();
     static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
-    auto kernel = fa::fa_fwd_persistent_kernel<DQK, DV>;
+    auto kernel = fa::fa_fwd_persistent_kernel<DQK, DV, kVarlen>;
     fa_status s = ensure_smem_attr(h, kernel, smem);
     if (s != FA_OK) return s;
     const long long n_items = p.head_pair ? static_cast<long long>(p.n_q_tiles) * (p.Hq / 2) * p.B
@@ -396,8 +396,10 @@ struct LaunchPlan {
     bool head_pair;                // pair kernel: the CTA's two tiles are one query tile of two adjacent heads of a group
     double pair_us, stream_us;     // the two estimates (0 when no estimate was needed)
 };
+// (packed batches: Sq is the longest query length, Sk the mean K/V length, total_q the sum of the query
+//  lengths if known, else 0)
 LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size_t scratch_bytes, bool varlen,
-                       int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal) {
+                       int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal, long long total_q = 0) {
     LaunchPlan pl;
     pl.kernel = kPlanPair;
     pl.kv_splits = 1;
@@ -449,10 +451,16 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     // longest item is: measured, lists of 3.5 items per SM are 4-6 % ahead with items of up to
     // 4 K/V tiles and 1-4 % behind with longer ones, and ahead again from 4.3 items per SM on.
     const long long n_items = static_cast<long long>((n_q_tiles + 1) / 2) * Hq * B;
-    const int longest = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, causal);
-    const bool persistent_ok = !varlen && pair_splits == 1 && dqk != 192 && !drop;
+    // (packed batches: the list has an item for every tile of the longest sequence, which Sq is;
+    //  the sequences a tile does not exist in pass through the kernel's item ring empty)
+    const int longest = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, (varlen && Sk < Sq) ? Sq : Sk, causal);
+    const bool persistent_ok = pair_splits == 1 && dqk != 192 && !drop;
     const long long min_items_per_sm = (!causal || longest <= 4) ? 3 : 4;
     bool persistent = persistent_ok && n_items >= min_items_per_sm * num_sms && longest <= 32;
+    // A packed batch of short sequences of mixed lengths (at most two query tiles, many of them
+    // absent or partly filled) gains nothing from it: an item of one or two rounds costs a
+    // persistent CTA as much as a fresh CTA (1024 sequences of 16..256 tokens: 760 vs 706 us).
+    if (varlen && n_q_tiles <= 2 && total_q > 0 && total_q * 8 < static_cast<long long>(B) * Sq * 7) persistent = false;
     if (flags & FA_FLAG_NO_PERSISTENT) persistent = false;
     if ((flags & FA_FLAG_FORCE_PERSISTENT) && persistent_ok) persistent = true;
     // One query tile per CTA (twice the CTAs, each with a shorter chain) wins where the pair
@@ -478,7 +486,7 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
             // CTAs and their fixed cost (B64 x 128 tokens, Hq 32 / Hkv 8: 57 vs 114 us)
             const bool paired_single_tiles = n_q_tiles == 1 && head_pair_ok && dqk != 192 && stream_splits == 1 &&
                                              static_cast<long long>(B) * Hq > num_sms;
-            stream = (dqk == 192) || (n_q_tiles == 1 && !paired_single_tiles);
+            stream = (dqk == 192) || (n_q_tiles == 1 && !paired_single_tiles && !persistent);
         } else if (!persistent) {
             const TilingEstimate e = estimate_tilings(num_sms, B, Hq, Sq, Sk, dqk, causal, n_q_tiles, pair_splits, stream_splits, head_pair_ok);
             pl.pair_us = e.pair_us;
@@ -569,6 +577,10 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
     }
     if (pl.kernel == kPlanPersistent) {
         h->last_kernel = "fa_fwd_persistent";
+        if (cu_q) {
+            if (dqk == 64) return launch_persistent<64, 64, true>(h, map_q, map_k, map_v, map_o, p, st);
+            return launch_persistent<128, 128, true>(h, map_q, map_k, map_v, map_o, p, st);
+        }
         if (dqk == 64) return launch_persistent<64, 64>(h, map_q, map_k, map_v, map_o, p, st);
         return launch_persistent<128, 128>(h, map_q, map_k, map_v, map_o, p, st);
     }
@@ -796,7 +808,7 @@ fa_status fa_forward_varlen(fa_handle* h, const void* Q, const void* K, const vo
     // packed [total, H, d]: one batch slice, rows H*d apart, heads d apart
     const int mean_sk = (total_k + B - 1) / B > 0 ? (total_k + B - 1) / B : 1;
     const LaunchPlan pl = plan_launch(h->num_sms, h->flags, h->kv_splits_cfg, h->scratch_bytes, true,
-                                      B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal ? 1 : 0);
+                                      B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal ? 1 : 0, total_q);
     // packed heads: the box of Q is the max_sq rows (from the sequence's first row) of pack_heads heads
     const int q_box_rows = pl.pack_heads > 1 ? max_sq : fa::kTileM;
     const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;

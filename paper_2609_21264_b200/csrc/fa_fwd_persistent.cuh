@@ -25,7 +25,9 @@
 //
 // Differences in the roles: warp 15 (idle in the non-persistent kernel) loads the Q tiles, warp
 // 14 only K and V; two K stages instead of three at d = 128 make room for the staging buffer.
-// Fixed-length problems without split-KV only.
+// No split-KV.  kVarlen = packed variable-length batch: an item's lengths and row offsets are read
+// from p.cu_q / p.cu_k when it is decoded; the list has an item for every tile (pair) of the
+// longest sequence, and the items a shorter sequence does not have pass through the ring empty.
 #pragma once
 
 #include "fa_fwd_pipelined.cuh"
@@ -73,11 +75,14 @@ constexpr int persist_smem_bytes() {
 // One work item, decoded from its place in the longest-first order.
 struct PersistItem {
     int b, hq, kvh;
+    int Sq, Sk;              // lengths of the item's sequence (the launch's, or the packed sequence's)
+    int q_row0, k_row0;      // first rows of the sequence in the packed tensors (0 with fixed lengths)
     int hq1;                 // query head of tile 1 (the same head, or the next one when heads are paired)
     int i0_0, i0_1;          // first rows of the two query tiles (128 rows apart, or equal when heads are paired)
     int nkv_0, nkv_1, n_max; // K/V tiles of tile 0, tile 1, and the larger of the two
 };
 
+template <bool kVarlen = false>
 __device__ __forceinline__ PersistItem persist_decode(const FwdParams& p, int idx) {
     // Groups of (batch, head) instances whose K/V fit in L2 together follow one another; inside a
     // group every head's last (with a causal mask: heaviest) pair comes first.
@@ -101,13 +106,20 @@ __device__ __forceinline__ PersistItem persist_decode(const FwdParams& p, int id
     it.kvh = it.hq / (p.Hq / p.Hkv);
     it.i0_0 = (hp ? pair : 2 * pair) * kTileM;
     it.i0_1 = hp ? it.i0_0 : it.i0_0 + kTileM;
-    it.nkv_0 = kv_tiles_for_q_tile(it.i0_0, kTileM, p.Sq, p.Sk, p.causal);
-    it.nkv_1 = (it.i0_1 < p.Sq) ? kv_tiles_for_q_tile(it.i0_1, kTileM, p.Sq, p.Sk, p.causal) : 0;
+    it.Sq = p.Sq; it.Sk = p.Sk; it.q_row0 = 0; it.k_row0 = 0;
+    if constexpr (kVarlen) {
+        it.q_row0 = p.cu_q[it.b];
+        it.k_row0 = p.cu_k[it.b];
+        it.Sq = p.cu_q[it.b + 1] - it.q_row0;
+        it.Sk = p.cu_k[it.b + 1] - it.k_row0;
+    }
+    it.nkv_0 = (it.i0_0 < it.Sq) ? kv_tiles_for_q_tile(it.i0_0, kTileM, it.Sq, it.Sk, p.causal) : 0;
+    it.nkv_1 = (it.i0_1 < it.Sq) ? kv_tiles_for_q_tile(it.i0_1, kTileM, it.Sq, it.Sk, p.causal) : 0;
     it.n_max = it.nkv_0 > it.nkv_1 ? it.nkv_0 : it.nkv_1;
     return it;
 }
 
-template <int DQK, int DV>
+template <int DQK, int DV, bool kVarlen = false>
 __global__ void __launch_bounds__(512, 1)
 fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                          const __grid_constant__ CUtensorMap tm_k,
@@ -194,7 +206,6 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
     const uint32_t tmem_base = sh.tmem_base;
     WaitCtx wctx{&sh.abort_flag, p.status, p.wait_limit_ns};
     const float c = p.scale_log2;
-    const int off = p.Sk - p.Sq;
 
     // Consumer side of the work-item ring: the k-th item of this CTA, or -1 at the end of the list
     // (or when a wait gave up).  The warp form is called by all lanes of a warp together.
@@ -237,17 +248,20 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
         for (int k = 0; ok; ++k) {
             const int idx = item_index(k);
             if (idx < 0) break;
-            int nkv_t, i0_t;
+            int nkv_t, i0_t, Sq, Sk;
             uint32_t my_use;           // this tile's place in the order of staging-buffer users
             {
-                const PersistItem item = persist_decode(p, idx);
+                const PersistItem item = persist_decode<kVarlen>(p, idx);
                 nkv_t = t == 0 ? item.nkv_0 : item.nkv_1;
                 i0_t = t == 0 ? item.i0_0 : item.i0_1;
+                Sq = item.Sq;
+                Sk = item.Sk;
                 my_use = uc + ((t == 1 && item.nkv_0 > 0) ? 1u : 0u);
                 uc += (item.nkv_0 > 0 ? 1u : 0u) + (item.nkv_1 > 0 ? 1u : 0u);
             }
             const int i_glob = i0_t + row;
-            int kmax_row = p.Sk - 1;
+            const int off = Sk - Sq;
+            int kmax_row = Sk - 1;
             if (p.causal && i_glob + off < kmax_row) kmax_row = i_glob + off;
 
             float m_ref = -INFINITY;   // reference maximum, raw score units
@@ -347,14 +361,16 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             if (!ok) break;
 
             // ---- epilogue of the item: O = G' / s (bf16), lse = u * scale + ln s
-            if (i0_t >= p.Sq) continue;
-            const PersistItem item = persist_decode(p, idx);     // again: nothing of it was kept live
+            if (i0_t >= Sq) continue;
+            const PersistItem item = persist_decode<kVarlen>(p, idx);     // again: nothing of it was kept live
             const int hq_t = t == 0 ? item.hq : item.hq1;
-            const size_t lse_row0 = (static_cast<size_t>(item.b) * p.Hq + hq_t) * p.Sq;
+            // fixed lengths: lse [B, Hq, Sq]; packed batches: lse [Hq, total_q], O rows q_row0 onwards
+            const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq_t) * p.total_q + item.q_row0
+                                            : (static_cast<size_t>(item.b) * p.Hq + hq_t) * p.Sq;
+            __nv_bfloat16* o_row = p.O + ((kVarlen ? item.q_row0 * p.o_stride_s : item.b * p.o_stride_b) + hq_t * p.o_stride_h +
+                                          static_cast<long long>(i_glob) * p.o_stride_s);
             if (nkv_t == 0) {             // no key visible to any row of this tile
-                if (i_glob < p.Sq) {
-                    __nv_bfloat16* o_row = p.O + (item.b * p.o_stride_b + hq_t * p.o_stride_h +
-                                                  static_cast<long long>(i_glob) * p.o_stride_s);
+                if (i_glob < Sq) {
                     const uint4 z = make_uint4(0, 0, 0, 0);
 #pragma unroll
                     for (int v = 0; v < DV / 8; ++v) reinterpret_cast<uint4*>(o_row)[v] = z;
@@ -367,8 +383,13 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             if (!ok) break;
             tc_fence_after_sync();
             const float inv_l = (l > 0.f) ? (1.f / l) : 0.f;
-            if (p.lse && i_glob < p.Sq)
+            if (p.lse && i_glob < Sq)
                 p.lse[lse_row0 + i_glob] = (l > 0.f) ? (m_ref * c * 0.6931471805599453f + logf(l)) : -INFINITY;
+            // A packed batch's last tile of a sequence is followed by the next sequence's rows, which a
+            // box store would overwrite: its rows go from registers to global memory one by one (it
+            // still takes its turn at the staging buffer, so that the order of users stays the list's;
+            // one 256-byte bulk copy per row out of the staging buffer measured 5-15 % slower).
+            const bool box_store = !kVarlen || (i0_t + kTileM <= Sq);
             // the previous user's TMA store must have read the staging buffer
             ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.stage_empty), (my_use & 1u) ^ 1u, wctx, kSiteEpiStaged));
             if (!ok) break;
@@ -379,14 +400,24 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 tmem_ld_x32(tO + cc * 32, r);
                 tc_wait_ld();
                 const uint32_t chunk = sO + (cc >> 1) * kChunkBytes;
+                if (box_store) {
 #pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    const uint32_t piece = static_cast<uint32_t>(((cc & 1) * 4 + v) ^ (row & 7)) << 4;
-                    st_shared_v4(chunk + piece,
-                                 pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
-                                 pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
-                                 pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
-                                 pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
+                    for (int v = 0; v < 4; ++v) {
+                        const uint32_t piece = static_cast<uint32_t>(((cc & 1) * 4 + v) ^ (row & 7)) << 4;
+                        st_shared_v4(chunk + piece,
+                                     pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
+                                     pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
+                                     pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
+                                     pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
+                    }
+                } else if (i_glob < Sq) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v)
+                        reinterpret_cast<uint4*>(o_row + cc * 32)[v] = make_uint4(
+                            pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
+                            pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
+                            pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
+                            pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
                 }
             }
             // O_t has been read: order the TMEM loads before the next item's MMAs into O_t and S_t
@@ -397,11 +428,14 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             if ((warp & 3) == 0 && lane == 0) {
                 ok = mbar_wait(smem_addr(&sh.stage_full), my_use & 1u, wctx, kSiteEpiStaged);
                 if (ok) {
+                    if (box_store) {
 #pragma unroll
-                    for (int ch = 0; ch < DV / kChunkCols; ++ch)
-                        tma_store_4d(&tm_o, sStage + ch * kChunkBytes, ch * kChunkCols, i0_t, hq_t, item.b);
-                    tma_store_commit();
-                    tma_store_wait_read_all();
+                        for (int ch = 0; ch < DV / kChunkCols; ++ch)
+                            tma_store_4d(&tm_o, sStage + ch * kChunkBytes, ch * kChunkCols, item.q_row0 + i0_t, hq_t,
+                                         kVarlen ? 0 : item.b);
+                        tma_store_commit();
+                        tma_store_wait_read_all();
+                    }
                     mbar_arrive(smem_addr(&sh.stage_empty));
                 }
             }
@@ -420,7 +454,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
         for (int k = 0; ok; ++k) {
             const int idx = item_index(k);
             if (idx < 0) break;
-            const PersistItem item = persist_decode(p, idx);
+            const PersistItem item = persist_decode<kVarlen>(p, idx);
 #pragma unroll 1
             for (int j = 0; j < item.n_max && ok; ++j) {
 #pragma unroll
@@ -510,7 +544,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 if (idx < 0) break;
                 int nkv_t, n_max;
                 {
-                    const PersistItem item = persist_decode(p, idx);
+                    const PersistItem item = persist_decode<kVarlen>(p, idx);
                     nkv_t = (t == 0) ? item.nkv_0 : item.nkv_1;
                     n_max = item.n_max;
                 }
@@ -581,7 +615,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 *reinterpret_cast<volatile int*>(&sh.item_ring[slot]) = idx;
                 mbar_arrive(smem_addr(&sh.item_full[slot]));
                 if (idx >= n_items) break;
-                const PersistItem item = persist_decode(p, idx);
+                const PersistItem item = persist_decode<kVarlen>(p, idx);
 #pragma unroll 1
                 for (int j = 0; j < item.n_max; ++j) {
                     const int j0 = j * kTileN;
@@ -594,7 +628,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                         for (int cc = 0; cc < Base::kQChunks; ++cc)
                             tma_load_4d(sK + s * Cfg::kKBytes + cc * kChunkBytes, &tm_k, bar, cc * kChunkCols,
-                                        j0, item.kvh, item.b);
+                                        item.k_row0 + j0, item.kvh, kVarlen ? 0 : item.b);
                         ++kc;
                     }
                     {
@@ -606,14 +640,15 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                         for (int cc = 0; cc < Base::kVChunks; ++cc)
                             tma_load_4d(sV + s * Cfg::kVBytes + cc * kChunkBytes, &tm_v, bar, cc * kChunkCols,
-                                        j0, item.kvh, item.b);
+                                        item.k_row0 + j0, item.kvh, kVarlen ? 0 : item.b);
                         ++vc;
                     }
                 }
                 // Draw the next item only now that the loads of this one are all issued (the rings
                 // keep this thread a tile or two ahead of the MMAs): an earlier draw would bind an
-                // item to this CTA long before it can start on it.  The launch makes n_items draws
-                // in all (n_items - G that return an item, one past the end per CTA).
+                // item to this CTA long before it can start on it (starting the atomic ahead of the
+                // loads of short items, to hide its round trip, measured 1-4 % slower).  The launch
+                // makes n_items draws in all (n_items - G that return an item, one past the end per CTA).
                 const unsigned int ticket = atomicAdd(p.sched_counter, 1u);
                 if (ticket == static_cast<unsigned int>(n_items) - 1u) atomicExch(p.sched_counter, 0u);
                 idx = G + static_cast<int>(ticket);
@@ -629,7 +664,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             for (int k = 0; ok; ++k) {
                 const int idx = item_index_thread(k);
                 if (idx < 0) break;
-                const PersistItem item = persist_decode(p, idx);
+                const PersistItem item = persist_decode<kVarlen>(p, idx);
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if ((t == 0 ? item.nkv_0 : item.nkv_1) == 0) continue;
@@ -641,7 +676,8 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                     for (int cc = 0; cc < Base::kQChunks; ++cc)
                         tma_load_4d(sQ + t * Cfg::kQBytes + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols,
-                                    t == 0 ? item.i0_0 : item.i0_1, t == 0 ? item.hq : item.hq1, item.b);
+                                    item.q_row0 + (t == 0 ? item.i0_0 : item.i0_1), t == 0 ? item.hq : item.hq1,
+                                    kVarlen ? 0 : item.b);
                     if (t == 0) ++qc0; else ++qc1;
                 }
             }

@@ -13,12 +13,13 @@ from parity_util import assert_parity, bf16_tensor_to_f64, to_torch_bf16
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module", params=["pipelined", "serial", "stream"])
+@pytest.fixture(scope="module", params=["pipelined", "serial", "stream", "persistent"])
 def handle(request):
     from paper_2609_21264_b200 import binding
     # the fixed-length comparison below wants the same tiling (hence rounding order) as the packed path
-    flags = {"serial": binding.FA_FLAG_SERIAL_KERNEL, "pipelined": binding.FA_FLAG_NO_STREAM_KERNEL,
-             "stream": binding.FA_FLAG_STREAM_KERNEL}[request.param]
+    flags = {"serial": binding.FA_FLAG_SERIAL_KERNEL, "pipelined": binding.FA_FLAG_NO_STREAM_KERNEL | binding.FA_FLAG_NO_PERSISTENT,
+             "stream": binding.FA_FLAG_STREAM_KERNEL,
+             "persistent": binding.FA_FLAG_NO_STREAM_KERNEL | binding.FA_FLAG_FORCE_PERSISTENT}[request.param]
     h = binding.fa_create(flags=flags)
     yield h
     binding.fa_destroy(h)

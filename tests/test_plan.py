@@ -103,11 +103,16 @@ def test_argument_errors():
         binding.fa_plan(0, 1, 2, 2, 128, 128, 128, 128, False)
 
 
-def test_many_single_tile_sequences_take_the_pair_kernel_with_paired_heads():
-    plan = lambda B, Hq, Hkv, d, **kw: binding.fa_plan(SMS, B, Hq, Hkv, 128, 128, d, 128 if d == 192 else d, True, varlen=True, **kw)
+def test_packed_batches_of_many_short_sequences():
+    plan = lambda B, Hq, Hkv, d, S=128, **kw: binding.fa_plan(SMS, B, Hq, Hkv, S, S, d, 128 if d == 192 else d, True, varlen=True, **kw)
+    # many items per SM: the persistent kernel, heads of a group paired (one item per tile and pair of heads)
     p = plan(64, 32, 8, 128)
+    assert p["kernel"] == "fa_fwd_persistent" and p["ctas"] == SMS and p["kv_splits"] == 1, p
+    assert plan(8, 32, 8, 128, S=2048)["kernel"] == "fa_fwd_persistent"
+    # without it: single tiles of two heads of a group share a CTA of the pair kernel
+    p = plan(64, 32, 8, 128, flags=binding.FA_FLAG_NO_PERSISTENT)
     assert p["kernel"] == "fa_fwd_pipelined" and p["ctas"] == 64 * 16 and p["kv_splits"] == 1, p
     assert plan(4, 32, 8, 128)["kernel"] == "fa_fwd_stream"              # 128 items: under a wave of single tiles
-    assert plan(64, 32, 32, 128)["kernel"] == "fa_fwd_stream"            # one head per K/V head: nothing to pair
+    assert plan(64, 32, 32, 128, flags=binding.FA_FLAG_NO_PERSISTENT)["kernel"] == "fa_fwd_stream"   # nothing to pair
     assert plan(64, 32, 8, 192)["kernel"] == "fa_fwd_stream"             # 192/128 stays on the stream kernel
-    assert plan(64, 32, 8, 128, flags=binding.FA_FLAG_NO_HEAD_PACKING)["kernel"] == "fa_fwd_stream"
+    assert plan(64, 32, 8, 128, flags=binding.FA_FLAG_NO_HEAD_PACKING | binding.FA_FLAG_NO_PERSISTENT)["kernel"] == "fa_fwd_stream"
