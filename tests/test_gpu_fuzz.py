@@ -1,6 +1,8 @@
 """Seeded fuzz over the entry points (contiguous, strided, block-scaled 8-bit, packed batches): small
 random problems of every kind through one default handle, each checked against the oracle, so that
-whatever kernel, tiling, split count and head sharing the library plans for a shape is exercised."""
+whatever kernel, tiling, split count and head sharing the library plans for a shape is exercised;
+and once more through a handle that takes the persistent kernel wherever it applies (small
+problems would never reach it by themselves)."""
 import numpy as np
 import pytest
 
@@ -12,11 +14,12 @@ pytestmark = pytest.mark.gpu
 N_CASES = 160
 
 
-@pytest.fixture(scope="module")
-def handle():
+@pytest.fixture(scope="module", params=["planned", "persistent_where_possible"])
+def handle(request):
     from paper_2609_21264_b200 import binding
-    h = binding.fa_create()
-    yield h
+    h = binding.fa_create(flags=0 if request.param == "planned" else binding.FA_FLAG_FORCE_PERSISTENT)
+    h_kind = request.param
+    yield h, h_kind
     binding.fa_destroy(h)
 
 
@@ -38,7 +41,8 @@ def _check(handle, name, O, lse, O_ref, lse_ref, Vd=None, G=1):
 def test_fuzz_all_entry_points(handle):
     import torch
     from paper_2609_21264_b200 import binding
-    rng = np.random.default_rng(20261127)
+    handle, handle_kind = handle
+    rng = np.random.default_rng(20261127 if handle_kind == "planned" else 20261128)
     seen = set()
     for it in range(N_CASES):
         kind = int(rng.integers(0, 4))           # 0 contiguous, 1 [B,S,H,d] strides, 2 e4m3, 3 packed batch
@@ -112,5 +116,8 @@ def test_fuzz_all_entry_points(handle):
     # the fuzz is only worth its time if it reaches the tilings: both kernels of the 16-bit path, with and without
     # split-KV, the 8-bit stream kernel and packed batches on the stream kernel
     kernels = {(k, n) for k, n, _ in seen}
-    assert {(0, "fa_fwd_stream"), (0, "fa_fwd_pipelined"), (2, "fa_fwd_fp8_stream"), (3, "fa_fwd_stream")} <= kernels, seen
+    if handle_kind == "planned":
+        assert {(0, "fa_fwd_stream"), (0, "fa_fwd_pipelined"), (2, "fa_fwd_fp8_stream"), (3, "fa_fwd_stream")} <= kernels, seen
+    else:
+        assert {(0, "fa_fwd_persistent"), (1, "fa_fwd_persistent"), (3, "fa_fwd_persistent"), (3, "fa_fwd_stream")} <= kernels, seen
     assert any(s for _, _, s in seen)
