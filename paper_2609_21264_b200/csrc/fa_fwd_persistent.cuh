@@ -386,9 +386,8 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             if (p.lse && i_glob < Sq)
                 p.lse[lse_row0 + i_glob] = (l > 0.f) ? (m_ref * c * 0.6931471805599453f + logf(l)) : -INFINITY;
             // A packed batch's last tile of a sequence is followed by the next sequence's rows, which a
-            // box store would overwrite: its rows go from registers to global memory one by one (it
-            // still takes its turn at the staging buffer, so that the order of users stays the list's;
-            // one 256-byte bulk copy per row out of the staging buffer measured 5-15 % slower).
+            // box store would overwrite: every warp copies the rows it staged to global memory itself
+            // (one 256-byte bulk copy per row out of the staging buffer measured 5-15 % slower).
             const bool box_store = !kVarlen || (i0_t + kTileM <= Sq);
             // the previous user's TMA store must have read the staging buffer
             ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.stage_empty), (my_use & 1u) ^ 1u, wctx, kSiteEpiStaged));
@@ -400,25 +399,21 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 tmem_ld_x32(tO + cc * 32, r);
                 tc_wait_ld();
                 const uint32_t chunk = sO + (cc >> 1) * kChunkBytes;
-                if (box_store) {
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        const uint32_t piece = static_cast<uint32_t>(((cc & 1) * 4 + v) ^ (row & 7)) << 4;
-                        st_shared_v4(chunk + piece,
-                                     pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
-                                     pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
-                                     pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
-                                     pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
-                    }
-                } else if (i_glob < Sq) {
-#pragma unroll
-                    for (int v = 0; v < 4; ++v)
-                        reinterpret_cast<uint4*>(o_row + cc * 32)[v] = make_uint4(
-                            pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
-                            pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
-                            pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
-                            pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
+                for (int v = 0; v < 4; ++v) {
+                    const uint32_t piece = static_cast<uint32_t>(((cc & 1) * 4 + v) ^ (row & 7)) << 4;
+                    st_shared_v4(chunk + piece,
+                                 pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
+                                 pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
+                                 pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
+                                 pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
                 }
+            }
+            if (!box_store) {
+                // every warp copies the 32 rows it staged itself, whole rows per instruction
+                __syncwarp();
+                store_staged_rows<DV>(sStage, (warp & 3) * 32, Sq - i0_t, o_row - static_cast<long long>(row) * p.o_stride_s,
+                                      p.o_stride_s, lane);
             }
             // O_t has been read: order the TMEM loads before the next item's MMAs into O_t and S_t
             tc_fence_before_sync();

@@ -407,7 +407,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 // A packed batch's last tile of a sequence is followed by the next sequence's rows,
                 // which a box store would overwrite: such tiles take the row-by-row path.
                 const bool box_store = !kVarlen || (i0_t + kTileM <= Sq);
-                if (box_store) {
+                {
                     // The tile goes through shared memory (the Q tile's space: its last reader, the
                     // final score MMA, is complete once o_final has fired) in the swizzled layout of
                     // a TMA box, and one thread stores it; rows past Sq are clipped by the TMA unit.
@@ -429,6 +429,8 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                                          pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
                         }
                     }
+                }
+                if (box_store) {
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_addr(&sh.o_staged[t]));
@@ -442,23 +444,10 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                         tma_store_wait_read_all();     // the CTA's shared memory outlives the reads
                     }
                 } else {
-#pragma unroll 1
-                    for (int cc = 0; cc < DV / 32; ++cc) {
-                        uint32_t r[32];
-                        tmem_ld_x32(tO + cc * 32, r);
-                        tc_wait_ld();
-                        if (i_glob < Sq) {
-                            uint32_t pk[16];
-#pragma unroll
-                            for (int e = 0; e < 32; e += 2)
-                                pk[e / 2] = pack_bf16x2(__uint_as_float(r[e]) * inv_l,
-                                                        __uint_as_float(r[e + 1]) * inv_l);
-#pragma unroll
-                            for (int v = 0; v < 4; ++v)
-                                reinterpret_cast<uint4*>(o_row + cc * 32)[v] =
-                                    make_uint4(pk[4 * v], pk[4 * v + 1], pk[4 * v + 2], pk[4 * v + 3]);
-                        }
-                    }
+                    // every warp copies the 32 rows it staged itself, whole rows per instruction
+                    __syncwarp();
+                    store_staged_rows<DV>(sQ + t * Cfg::kQBytes, (warp & 3) * 32, Sq - i0_t,
+                                          o_row - static_cast<long long>(row) * p.o_stride_s, p.o_stride_s, lane);
                 }
             }
         }

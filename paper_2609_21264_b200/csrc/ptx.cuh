@@ -205,6 +205,32 @@ FA_DEVI void tma_store_4d(const CUtensorMap* map, uint32_t src_smem, int c0, int
 FA_DEVI void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
+FA_DEVI uint4 ld_shared_v4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+// A warp's 32 rows of a bf16 output tile, staged in the swizzled layout of a TMA box (64-column
+// chunks of 128 rows x 128 bytes, 16-byte pieces XORed with the row's low three bits), go to global
+// memory coalesced: consecutive lanes take consecutive 16-byte pieces of a row, so one instruction
+// covers whole rows instead of 32 rows' pieces.  Rows from `valid_rows` on are skipped.  For the
+// tiles that cannot leave as one TMA box (the last, partly filled tile of a packed sequence).
+// tile_smem: the tile's staging area; row0: the warp's first row in it; tile_global: address of
+// the tile's row 0, column 0; stride: elements between rows.  The caller has synchronised the warp
+// after its own stores into the staging area (every lane staged row0 + lane).
+template <int DV>
+FA_DEVI void store_staged_rows(uint32_t tile_smem, int row0, int valid_rows, __nv_bfloat16* tile_global,
+                               long long stride, int lane) {
+    constexpr int kPieces = DV / 8;                  // 16-byte pieces per row
+    constexpr int kRowsPerPass = 32 / kPieces;
+    const int piece = lane % kPieces;
+#pragma unroll 4
+    for (int rr = 0; rr < 32; rr += kRowsPerPass) {
+        const int r = row0 + rr + lane / kPieces;
+        const uint4 v = ld_shared_v4(tile_smem + (piece >> 3) * (128 * 128) + r * 128 + (((piece & 7) ^ (r & 7)) << 4));
+        if (r < valid_rows) *reinterpret_cast<uint4*>(tile_global + r * stride + piece * 8) = v;
+    }
+}
 FA_DEVI void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 FA_DEVI void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 FA_DEVI void tma_store_wait_read_all() {
