@@ -238,7 +238,10 @@ fa_status fa_forward_fp8(fa_handle* h,
  * many CTAs, and the two run-time estimates behind the choice (0 when none was needed).  A pure
  * host function: no handle, no device, no CUDA call; `num_sms` is the SM count to plan for (148 on
  * B200) and `cfg` the creation parameters a handle would have (NULL = defaults; its device field is
- * ignored).  `varlen` != 0 plans fa_forward_varlen with Sq = max_sq and Sk = the mean key length.
+ * ignored).  `varlen` != 0 plans fa_forward_varlen with Sq = max_sq and Sk = the mean key length,
+ * as for a batch whose sequences all have max_sq queries (the launch also knows total_q: with at
+ * most two query tiles per sequence and total_q below 7/8 of B * max_sq it keeps the batch off the
+ * persistent kernel).
  * The tile schedule is the first step of the path (one CTA per pair of query tiles in the paper's
  * mapping, Section 4); here it is chosen per launch, and this call makes the choice inspectable.
  * Returns FA_ERR_UNSUPPORTED for head sizes the kernels do not have, FA_ERR_INVALID_ARG otherwise.
