@@ -395,7 +395,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the short timing of the other configs")
     ap.add_argument("--table6", action="store_true",
                     help="also time the twelve attention shapes of the paper's Table 6 (key 'table6')")
-    ap.add_argument("--no-decode", action="store_true", help="skip the grouped-head decode step (key 'decode')")
+    ap.add_argument("--no-decode", action="store_true", help="skip the grouped-head decode step and the packed batches (keys 'decode', 'packed_batches')")
     ap.add_argument("--libraries", action="store_true",
                     help="also time the attention kernels of the libraries in the image (torch SDPA back ends, flash_attn) "
                          "on the five configurations and a few decode shapes, for context (key 'libraries')")
@@ -557,6 +557,36 @@ def main():
                                    "frac_of_measured_hbm": bytes8 / t8 / 1e9 / peaks["hbm_gbs"]},
                           "note": "inputs larger than L2 (1.07 GB / 0.54 GB of K and V); 20 launches each after 3 warm-up launches"}
         del qd, kd, vd, od, ld, q8, k8, v8
+        torch.cuda.empty_cache()
+
+        # Packed batches of sequences of different lengths (fa_forward_varlen; Hq 32 / Hkv 8, d 128, causal):
+        # one batch of equal sequences (comparable with the fixed-length call) and one of mixed lengths.
+        import numpy as np
+        packed = []
+        for pname, lens in (("8 x 2048 tokens", [2048] * 8),
+                            ("64 sequences of 64..2048 tokens", [int(x) for x in np.random.RandomState(5).randint(64, 2049, 64)])):
+            tq = int(sum(lens))
+            qp = torch.randn((tq, 32, 128), generator=gen, device=device).to(torch.bfloat16)
+            kp = torch.randn((tq, 8, 128), generator=gen, device=device).to(torch.bfloat16)
+            vp = torch.randn((tq, 8, 128), generator=gen, device=device).to(torch.bfloat16)
+            op = torch.empty_like(qp)
+            lp = torch.empty((32, tq), dtype=torch.float32, device=device)
+            cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device=device)
+
+            def packed_call():
+                st = binding.fa_forward_varlen(h, qp.data_ptr(), kp.data_ptr(), vp.data_ptr(), op.data_ptr(), lp.data_ptr(),
+                                               cu.data_ptr(), cu.data_ptr(), len(lens), tq, tq, max(lens), 32, 8, 128, 128,
+                                               True, 0.0, cs)
+                if st != binding.FA_OK:
+                    raise binding.FaError(st, "fa_forward_varlen")
+
+            tp = timed_launches(packed_call)
+            flp = 4.0 * 128 * 32 * sum(l * (l + 1) // 2 for l in lens)
+            packed.append({"workload": pname, "total_tokens": tq, "us": tp * 1e6, "tflops_algorithmic": flp / tp / 1e12,
+                           "kernel": binding.fa_last_kernel_name(h)})
+            del qp, kp, vp, op, lp, cu
+        line["packed_batches"] = {"cases": packed, "note": "Hq 32 / Hkv 8, d 128, causal, lengths on the device; "
+                                  "20 launches each after 3 warm-up launches"}
         torch.cuda.empty_cache()
 
     if not args.no_e2e:
