@@ -70,8 +70,8 @@ typedef enum fa_status {
  * completion-to-launch latency (a few microseconds per launch). */
 #define FA_FLAG_NO_DEPENDENT_LAUNCH 4u
 /* fa_config.flags: kernel choice.  The library runs problems with many short work items (at
- * least three pairs of query tiles per SM, four under a causal mask with more than 4 K/V tiles
- * each, at most 32 K/V tiles each; packed batches counted by their longest sequence) on a
+ * least three pairs of query tiles per SM, at most 32 K/V tiles each; packed batches counted by
+ * their longest sequence) on a
  * persistent variant of the pipelined kernel (one CTA per SM walking a list of items) and
  * everything else on the one-item-per-CTA kernel.  These two flags override the choice where
  * both kernels apply (head sizes 64 and 128, no split-KV); results are bit-identical. */
@@ -238,10 +238,7 @@ fa_status fa_forward_fp8(fa_handle* h,
  * many CTAs, and the two run-time estimates behind the choice (0 when none was needed).  A pure
  * host function: no handle, no device, no CUDA call; `num_sms` is the SM count to plan for (148 on
  * B200) and `cfg` the creation parameters a handle would have (NULL = defaults; its device field is
- * ignored).  `varlen` != 0 plans fa_forward_varlen with Sq = max_sq and Sk = the mean key length,
- * as for a batch whose sequences all have max_sq queries (the launch also knows total_q: with at
- * most two query tiles per sequence and total_q below 7/8 of B * max_sq it keeps the batch off the
- * persistent kernel).
+ * ignored).  `varlen` != 0 plans fa_forward_varlen with Sq = max_sq and Sk = the mean key length.
  * The tile schedule is the first step of the path (one CTA per pair of query tiles in the paper's
  * mapping, Section 4); here it is chosen per launch, and this call makes the choice inspectable.
  * Returns FA_ERR_UNSUPPORTED for head sizes the kernels do not have, FA_ERR_INVALID_ARG otherwise.

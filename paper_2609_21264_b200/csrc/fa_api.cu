@@ -396,10 +396,9 @@ struct LaunchPlan {
     bool head_pair;                // pair kernel: the CTA's two tiles are one query tile of two adjacent heads of a group
     double pair_us, stream_us;     // the two estimates (0 when no estimate was needed)
 };
-// (packed batches: Sq is the longest query length, Sk the mean K/V length, total_q the sum of the query
-//  lengths if known, else 0)
+// (packed batches: Sq is the longest query length, Sk the mean K/V length)
 LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size_t scratch_bytes, bool varlen,
-                       int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal, long long total_q = 0) {
+                       int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv, int causal) {
     LaunchPlan pl;
     pl.kernel = kPlanPair;
     pl.kv_splits = 1;
@@ -447,20 +446,12 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     // every SM gets several items: measured on B200 it is 5-20 % faster from about three items per
     // SM on, level at 64-tile items and a few per cent slower below two items per SM (its one-time
     // set-up and the coarser balance of a short list).  d = 192 has no room for its staging buffer.
-    // Under a causal mask the items differ in length and the list balances worse the longer its
-    // longest item is: measured, lists of 3.5 items per SM are 4-6 % ahead with items of up to
-    // 4 K/V tiles and 1-4 % behind with longer ones, and ahead again from 4.3 items per SM on.
     const long long n_items = static_cast<long long>((n_q_tiles + 1) / 2) * Hq * B;
     // (packed batches: the list has an item for every tile of the longest sequence, which Sq is;
     //  the sequences a tile does not exist in pass through the kernel's item ring empty)
     const int longest = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, (varlen && Sk < Sq) ? Sq : Sk, causal);
     const bool persistent_ok = pair_splits == 1 && dqk != 192 && !drop;
-    const long long min_items_per_sm = (!causal || longest <= 4) ? 3 : 4;
-    bool persistent = persistent_ok && n_items >= min_items_per_sm * num_sms && longest <= 32;
-    // A packed batch of short sequences of mixed lengths (at most two query tiles, many of them
-    // absent or partly filled) gains nothing from it: an item of one or two rounds costs a
-    // persistent CTA as much as a fresh CTA (1024 sequences of 16..256 tokens: 760 vs 706 us).
-    if (varlen && n_q_tiles <= 2 && total_q > 0 && total_q * 8 < static_cast<long long>(B) * Sq * 7) persistent = false;
+    bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= 32;
     if (flags & FA_FLAG_NO_PERSISTENT) persistent = false;
     if ((flags & FA_FLAG_FORCE_PERSISTENT) && persistent_ok) persistent = true;
     // One query tile per CTA (twice the CTAs, each with a shorter chain) wins where the pair
@@ -808,7 +799,7 @@ fa_status fa_forward_varlen(fa_handle* h, const void* Q, const void* K, const vo
     // packed [total, H, d]: one batch slice, rows H*d apart, heads d apart
     const int mean_sk = (total_k + B - 1) / B > 0 ? (total_k + B - 1) / B : 1;
     const LaunchPlan pl = plan_launch(h->num_sms, h->flags, h->kv_splits_cfg, h->scratch_bytes, true,
-                                      B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal ? 1 : 0, total_q);
+                                      B, Hq, Hkv, max_sq, mean_sk, dqk, dv, causal ? 1 : 0);
     // packed heads: the box of Q is the max_sq rows (from the sequence's first row) of pack_heads heads
     const int q_box_rows = pl.pack_heads > 1 ? max_sq : fa::kTileM;
     const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;

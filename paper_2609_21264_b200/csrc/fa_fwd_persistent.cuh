@@ -16,7 +16,8 @@
 //
 // Items are ordered longest first (as in the non-persistent grid).  CTA c starts with item c;
 // every further item is drawn from a global ticket counter by the K/V load thread once the loads
-// of the current item are all issued, and handed to the other roles through a four-slot ring in
+// of the current item are all issued, decoded by that thread (the divisions of the decode take a
+// lone thread over a thousand cycles) and handed to the other roles through a four-slot ring in
 // shared memory, so a CTA that got short items simply takes more of them.  Every CTA draws
 // exactly one ticket past the end of the list, which makes the total number of draws known: the
 // CTA that takes the last one puts the counter back to zero for the next launch.  All mbarrier
@@ -46,6 +47,18 @@ struct PersistCfg {
     static constexpr int kTileBytes = 2 * kQBytes + kKStages * kKBytes + kVStages * kVBytes + kOBytes;
 };
 
+// One work item, decoded from its place in the longest-first order.
+struct alignas(16) PersistItem {
+    int b, hq, kvh;
+    int Sq, Sk;              // lengths of the item's sequence (the launch's, or the packed sequence's)
+    int q_row0, k_row0;      // first rows of the sequence in the packed tensors (0 with fixed lengths)
+    int hq1;                 // query head of tile 1 (the same head, or the next one when heads are paired)
+    int i0_0, i0_1;          // first rows of the two query tiles (128 rows apart, or equal when heads are paired)
+    int nkv_0, nkv_1, n_max; // K/V tiles of tile 0, tile 1, and the larger of the two
+    int pad[3];
+};
+static_assert(sizeof(PersistItem) == 64, "the item ring moves items as four 16-byte words");
+
 struct PersistShared {
     uint64_t q_full[2];      // Q loader -> MMA thread t: Q_t of the item is in shared memory
     uint64_t q_empty[2];     // MMA thread t -> Q loader: last score MMA of the item has read Q_t
@@ -61,7 +74,8 @@ struct PersistShared {
     uint64_t stage_empty;    // storing thread -> softmax warps: the TMA store has read the staging buffer
     uint64_t item_full[4];   // K/V load thread -> every role: item_ring[slot] holds the next work item
     uint64_t item_empty[4];  // every role -> K/V load thread: slot read (8 + 4 warps, 2 MMA threads, Q loader)
-    int item_ring[4];
+    int item_ring[4];        // index of the item in the list (>= the list's length: the end mark)
+    PersistItem items[4];    // the item itself, decoded once by the K/V load thread
     float alpha[2][2][kTileM];   // [tile][iteration & 1][row]
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -71,16 +85,6 @@ template <int DQK, int DV>
 constexpr int persist_smem_bytes() {
     return PersistCfg<DQK, DV>::kTileBytes + static_cast<int>(sizeof(PersistShared));
 }
-
-// One work item, decoded from its place in the longest-first order.
-struct PersistItem {
-    int b, hq, kvh;
-    int Sq, Sk;              // lengths of the item's sequence (the launch's, or the packed sequence's)
-    int q_row0, k_row0;      // first rows of the sequence in the packed tensors (0 with fixed lengths)
-    int hq1;                 // query head of tile 1 (the same head, or the next one when heads are paired)
-    int i0_0, i0_1;          // first rows of the two query tiles (128 rows apart, or equal when heads are paired)
-    int nkv_0, nkv_1, n_max; // K/V tiles of tile 0, tile 1, and the larger of the two
-};
 
 template <bool kVarlen = false>
 __device__ __forceinline__ PersistItem persist_decode(const FwdParams& p, int idx) {
@@ -209,21 +213,35 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
 
     // Consumer side of the work-item ring: the k-th item of this CTA, or -1 at the end of the list
     // (or when a wait gave up).  The warp form is called by all lanes of a warp together.
-    auto item_index_thread = [&](int k) -> int {
+    // A consumer waits for slot k & 3, copies what it needs (item_at) and releases the slot; the softmax
+    // warps, which need the item again in their epilogue, release it at the end of the item instead.
+    auto item_wait_thread = [&](int k) -> int {
         const int slot = k & 3;
         if (!mbar_wait(smem_addr(&sh.item_full[slot]), (static_cast<uint32_t>(k) >> 2) & 1u, wctx, kSiteItem)) return -1;
         const int idx = *reinterpret_cast<volatile int*>(&sh.item_ring[slot]);
-        mbar_arrive(smem_addr(&sh.item_empty[slot]));
         return idx < n_items ? idx : -1;
     };
-    auto item_index = [&](int k) -> int {
+    auto item_wait = [&](int k) -> int {
         const int slot = k & 3;
         if (!__all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.item_full[slot]), (static_cast<uint32_t>(k) >> 2) & 1u,
                                                wctx, kSiteItem))) return -1;
         const int idx = *reinterpret_cast<volatile int*>(&sh.item_ring[slot]);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_addr(&sh.item_empty[slot]));
         return idx < n_items ? idx : -1;
+    };
+    auto item_at = [&](int k) -> PersistItem {
+        PersistItem it_;
+        const volatile int4* src = reinterpret_cast<const volatile int4*>(&sh.items[k & 3]);
+        int4* dst = reinterpret_cast<int4*>(&it_);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            dst[i].x = src[i].x; dst[i].y = src[i].y; dst[i].z = src[i].z; dst[i].w = src[i].w;
+        }
+        return it_;
+    };
+    auto item_release_thread = [&](int k) { mbar_arrive(smem_addr(&sh.item_empty[k & 3])); };
+    auto item_release = [&](int k) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_addr(&sh.item_empty[k & 3]));
     };
 
     if (warp < 8) {
@@ -245,13 +263,12 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
         bool ok = true;
 
 #pragma unroll 1
-        for (int k = 0; ok; ++k) {
-            const int idx = item_index(k);
-            if (idx < 0) break;
+        for (int k = 0; ok; item_release(k), ++k) {      // (the slot is kept until the item's epilogue has read it again)
+            if (item_wait(k) < 0) break;
             int nkv_t, i0_t, Sq, Sk;
             uint32_t my_use;           // this tile's place in the order of staging-buffer users
             {
-                const PersistItem item = persist_decode<kVarlen>(p, idx);
+                const PersistItem item = item_at(k);
                 nkv_t = t == 0 ? item.nkv_0 : item.nkv_1;
                 i0_t = t == 0 ? item.i0_0 : item.i0_1;
                 Sq = item.Sq;
@@ -362,7 +379,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
 
             // ---- epilogue of the item: O = G' / s (bf16), lse = u * scale + ln s
             if (i0_t >= Sq) continue;
-            const PersistItem item = persist_decode<kVarlen>(p, idx);     // again: nothing of it was kept live
+            const PersistItem item = item_at(k);     // again: nothing of it was kept live
             const int hq_t = t == 0 ? item.hq : item.hq1;
             // fixed lengths: lse [B, Hq, Sq]; packed batches: lse [Hq, total_q], O rows q_row0 onwards
             const size_t lse_row0 = kVarlen ? static_cast<size_t>(hq_t) * p.total_q + item.q_row0
@@ -447,9 +464,9 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
         bool ok = true;
 #pragma unroll 1
         for (int k = 0; ok; ++k) {
-            const int idx = item_index(k);
-            if (idx < 0) break;
-            const PersistItem item = persist_decode<kVarlen>(p, idx);
+            if (item_wait(k) < 0) break;
+            const PersistItem item = item_at(k);
+            item_release(k);
 #pragma unroll 1
             for (int j = 0; j < item.n_max && ok; ++j) {
 #pragma unroll
@@ -535,14 +552,14 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             bool ok = true;
 #pragma unroll 1
             for (int k = 0; ok; ++k) {
-                const int idx = item_index_thread(k);
-                if (idx < 0) break;
+                if (item_wait_thread(k) < 0) break;
                 int nkv_t, n_max;
                 {
-                    const PersistItem item = persist_decode<kVarlen>(p, idx);
+                    const PersistItem item = item_at(k);
                     nkv_t = (t == 0) ? item.nkv_0 : item.nkv_1;
                     n_max = item.n_max;
                 }
+                item_release_thread(k);
                 if (n_max == 0) continue;
                 // First block of the item: S_t(0) = Q_t K_0^T.  It is issued as soon as its operands
                 // are there, outside the alternation of the two threads: the other thread may still
@@ -607,10 +624,20 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 const int slot = k & 3;
                 if (k >= 4) ok = mbar_wait(smem_addr(&sh.item_empty[slot]), ((static_cast<uint32_t>(k) >> 2) - 1u) & 1u, wctx, kSiteItem);
                 if (!ok) break;
+                PersistItem item;
+                if (idx < n_items) {
+                    item = persist_decode<kVarlen>(p, idx);
+                    item.pad[0] = item.pad[1] = item.pad[2] = 0;
+                    const int4* src = reinterpret_cast<const int4*>(&item);
+                    volatile int4* dst = reinterpret_cast<volatile int4*>(&sh.items[slot]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        dst[i].x = src[i].x; dst[i].y = src[i].y; dst[i].z = src[i].z; dst[i].w = src[i].w;
+                    }
+                }
                 *reinterpret_cast<volatile int*>(&sh.item_ring[slot]) = idx;
-                mbar_arrive(smem_addr(&sh.item_full[slot]));
+                mbar_arrive(smem_addr(&sh.item_full[slot]));       // (release: the stores above are visible to whoever sees the phase)
                 if (idx >= n_items) break;
-                const PersistItem item = persist_decode<kVarlen>(p, idx);
 #pragma unroll 1
                 for (int j = 0; j < item.n_max; ++j) {
                     const int j0 = j * kTileN;
@@ -657,9 +684,9 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             bool ok = true;
 #pragma unroll 1
             for (int k = 0; ok; ++k) {
-                const int idx = item_index_thread(k);
-                if (idx < 0) break;
-                const PersistItem item = persist_decode<kVarlen>(p, idx);
+                if (item_wait_thread(k) < 0) break;
+                const PersistItem item = item_at(k);
+                item_release_thread(k);
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if ((t == 0 ? item.nkv_0 : item.nkv_1) == 0) continue;

@@ -34,13 +34,14 @@ def test_table6_rows():
     assert got["deepseek_67b_gqa_s4096"] == "fa_fwd_persistent"  # 1024 short items
 
 
-def test_persistent_kernel_needs_more_items_per_sm_under_a_causal_mask_with_long_items():
+def test_persistent_kernel_from_three_items_per_sm():
     kernel = lambda B, Hq, Hkv, S, causal: binding.fa_plan(SMS, B, Hq, Hkv, S, S, 128, 128, causal)["kernel"]
-    assert kernel(2, 32, 8, 2048, True) == "fa_fwd_pipelined"       # 512 items of up to 16 K/V tiles: 3.5 per SM
-    assert kernel(2, 32, 32, 2048, True) == "fa_fwd_pipelined"
-    assert kernel(3, 32, 8, 2048, True) == "fa_fwd_persistent"      # 768 items: 5.2 per SM
+    assert kernel(2, 32, 8, 2048, True) == "fa_fwd_persistent"      # 512 items of up to 16 K/V tiles: 3.5 per SM
+    assert kernel(2, 32, 32, 2048, True) == "fa_fwd_persistent"
     assert kernel(8, 32, 8, 512, True) == "fa_fwd_persistent"       # 512 items of up to 4 tiles
-    assert kernel(2, 32, 8, 2048, False) == "fa_fwd_persistent"     # equal items: three per SM are enough
+    assert kernel(2, 32, 8, 2048, False) == "fa_fwd_persistent"
+    assert kernel(1, 32, 8, 2048, True) == "fa_fwd_pipelined"       # 256 items: under two per SM
+    assert kernel(1, 32, 8, 8192, True) == "fa_fwd_pipelined"       # items of 64 K/V tiles
 
 
 def test_decode_like_shapes_split_the_kv_range_on_the_stream_kernel():
@@ -89,7 +90,8 @@ def test_flags_and_configuration_override_the_choice():
 
 
 def test_packed_batches_and_head_size_192():
-    assert binding.fa_plan(SMS, 4, 16, 4, 2048, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_pipelined"
+    assert binding.fa_plan(SMS, 2, 16, 4, 2048, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_pipelined"    # 256 items
+    assert binding.fa_plan(SMS, 4, 16, 4, 2048, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_persistent"   # 512 items
     assert binding.fa_plan(SMS, 4, 16, 4, 2048, 1024, 192, 128, True, varlen=True)["kernel"] == "fa_fwd_stream"
     assert binding.fa_plan(SMS, 1, 16, 16, 2048, 2048, 192, 128, True)["kernel"] == "fa_fwd_stream"
 
