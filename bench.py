@@ -611,7 +611,8 @@ def main():
             tr, bd = metrics.roofline_seconds(fa, nb, pk, peaks["hbm_gbs"])
             per.append({"config": idx, "workload": wc.name, "us": t * 1e6, "tflops_algorithmic": fa / t / 1e12,
                         "tflops_paper_convention": fp / t / 1e12, "bound": bd, "roofline_frac": tr / t,
-                        "frac_of_nominal_2250": fa / t / 2.25e15, "steps": k})
+                        "frac_of_nominal_2250": fa / t / 2.25e15, "steps": k,
+                        "kernel": binding.fa_last_kernel_name(h)})
             del ss
             torch.cuda.empty_cache()
         line["per_config"] = per

@@ -444,14 +444,15 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     const int pair_splits = varlen ? 1 : choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles);
     // The persistent kernel wins where a CTA's fixed cost is a visible share of an item's time and
     // every SM gets several items: measured on B200 it is 5-20 % faster from about three items per
-    // SM on, level at 64-tile items and a few per cent slower below two items per SM (its one-time
-    // set-up and the coarser balance of a short list).  d = 192 has no room for its staging buffer.
+    // SM on, still 2 % faster at 64-tile items (d = 128; level at d = 64), 1-2 % slower at 128-tile
+    // items and a few per cent slower below two items per SM (its one-time set-up and the coarser
+    // balance of a short list).  d = 192 has no room for its staging buffer.
     const long long n_items = static_cast<long long>((n_q_tiles + 1) / 2) * Hq * B;
     // (packed batches: the list has an item for every tile of the longest sequence, which Sq is;
     //  the sequences a tile does not exist in pass through the kernel's item ring empty)
     const int longest = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, (varlen && Sk < Sq) ? Sq : Sk, causal);
     const bool persistent_ok = pair_splits == 1 && dqk != 192 && !drop;
-    bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= 32;
+    bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= (dqk == 64 ? 32 : 64);
     if (flags & FA_FLAG_NO_PERSISTENT) persistent = false;
     if ((flags & FA_FLAG_FORCE_PERSISTENT) && persistent_ok) persistent = true;
     // One query tile per CTA (twice the CTAs, each with a shorter chain) wins where the pair

@@ -14,7 +14,8 @@ def plan(w, **kw):
 
 
 def test_benchmark_configurations():
-    expect = ["fa_fwd_stream", "fa_fwd_pipelined", "fa_fwd_pipelined", "fa_fwd_stream", "fa_fwd_pipelined"]
+    # (config 3: 4096 items of up to 64 K/V tiles, the longest the persistent kernel is chosen for)
+    expect = ["fa_fwd_stream", "fa_fwd_pipelined", "fa_fwd_persistent", "fa_fwd_stream", "fa_fwd_pipelined"]
     for w, kernel in zip(W.CONFIGS, expect):
         p = plan(w)
         assert p["kernel"] == kernel, (w.name, p)
@@ -41,7 +42,11 @@ def test_persistent_kernel_from_three_items_per_sm():
     assert kernel(8, 32, 8, 512, True) == "fa_fwd_persistent"       # 512 items of up to 4 tiles
     assert kernel(2, 32, 8, 2048, False) == "fa_fwd_persistent"
     assert kernel(1, 32, 8, 2048, True) == "fa_fwd_pipelined"       # 256 items: under two per SM
-    assert kernel(1, 32, 8, 8192, True) == "fa_fwd_pipelined"       # items of 64 K/V tiles
+    assert kernel(1, 32, 8, 8192, True) == "fa_fwd_persistent"      # items of 64 K/V tiles: the limit at d = 128
+    assert kernel(4, 32, 32, 8192, True) == "fa_fwd_persistent"
+    assert kernel(1, 32, 8, 16384, True) == "fa_fwd_pipelined"      # items of 128 K/V tiles
+    assert binding.fa_plan(SMS, 4, 16, 16, 4096, 4096, 64, 64, True)["kernel"] == "fa_fwd_persistent"   # d = 64: up to 32 tiles
+    assert binding.fa_plan(SMS, 4, 16, 16, 8192, 8192, 64, 64, True)["kernel"] != "fa_fwd_persistent"
 
 
 def test_decode_like_shapes_split_the_kv_range_on_the_stream_kernel():
