@@ -46,6 +46,12 @@ struct PipeCfg {
     static constexpr int kTileBytes = 2 * kQBytes + kKStages * kKBytes + kVStages * kVBytes;
     static constexpr int kTmemCols = 512;
     static constexpr int kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 384;
+    // At head size 64 an O accumulator takes 64 columns and the 64 behind it hold P_t, so that
+    // P_t(j) does not overlay S_t: the score MMA of K/V tile j+1 is then issued as soon as the softmax
+    // warps hold S_t(j) in registers, and a tile's chain is softmax -> softmax instead of
+    // softmax -> PV -> QK.  (At 128 the 512 columns are taken by 2 x (S + O) and P_t overlays S_t.)
+    static constexpr bool kSeparateP = (DV == 64);
+    static constexpr int kColP0 = kSeparateP ? kColO0 + 64 : kColS0, kColP1 = kSeparateP ? kColO1 + 64 : kColS1;
     static constexpr int kThreads = 512;
 };
 
@@ -68,6 +74,8 @@ struct PipeShared {
     uint64_t o_final[2];     // MMA -> softmax: last PV of tile t done, O_t is final
     uint64_t turn[2];        // MMA thread 1-t -> MMA thread t: your turn to issue
     uint64_t o_staged[2];    // softmax warps -> storing thread: the bf16 O_t tile is in shared memory
+    uint64_t pv_done[2];     // MMA -> softmax, correction (separate P only): PV of iteration j complete, P_t and O_t may be written
+    uint64_t s_read[2];      // softmax -> MMA (separate P only): S_t(j) is in registers, the next score block may be issued
     float alpha[2][2][kTileM];   // [tile][j & 1][row]
     uint32_t tmem_base;
     uint32_t abort_flag;
@@ -196,6 +204,8 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             mbar_init(smem_addr(&sh.o_final[t]), 1);
             mbar_init(smem_addr(&sh.turn[t]), 1);
             mbar_init(smem_addr(&sh.o_staged[t]), 4);     // 4 softmax warps
+            mbar_init(smem_addr(&sh.pv_done[t]), 1);
+            mbar_init(smem_addr(&sh.s_read[t]), 4);       // 4 softmax warps
         }
 #pragma unroll
         for (int s = 0; s < 4; ++s) {
@@ -232,6 +242,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         const int row = tid & (kTileM - 1);
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1) + lane_sel;
+        const uint32_t tP = tmem_base + (t == 0 ? Cfg::kColP0 : Cfg::kColP1) + lane_sel;
         const uint32_t bar_s = smem_addr(&sh.s_full[t]);
         const uint32_t bar_p = smem_addr(&sh.p_full[t]);
         const uint32_t bar_ph = smem_addr(&sh.p_half[t]);
@@ -283,7 +294,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                     pk[e / 2] = pack_bf16x2(v0.x, v0.y);
                     pk[e / 2 + 1] = pack_bf16x2(v1.x, v1.y);
                 }
-                tmem_st_x16(tS + q * 16, pk);
+                tmem_st_x16(tP + q * 16, pk);
             };
             // The exponentials do not wait for the row maximum: they start against the reference
             // maximum carried over from earlier tiles while the maximum of this tile is reduced on
@@ -325,6 +336,21 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 }
             }
             sh.alpha[t][j & 1][row] = alpha;
+            if constexpr (Cfg::kSeparateP) {
+                // S_t(j) is in registers: the next score block may overwrite it.
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_addr(&sh.s_read[t]));
+                // P_t(j-1) is still being read by its PV product unless that has completed.  The wait
+                // comes before the rescale factor is published, not just before the first store of
+                // P_t(j): the softmax no longer follows the PV product on the tensor pipe, and without it
+                // scale_full could run two phases ahead of the correction warps.
+                if (j > 0) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.pv_done[t]), (j - 1) & 1, wctx, kSiteSoftmaxSFull));
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                }
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_scale);
             if (lane == 0 && ((warp & 3) == 0 || (warp & 3) == 2)) FA_TRACE_STAMP(t + ((warp & 3) == 2 ? 4 : 0), j, 2);
@@ -465,6 +491,13 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                        kSiteCorrScale));
                 if (!ok) break;
                 const float alpha = sh.alpha[t][j & 1][row];
+                if constexpr (Cfg::kSeparateP) {
+                    // the score block of iteration j no longer follows the PV product of j-1 on the tensor pipe
+                    if (j > 0) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.pv_done[t]), (j - 1) & 1, wctx, kSiteCorrScale));
+                        if (!ok) break;
+                    }
+                }
                 if (lane == 0 && (warp & 3) == 0) FA_TRACE_STAMP(3, j, t * 4 + 0);
                 if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
                     tc_fence_after_sync();
@@ -505,7 +538,8 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
             const uint32_t q_lo = (((sQ + t * Cfg::kQBytes) & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((static_cast<uint32_t>(kChunkBytes) >> 4) << 16);
-            const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1);   // P_t overlays it
+            const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1);   // P_t overlays it unless kSeparateP
+            const uint32_t tP = tmem_base + (t == 0 ? Cfg::kColP0 : Cfg::kColP1);
             const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1);
             const uint32_t bar_s = smem_addr(&sh.s_full[t]);
             const uint32_t bar_ph = smem_addr(&sh.p_half[t]);
@@ -527,7 +561,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 const uint32_t vlo = v_lo0 + stage * (Cfg::kVBytes >> 4);
 #pragma unroll
                 for (int kk = 4 * half; kk < 4 * half + 4; ++kk)
-                    mma_ts(tO, tS + kk * 8, desc(vlo + kk * (2048 >> 4)), kIdescPV,
+                    mma_ts(tO, tP + kk * 8, desc(vlo + kk * (2048 >> 4)), kIdescPV,
                            (half == 0 && kk == 0) ? accumulate : 1u);
             };
             // The two issuing threads alternate strictly, one block of MMAs each (round r of thread
@@ -565,6 +599,18 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 // tile, so that neither arrives twice in one phase of an "empty" barrier.
                 ok = mbar_wait(smem_addr(&sh.v_full[sv]), ph_v, wctx, kSiteMmaKvFull);
                 if (ok && j + 1 < n_max) ok = mbar_wait(smem_addr(&sh.k_full[sk]), ph_k, wctx, kSiteMmaKvFull);
+                if constexpr (Cfg::kSeparateP) {
+                    // Next score block first, outside the alternation: it needs S_t(j) to have been read, not P_t(j).
+                    if (ok && j + 1 < nkv_t) {
+                        ok = mbar_wait(smem_addr(&sh.s_read[t]), j & 1, wctx, kSiteMmaPFull);
+                        if (ok) {
+                            tc_fence_after_sync();
+                            issue_qk(sk);
+                            tc_commit(bar_s);
+                        }
+                    }
+                    if (ok && j + 1 < n_max) tc_commit(bar_ke);   // arrives at once if nothing was issued
+                }
                 if (ok && j < nkv_t) {
                     FA_TRACE_STAMP(2, j, t * 4 + 0);
                     ok = mbar_wait(bar_ph, j & 1, wctx, kSiteMmaPFull);
@@ -581,9 +627,10 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                     if (!ok) break;
                     tc_fence_after_sync();
                     issue_pv_half(IntC<1>{}, sv, 1u);
+                    if constexpr (Cfg::kSeparateP) tc_commit(smem_addr(&sh.pv_done[t]));
                     FA_TRACE_STAMP(2, j, t * 4 + 2);
                 }
-                if (j + 1 < nkv_t) {
+                if (!Cfg::kSeparateP && j + 1 < nkv_t) {
                     issue_qk(sk);
                     tc_commit(bar_s);
                     FA_TRACE_STAMP(2, j, t * 4 + 3);
@@ -591,7 +638,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                     tc_commit(smem_addr(&sh.o_final[t]));
                 }
                 tc_commit(bar_ve);
-                if (j + 1 < n_max) tc_commit(bar_ke);
+                if (!Cfg::kSeparateP && j + 1 < n_max) tc_commit(bar_ke);
                 pass_turn();
                 if (++sv == NV) { sv = 0; ph_v ^= 1u; }
                 if (++sk == NK) { sk = 0; ph_k ^= 1u; }
