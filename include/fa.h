@@ -70,7 +70,7 @@ typedef enum fa_status {
  * completion-to-launch latency (a few microseconds per launch). */
 #define FA_FLAG_NO_DEPENDENT_LAUNCH 4u
 /* fa_config.flags: kernel choice.  The library runs problems with many short work items (at
- * least three pairs of query tiles per SM, at most 64 K/V tiles each, 32 at head size 64;
+ * least three pairs of query tiles per SM, at most 64 K/V tiles each, 16 at head size 64;
  * packed batches counted by their longest sequence) on a persistent variant of the pipelined
  * kernel (one CTA per SM walking a list of items) and everything else on the one-item-per-CTA kernel.  These two flags override the choice where
  * both kernels apply (head sizes 64 and 128, no split-KV); results are bit-identical. */

@@ -444,15 +444,16 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     const int pair_splits = varlen ? 1 : choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles);
     // The persistent kernel wins where a CTA's fixed cost is a visible share of an item's time and
     // every SM gets several items: measured on B200 it is 5-20 % faster from about three items per
-    // SM on, still 2 % faster at 64-tile items (d = 128; level at d = 64), 1-2 % slower at 128-tile
-    // items and a few per cent slower below two items per SM (its one-time set-up and the coarser
-    // balance of a short list).  d = 192 has no room for its staging buffer.
+    // SM on, still 2 % faster at 64-tile items at d = 128, 1-2 % slower at 128-tile items; at d = 64,
+    // where the pair kernel keeps P in TMEM columns of its own and has the shorter chain per K/V tile,
+    // it is 5-12 % faster up to 8-tile items, level at 16 and 4-5 % slower at 32; and it is a few per
+    // cent slower below two items per SM (its one-time set-up and the coarser balance of a short list).  d = 192 has no room for its staging buffer.
     const long long n_items = static_cast<long long>((n_q_tiles + 1) / 2) * Hq * B;
     // (packed batches: the list has an item for every tile of the longest sequence, which Sq is;
     //  the sequences a tile does not exist in pass through the kernel's item ring empty)
     const int longest = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, (varlen && Sk < Sq) ? Sq : Sk, causal);
     const bool persistent_ok = pair_splits == 1 && dqk != 192 && !drop;
-    bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= (dqk == 64 ? 32 : 64);
+    bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= (dqk == 64 ? 16 : 64);
     if (flags & FA_FLAG_NO_PERSISTENT) persistent = false;
     if ((flags & FA_FLAG_FORCE_PERSISTENT) && persistent_ok) persistent = true;
     // One query tile per CTA (twice the CTAs, each with a shorter chain) wins where the pair
@@ -484,9 +485,10 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
             pl.pair_us = e.pair_us;
             pl.stream_us = e.stream_us;
             stream = e.stream_us < 0.9 * e.pair_us;
-            // at d = 64 the stream kernel is also 3-7 % ahead on long items (measured from 64
-            // K/V tiles per query tile on), closer than the estimate can tell
-            if (dqk == 64 && longest >= 32 && pair_splits == 1 && stream_splits == 1) stream = true;
+            // at d = 64 the stream kernel is also ahead on long items, closer than the estimate can
+            // tell: 10 % without a mask (64 K/V tiles per query tile), 3-4 % under a causal mask from
+            // 256 tiles on; with shorter causal items the pair kernel is 2-9 % ahead
+            if (dqk == 64 && longest >= (causal ? 192 : 32) && pair_splits == 1 && stream_splits == 1) stream = true;
         }
     }
     if (stream) {

@@ -45,8 +45,8 @@ def test_persistent_kernel_from_three_items_per_sm():
     assert kernel(1, 32, 8, 8192, True) == "fa_fwd_persistent"      # items of 64 K/V tiles: the limit at d = 128
     assert kernel(4, 32, 32, 8192, True) == "fa_fwd_persistent"
     assert kernel(1, 32, 8, 16384, True) == "fa_fwd_pipelined"      # items of 128 K/V tiles
-    assert binding.fa_plan(SMS, 4, 16, 16, 4096, 4096, 64, 64, True)["kernel"] == "fa_fwd_persistent"   # d = 64: up to 32 tiles
-    assert binding.fa_plan(SMS, 4, 16, 16, 8192, 8192, 64, 64, True)["kernel"] != "fa_fwd_persistent"
+    assert binding.fa_plan(SMS, 8, 16, 16, 2048, 2048, 64, 64, True)["kernel"] == "fa_fwd_persistent"   # d = 64: up to 16 tiles
+    assert binding.fa_plan(SMS, 4, 16, 16, 4096, 4096, 64, 64, True)["kernel"] == "fa_fwd_pipelined"
 
 
 def test_decode_like_shapes_split_the_kv_range_on_the_stream_kernel():
