@@ -35,6 +35,10 @@ CASES = [
     _wl("more_queries_than_keys", 1, 150, 150, 400, 140, 128, True, 1204),   # tiles with no visible key
     _wl("fewer_items_than_sms", 1, 4, 2, 700, 700, 128, True, 1205),         # 12 items: short grid
     _wl("single_tile_items", 1, 300, 300, 100, 260, 64, False, 1206),        # tile 1 never exists
+    # head size 64: the per-item kernel keeps P in TMEM columns of its own and issues score blocks ahead of
+    # the PV products, the persistent kernel does not; items long enough for the hand-offs to wrap many times
+    _wl("long_causal_items_d64", 2, 12, 12, 2048, 2048, 64, True, 1207),     # up to 16 K/V tiles, tile 0 one short of tile 1
+    _wl("long_full_items_d64", 1, 20, 4, 1100, 2300, 64, False, 1208),       # 18 K/V tiles, ragged tails
 ]
 
 
