@@ -346,7 +346,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 // P_t(j): the softmax no longer follows the PV product on the tensor pipe, and without it
                 // scale_full could run two phases ahead of the correction warps.
                 if (j > 0) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.pv_done[t]), (j - 1) & 1, wctx, kSiteSoftmaxSFull));
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.pv_done[t]), (j - 1) & 1, wctx, kSiteSoftmaxPFree));
                     if (!ok) break;
                     tc_fence_after_sync();
                 }
@@ -494,7 +494,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 if constexpr (Cfg::kSeparateP) {
                     // the score block of iteration j no longer follows the PV product of j-1 on the tensor pipe
                     if (j > 0) {
-                        ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.pv_done[t]), (j - 1) & 1, wctx, kSiteCorrScale));
+                        ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.pv_done[t]), (j - 1) & 1, wctx, kSiteCorrPvDone));
                         if (!ok) break;
                     }
                 }
@@ -602,7 +602,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
                 if constexpr (Cfg::kSeparateP) {
                     // Next score block first, outside the alternation: it needs S_t(j) to have been read, not P_t(j).
                     if (ok && j + 1 < nkv_t) {
-                        ok = mbar_wait(smem_addr(&sh.s_read[t]), j & 1, wctx, kSiteMmaPFull);
+                        ok = mbar_wait(smem_addr(&sh.s_read[t]), j & 1, wctx, kSiteMmaSFree);
                         if (ok) {
                             tc_fence_after_sync();
                             issue_qk(sk);
