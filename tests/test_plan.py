@@ -123,3 +123,14 @@ def test_packed_batches_of_many_short_sequences():
     assert plan(64, 32, 32, 128, flags=binding.FA_FLAG_NO_PERSISTENT)["kernel"] == "fa_fwd_stream"   # nothing to pair
     assert plan(64, 32, 8, 192)["kernel"] == "fa_fwd_stream"             # 192/128 stays on the stream kernel
     assert plan(64, 32, 8, 128, flags=binding.FA_FLAG_NO_HEAD_PACKING | binding.FA_FLAG_NO_PERSISTENT)["kernel"] == "fa_fwd_stream"
+
+
+def test_head_size_64_long_items():
+    # The pair kernel at head size 64 keeps P in TMEM columns of its own and is ahead of the stream
+    # kernel on causal items of up to 128 K/V tiles; without a mask, and on longer causal items, the
+    # stream kernel stays ahead.
+    kernel = lambda S, causal: binding.fa_plan(SMS, 1, 16, 16, S, S, 64, 64, causal)["kernel"]
+    assert kernel(8192, True) == "fa_fwd_pipelined"
+    assert kernel(16384, True) == "fa_fwd_pipelined"
+    assert kernel(32768, True) == "fa_fwd_stream"
+    assert kernel(8192, False) == "fa_fwd_stream"
