@@ -95,6 +95,11 @@ typedef enum fa_status {
  * number of query tiles: the CTA's tiles are the same query tile of two adjacent heads of a
  * group instead of two adjacent query tiles of one head; results bit-identical either way). */
 #define FA_FLAG_NO_HEAD_PACKING 128u
+/* fa_config.flags: at head size 128 the one-item-per-CTA tiling with two query tiles per CTA has two
+ * kernels: csrc/fa_fwd_pair.cuh (the default: one MMA-issuing thread that probes its barriers from
+ * inside the blocks of MMAs, no correction warpgroup) and the older csrc/fa_fwd_pipelined.cuh, which
+ * this flag selects.  Same results up to fp32 rounding order.  Meant for tests and A/B timing. */
+#define FA_FLAG_LEGACY_PAIR_KERNEL 256u
 
 /* Optional creation parameters.  Zero-initialise, set struct_size = sizeof(fa_config). */
 typedef struct fa_config {

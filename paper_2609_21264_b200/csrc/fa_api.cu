@@ -13,6 +13,7 @@
 #include "../../include/fa.h"
 #include "fa_common.cuh"
 #include "fa_fwd_pipelined.cuh"
+#include "fa_fwd_pair.cuh"
 #include "fa_fwd_persistent.cuh"
 #include "fa_fwd_stream.cuh"
 #include "fa_fwd_fp8.cuh"
@@ -157,16 +158,15 @@ fa_status launch_simple(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& 
     return FA_OK;
 }
 
-template <int DQK, int DV, bool kVarlen, bool kHeadPair = false>
-fa_status launch_pipelined(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& mk,
-                           const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
-    constexpr int smem = fa::pipe_smem_bytes<DQK, DV>();
-    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
-    auto kernel = fa::fa_fwd_pipelined_kernel<DQK, DV, kVarlen, kHeadPair>;
+// Launch of a kernel with two query tiles per CTA (and of the combine kernel behind it with split-KV).
+template <int DV, typename Kernel>
+fa_status launch_two_tile(fa_handle* h, Kernel kernel, int smem, int threads, bool head_pair, const CUtensorMap& mq,
+                          const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p,
+                          cudaStream_t st) {
     fa_status s = ensure_smem_attr(h, kernel, smem);
     if (s != FA_OK) return s;
     // items: pairs of adjacent query tiles of a head, or one query tile of a pair of adjacent heads
-    const long long n_ctas = (kHeadPair ? static_cast<long long>(p.n_q_tiles) * (p.Hq / 2)
+    const long long n_ctas = (head_pair ? static_cast<long long>(p.n_q_tiles) * (p.Hq / 2)
                                         : static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq) * p.B * p.kv_splits;
     if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
     // Programmatic stream serialisation: the kernel may be scheduled while its predecessor in the
@@ -177,7 +177,7 @@ fa_status launch_pipelined(fa_handle* h, const CUtensorMap& mq, const CUtensorMa
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
-    cfg.blockDim = dim3(fa::PipeCfg<DQK, DV>::kThreads, 1, 1);
+    cfg.blockDim = dim3(threads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cfg.attrs = attr;
@@ -197,6 +197,26 @@ fa_status launch_pipelined(fa_handle* h, const CUtensorMap& mq, const CUtensorMa
         h->launches += 1;
     }
     return FA_OK;
+}
+
+// Two query tiles per CTA, one item per CTA: at head size 128 the kernel of fa_fwd_pair.cuh, otherwise
+// (and with FA_FLAG_LEGACY_PAIR_KERNEL) the one of fa_fwd_pipelined.cuh.
+template <int DQK, int DV, bool kVarlen, bool kHeadPair = false>
+fa_status launch_pipelined(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& mk,
+                           const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
+    if constexpr (DQK == 128 && DV == 128) {
+        if (!(h->flags & FA_FLAG_LEGACY_PAIR_KERNEL)) {
+            constexpr int smem = fa::pair_smem_bytes<DQK, DV>();
+            static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+            h->last_kernel = "fa_fwd_pair";
+            return launch_two_tile<DV>(h, fa::fa_fwd_pair_kernel<DQK, DV, kVarlen, kHeadPair>, smem,
+                                       fa::PairCfg<DQK, DV>::kThreads, kHeadPair, mq, mk, mv, mo, p, st);
+        }
+    }
+    constexpr int smem = fa::pipe_smem_bytes<DQK, DV>();
+    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+    return launch_two_tile<DV>(h, fa::fa_fwd_pipelined_kernel<DQK, DV, kVarlen, kHeadPair>, smem,
+                               fa::PipeCfg<DQK, DV>::kThreads, kHeadPair, mq, mk, mv, mo, p, st);
 }
 
 // Number of K/V splits for a problem: 1 unless the query tiles alone leave most SMs idle and the
@@ -639,7 +659,7 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg) {
         if (cfg->struct_size >= sizeof(fa_config)) scratch_bytes = cfg->scratch_bytes;
         if (flags & ~(FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD | FA_FLAG_NO_DEPENDENT_LAUNCH |
                       FA_FLAG_NO_PERSISTENT | FA_FLAG_FORCE_PERSISTENT | FA_FLAG_STREAM_KERNEL |
-                      FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)) return FA_ERR_INVALID_ARG;
+                      FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING | FA_FLAG_LEGACY_PAIR_KERNEL)) return FA_ERR_INVALID_ARG;
         if (kv_splits_cfg > 256) return FA_ERR_INVALID_ARG;
     }
     if (scratch_bytes == 0) scratch_bytes = 32ull << 20;

@@ -70,6 +70,25 @@ constexpr int kTraceIters = 64, kTraceEvents = 16, kTraceRoles = 6;   // roles: 
 #define FA_TRACE_STAMP(role, iter, ev) do { } while (0)
 #endif
 
+// -DFA_TRACE -DFA_TRACE_PHASES: every softmax warp of the pair kernel adds up the cycles it spends in each part of
+// its loop (clock reads at the points where the warp synchronises anyway) and leaves the sums in the trace buffer.
+#if defined(FA_TRACE) && defined(FA_TRACE_PHASES)
+#define FA_PHASE_DECL() uint32_t ph_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, ph_last; asm volatile("mov.u32 %0, %%clock;" : "=r"(ph_last))
+#define FA_PHASE(k) do { uint32_t c_; asm volatile("mov.u32 %0, %%clock;" : "=r"(c_)); ph_acc[k] += c_ - ph_last; ph_last = c_; } while (0)
+#define FA_PHASE_STORE(nphases, count)                                                                       \
+    do {                                                                                                     \
+        if (lane == 0 && p.trace) {                                                                          \
+            uint32_t* o_ = reinterpret_cast<uint32_t*>(p.trace) + (static_cast<size_t>(blockIdx.x) * 16 + warp) * 8; \
+            for (int k_ = 0; k_ < (nphases); ++k_) o_[k_] = ph_acc[k_];                                      \
+            o_[7] = (count);                                                                                 \
+        }                                                                                                    \
+    } while (0)
+#else
+#define FA_PHASE_DECL() do { } while (0)
+#define FA_PHASE(k) do { } while (0)
+#define FA_PHASE_STORE(nphases, count) do { } while (0)
+#endif
+
 // Number of K/V tiles a query tile starting at row i0 (covering `rows` rows) has to visit.
 // Key j is visible to query i iff j <= i + (Sk - Sq) in causal mode.
 __host__ __device__ inline int kv_tiles_for_q_tile(int i0, int rows, int Sq, int Sk, int causal) {

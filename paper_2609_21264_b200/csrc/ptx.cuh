@@ -42,6 +42,44 @@ FA_DEVI float exp2_approx(float x) {
     return y;
 }
 
+// exp2 of two values on the FMA pipe instead of the MUFU: the integer part n = floor(x) is taken with the
+// 1.5 * 2^23 trick (an addition rounded towards minus infinity leaves n in the low mantissa bits), the fraction
+// f = x - n in [0, 1) goes through a cubic (minimax fit of 2^f, relative error 7.5e-5, far below the bf16 rounding
+// of P that follows), and n is put back with a shift and an integer add into the exponent field.  Valid for
+// x < 127; x below -127 is clamped there and comes out as a denormal (below 1.2e-38), which the row sum's
+// flushing additions read as zero.
+FA_DEVI float2 exp2_poly2(float2 x) {
+    const float kMagic = 12582912.f;
+    x.x = fmaxf(x.x, -127.f);
+    x.y = fmaxf(x.y, -127.f);
+    unsigned long long xb, yb, mb;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(xb) : "f"(x.x), "f"(x.y));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(mb) : "f"(kMagic));
+    asm("add.rm.ftz.f32x2 %0, %1, %2;" : "=l"(yb) : "l"(xb), "l"(mb));
+    float2 y;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(y.x), "=f"(y.y) : "l"(yb));
+    const float2 nf = __fadd2_rn(y, make_float2(-kMagic, -kMagic));
+    const float2 f = __fadd2_rn(x, make_float2(-nf.x, -nf.y));
+    float2 p = __ffma2_rn(make_float2(7.8024521470e-02f, 7.8024521470e-02f), f, make_float2(2.2606717050e-01f, 2.2606717050e-01f));
+    p = __ffma2_rn(p, f, make_float2(6.9583350420e-01f, 6.9583350420e-01f));
+    p = __ffma2_rn(p, f, make_float2(9.9992519617e-01f, 9.9992519617e-01f));
+    float2 r;
+    r.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(y.x) << 23));
+    r.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(y.y) << 23));
+    return r;
+}
+
+// a + b on two lanes, denormal inputs and results flushed to zero
+FA_DEVI float2 fadd2_ftz(float2 a, float2 b) {
+    unsigned long long ab, bb, rb;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ab) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(bb) : "f"(b.x), "f"(b.y));
+    asm("add.rn.ftz.f32x2 %0, %1, %2;" : "=l"(rb) : "l"(ab), "l"(bb));
+    float2 r;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(r.x), "=f"(r.y) : "l"(rb));
+    return r;
+}
+
 FA_DEVI float fmax3(float a, float b, float c) {
     float y;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
