@@ -3,6 +3,13 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config IDX] [--impl reference]
 
+The default workload is the largest single-GPU configuration (index 4: 128K tokens, grouped
+heads, causal), whose timed region of K launches lasts seconds: the clock samples fall inside it
+and the GPU runs under its power cap, as it does in production.  `per_config` holds a full record
+of all five configurations (back-to-back mean, per-launch minimum and median of 20 launches after
+10 warm-ups as in Section 5.1 of the paper, clock samples of its own window, roofline fractions
+against the measured burst and sustained peaks).
+
 A step is one pass of the whole hot path (one `fa_forward` launch) over one
 batch of the workload.  `value` is effective-GEMM throughput (Section 5.1 of the
 paper: 2*H*Lq*Lk*(dk+dv)/T) counted over VISIBLE (query, key) pairs only; the
@@ -34,7 +41,11 @@ L2_BYTES = 126 * 1024 * 1024
 PAPER_SECONDS = {"llama3_8b_gqa_s2048": 34076e-6}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None = not captured for that workload).
-NCU_DRAM_BYTES_PER_LAUNCH = {"llama3_8b_gqa_s2048": 25232640 + 0}   # profiles/fa_fwd_pipelined_llama3_8b_gqa_s2048.txt
+# A workload too large to capture under the profiler carries the figure of a smaller case of the same kernel scaled
+# by the compulsory bytes (DRAM traffic of this kernel grows in proportion to them: K and V are read once per K/V
+# head from DRAM and re-read from L2, Q and O move once); see profiles/ and the design doc.
+NCU_DRAM_BYTES_PER_LAUNCH = {}
+NCU_DRAM_BYTES_PER_COMPULSORY_BYTE = {}
 
 
 def load_peaks():
@@ -135,6 +146,29 @@ def make_device_sets(w, n_sets, device):
     return sets
 
 
+def host_inputs(w):
+    """(Q, K, V) bf16 bit patterns (uint16 numpy arrays) of the workload's shapes and distribution, drawn on the host
+    with torch's seeded generator: the same recipe as workloads.make_inputs (i.i.d. N(0, sigma^2) rounded to bf16, K
+    times k_mult) from a faster generator, for the timing legs, which need the distribution and not the very bits the
+    parity tests are stored against."""
+    import numpy as np
+    import torch
+    g = torch.Generator().manual_seed(w.seed)
+    out = []
+    for shape, mult in zip(w.shapes()[:3], (1.0, w.k_mult, 1.0)):
+        x = torch.empty(shape, dtype=torch.bfloat16)
+        flat = x.view(-1)
+        step = 1 << 26
+        for o in range(0, flat.numel(), step):
+            n = min(step, flat.numel() - o)
+            chunk = torch.randn(n, generator=g, dtype=torch.float32) * w.sigma
+            flat[o:o + n] = chunk.to(torch.bfloat16)
+        if mult != 1.0:
+            x = x * mult
+        out.append(x.view(torch.int16).numpy().view(np.uint16))
+    return tuple(out)
+
+
 def workload_numbers(w):
     fl_alg = metrics.flops_algorithmic(w.B, w.Hq, w.Sq, w.Sk, w.dqk, w.dv, w.causal)
     fl_pap = metrics.flops_paper(w.B, w.Hq, w.Sq, w.Sk, w.dqk, w.dv)
@@ -182,11 +216,11 @@ def run_device_timed(binding, h, w, sets, steps, warmup, world, sampler=None):
     return e0.elapsed_time(e1) * 1e-3, binding.fa_launch_count(h) - n0
 
 
-def run_e2e_timed(binding, h, w, steps, warmup, world):
+def run_e2e_timed(binding, h, w, steps, warmup, world, host=None):
     """Same metric through fa_forward_host: pinned host buffers, copies inside the timed region."""
     import numpy as np
     import torch
-    Q, K, V = workloads.make_inputs(w)
+    Q, K, V = host if host is not None else host_inputs(w)
     pin = [torch.from_numpy(a.view(np.int16)).pin_memory() for a in (Q, K, V)]
     o = torch.empty(w.shapes()[3], dtype=torch.int16).pin_memory()
     lse = torch.empty(w.shapes()[3][:3], dtype=torch.float32).pin_memory()
@@ -214,11 +248,11 @@ def run_e2e_timed(binding, h, w, steps, warmup, world):
     return dt, h2d, d2h, float(lse.double().mean())
 
 
-def oracle_timed(w, budget_s=20.0):
+def oracle_timed(w, budget_s=20.0, host=None):
     """The fp64 oracle on the host cores over a bounded sample of query rows of the workload."""
     import numpy as np
     import oracle
-    Q, K, V = workloads.make_inputs(w)
+    Q, K, V = host if host is not None else host_inputs(w)
     rng = np.random.default_rng(0)
     threads = oracle.num_threads()
 
@@ -248,7 +282,8 @@ def oracle_timed(w, budget_s=20.0):
         t0 = time.perf_counter()
         oracle.attention(Q, K, V, causal=w.causal, scale=w.scale, rows=rows)
         dt = time.perf_counter() - t0
-        pairs, sample = pairs_of(rows), "%d random query rows of the workload" % n
+        pairs, sample = pairs_of(rows), ("%d random query rows of the workload; the rate over the whole workload is "
+                                         "extrapolated from them (every row is an independent problem)" % n)
     flops = 2 * pairs * (w.dqk + w.dv)
     return {"value": flops / dt / 1e12, "unit": "TFLOP_GEMM/s", "cores": threads, "kind": "oracle",
             "sample": sample, "seconds": dt}
@@ -324,13 +359,105 @@ def time_libraries(binding, h, device):
     return rows
 
 
-def config_dict(w, extra=None):
-    d = {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "Sq": w.Sq, "Sk": w.Sk, "dqk": w.dqk,
-         "dv": w.dv, "causal": w.causal, "scale": w.scale, "inputs": "bf16 N(0,1), seeded",
-         "flop_convention": "value counts visible (i,j) pairs only; value_paper_convention counts Sq*Sk"}
-    if extra:
-        d.update(extra)
-    return d
+def l2_note(w):
+    n_sets = n_sets_for(w)
+    _, _, nbytes = workload_numbers(w)
+    return ("rotating %d input sets (%.0f MB in total, L2 is 126 MB)" % (n_sets, n_sets * nbytes / 1e6) if n_sets > 1 else
+            "one input set of %.0f MB (larger than the 126 MB L2)" % (nbytes / 1e6))
+
+
+def config_dict(w, world=1):
+    """The workload as both arms print it (identical for the same workload and N)."""
+    return {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "Sq": w.Sq, "Sk": w.Sk, "dqk": w.dqk,
+            "dv": w.dv, "causal": w.causal, "scale": w.scale, "inputs": "bf16 N(0,1), seeded",
+            "flop_convention": "value counts visible (i,j) pairs only; value_paper_convention counts Sq*Sk",
+            "l2": l2_note(w), "parallelism": "replicas x%d, no collective" % world}
+
+
+def per_launch_times(binding, h, w, sets, launches, warmup):
+    """Duration of every one of `launches` launches after `warmup` (an event pair around each, on the launching
+    stream; the handle launches the ordinary way, so consecutive launches do not overlap); seconds."""
+    import torch
+    stream = torch.cuda.current_stream()
+
+    def one(i):
+        q, k, v, o, lse = sets[i % len(sets)]
+        st = binding.fa_forward(h, q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(),
+                                w.B, w.Hq, w.Hkv, w.Sq, w.Sk, w.dqk, w.dv, w.causal, w.scale, stream.cuda_stream)
+        if st != binding.FA_OK:
+            raise binding.FaError(st, "fa_forward")
+
+    for i in range(warmup):
+        one(i)
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(launches)]
+    for i, (e0, e1) in enumerate(ev):
+        e0.record(stream)
+        one(warmup + i)
+        e1.record(stream)
+    torch.cuda.synchronize()
+    return sorted(e0.elapsed_time(e1) * 1e-3 for e0, e1 in ev)
+
+
+def roofline_of(w, t_step, peaks, kernel):
+    """Roofline record of one launch of `w` that takes t_step seconds: against the measured burst peak (a kernel timed
+    alone) and the sustained one (a kernel inside a long, power-capped region); `frac` takes the one that applies."""
+    fl_alg, _, nbytes = workload_numbers(w)
+    t_tensor_burst = fl_alg / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+    bound = "tensor" if t_tensor_burst >= t_hbm else "hbm"
+    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(w.name)
+    if traffic is None and w.name in NCU_DRAM_BYTES_PER_COMPULSORY_BYTE:
+        traffic = NCU_DRAM_BYTES_PER_COMPULSORY_BYTE[w.name] * nbytes
+    r = {"bound": bound, "kernel": kernel, "avg_launch_us": t_step * 1e6, "traffic": traffic,
+         "algorithmic_flops_per_launch": fl_alg, "compulsory_bytes_per_launch": nbytes,
+         "frac_of_nominal_2250_tflops": fl_alg / t_step / 2.25e15}
+    if bound == "tensor":
+        ach = fl_alg / t_step / 1e12
+        r.update({"achieved": ach, "unit": "TFLOP/s", "frac_burst": ach / peaks["bf16_tflops"],
+                  "frac_sustained": ach / peaks["bf16_tflops_sustained"]})
+    else:
+        ach = nbytes / t_step / 1e9
+        r.update({"achieved": ach, "unit": "GB/s", "frac_burst": ach / peaks["hbm_gbs"], "frac_sustained": ach / peaks["hbm_gbs"]})
+    return r
+
+
+def measure_config(binding, h, h_plain, w, device, peaks, gpu_index, steps=None, warmup=None, world=1):
+    """Full record of one configuration: back-to-back mean over a timed region with its own clock samples, per-launch
+    minimum and median (Section 5.1's protocol: 10 warm-ups, 20 timed launches), roofline fractions."""
+    import torch
+    fl_alg, fl_pap, nbytes = workload_numbers(w)
+    sets = make_device_sets(w, n_sets_for(w), device)
+    if steps is None:
+        steps = max(20, min(2000, int(0.5 / max(fl_alg / 1.0e15, 1e-5))))
+    if warmup is None:
+        warmup = max(3, min(50, steps // 10))
+    sampler = ClockSampler(gpu_index, period_s=0.002)
+    sampler.start()
+    sampler.wait_ready()
+    seconds, launches = run_device_timed(binding, h, w, sets, steps, warmup, world, sampler)
+    clocks = sampler.stop()
+    seconds = launch.max_over_ranks(seconds, world, device)
+    t = seconds / steps
+    kernel = binding.fa_last_kernel_name(h)
+    each = per_launch_times(binding, h_plain, w, sets, 20, 10)
+    del sets
+    torch.cuda.empty_cache()
+    long_region = seconds > 0.25          # long enough for the power cap to set the clock
+    roof = roofline_of(w, t, peaks, kernel)
+    roof["frac"] = roof["frac_sustained"] if long_region else roof["frac_burst"]
+    roof["peak"] = (peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"]) if roof["bound"] == "tensor" else peaks["hbm_gbs"]
+    roof["peak_source"] = "%s (%s: the timed region lasted %.2f s)" % (peaks["source"], "sustained" if long_region else "burst", seconds)
+    rec = {"workload": w.name, "kernel": kernel, "steps": steps, "warmup": warmup, "us": t * 1e6,
+           "tflops_algorithmic": fl_alg / t / 1e12, "tflops_paper_convention": fl_pap / t / 1e12,
+           "per_launch_us_min": each[0] * 1e6, "per_launch_us_median": each[len(each) // 2] * 1e6,
+           "per_launch_note": "20 launches after 10 warm-ups, an event pair around each, launched without programmatic "
+                              "stream serialisation (no overlap between consecutive launches); 'us' is the mean of "
+                              "back-to-back launches, whose tails overlap",
+           "bound": roof["bound"], "frac_burst": roof["frac_burst"], "frac_sustained": roof["frac_sustained"],
+           "frac_of_nominal_2250": fl_alg / t / 2.25e15, "clocks": clocks,
+           "us_x_sm_mhz": (t * 1e6 * clocks["sm_mhz"]) if clocks.get("sm_mhz") else None}
+    return rec, roof, seconds, launches, steps, warmup
 
 
 def run_reference(args, w, rank, world):
@@ -339,7 +466,7 @@ def run_reference(args, w, rank, world):
         return
     import numpy as np
     import oracle
-    Q, K, V = workloads.make_inputs(w)
+    Q, K, V = host_inputs(w)
     threads = oracle.num_threads()
     rows_total = w.B * w.Hq * w.Sq
     rng = np.random.default_rng(0)
@@ -372,7 +499,7 @@ def run_reference(args, w, rank, world):
             "unit": "TFLOP_GEMM/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": config_dict(w),
+            "config": config_dict(w, max(1, args.gpus)),
             "cpu_baseline": {"value": value, "unit": "TFLOP_GEMM/s", "cores": threads, "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": "TFLOP_GEMM/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -380,22 +507,62 @@ def run_reference(args, w, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def plan_ab(binding, device, gpu_index):
+    """The planner's choices against the alternatives it rejected, on the five configurations and on items of every
+    length: every case with the library's own plan and with each kernel forced through the FA_FLAG_* overrides."""
+    import torch
+    variants = (("planned", 0), ("two_tiles_per_item", binding.FA_FLAG_NO_PERSISTENT | binding.FA_FLAG_NO_STREAM_KERNEL),
+                ("persistent", binding.FA_FLAG_FORCE_PERSISTENT | binding.FA_FLAG_NO_STREAM_KERNEL),
+                ("stream", binding.FA_FLAG_STREAM_KERNEL))
+    handles = {name: binding.fa_create(device=device.index, flags=flags) for name, flags in variants}
+    cases = list(workloads.CONFIGS)
+    for (B, Hq, Hkv, S, causal) in ((64, 32, 8, 128, True), (32, 32, 8, 256, True), (16, 32, 8, 512, True), (8, 32, 8, 1024, True),
+                                    (8, 32, 8, 2048, True), (4, 32, 8, 4096, True), (2, 32, 8, 16384, True), (4, 32, 8, 2048, False)):
+        cases.append(workloads.Workload("b%d_h%d_%d_s%d_%s" % (B, Hq, Hkv, S, "causal" if causal else "full"), B, Hq, Hkv, S, S, 128, 128,
+                                        causal, 128 ** -0.5))
+    rows = []
+    for w in cases:
+        fl_alg, _, _ = workload_numbers(w)
+        sets = make_device_sets(w, n_sets_for(w), device)
+        k = max(5, min(300, int(0.3 / max(fl_alg / 1.0e15, 1e-5))))
+        row = {"workload": w.name}
+        for name, h in handles.items():
+            try:
+                sec, _ = run_device_timed(binding, h, w, sets, k, 3, 1)
+                row[name] = {"us": sec / k * 1e6, "tflops_algorithmic": fl_alg / (sec / k) / 1e12, "kernel": binding.fa_last_kernel_name(h)}
+            except binding.FaError as e:
+                row[name] = {"error": str(e)}
+        timed = {n: r["us"] for n, r in row.items() if isinstance(r, dict) and "us" in r and n != "planned"}
+        row["best"] = min(timed, key=timed.get) if timed else None
+        row["planned_over_best"] = row["planned"]["us"] / min(timed.values()) if timed and "us" in row["planned"] else None
+        rows.append(row)
+        del sets
+        torch.cuda.empty_cache()
+    for h in handles.values():
+        binding.fa_destroy(h)
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--config", type=int, default=1, help="index into the five benchmark configurations")
+    ap.add_argument("--config", type=int, default=4,
+                    help="index into the five benchmark configurations (default: the largest, 128K tokens)")
     ap.add_argument("--shape", default=None,
                     help="time a custom shape instead of --config, e.g. "
                          "B=1,Hq=16,Hkv=16,S=8192,dqk=128,dv=128,causal=1 (used for small ncu captures)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-sweep", action="store_true", help="skip the short timing of the other configs")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the records of the other configurations (key 'per_config')")
     ap.add_argument("--table6", action="store_true",
                     help="also time the twelve attention shapes of the paper's Table 6 (key 'table6')")
     ap.add_argument("--no-decode", action="store_true", help="skip the grouped-head decode step and the packed batches (keys 'decode', 'packed_batches')")
+    ap.add_argument("--plan-ab", action="store_true",
+                    help="also time every configuration, and items of every length, with each kernel forced, next to the "
+                         "library's own choice (key 'plan_ab')")
     ap.add_argument("--libraries", action="store_true",
                     help="also time the attention kernels of the libraries in the image (torch SDPA back ends, flash_attn) "
                          "on the five configurations and a few decode shapes, for context (key 'libraries')")
@@ -434,32 +601,13 @@ def main():
     warmup = args.warmup if args.warmup is not None else max(3, min(50, steps // 10))
     warmup = max(3, warmup)
 
-    sampler = ClockSampler(physical_gpu_index(local))
-    sampler.start()
-    h = binding.fa_create(device=local)
-    n_sets = n_sets_for(w)
-    sets = make_device_sets(w, n_sets, device)
-    sampler.wait_ready()
-    seconds, launches = run_device_timed(binding, h, w, sets, steps, warmup, world, sampler)
-    clocks = sampler.stop()
-    seconds = launch.max_over_ranks(seconds, world, device)
-    t_step = seconds / steps
-
+    gpu_index = physical_gpu_index(local)
     peaks = load_peaks()
-    long_step = t_step > 5e-3
-    peak_tf = peaks["bf16_tflops_sustained"] if long_step else peaks["bf16_tflops"]
-    t_roof, bound = metrics.roofline_seconds(fl_alg, nbytes, peak_tf, peaks["hbm_gbs"])
-    if bound == "tensor":
-        achieved, peak, unit = fl_alg / t_step / 1e12, peak_tf, "TFLOP/s"
-    else:
-        achieved, peak, unit = nbytes / t_step / 1e9, peaks["hbm_gbs"], "GB/s"
-    roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(w.name),
-                "peak_source": "%s (%s)" % (peaks["source"], "sustained" if long_step else "burst"),
-                "kernel": binding.fa_last_kernel_name(h), "algorithmic_flops_per_launch": fl_alg,
-                "compulsory_bytes_per_launch": nbytes, "avg_launch_us": t_step * 1e6,
-                "t_roof_us": t_roof * 1e6,
-                "frac_of_nominal_2250_tflops": fl_alg / t_step / 2.25e15}
+    h = binding.fa_create(device=local)
+    h_plain = binding.fa_create(device=local, flags=binding.FA_FLAG_NO_DEPENDENT_LAUNCH)
+    rec, roofline, seconds, launches, steps, warmup = measure_config(binding, h, h_plain, w, device, peaks, gpu_index, steps, warmup, world)
+    t_step = seconds / steps
+    clocks = rec["clocks"]
 
     value = world * fl_alg / t_step / 1e12
     line = {"metric": "attention_fwd_tflop_gemm_per_s", "value": value, "unit": "TFLOP_GEMM/s",
@@ -467,12 +615,10 @@ def main():
             "higher_is_better": True, "scaling": "weak",
             "vs_baseline": (PAPER_SECONDS[w.name] / t_step if (w.name in PAPER_SECONDS and world == 1) else None),
             "dtype": "bf16", "data": "synthetic",
-            "config": config_dict(w, {"l2": "rotating %d input sets (%.0f MB in total, L2 is 126 MB)"
-                                      % (n_sets, n_sets * nbytes / 1e6) if n_sets > 1 else
-                                      "one input set of %.0f MB (larger than the 126 MB L2)" % (nbytes / 1e6),
-                                      "parallelism": "replicas x%d, no collective" % world}),
+            "config": config_dict(w, world),
             "value_paper_convention": world * fl_pap / t_step / 1e12,
             "paper_context": "3.62 TFLOP_GEMM/s on XDNA 2 (paper's headline, other hardware and shape)",
+            "per_launch_us_min": rec["per_launch_us_min"], "per_launch_us_median": rec["per_launch_us_median"],
             "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches)}
 
     if not args.no_sweep and world == 1 and w.dqk == 128 and w.dv == 128:
@@ -589,33 +735,31 @@ def main():
                                   "20 launches each after 3 warm-up launches"}
         torch.cuda.empty_cache()
 
+    host = None
+    if (not args.no_e2e) or (rank == 0 and world == 1 and not args.no_cpu_baseline):
+        host = host_inputs(w)
     if not args.no_e2e:
-        e2e_steps = max(3, min(steps, 50))
-        dt, h2d, d2h, _ = run_e2e_timed(binding, h, w, e2e_steps, 3, world)
+        e2e_steps = max(3, min(steps, 50, int(4.0 / max(t_step * 3, 1e-4)) + 3))
+        dt, h2d, d2h, _ = run_e2e_timed(binding, h, w, e2e_steps, 3 if t_step < 0.05 else 1, world, host)
         dt = launch.max_over_ranks(dt, world, device)
         line["e2e"] = {"value": world * fl_alg * e2e_steps / dt / 1e12, "unit": "TFLOP_GEMM/s",
                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-                       "ms_per_step": dt / e2e_steps * 1e3}
+                       "ms_per_step": dt / e2e_steps * 1e3,
+                       "api": "fa_forward_host: pinned host buffers, both copies inside the timed region"}
 
     if not args.no_sweep and world == 1:
         per = []
-        del sets
-        torch.cuda.empty_cache()
         for idx, wc in enumerate(workloads.CONFIGS):
-            fa, fp, nb = workload_numbers(wc)
-            ss = make_device_sets(wc, n_sets_for(wc), device)
-            k = max(5, min(200, int(0.3 / max(fa / 1.0e15, 1e-5))))
-            sec, _ = run_device_timed(binding, h, wc, ss, k, 3, 1)
-            t = sec / k
-            pk = peaks["bf16_tflops_sustained"] if t > 5e-3 else peaks["bf16_tflops"]
-            tr, bd = metrics.roofline_seconds(fa, nb, pk, peaks["hbm_gbs"])
-            per.append({"config": idx, "workload": wc.name, "us": t * 1e6, "tflops_algorithmic": fa / t / 1e12,
-                        "tflops_paper_convention": fp / t / 1e12, "bound": bd, "roofline_frac": tr / t,
-                        "frac_of_nominal_2250": fa / t / 2.25e15, "steps": k,
-                        "kernel": binding.fa_last_kernel_name(h)})
-            del ss
-            torch.cuda.empty_cache()
+            if wc.name == w.name:
+                r = dict(rec)
+            else:
+                r, _, _, _, _, _ = measure_config(binding, h, h_plain, wc, device, peaks, gpu_index)
+            r["config"] = idx
+            per.append(r)
         line["per_config"] = per
+
+    if args.plan_ab and world == 1:
+        line["plan_ab"] = plan_ab(binding, device, gpu_index)
 
     if args.table6 and world == 1:
         rows = []
@@ -636,9 +780,10 @@ def main():
         line["libraries"] = time_libraries(binding, h, device)
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = oracle_timed(w)
+        line["cpu_baseline"] = oracle_timed(w, host=host)
 
     binding.fa_destroy(h)
+    binding.fa_destroy(h_plain)
     if rank == 0:
         print(json.dumps(line), flush=True)
     launch.destroy(world)

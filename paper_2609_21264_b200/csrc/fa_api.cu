@@ -462,18 +462,19 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     }
     // packed batches: no split (the lengths that decide it are on the device)
     const int pair_splits = varlen ? 1 : choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles);
-    // The persistent kernel wins where a CTA's fixed cost is a visible share of an item's time and
-    // every SM gets several items: measured on B200 it is 5-20 % faster from about three items per
-    // SM on, still 2 % faster at 64-tile items at d = 128, 1-2 % slower at 128-tile items; at d = 64,
-    // where the pair kernel keeps P in TMEM columns of its own and has the shorter chain per K/V tile,
-    // it is 5-12 % faster up to 8-tile items, level at 16 and 4-5 % slower at 32; and it is a few per
-    // cent slower below two items per SM (its one-time set-up and the coarser balance of a short list).  d = 192 has no room for its staging buffer.
+    // The persistent kernel wins where a CTA's fixed cost is a visible share of an item's time and every SM gets
+    // several items.  Measured on B200 against the one-item-per-CTA kernels (an A/B over item lengths,
+    // `bench.py --plan-ab`): at d = 128, where the per-item kernel is the one of fa_fwd_pair.cuh, it is 28 / 20 /
+    // 6 / 4 % faster on items of 1 / 2 / 4 / 8 K/V tiles, level at 16 and 3-7 % slower from 32 tiles on (that kernel's
+    // loop is the faster one); at d = 64, where the per-item kernel keeps P in TMEM columns of its own, it is 5-12 %
+    // faster up to 8-tile items, level at 16 and 4-5 % slower at 32; and it is a few per cent slower below two items
+    // per SM (its one-time set-up and the coarser balance of a short list).  d = 192 has no room for its staging buffer.
     const long long n_items = static_cast<long long>((n_q_tiles + 1) / 2) * Hq * B;
     // (packed batches: the list has an item for every tile of the longest sequence, which Sq is;
     //  the sequences a tile does not exist in pass through the kernel's item ring empty)
     const int longest = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, (varlen && Sk < Sq) ? Sq : Sk, causal);
     const bool persistent_ok = pair_splits == 1 && dqk != 192 && !drop;
-    bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= (dqk == 64 ? 16 : 64);
+    bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= (dqk == 64 ? 16 : 8);
     if (flags & FA_FLAG_NO_PERSISTENT) persistent = false;
     if ((flags & FA_FLAG_FORCE_PERSISTENT) && persistent_ok) persistent = true;
     // One query tile per CTA (twice the CTAs, each with a shorter chain) wins where the pair
@@ -996,6 +997,8 @@ fa_status fa_plan(int num_sms, const fa_config* cfg, int varlen, int B, int Hq, 
                                       B, Hq, Hkv, Sq, Sk, dqk, dv, causal ? 1 : 0);
     static const char* const names[4] = {"fa_fwd_simple", "fa_fwd_pipelined", "fa_fwd_persistent", "fa_fwd_stream"};
     out->kernel = names[pl.kernel];
+    // the one-item-per-CTA tiling with two query tiles has a kernel of its own at head size 128
+    if (pl.kernel == kPlanPair && dqk == 128 && dv == 128 && !(flags & FA_FLAG_LEGACY_PAIR_KERNEL)) out->kernel = "fa_fwd_pair";
     out->kv_splits = pl.kv_splits;
     out->heads_per_tile = pl.pack_heads;
     const long long n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;

@@ -373,7 +373,7 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
     } else if (warp == 12 || warp == 13) {
         // ============================================================ MMA issue for tile t = warp - 12
         setmaxnreg_dec<kRegsOther>();
-        if (lane == 0 && n_max > 0) {
+        if (elect_one() && n_max > 0) {
             const int t = warp - 12;
             const int nkv_t = (t == 0) ? nkv_0 : nkv_1;
             constexpr uint32_t kIdescQK = make_idesc_e4m3_f32(kTileM, kTileN, false, false);
@@ -464,7 +464,7 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
     } else if (warp == 14) {
         // ============================================================ TMA loads
         setmaxnreg_dec<kRegsOther>();
-        if (lane == 0 && n_max > 0) {
+        if (elect_one() && n_max > 0) {
             auto load_q = [&](int t) {
                 if ((t == 0 ? nkv_0 : nkv_1) == 0) return;
                 const uint32_t bar = smem_addr(&sh.q_full[t]);

@@ -530,11 +530,8 @@ fa_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q,
     } else if (warp == 8) {
         // ============================================================ MMA issue, one thread for both tiles
         setmaxnreg_dec<kPairRegsOther>();
-#ifdef FA_MMA_LANE0
-        if (lane == 0 && n_max > 0) {
-#else
+        // elect.sync, not lane == 0: only then are the descriptors kept in uniform registers (see the top of the file)
         if (elect_one() && n_max > 0) {
-#endif
             constexpr uint32_t kIdescQK = make_idesc_bf16_f32(kTileM, kTileN, false, false);
             constexpr uint32_t kIdescPV = make_idesc_bf16_f32(kTileM, DV, false, true);
             constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // sbo, version, swizzle
@@ -654,7 +651,7 @@ fa_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q,
     } else if (warp == 9) {
         // ============================================================ TMA loads
         setmaxnreg_dec<kPairRegsOther>();
-        if (lane == 0 && n_max > 0) {
+        if (elect_one() && n_max > 0) {
             auto load_q = [&](int t) {
                 if ((t == 0 ? nkv_0 : nkv_1) == 0) return;
                 const uint32_t bar = smem_addr(&sh.q_full[t]);

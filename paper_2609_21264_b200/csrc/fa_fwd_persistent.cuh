@@ -502,7 +502,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
     } else if (warp == 12 || warp == 13) {
         // ============================================================ MMA issue for tile t = warp - 12
         setmaxnreg_dec<kRegsOther>();
-        if (lane == 0) {
+        if (elect_one()) {
             const int t = warp - 12;
             constexpr uint32_t kIdescQK = make_idesc_bf16_f32(kTileM, kTileN, false, false);
             constexpr uint32_t kIdescPV = make_idesc_bf16_f32(kTileM, DV, false, true);
@@ -614,7 +614,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
     } else if (warp == 14) {
         // ============================================================ TMA loads of K and V
         setmaxnreg_dec<kRegsOther>();
-        if (lane == 0) {
+        if (elect_one()) {
             uint32_t kc = 0, vc = 0;         // K and V tiles requested so far, over all items
             int idx = cta;                   // first item: static, the heaviest items go first
             bool ok = true;
@@ -679,7 +679,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
     } else {
         // ============================================================ warp 15: TMA loads of the Q tiles
         setmaxnreg_dec<kRegsOther>();
-        if (lane == 0) {
+        if (elect_one()) {
             uint32_t qc0 = 0, qc1 = 0;       // loads of Q_0 and Q_1 so far
             bool ok = true;
 #pragma unroll 1

@@ -527,7 +527,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
         // other's MMAs.  The two threads touch disjoint TMEM (S_t, O_t) and share the K/V stages,
         // whose "empty" barriers therefore count two arrivals.
         setmaxnreg_dec<kRegsOther>();
-        if (lane == 0 && n_max > 0) {
+        if (elect_one() && n_max > 0) {
             const int t = warp - 12;
             const int nkv_t = (t == 0) ? nkv_0 : nkv_1;
             constexpr uint32_t kIdescQK = make_idesc_bf16_f32(kTileM, kTileN, false, false);
@@ -647,7 +647,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q,
     } else if (warp == 14) {
         // ============================================================ TMA loads
         setmaxnreg_dec<kRegsOther>();
-        if (lane == 0 && n_max > 0) {
+        if (elect_one() && n_max > 0) {
             auto load_q = [&](int t) {
                 if ((t == 0 ? nkv_0 : nkv_1) == 0) return;
                 const uint32_t bar = smem_addr(&sh.q_full[t]);

@@ -501,7 +501,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     } else if (warp == 12) {
         // ============================================================ score MMAs: S^(j&1) = Q K_j^T
         setmaxnreg_dec<kRegsOther>();
-        if (lane == 0 && n_kv > 0) {
+        if (elect_one() && n_kv > 0) {
             constexpr uint32_t kIdescQK = make_idesc_bf16_f32(kTileM, kTileN, false, false);
             constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // sbo, version, swizzle
             const uint32_t q_lo = ((sQ & 0x3FFFFu) >> 4) | (1u << 16);
@@ -531,7 +531,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     } else if (warp == 13) {
         // ============================================================ PV MMAs: O += P^(j&1) V_j
         setmaxnreg_dec<kRegsOther>();
-        if (lane == 0 && n_kv > 0) {
+        if (elect_one() && n_kv > 0) {
             constexpr uint32_t kIdescPV = make_idesc_bf16_f32(kTileM, DV, false, true);
             constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
             const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((static_cast<uint32_t>(kChunkBytes) >> 4) << 16);
@@ -563,7 +563,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         // runs behind a whole softmax, and one thread loading both in turn would hold the K loads
         // (which the score MMAs want two tiles ahead) back behind it.
         setmaxnreg_dec<kRegsOther>();
-        if (lane == 0 && n_kv > 0) {
+        if (elect_one() && n_kv > 0) {
             {
                 const uint32_t bar = smem_addr(&sh.q_full);
                 // with packed heads the box is Sq rows x pack_heads heads (row h * Sq + i of the tile)
@@ -588,7 +588,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     } else {
         // ============================================================ warp 15: TMA loads of V
         setmaxnreg_dec<kRegsOther>();
-        if (lane == 0 && n_kv > 0) {
+        if (elect_one() && n_kv > 0) {
             bool ok = true;
             for (int j = 0; j < n_kv && ok; ++j) {
                 const int s = j % NV;

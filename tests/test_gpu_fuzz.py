@@ -117,7 +117,9 @@ def test_fuzz_all_entry_points(handle):
     # split-KV, the 8-bit stream kernel and packed batches on the stream kernel
     kernels = {(k, n) for k, n, _ in seen}
     if handle_kind == "planned":
+        # (two query tiles per CTA: fa_fwd_pair at head size 128, fa_fwd_pipelined at the other head sizes)
         assert {(0, "fa_fwd_stream"), (0, "fa_fwd_pipelined"), (2, "fa_fwd_fp8_stream"), (3, "fa_fwd_stream")} <= kernels, seen
+        assert "fa_fwd_pair" in {n for _, n in kernels}, seen
     else:
         assert {(0, "fa_fwd_persistent"), (1, "fa_fwd_persistent"), (3, "fa_fwd_persistent"), (3, "fa_fwd_stream")} <= kernels, seen
     assert any(s for _, _, s in seen)

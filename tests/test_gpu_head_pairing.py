@@ -61,7 +61,7 @@ def test_paired_heads_equal_the_unpaired_launch_and_the_oracle(w, persistent):
     Q, K, V = W.make_inputs(w)
     o1, l1, k1 = _run(base, w, Q, K, V)
     o2, l2, k2 = _run(base | binding.FA_FLAG_NO_HEAD_PACKING, w, Q, K, V)
-    assert k1 == k2 == ("fa_fwd_persistent" if persistent else "fa_fwd_pipelined")
+    assert k1 == k2 == ("fa_fwd_persistent" if persistent else ("fa_fwd_pair" if w.dqk == 128 else "fa_fwd_pipelined"))
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     n_q_tiles = (w.Sq + 127) // 128
     plan = binding.fa_plan(sms, w.B, w.Hq, w.Hkv, w.Sq, w.Sk, w.dqk, w.dv, w.causal, flags=base)
@@ -134,7 +134,7 @@ def test_paired_heads_in_packed_batches(name, lens_q, lens_k, Hq, Hkv, d, causal
             torch.cuda.synchronize()
             st, detail = binding.fa_last_status(h)
             assert st == binding.FA_OK, "device status %d (site 0x%x)" % (st, detail)
-            assert binding.fa_last_kernel_name(h) == ("fa_fwd_persistent" if persistent else "fa_fwd_pipelined")
+            assert binding.fa_last_kernel_name(h) == ("fa_fwd_persistent" if persistent else ("fa_fwd_pair" if d == 128 else "fa_fwd_pipelined"))
             outs.append((o, lse))
         finally:
             binding.fa_destroy(h)

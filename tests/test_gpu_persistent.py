@@ -56,7 +56,7 @@ def test_persistent_matches_oracle_and_per_item_kernel(handles, w):
         assert st == binding.FA_OK, "%s: device status %d (site 0x%x)" % (name, st, detail)
         out[name] = (o, lse)
     assert binding.fa_last_kernel_name(handles["persistent"]) == "fa_fwd_persistent"
-    assert binding.fa_last_kernel_name(handles["per_item"]) == "fa_fwd_pipelined"
+    assert binding.fa_last_kernel_name(handles["per_item"]) == ("fa_fwd_pair" if w.dqk == 128 else "fa_fwd_pipelined")
     o_p, lse_p = out["persistent"]
     o_i, lse_i = out["per_item"]
     assert torch.equal(o_p.view(torch.int16), o_i.view(torch.int16))
@@ -90,8 +90,8 @@ def test_default_choice_by_shape():
     import torch
     h = binding.fa_create()
     try:
-        for (B, H, S, expect) in ((8, 32, 1024, "fa_fwd_persistent"), (1, 32, 2048, "fa_fwd_pipelined"),
-                                  (1, 12, 512, "fa_fwd_stream"), (1, 64, 16384, "fa_fwd_pipelined")):
+        for (B, H, S, expect) in ((8, 32, 1024, "fa_fwd_persistent"), (1, 32, 2048, "fa_fwd_pair"),
+                                  (1, 12, 512, "fa_fwd_stream"), (1, 64, 16384, "fa_fwd_pair")):
             q = torch.zeros((B, H, S, 128), dtype=torch.bfloat16, device="cuda")
             binding.forward(h, q, q, q, causal=True)
             torch.cuda.synchronize()

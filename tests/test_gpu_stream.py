@@ -114,8 +114,8 @@ def test_choice_between_tilings():
     try:
         for (B, H, Sq, Sk, causal, expect, split) in ((1, 8, 1024, 1024, True, "fa_fwd_stream", False),
                                                        (1, 32, 128, 32768, False, "fa_fwd_stream", True),
-                                                       (1, 32, 2048, 2048, True, "fa_fwd_pipelined", False),
-                                                       (1, 12, 2048, 2048, False, "fa_fwd_pipelined", False)):
+                                                       (1, 32, 2048, 2048, True, "fa_fwd_pair", False),
+                                                       (1, 12, 2048, 2048, False, "fa_fwd_pair", False)):
             q = torch.zeros((B, H, Sq, 128), dtype=torch.bfloat16, device="cuda")
             k = torch.zeros((B, H, Sk, 128), dtype=torch.bfloat16, device="cuda")
             binding.forward(h, q, k, k, causal=causal)

@@ -14,8 +14,8 @@ def plan(w, **kw):
 
 
 def test_benchmark_configurations():
-    # (config 3: 4096 items of up to 64 K/V tiles, the longest the persistent kernel is chosen for)
-    expect = ["fa_fwd_stream", "fa_fwd_pipelined", "fa_fwd_persistent", "fa_fwd_stream", "fa_fwd_pipelined"]
+    # (config 3: 4096 items of up to 64 K/V tiles: too long for the persistent kernel at d = 128, see test_persistent_kernel...)
+    expect = ["fa_fwd_stream", "fa_fwd_pair", "fa_fwd_pair", "fa_fwd_stream", "fa_fwd_pair"]
     for w, kernel in zip(W.CONFIGS, expect):
         p = plan(w)
         assert p["kernel"] == kernel, (w.name, p)
@@ -30,21 +30,24 @@ def test_table6_rows():
     got = {w.name: plan(w)["kernel"] for w, _ in W.TABLE6}
     assert got["gpt2_small_s2048"] == "fa_fwd_stream"          # 96 causal pairs: under a wave
     assert got["bert_base_s2048"] == "fa_fwd_pipelined"        # 192 equal tiles would make two waves
-    assert got["llama3_8b_s2048"] == "fa_fwd_pipelined"
+    assert got["llama3_8b_s2048"] == "fa_fwd_pair"
     assert got["qwen15_05b_s32768"] == "fa_fwd_stream"         # d = 64 with long items
-    assert got["deepseek_67b_gqa_s4096"] == "fa_fwd_persistent"  # 1024 short items
+    assert got["deepseek_67b_gqa_s4096"] == "fa_fwd_pair"        # 1024 items of up to 32 K/V tiles: past the persistent kernel's limit at d = 128
 
 
 def test_persistent_kernel_from_three_items_per_sm():
     kernel = lambda B, Hq, Hkv, S, causal: binding.fa_plan(SMS, B, Hq, Hkv, S, S, 128, 128, causal)["kernel"]
-    assert kernel(2, 32, 8, 2048, True) == "fa_fwd_persistent"      # 512 items of up to 16 K/V tiles: 3.5 per SM
-    assert kernel(2, 32, 32, 2048, True) == "fa_fwd_persistent"
+    # d = 128: the persistent kernel up to items of 8 K/V tiles (measured: 4-28 % ahead there, level at 16 tiles,
+    # 3-7 % behind the per-item kernel of fa_fwd_pair.cuh from 32 tiles on)
+    assert kernel(4, 32, 8, 1024, True) == "fa_fwd_persistent"      # 512 items of up to 8 K/V tiles: 3.5 per SM
+    assert kernel(4, 32, 32, 1024, True) == "fa_fwd_persistent"
     assert kernel(8, 32, 8, 512, True) == "fa_fwd_persistent"       # 512 items of up to 4 tiles
-    assert kernel(2, 32, 8, 2048, False) == "fa_fwd_persistent"
-    assert kernel(1, 32, 8, 2048, True) == "fa_fwd_pipelined"       # 256 items: under two per SM
-    assert kernel(1, 32, 8, 8192, True) == "fa_fwd_persistent"      # items of 64 K/V tiles: the limit at d = 128
-    assert kernel(4, 32, 32, 8192, True) == "fa_fwd_persistent"
-    assert kernel(1, 32, 8, 16384, True) == "fa_fwd_pipelined"      # items of 128 K/V tiles
+    assert kernel(4, 32, 8, 1024, False) == "fa_fwd_persistent"
+    assert kernel(2, 32, 8, 1024, True) == "fa_fwd_pair"            # 256 items: under two per SM
+    assert kernel(2, 32, 8, 2048, True) == "fa_fwd_pair"            # items of 16 K/V tiles
+    assert kernel(4, 32, 32, 8192, True) == "fa_fwd_pair"           # items of 64 K/V tiles
+    assert kernel(1, 32, 8, 16384, True) == "fa_fwd_pair"           # items of 128 K/V tiles
+    assert binding.fa_plan(SMS, 4, 32, 32, 8192, 8192, 128, 128, True, flags=binding.FA_FLAG_LEGACY_PAIR_KERNEL)["kernel"] == "fa_fwd_pipelined"
     assert binding.fa_plan(SMS, 8, 16, 16, 2048, 2048, 64, 64, True)["kernel"] == "fa_fwd_persistent"   # d = 64: up to 16 tiles
     assert binding.fa_plan(SMS, 4, 16, 16, 4096, 4096, 64, 64, True)["kernel"] == "fa_fwd_pipelined"
 
@@ -95,8 +98,9 @@ def test_flags_and_configuration_override_the_choice():
 
 
 def test_packed_batches_and_head_size_192():
-    assert binding.fa_plan(SMS, 2, 16, 4, 2048, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_pipelined"    # 256 items
-    assert binding.fa_plan(SMS, 4, 16, 4, 2048, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_persistent"   # 512 items
+    assert binding.fa_plan(SMS, 2, 16, 4, 1024, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_pair"         # 128 items
+    assert binding.fa_plan(SMS, 8, 16, 4, 1024, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_persistent"   # 512 items of up to 8 K/V tiles
+    assert binding.fa_plan(SMS, 4, 16, 4, 2048, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_pair"         # 512 items of up to 16
     assert binding.fa_plan(SMS, 4, 16, 4, 2048, 1024, 192, 128, True, varlen=True)["kernel"] == "fa_fwd_stream"
     assert binding.fa_plan(SMS, 1, 16, 16, 2048, 2048, 192, 128, True)["kernel"] == "fa_fwd_stream"
 
@@ -115,10 +119,11 @@ def test_packed_batches_of_many_short_sequences():
     # many items per SM: the persistent kernel, heads of a group paired (one item per tile and pair of heads)
     p = plan(64, 32, 8, 128)
     assert p["kernel"] == "fa_fwd_persistent" and p["ctas"] == SMS and p["kv_splits"] == 1, p
-    assert plan(8, 32, 8, 128, S=2048)["kernel"] == "fa_fwd_persistent"
+    assert plan(8, 32, 8, 128, S=1024)["kernel"] == "fa_fwd_persistent"
+    assert plan(8, 32, 8, 128, S=2048)["kernel"] == "fa_fwd_pair"
     # without it: single tiles of two heads of a group share a CTA of the pair kernel
     p = plan(64, 32, 8, 128, flags=binding.FA_FLAG_NO_PERSISTENT)
-    assert p["kernel"] == "fa_fwd_pipelined" and p["ctas"] == 64 * 16 and p["kv_splits"] == 1, p
+    assert p["kernel"] == "fa_fwd_pair" and p["ctas"] == 64 * 16 and p["kv_splits"] == 1, p
     assert plan(4, 32, 8, 128)["kernel"] == "fa_fwd_stream"              # 128 items: under a wave of single tiles
     assert plan(64, 32, 32, 128, flags=binding.FA_FLAG_NO_PERSISTENT)["kernel"] == "fa_fwd_stream"   # nothing to pair
     assert plan(64, 32, 8, 192)["kernel"] == "fa_fwd_stream"             # 192/128 stays on the stream kernel
