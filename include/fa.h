@@ -56,11 +56,13 @@ typedef enum fa_status {
  * between loads, MMAs and softmax) instead of the pipelined one.  Same results up to
  * rounding order; much slower.  Meant for tests. */
 #define FA_FLAG_SERIAL_KERNEL 1u
-/* fa_config.flags, test hook for the failure path: the load warp of the pipelined kernel leaves
- * out the load of the first V tile, so the wait for it runs into the device-side limit
+/* fa_config.flags, test hook for the failure path: the loading thread of whichever kernel runs
+ * (every attention kernel of the library honours it, the 8-bit ones included) leaves out the load
+ * of its CTA's first V tile, so the wait for it runs into the device-side limit
  * (fa_config.wait_limit_ms).  The kernel then returns normally, results are invalid and
- * fa_last_status reports FA_ERR_DEVICE_TIMEOUT; the context stays usable.  Nothing faults,
- * traps or spins without bound.  Use with a short wait_limit_ms on a tiny problem. */
+ * fa_last_status reports FA_ERR_DEVICE_TIMEOUT; the context and the handle stay usable.  Nothing
+ * faults, traps or spins without bound.  Use with a short wait_limit_ms on a tiny problem.
+ * fa_debug_set_drop_v_load switches the hook on and off for an existing handle. */
 #define FA_FLAG_DEBUG_DROP_V_LOAD 2u
 /* fa_config.flags: launch the kernels the ordinary way.  By default the pipelined kernel (and the
  * split-KV combine kernel) are launched with programmatic stream serialisation: the GPU may
@@ -283,6 +285,12 @@ fa_status fa_forward_host(fa_handle* h,
  */
 fa_status fa_last_status(fa_handle* h, uint32_t* detail);
 
+/* Test hook: switches FA_FLAG_DEBUG_DROP_V_LOAD on (enabled != 0) or off for launches made through `h` from now on,
+ * so that a test can make one launch run into its wait limit and check that the next one through the same handle
+ * is correct.  When fa_last_status reports an error it also puts the persistent kernel's work-item counter, which a
+ * launch that gave up leaves half-way, back to zero: call it (after synchronising) before launching again. */
+fa_status fa_debug_set_drop_v_load(fa_handle* h, int enabled);
+
 /* Free everything the handle owns.  fa_destroy(NULL) returns FA_OK. */
 fa_status fa_destroy(fa_handle* h);
 
@@ -320,11 +328,15 @@ int fa_last_kv_splits(const fa_handle* h);   /* K/V splits the last fa_forward u
  *     different streams, or different host threads -- race on it: serialise them;
  *   - the first call on a device performs a one-time set-up for that device (looks up the array's
  *     device address, the driver's tensor-map encoder, raises the kernels' shared-memory limit).
- *     Make that first call with the device current and before any stream capture begins.
- * No call made here allocates host or device memory.  Arguments as for fa_forward; kv_splits in
- * [2, 64]; device pointers; the work is enqueued on `stream` of the CURRENT device and the call
- * returns without synchronising.  A device-side wait that runs out is not reported (there is no
- * status word); results are then undefined, as with fa_forward.
+ *     Make that first call with the device current and before any stream capture begins.  With CUDA's
+ *     lazy module loading that first call is also when the driver places this part of the library on
+ *     the device, code and the 8 MiB array included: a caller that hands all of the device's memory to
+ *     its own pools should make one small call BEFORE it freezes its memory plan.  Later calls do not
+ *     allocate.
+ * The library itself calls no allocating routine here (no cudaMalloc, no host heap).  Arguments as for
+ * fa_forward; kv_splits in [2, 64]; device pointers; the work is enqueued on `stream` of the CURRENT
+ * device and the call returns without synchronising.  A device-side wait that runs out is recorded in a
+ * status word that also lives in the library's device data; fa_noalloc_last_status reads it.
  */
 #define FA_NOALLOC_SCRATCH_BYTES (8u << 20)
 fa_status fa_forward_split_noalloc(const void* Q, const void* K, const void* V,
@@ -332,6 +344,10 @@ fa_status fa_forward_split_noalloc(const void* Q, const void* K, const void* V,
                                    int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv,
                                    int causal, float scale, int kv_splits, void* stream);
 size_t fa_noalloc_scratch_bytes(void);   /* FA_NOALLOC_SCRATCH_BYTES as built into the library */
+/* (no paper counterpart) Status of the fa_forward_split_noalloc calls on the CURRENT device since the last call of this
+ * function: synchronises the device, returns FA_OK or FA_ERR_DEVICE_TIMEOUT (with the wait site in *detail when
+ * detail is not NULL) and clears the word.  Allocates nothing.  The word is shared by all calls, like the array. */
+fa_status fa_noalloc_last_status(uint32_t* detail);
 
 #ifdef __cplusplus
 }

@@ -32,7 +32,7 @@ FA_FLAG_LEGACY_PAIR_KERNEL = 256
 
 EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_varlen", "fa_forward_fp8", "fa_plan", "fa_forward_host", "fa_last_status", "fa_destroy",
            "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits",
-           "fa_forward_split_noalloc", "fa_noalloc_scratch_bytes")
+           "fa_forward_split_noalloc", "fa_noalloc_scratch_bytes", "fa_noalloc_last_status", "fa_debug_set_drop_v_load")
 
 
 class FaError(RuntimeError):
@@ -101,6 +101,10 @@ def load():
     lib.fa_forward_split_noalloc.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, i32, f32, i32, vp]
     lib.fa_noalloc_scratch_bytes.restype = ctypes.c_size_t
     lib.fa_noalloc_scratch_bytes.argtypes = []
+    lib.fa_debug_set_drop_v_load.restype = i32
+    lib.fa_debug_set_drop_v_load.argtypes = [vp, i32]
+    lib.fa_noalloc_last_status.restype = i32
+    lib.fa_noalloc_last_status.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
     _lib = lib
     return lib
 
@@ -190,8 +194,19 @@ def fa_forward_split_noalloc(Q, K, V, O, lse, B, Hq, Hkv, Sq, Sk, dqk, dv, causa
                                            int(bool(causal)), float(scale), int(kv_splits), stream)
 
 
+def fa_debug_set_drop_v_load(h, enabled) -> int:
+    return int(load().fa_debug_set_drop_v_load(h, int(bool(enabled))))
+
+
 def fa_noalloc_scratch_bytes() -> int:
     return int(load().fa_noalloc_scratch_bytes())
+
+
+def fa_noalloc_last_status():
+    """(status, wait site) of the allocation-free calls on the current device since the last query; synchronises."""
+    detail = ctypes.c_uint32(0)
+    st = load().fa_noalloc_last_status(ctypes.byref(detail))
+    return int(st), int(detail.value)
 
 
 def fa_last_kv_splits(h) -> int:

@@ -427,7 +427,6 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     pl.head_pair = false;
     pl.pair_us = pl.stream_us = 0.0;
     const int n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
-    const bool drop = (flags & FA_FLAG_DEBUG_DROP_V_LOAD) != 0;
     int max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;           // K/V tiles of the longest query tile
     if (causal) {
         const int t = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, Sk, 1);
@@ -446,7 +445,7 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     // h the largest divisor of the group size that fits, and every K/V tile is read and
     // multiplied once for all of them.  Only the stream kernel has this mode.
     // (Packed batches: Sq is the longest query of the batch and there is no split.)
-    if (!drop && !(flags & (FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)) && Sq <= fa::kTileM / 2 &&
+    if (!(flags & (FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)) && Sq <= fa::kTileM / 2 &&
         Hq / Hkv >= 2) {
         const int group = Hq / Hkv;
         int hp = 1;
@@ -473,7 +472,7 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     // (packed batches: the list has an item for every tile of the longest sequence, which Sq is;
     //  the sequences a tile does not exist in pass through the kernel's item ring empty)
     const int longest = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, (varlen && Sk < Sq) ? Sq : Sk, causal);
-    const bool persistent_ok = pair_splits == 1 && dqk != 192 && !drop;
+    const bool persistent_ok = pair_splits == 1 && dqk != 192;
     bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= (dqk == 64 ? 16 : 8);
     if (flags & FA_FLAG_NO_PERSISTENT) persistent = false;
     if ((flags & FA_FLAG_FORCE_PERSISTENT) && persistent_ok) persistent = true;
@@ -484,11 +483,11 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     // tiles of a pair-kernel CTA the same number of K/V tiles (no round that one of them runs alone).
     // (Without a mask it only matters for an odd number of query tiles, whose last tile would be alone.)
     // (Packed batches: every sequence's tiles pair up the same way; n_q_tiles is the longest one's.)
-    const bool head_pair_ok = !drop && (causal || (n_q_tiles & 1)) && pair_splits == 1 && (Hq / Hkv) % 2 == 0 &&
+    const bool head_pair_ok = (causal || (n_q_tiles & 1)) && pair_splits == 1 && (Hq / Hkv) % 2 == 0 &&
                               !(flags & FA_FLAG_NO_HEAD_PACKING);
     bool stream = false;
     int stream_splits = 1;
-    if (!drop && !(flags & FA_FLAG_NO_STREAM_KERNEL)) {
+    if (!(flags & FA_FLAG_NO_STREAM_KERNEL)) {
         // packed batches split only with a single query tile per sequence (decode-like), by the mean K/V length
         if (!varlen || n_q_tiles == 1) stream_splits = choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles, true);
         if (flags & FA_FLAG_STREAM_KERNEL) {
@@ -752,8 +751,25 @@ fa_status fa_last_status(fa_handle* h, uint32_t* detail) {
     const uint32_t code = sw[0];
     const uint32_t who = sw[1];
     if (detail) *detail = code ? who : 0u;
-    if (code) { sw[0] = 0; sw[1] = 0; }
+    if (code) {
+        sw[0] = 0;
+        sw[1] = 0;
+        // A persistent launch that gave up has not made all of its draws from the ticket counter, which the last
+        // draw of a complete launch puts back to zero: zero it here, or the next persistent launch would start in the
+        // middle of its item list.  (The caller synchronised before asking, so no launch is using the counter.)
+        if (h->sched_counter) {
+            DeviceGuard guard(h->device);
+            if (guard.ok()) cudaMemset(h->sched_counter, 0, sizeof(unsigned int));
+        }
+    }
     return code == 0 ? FA_OK : (code == FA_ERR_DEVICE_TIMEOUT ? FA_ERR_DEVICE_TIMEOUT : FA_ERR_CUDA);
+}
+
+fa_status fa_debug_set_drop_v_load(fa_handle* h, int enabled) {
+    if (!h) return FA_ERR_INVALID_ARG;
+    if (enabled) h->flags |= FA_FLAG_DEBUG_DROP_V_LOAD;
+    else h->flags &= ~FA_FLAG_DEBUG_DROP_V_LOAD;
+    return FA_OK;
 }
 
 uint64_t fa_launch_count(const fa_handle* h) { return h ? h->launches : 0; }
@@ -855,7 +871,7 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     if (s != FA_OK) return s;
     if ((q_scale && misaligned(q_scale, 4)) || (k_scale && misaligned(k_scale, 4)) || (v_scale && misaligned(v_scale, 4)))
         return FA_ERR_INVALID_ARG;
-    if (h->flags & (FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD)) return FA_ERR_UNSUPPORTED;
+    if (h->flags & FA_FLAG_SERIAL_KERNEL) return FA_ERR_UNSUPPORTED;
     DeviceGuard guard(h->device);
     if (!guard.ok()) return FA_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -893,6 +909,7 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     p.heads_per_group = heads_per_group(static_cast<long long>(Sk) * 2 * d, B, Hq, Hkv);      // one byte per element
     p.status = h->status_dev;
     p.wait_limit_ns = h->wait_limit_ns;
+    p.debug_drop_v_load = (h->flags & FA_FLAG_DEBUG_DROP_V_LOAD) ? 1 : 0;
     fa::Fp8Params f;
     f.q_scale = q_scale; f.k_scale = k_scale; f.v_scale = v_scale;
     f.n_kv_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;

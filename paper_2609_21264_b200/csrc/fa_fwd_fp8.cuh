@@ -484,7 +484,7 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
                     tma_load_4d(sK + s * kTile8, &tm_k, bar, 0, j0, kvh, b);
                     if (j == 0) load_q(1);
                 }
-                {
+                if (!(p.debug_drop_v_load && j == 0)) {       // (test hook: see FA_FLAG_DEBUG_DROP_V_LOAD)
                     const int s = j % NV;
                     ok = mbar_wait(smem_addr(&sh.v_empty[s]), ((j / NV) & 1) ^ 1, wctx, kSiteLoadKvEmpty);
                     if (!ok) break;

@@ -653,7 +653,7 @@ fa_fwd_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                                         item.k_row0 + j0, item.kvh, kVarlen ? 0 : item.b);
                         ++kc;
                     }
-                    {
+                    if (!(p.debug_drop_v_load && k == 0 && j == 0)) {      // (test hook: see FA_FLAG_DEBUG_DROP_V_LOAD)
                         const uint32_t s = vc % NV;
                         ok = mbar_wait(smem_addr(&sh.v_empty[s]), ((vc / NV) & 1u) ^ 1u, wctx, kSiteLoadKvEmpty);
                         if (!ok) break;

@@ -591,6 +591,7 @@ fa_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         if (elect_one() && n_kv > 0) {
             bool ok = true;
             for (int j = 0; j < n_kv && ok; ++j) {
+                if (p.debug_drop_v_load && j == 0) continue;      // (test hook: see FA_FLAG_DEBUG_DROP_V_LOAD)
                 const int s = j % NV;
                 ok = mbar_wait(smem_addr(&sh.v_empty[s]), ((j / NV) & 1) ^ 1, wctx, kSiteLoadKvEmpty);
                 if (!ok) break;

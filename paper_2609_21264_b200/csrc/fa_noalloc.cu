@@ -31,6 +31,9 @@ constexpr size_t kStaticScratchBytes = FA_NOALLOC_SCRATCH_BYTES;
 // array directly; host code may not pass it to a kernel (on the host the name is a stand-in,
 // not a device address) and gets the address with cudaGetSymbolAddress instead.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+// Status of the kernels launched from here ([0] = fa_status, [1] = wait site), written by a device-side wait that runs
+// out; the same rule applies: host code asks for its address, kernels get that address.
+static __device__ uint32_t g_static_status[2];
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
                                    const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -42,6 +45,7 @@ constexpr int kMaxDevices = 64;
 struct DeviceState {          // fixed-size host bookkeeping: no heap
     bool ready = false;
     unsigned char* scratch = nullptr;     // device address of g_static_scratch on this device
+    uint32_t* status = nullptr;           // device address of g_static_status on this device
     EncodeTiledFn encode = nullptr;
 };
 DeviceState g_dev[kMaxDevices];
@@ -55,7 +59,8 @@ bool raise_smem_limit() {
 }
 
 // One-time set-up for the CURRENT device: address of the scratch array on this device, the
-// driver's tensor-map encoder, the kernels' shared-memory limit.  Nothing here allocates.
+// driver's tensor-map encoder, the kernels' shared-memory limit.  No allocating routine is called; with lazy
+// module loading the driver places this translation unit's code and data (the 8 MiB array) on the device now.
 fa_status setup_current_device(int device) {
     std::lock_guard<std::mutex> lock(g_dev_mutex);
     DeviceState& d = g_dev[device];
@@ -65,6 +70,11 @@ fa_status setup_current_device(int device) {
     if (major != 10) return FA_ERR_NO_DEVICE;
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) {
+        cudaGetLastError();
+        return FA_ERR_CUDA;
+    }
+    void* sptr = nullptr;
+    if (cudaGetSymbolAddress(&sptr, g_static_status) != cudaSuccess || sptr == nullptr) {
         cudaGetLastError();
         return FA_ERR_CUDA;
     }
@@ -80,6 +90,7 @@ fa_status setup_current_device(int device) {
         return FA_ERR_CUDA;
     }
     d.scratch = static_cast<unsigned char*>(ptr);
+    d.status = static_cast<uint32_t*>(sptr);
     d.encode = reinterpret_cast<EncodeTiledFn>(fn);
     d.ready = true;
     return FA_OK;
@@ -180,7 +191,7 @@ fa_status fa_forward_split_noalloc(const void* Q, const void* K, const void* V, 
     p.scale_log2 = scale * 1.4426950408889634f;
     p.n_q_tiles = n_q_tiles;
     p.heads_per_group = B * Hq;                 // short problems: everything fits in L2
-    p.status = nullptr;                         // no status word: device-side timeouts are not reported here
+    p.status = dev.status;                      // a wait that runs out leaves its code here (fa_noalloc_last_status)
     p.wait_limit_ns = 2000ull * 1000000ull;
     p.kv_splits = splits;
     p.tiles_per_split = (max_tiles + splits - 1) / splits;
@@ -193,6 +204,23 @@ fa_status fa_forward_split_noalloc(const void* Q, const void* K, const void* V, 
     if (dqk == 64) return launch<64, 64>(mq, mk, mv, mo, p, st);
     if (dqk == 128) return launch<128, 128>(mq, mk, mv, mo, p, st);
     return launch<192, 128>(mq, mk, mv, mo, p, st);
+}
+
+fa_status fa_noalloc_last_status(uint32_t* detail) {
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return FA_ERR_NO_DEVICE; }
+    if (device < 0 || device >= kMaxDevices) return FA_ERR_UNSUPPORTED;
+    if (detail) *detail = 0;
+    if (!g_dev[device].ready) return FA_OK;      // nothing has been launched from here on this device
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return FA_ERR_CUDA; }
+    uint32_t words[2] = {0, 0};
+    if (cudaMemcpyFromSymbol(words, g_static_status, sizeof words) != cudaSuccess) { cudaGetLastError(); return FA_ERR_CUDA; }
+    if (words[0] != 0) {
+        const uint32_t zero[2] = {0, 0};
+        if (cudaMemcpyToSymbol(g_static_status, zero, sizeof zero) != cudaSuccess) { cudaGetLastError(); return FA_ERR_CUDA; }
+    }
+    if (detail) *detail = words[1];
+    return static_cast<fa_status>(words[0]);
 }
 
 }  // extern "C"

@@ -1,4 +1,4 @@
-"""The allocation-free split-KV entry point against the handle-based one.
+"""The allocation-free split-KV entry point against the oracle and against the handle-based one.
 
 `fa_forward_split_noalloc` is for callers that may not allocate device memory (a server whose
 memory plan is frozen, a real-time loop, a plug-in limited to its host's buffers): it takes no
@@ -9,8 +9,9 @@ other test; it also passes when run alone in a fresh process (it does its own se
 import numpy as np
 import pytest
 
+import oracle
 from paper_2609_21264_b200 import workloads as W
-from parity_util import LSE_MAX_ABS, O_MAX_ABS, O_MEAN_ABS, bf16_tensor_to_f64, to_torch_bf16
+from parity_util import LSE_MAX_ABS, O_MAX_ABS, O_MEAN_ABS, assert_parity, bf16_tensor_to_f64, to_torch_bf16
 
 pytestmark = pytest.mark.gpu
 
@@ -59,6 +60,52 @@ def test_no_alloc_entry_point_matches_handle_path_on_two_calls_in_a_row():
         assert st == b.FA_OK
     finally:
         b.fa_destroy(h)
+
+
+def _no_alloc(w, splits, want_lse=True):
+    import torch
+    from paper_2609_21264_b200 import binding as b
+    Q, K, V = W.make_inputs(w)
+    q, k, v = to_torch_bf16(Q), to_torch_bf16(K), to_torch_bf16(V)
+    o = torch.full((w.B, w.Hq, w.Sq, w.dv), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((w.B, w.Hq, w.Sq), float("nan"), dtype=torch.float32, device="cuda") if want_lse else None
+    st = b.fa_forward_split_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr() if want_lse else None,
+                                    w.B, w.Hq, w.Hkv, w.Sq, w.Sk, w.dqk, w.dv, w.causal, w.scale, splits,
+                                    torch.cuda.current_stream().cuda_stream)
+    assert st == b.FA_OK, b.fa_strerror(st)
+    torch.cuda.synchronize()
+    assert b.fa_noalloc_last_status() == (b.FA_OK, 0)
+    return (Q, K, V), bf16_tensor_to_f64(o), (lse.double().cpu().numpy() if want_lse else None)
+
+
+# Shapes chosen for what the shared array and the split path can get wrong: later splits that are empty under a causal
+# mask, a forced empty split (fewer K/V tiles than splits), the asymmetric head sizes, an odd number of query tiles,
+# more queries than keys (rows with no visible key at all), and partials that fill the 8 MiB array to the last byte.
+ORACLE_CASES = [
+    (W.Workload("causal_multi_tile_empty_late_splits", 1, 4, 2, 384, 384, 128, 128, True, 128 ** -0.5, seed=41), 3),
+    (W.Workload("one_kv_tile_two_splits", 1, 6, 3, 100, 128, 64, 64, False, 64 ** -0.5, seed=42), 2),
+    (W.Workload("d192_dv128", 1, 4, 2, 200, 1000, 192, 128, True, 192 ** -0.5, seed=43), 4),
+    (W.Workload("odd_number_of_query_tiles", 1, 2, 2, 300, 2100, 128, 128, False, 128 ** -0.5, seed=44), 5),
+    (W.Workload("more_queries_than_keys", 1, 2, 1, 333, 200, 128, 128, True, 128 ** -0.5, seed=45), 2),
+    # 2 splits x (1 x 8 x 1016) rows x 129 floats x 4 bytes = 8 388 096 bytes + ... : the largest row count that fits
+    (W.Workload("partials_at_the_limit", 1, 8, 4, (8 << 20) // (2 * 8 * 129 * 4), 700, 128, 128, False, 128 ** -0.5, seed=46), 2),
+]
+
+
+@pytest.mark.parametrize("w,splits", ORACLE_CASES, ids=[c[0].name for c in ORACLE_CASES])
+def test_no_alloc_entry_point_against_the_oracle(w, splits):
+    from paper_2609_21264_b200 import binding as b
+    if w.name == "partials_at_the_limit":
+        need = splits * w.B * w.Hq * w.Sq * (w.dv + 1) * 4
+        assert need <= b.fa_noalloc_scratch_bytes() < splits * w.B * w.Hq * (w.Sq + 1) * (w.dv + 1) * 4
+    (Q, K, V), O, lse = _no_alloc(w, splits)
+    O_ref, lse_ref = oracle.attention(Q, K, V, causal=w.causal, scale=w.scale)
+    assert_parity(O, lse, O_ref, lse_ref, w.name)
+    if w.name == "more_queries_than_keys":
+        assert np.isneginf(lse_ref).any() and (O[np.isneginf(lse_ref)] == 0).all()
+    # once more without the log-sum-exp output (a NULL pointer is legal), on what the first call left in the array
+    _, O2, _ = _no_alloc(w, splits, want_lse=False)
+    np.testing.assert_array_equal(O, O2)
 
 
 def test_no_alloc_entry_point_rejects_what_does_not_fit_and_bad_arguments():
