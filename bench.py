@@ -39,13 +39,18 @@ from paper_2609_21264_b200 import launch, metrics, workloads  # noqa: E402
 L2_BYTES = 126 * 1024 * 1024
 # Paper, Table 6: Llama-3 8B shape (32/8 heads, d=128, causal, S=2048) on XDNA 2: 34076 us.
 PAPER_SECONDS = {"llama3_8b_gqa_s2048": 34076e-6}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (None = not captured for that workload).
-# A workload too large to capture under the profiler carries the figure of a smaller case of the same kernel scaled
-# by the compulsory bytes (DRAM traffic of this kernel grows in proportion to them: K and V are read once per K/V
-# head from DRAM and re-read from L2, Q and O move once); see profiles/ and the design doc.
-NCU_DRAM_BYTES_PER_LAUNCH = {}
-NCU_DRAM_BYTES_PER_COMPULSORY_BYTE = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on each configuration, each taken
+# from a one-pass ncu capture of this program on that configuration at full size (a one-pass metric list saves and
+# restores no device memory, so the full workload can be captured); the commands and figures are under profiles/.
+# Reads below the compulsory bytes mean that part of a rotating input set was still in L2; writes below the output
+# size mean that the launch ended with its last outputs still in L2.
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    "bert_base_mha_s512": 2.42e6 + 0.0,
+    "llama3_8b_gqa_s2048": 25.23e6 + 0.0,
+    "llama2_7b_mha_b4_s8192": 922.56e6 + 256.61e6,
+    "deepseek_v2_mha_s4096_d192_128": 579.18e6 + 124.12e6,
+    "long_context_gqa_s131072": 3.14e9 + 1.06e9,
+}
 
 
 def load_peaks():
@@ -407,8 +412,6 @@ def roofline_of(w, t_step, peaks, kernel):
     t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
     bound = "tensor" if t_tensor_burst >= t_hbm else "hbm"
     traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(w.name)
-    if traffic is None and w.name in NCU_DRAM_BYTES_PER_COMPULSORY_BYTE:
-        traffic = NCU_DRAM_BYTES_PER_COMPULSORY_BYTE[w.name] * nbytes
     r = {"bound": bound, "kernel": kernel, "avg_launch_us": t_step * 1e6, "traffic": traffic,
          "algorithmic_flops_per_launch": fl_alg, "compulsory_bytes_per_launch": nbytes,
          "frac_of_nominal_2250_tflops": fl_alg / t_step / 2.25e15}
