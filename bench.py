@@ -458,7 +458,8 @@ def measure_config(binding, h, h_plain, w, device, peaks, gpu_index, steps=None,
                               "stream serialisation (no overlap between consecutive launches); 'us' is the mean of "
                               "back-to-back launches, whose tails overlap",
            "bound": roof["bound"], "frac_burst": roof["frac_burst"], "frac_sustained": roof["frac_sustained"],
-           "frac_of_nominal_2250": fl_alg / t / 2.25e15, "clocks": clocks,
+           "frac_of_nominal_2250": fl_alg / t / 2.25e15,
+           "dram_traffic_bytes_per_launch": roof["traffic"], "compulsory_bytes_per_launch": nbytes, "clocks": clocks,
            "us_x_sm_mhz": (t * 1e6 * clocks["sm_mhz"]) if clocks.get("sm_mhz") else None}
     return rec, roof, seconds, launches, steps, warmup
 
