@@ -97,11 +97,18 @@ typedef enum fa_status {
  * number of query tiles: the CTA's tiles are the same query tile of two adjacent heads of a
  * group instead of two adjacent query tiles of one head; results bit-identical either way). */
 #define FA_FLAG_NO_HEAD_PACKING 128u
-/* fa_config.flags: at head size 128 the one-item-per-CTA tiling with two query tiles per CTA has two
- * kernels: csrc/fa_fwd_pair.cuh (the default: one MMA-issuing thread that probes its barriers from
- * inside the blocks of MMAs, no correction warpgroup) and the older csrc/fa_fwd_pipelined.cuh, which
- * this flag selects.  Same results up to fp32 rounding order.  Meant for tests and A/B timing. */
+/* fa_config.flags: at head size 128 the tilings with two query tiles per CTA have two generations of
+ * kernels: csrc/fa_fwd_pair.cuh and its persistent form csrc/fa_fwd_pair_persistent.cuh (the default:
+ * one MMA-issuing thread that probes its barriers from inside the blocks of MMAs, no correction
+ * warpgroup) and the older csrc/fa_fwd_pipelined.cuh and csrc/fa_fwd_persistent.cuh, which this flag
+ * selects.  Same results, bit for bit.  Meant for tests and A/B timing. */
 #define FA_FLAG_LEGACY_PAIR_KERNEL 256u
+/* fa_config.flags: run fixed-length problems without split-KV at head sizes 128 and 192/128 on the
+ * kernel that pairs two SMs (a cluster of two CTAs with one query tile each, every MMA issued once
+ * for both as a two-CTA tcgen05.mma, each CTA holding half of every K/V tile).  Its two softmax
+ * warpgroups keep separate partial results for the even and the odd K/V tiles and merge them at
+ * the end, so its output agrees with the other kernels' to rounding, not bit for bit. */
+#define FA_FLAG_TWO_CTA_KERNEL 512u
 
 /* Optional creation parameters.  Zero-initialise, set struct_size = sizeof(fa_config). */
 typedef struct fa_config {

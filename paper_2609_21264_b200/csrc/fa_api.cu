@@ -14,6 +14,8 @@
 #include "fa_common.cuh"
 #include "fa_fwd_pipelined.cuh"
 #include "fa_fwd_pair.cuh"
+#include "fa_fwd_duo.cuh"
+#include "fa_fwd_pair_persistent.cuh"
 #include "fa_fwd_persistent.cuh"
 #include "fa_fwd_stream.cuh"
 #include "fa_fwd_fp8.cuh"
@@ -219,6 +221,34 @@ fa_status launch_pipelined(fa_handle* h, const CUtensorMap& mq, const CUtensorMa
                                fa::PipeCfg<DQK, DV>::kThreads, kHeadPair, mq, mk, mv, mo, p, st);
 }
 
+// One query tile per CTA on pairs of CTAs (clusters of two, two-CTA MMAs): fa_fwd_duo.cuh.
+template <int DQK, int DV, bool kHeadPair>
+fa_status launch_duo(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                     const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
+    constexpr int smem = fa::duo_smem_bytes<DQK, DV>();
+    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+    auto kernel = fa::fa_fwd_duo_kernel<DQK, DV, kHeadPair>;
+    fa_status s = ensure_smem_attr(h, kernel, smem);
+    if (s != FA_OK) return s;
+    // one cluster per item: two adjacent query tiles of a head, or one query tile of two adjacent heads
+    const long long n_ctas = 2 * (kHeadPair ? static_cast<long long>(p.n_q_tiles) * (p.Hq / 2)
+                                            : static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq) * p.B;
+    if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);       // the kernel carries __cluster_dims__(2, 1, 1)
+    cfg.blockDim = dim3(fa::DuoCfg<DQK, DV>::kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = (h->flags & FA_FLAG_NO_DEPENDENT_LAUNCH) ? 0 : 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mo, p) != cudaSuccess) return FA_ERR_CUDA;
+    h->launches += 1;
+    return FA_OK;
+}
+
 // Number of K/V splits for a problem: 1 unless the query tiles alone leave most SMs idle and the
 // K/V range is long enough to cut; never more than the scratch buffer can hold partials for.
 int choose_kv_splits(int num_sms, uint32_t kv_splits_cfg, size_t scratch_bytes, int B, int Hq, int Sq, int Sk, int dv,
@@ -294,11 +324,6 @@ int heads_per_group(long long kv_bytes_per_head, int B, int Hq, int Hkv) {
 template <int DQK, int DV, bool kVarlen = false>
 fa_status launch_persistent(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& mk,
                             const CUtensorMap& mv, const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
-    constexpr int smem = fa::persist_smem_bytes<DQK, DV>();
-    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
-    auto kernel = fa::fa_fwd_persistent_kernel<DQK, DV, kVarlen>;
-    fa_status s = ensure_smem_attr(h, kernel, smem);
-    if (s != FA_OK) return s;
     const long long n_items = p.head_pair ? static_cast<long long>(p.n_q_tiles) * (p.Hq / 2) * p.B
                                           : static_cast<long long>((p.n_q_tiles + 1) / 2) * p.Hq * p.B;
     if (n_items > 0x3fffffffLL) return FA_ERR_UNSUPPORTED;
@@ -307,11 +332,31 @@ fa_status launch_persistent(fa_handle* h, const CUtensorMap& mq, const CUtensorM
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(n_items < h->num_sms ? n_items : h->num_sms), 1, 1);
-    cfg.blockDim = dim3(fa::PipeCfg<DQK, DV>::kThreads, 1, 1);
-    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = (h->flags & FA_FLAG_NO_DEPENDENT_LAUNCH) ? 0 : 1;
+    if constexpr (DQK == 128 && DV == 128) {
+        // head size 128: the persistent form of the kernel of fa_fwd_pair.cuh (FA_FLAG_LEGACY_PAIR_KERNEL: the earlier one)
+        if (!(h->flags & FA_FLAG_LEGACY_PAIR_KERNEL)) {
+            constexpr int smem = fa::pair_persist_smem_bytes();
+            static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+            auto kernel = fa::fa_fwd_pair_persistent_kernel<kVarlen>;
+            fa_status s = ensure_smem_attr(h, kernel, smem);
+            if (s != FA_OK) return s;
+            cfg.blockDim = dim3(fa::PairPersistCfg::kThreads, 1, 1);
+            cfg.dynamicSmemBytes = smem;
+            if (cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mo, p) != cudaSuccess) return FA_ERR_CUDA;
+            h->launches += 1;
+            return FA_OK;
+        }
+    }
+    constexpr int smem = fa::persist_smem_bytes<DQK, DV>();
+    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+    auto kernel = fa::fa_fwd_persistent_kernel<DQK, DV, kVarlen>;
+    fa_status s = ensure_smem_attr(h, kernel, smem);
+    if (s != FA_OK) return s;
+    cfg.blockDim = dim3(fa::PipeCfg<DQK, DV>::kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
     if (cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mo, p) != cudaSuccess) return FA_ERR_CUDA;
     h->launches += 1;
     return FA_OK;
@@ -407,7 +452,7 @@ TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int 
 
 // Which kernel a launch uses and how its K/V range is split: a pure function of the problem, the
 // handle's configuration and the SM count (fa_plan exposes it).
-enum PlanKernel { kPlanSerial = 0, kPlanPair = 1, kPlanPersistent = 2, kPlanStream = 3 };
+enum PlanKernel { kPlanSerial = 0, kPlanPair = 1, kPlanPersistent = 2, kPlanStream = 3, kPlanDuo = 4 };
 struct LaunchPlan {
     int kernel;
     int kv_splits;
@@ -463,17 +508,17 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     const int pair_splits = varlen ? 1 : choose_kv_splits(num_sms, kv_splits_cfg, scratch_bytes, B, Hq, Sq, Sk, dv, causal, n_q_tiles);
     // The persistent kernel wins where a CTA's fixed cost is a visible share of an item's time and every SM gets
     // several items.  Measured on B200 against the one-item-per-CTA kernels (an A/B over item lengths,
-    // `bench.py --plan-ab`): at d = 128, where the per-item kernel is the one of fa_fwd_pair.cuh, it is 28 / 20 /
-    // 6 / 4 % faster on items of 1 / 2 / 4 / 8 K/V tiles, level at 16 and 3-7 % slower from 32 tiles on (that kernel's
-    // loop is the faster one); at d = 64, where the per-item kernel keeps P in TMEM columns of its own, it is 5-12 %
-    // faster up to 8-tile items, level at 16 and 4-5 % slower at 32; and it is a few per cent slower below two items
-    // per SM (its one-time set-up and the coarser balance of a short list).  d = 192 has no room for its staging buffer.
+    // `bench.py --plan-ab`): at d = 128, where both are built on the loop of fa_fwd_pair.cuh, it is 35 / 26 / 11 / 9 /
+    // 7 / 3 % faster on items of 1 / 2 / 4 / 8 / 16 / 32 K/V tiles, 2 % at 64 and level at 128 and beyond; at d = 64,
+    // where the per-item kernel keeps P in TMEM columns of its own, it is 5-12 % faster up to 8-tile items, level
+    // at 16 and 4-5 % slower at 32; and it is a few per cent slower below two items per SM (its one-time set-up
+    // and the coarser balance of a short list).  d = 192 has no room for its staging buffer.
     const long long n_items = static_cast<long long>((n_q_tiles + 1) / 2) * Hq * B;
     // (packed batches: the list has an item for every tile of the longest sequence, which Sq is;
     //  the sequences a tile does not exist in pass through the kernel's item ring empty)
     const int longest = fa::kv_tiles_for_q_tile((n_q_tiles - 1) * fa::kTileM, fa::kTileM, Sq, (varlen && Sk < Sq) ? Sq : Sk, causal);
     const bool persistent_ok = pair_splits == 1 && dqk != 192;
-    bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= (dqk == 64 ? 16 : 8);
+    bool persistent = persistent_ok && n_items >= 3ll * num_sms && longest <= (dqk == 64 ? 16 : 128);
     if (flags & FA_FLAG_NO_PERSISTENT) persistent = false;
     if ((flags & FA_FLAG_FORCE_PERSISTENT) && persistent_ok) persistent = true;
     // One query tile per CTA (twice the CTAs, each with a shorter chain) wins where the pair
@@ -511,7 +556,15 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
             if (dqk == 64 && longest >= (causal ? 192 : 32) && pair_splits == 1 && stream_splits == 1) stream = true;
         }
     }
-    if (stream) {
+    // Pairs of CTAs with two-CTA MMAs (fa_fwd_duo.cuh): fixed-length launches without split-KV at head sizes
+    // 128 and 192/128.
+    const bool duo_ok = !varlen && dqk != 64 && pair_splits == 1 && stream_splits == 1;
+    bool duo = false;
+    if ((flags & FA_FLAG_TWO_CTA_KERNEL) && duo_ok) duo = true;
+    if (duo) {
+        pl.kernel = kPlanDuo;
+        pl.head_pair = head_pair_ok;
+    } else if (stream) {
         pl.kernel = kPlanStream;
         with_splits(stream_splits);
     } else if (persistent) {
@@ -619,6 +672,15 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
         if (dqk == 128) return launch_pipelined<128, 128, false>(h, map_q, map_k, map_v, map_o, p, st);
         return launch_pipelined<192, 128, false>(h, map_q, map_k, map_v, map_o, p, st);
     }
+    if (pl.kernel == kPlanDuo) {
+        h->last_kernel = "fa_fwd_duo";
+        if (pl.head_pair) {
+            if (dqk == 128) return launch_duo<128, 128, true>(h, map_q, map_k, map_v, map_o, p, st);
+            return launch_duo<192, 128, true>(h, map_q, map_k, map_v, map_o, p, st);
+        }
+        if (dqk == 128) return launch_duo<128, 128, false>(h, map_q, map_k, map_v, map_o, p, st);
+        return launch_duo<192, 128, false>(h, map_q, map_k, map_v, map_o, p, st);
+    }
     h->last_kernel = "fa_fwd_simple";
     if (dqk == 64) return launch_simple<64, 64>(h, map_q, map_k, map_v, p, st);
     if (dqk == 128) return launch_simple<128, 128>(h, map_q, map_k, map_v, p, st);
@@ -659,7 +721,8 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg) {
         if (cfg->struct_size >= sizeof(fa_config)) scratch_bytes = cfg->scratch_bytes;
         if (flags & ~(FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD | FA_FLAG_NO_DEPENDENT_LAUNCH |
                       FA_FLAG_NO_PERSISTENT | FA_FLAG_FORCE_PERSISTENT | FA_FLAG_STREAM_KERNEL |
-                      FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING | FA_FLAG_LEGACY_PAIR_KERNEL)) return FA_ERR_INVALID_ARG;
+                      FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING | FA_FLAG_LEGACY_PAIR_KERNEL |
+                      FA_FLAG_TWO_CTA_KERNEL)) return FA_ERR_INVALID_ARG;
         if (kv_splits_cfg > 256) return FA_ERR_INVALID_ARG;
     }
     if (scratch_bytes == 0) scratch_bytes = 32ull << 20;
@@ -800,7 +863,9 @@ fa_status fa_forward_strided(fa_handle* h, const void* Q, const void* K, const v
     const int q_box_rows = pl.pack_heads > 1 ? Sq : fa::kTileM;
     if ((s = get_map(h, Q, dqk, Sq, Hq, B, q_strides[0], q_strides[1], q_strides[2], q_box_rows, &mq, 2, pl.pack_heads)) != FA_OK) return s;
     CUtensorMap map_q = *mq;   // copies: a later insertion may evict or move cache entries
-    if ((s = get_map(h, K, dqk, Sk, Hkv, B, k_strides[0], k_strides[1], k_strides[2], fa::kTileN, &mk)) != FA_OK) return s;
+    // (the two-CTA kernel loads K in boxes of 64 keys: each CTA of a pair keeps half of a K tile)
+    const int k_box_rows = pl.kernel == kPlanDuo ? fa::kTileN / 2 : fa::kTileN;
+    if ((s = get_map(h, K, dqk, Sk, Hkv, B, k_strides[0], k_strides[1], k_strides[2], k_box_rows, &mk)) != FA_OK) return s;
     CUtensorMap map_k = *mk;
     if ((s = get_map(h, V, dv, Sk, Hkv, B, v_strides[0], v_strides[1], v_strides[2], fa::kTileN, &mv)) != FA_OK) return s;
     CUtensorMap map_v = *mv;
@@ -1012,7 +1077,7 @@ fa_status fa_plan(int num_sms, const fa_config* cfg, int varlen, int B, int Hq, 
     }
     const LaunchPlan pl = plan_launch(num_sms, flags, splits_cfg, static_cast<size_t>(scratch), varlen != 0,
                                       B, Hq, Hkv, Sq, Sk, dqk, dv, causal ? 1 : 0);
-    static const char* const names[4] = {"fa_fwd_simple", "fa_fwd_pipelined", "fa_fwd_persistent", "fa_fwd_stream"};
+    static const char* const names[5] = {"fa_fwd_simple", "fa_fwd_pipelined", "fa_fwd_persistent", "fa_fwd_stream", "fa_fwd_duo"};
     out->kernel = names[pl.kernel];
     // the one-item-per-CTA tiling with two query tiles has a kernel of its own at head size 128
     if (pl.kernel == kPlanPair && dqk == 128 && dv == 128 && !(flags & FA_FLAG_LEGACY_PAIR_KERNEL)) out->kernel = "fa_fwd_pair";
@@ -1023,6 +1088,7 @@ fa_status fa_plan(int num_sms, const fa_config* cfg, int varlen, int B, int Hq, 
     switch (pl.kernel) {
         case kPlanSerial: ctas = n_q_tiles * Hq * B; break;
         case kPlanPair: ctas = (pl.head_pair ? n_q_tiles * (Hq / 2) : ((n_q_tiles + 1) / 2) * Hq) * B * pl.kv_splits; break;
+        case kPlanDuo: ctas = 2 * (pl.head_pair ? n_q_tiles * (Hq / 2) : ((n_q_tiles + 1) / 2) * Hq) * B; break;
         case kPlanPersistent:
             ctas = (pl.head_pair ? n_q_tiles * (Hq / 2) : ((n_q_tiles + 1) / 2) * Hq) * B;
             if (ctas > num_sms) ctas = num_sms;

@@ -20,7 +20,7 @@ enum WaitSite : uint32_t {
     kSiteMmaOReady = 0x0304, kSiteMmaSFree = 0x0305, kSiteMmaTurn = 0x0306,
     kSiteSoftmaxSFull = 0x0401, kSiteSoftmaxPFree = 0x0402, kSiteSoftmaxCorrFree = 0x0403,
     kSiteCorrScale = 0x0501, kSiteCorrPvDone = 0x0502, kSiteCorrFinal = 0x0503,
-    kSiteEpiOFull = 0x0601, kSiteEpiStaged = 0x0602,
+    kSiteEpiOFull = 0x0601, kSiteEpiStaged = 0x0602, kSiteEpiState = 0x0603,
     kSiteSmemAlign = 0x0701,
     kSiteItem = 0x0801,
 };

@@ -467,5 +467,133 @@ FA_DEVI void tmem_st_x32(uint32_t taddr, const uint32_t (&r)[32]) {
         : "memory");
 }
 
+// ------------------------------------------------------------------ pairs of CTAs (cluster of two, tcgen05 cta_group::2)
+
+FA_DEVI uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the variable that sits at `addr` (a shared::cta address) in CTA `rank` of the cluster
+FA_DEVI uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+// All threads of the cluster execute both.  The wait returns once every thread of the cluster that has not exited
+// has arrived.
+FA_DEVI void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+FA_DEVI void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// Arrive on an mbarrier of any CTA of the cluster (shared::cluster address).  The plain form, as for a local
+// barrier: what is handed over with it here lives in TMEM and is ordered by the tcgen05 fences around the barrier
+// (tcgen05.wait::st, tcgen05.fence::before_thread_sync on this side, fence::after_thread_sync on the waiter's).
+// Measured on B200, round trip between the two CTAs of a pair: 359 cycles with this form and a plain try_wait, 943
+// with .release.cluster on the arrive and .acquire.cluster on the wait.
+FA_DEVI void mbar_arrive_cluster(uint32_t bar_cluster) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+FA_DEVI void st_shared_cluster_u32(uint32_t addr_cluster, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr_cluster), "r"(v) : "memory");
+}
+// 4-D tiled load into this CTA's shared memory whose bytes are counted on an mbarrier that may sit in the partner
+// CTA (shared::cluster address).  No multicast: every CTA fetches its own box.
+FA_DEVI void tma_load_4d_2cta(uint32_t dst_smem, const CUtensorMap* map, uint32_t bar_cluster,
+                              int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster),
+          "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+// TMEM of both CTAs of a pair: warp w of BOTH CTAs executes each of these.
+FA_DEVI void tmem_alloc_2cta(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+FA_DEVI void tmem_relinquish_alloc_permit_2cta() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+FA_DEVI void tmem_dealloc_2cta(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
+                 : "memory");
+}
+// Arrive (count 1) on the mbarrier at this offset in every CTA of `cta_mask` once every tcgen05 async op
+// issued so far by this thread has completed.
+FA_DEVI void tc_commit_2cta(uint32_t bar, uint16_t cta_mask) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(cta_mask) : "memory");
+}
+// 256 x N x 16 MMAs over a CTA pair, issued by ONE thread of the even CTA: rows 0..127 of A and D belong to the
+// even CTA, rows 128..255 to the odd one; each CTA supplies N/2 columns of B from its own shared memory (same
+// offsets in both CTAs).
+FA_DEVI void mma2_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+FA_DEVI void mma2_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// One asm statement: probe up to three mbarriers, issue three SS MMAs (all accumulating),
+// then read the probes' predicates; bit i of the result = probe i found its phase complete.
+FA_DEVI uint32_t probe3_mma2_ss3(uint32_t bar0, uint32_t par0, uint32_t bar1, uint32_t par1, uint32_t bar2, uint32_t par2,
+                                 uint32_t d_tmem, uint64_t a0, uint64_t b0, uint64_t a1, uint64_t b1, uint64_t a2, uint64_t b2,
+                                 uint32_t idesc) {
+    uint32_t r;
+    asm volatile(
+        "{\n"
+        ".reg .pred p0, p1, p2, q;\n"
+        ".reg .b32 t0, t1, t2;\n"
+        "setp.ne.b32 q, 1, 0;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p0, [%1], %2;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p1, [%3], %4;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p2, [%5], %6;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%7], %8, %9, %14, q;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%7], %10, %11, %14, q;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%7], %12, %13, %14, q;\n"
+        "selp.u32 t0, 1, 0, p0;\n"
+        "selp.u32 t1, 2, 0, p1;\n"
+        "selp.u32 t2, 4, 0, p2;\n"
+        "or.b32 t0, t0, t1;\n"
+        "or.b32 %0, t0, t2;\n"
+        "}\n"
+        : "=r"(r)
+        : "r"(bar0), "r"(par0), "r"(bar1), "r"(par1), "r"(bar2), "r"(par2), "r"(d_tmem), "l"(a0), "l"(b0), "l"(a1),
+          "l"(b1), "l"(a2), "l"(b2), "r"(idesc)
+        : "memory");
+    return r;
+}
+// Probe one mbarrier, issue two TS MMAs (accumulating), then read the predicate.
+FA_DEVI uint32_t probe_mma2_ts2(uint32_t bar, uint32_t par, uint32_t d_tmem, uint32_t a0_tmem, uint64_t b0, uint32_t a1_tmem,
+                                uint64_t b1, uint32_t idesc) {
+    uint32_t r;
+    asm volatile(
+        "{\n"
+        ".reg .pred p0, q;\n"
+        "setp.ne.b32 q, 1, 0;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p0, [%1], %2;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%3], [%4], %5, %8, q;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%3], [%6], %7, %8, q;\n"
+        "selp.u32 %0, 1, 0, p0;\n"
+        "}\n"
+        : "=r"(r)
+        : "r"(bar), "r"(par), "r"(d_tmem), "r"(a0_tmem), "l"(b0), "r"(a1_tmem), "l"(b1), "r"(idesc)
+        : "memory");
+    return r;
+}
+
 }  // namespace ptx
 }  // namespace fa

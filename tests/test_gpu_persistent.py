@@ -91,7 +91,8 @@ def test_default_choice_by_shape():
     h = binding.fa_create()
     try:
         for (B, H, S, expect) in ((8, 32, 1024, "fa_fwd_persistent"), (1, 32, 2048, "fa_fwd_pair"),
-                                  (1, 12, 512, "fa_fwd_stream"), (1, 64, 16384, "fa_fwd_pair")):
+                                  (1, 12, 512, "fa_fwd_stream"), (1, 64, 16384, "fa_fwd_persistent"),
+                                  (1, 16, 32768, "fa_fwd_pair")):     # items of 256 K/V tiles: past the persistent kernel's range
             q = torch.zeros((B, H, S, 128), dtype=torch.bfloat16, device="cuda")
             binding.forward(h, q, q, q, causal=True)
             torch.cuda.synchronize()

@@ -14,8 +14,8 @@ def plan(w, **kw):
 
 
 def test_benchmark_configurations():
-    # (config 3: 4096 items of up to 64 K/V tiles: too long for the persistent kernel at d = 128, see test_persistent_kernel...)
-    expect = ["fa_fwd_stream", "fa_fwd_pair", "fa_fwd_pair", "fa_fwd_stream", "fa_fwd_pair"]
+    # (config 3: 4096 items of up to 64 K/V tiles, 27 per SM: the persistent kernel; config 5: items of 1024 tiles)
+    expect = ["fa_fwd_stream", "fa_fwd_pair", "fa_fwd_persistent", "fa_fwd_stream", "fa_fwd_pair"]
     for w, kernel in zip(W.CONFIGS, expect):
         p = plan(w)
         assert p["kernel"] == kernel, (w.name, p)
@@ -32,22 +32,24 @@ def test_table6_rows():
     assert got["bert_base_s2048"] == "fa_fwd_pipelined"        # 192 equal tiles would make two waves
     assert got["llama3_8b_s2048"] == "fa_fwd_pair"
     assert got["qwen15_05b_s32768"] == "fa_fwd_stream"         # d = 64 with long items
-    assert got["deepseek_67b_gqa_s4096"] == "fa_fwd_pair"        # 1024 items of up to 32 K/V tiles: past the persistent kernel's limit at d = 128
+    assert got["deepseek_67b_gqa_s4096"] == "fa_fwd_persistent"  # 1024 items of up to 32 K/V tiles, 7 per SM
 
 
 def test_persistent_kernel_from_three_items_per_sm():
     kernel = lambda B, Hq, Hkv, S, causal: binding.fa_plan(SMS, B, Hq, Hkv, S, S, 128, 128, causal)["kernel"]
-    # d = 128: the persistent kernel up to items of 8 K/V tiles (measured: 4-28 % ahead there, level at 16 tiles,
-    # 3-7 % behind the per-item kernel of fa_fwd_pair.cuh from 32 tiles on)
+    # d = 128: the persistent kernel up to items of 128 K/V tiles (measured against the per-item kernel with the same
+    # loop: 35 % ahead on 1-tile items, 9 % at 8, 3 % at 32, level at 128)
     assert kernel(4, 32, 8, 1024, True) == "fa_fwd_persistent"      # 512 items of up to 8 K/V tiles: 3.5 per SM
     assert kernel(4, 32, 32, 1024, True) == "fa_fwd_persistent"
     assert kernel(8, 32, 8, 512, True) == "fa_fwd_persistent"       # 512 items of up to 4 tiles
     assert kernel(4, 32, 8, 1024, False) == "fa_fwd_persistent"
     assert kernel(2, 32, 8, 1024, True) == "fa_fwd_pair"            # 256 items: under two per SM
-    assert kernel(2, 32, 8, 2048, True) == "fa_fwd_pair"            # items of 16 K/V tiles
-    assert kernel(4, 32, 32, 8192, True) == "fa_fwd_pair"           # items of 64 K/V tiles
-    assert kernel(1, 32, 8, 16384, True) == "fa_fwd_pair"           # items of 128 K/V tiles
-    assert binding.fa_plan(SMS, 4, 32, 32, 8192, 8192, 128, 128, True, flags=binding.FA_FLAG_LEGACY_PAIR_KERNEL)["kernel"] == "fa_fwd_pipelined"
+    assert kernel(1, 32, 8, 2048, True) == "fa_fwd_pair"            # 256 items of up to 16 K/V tiles: under two per SM
+    assert kernel(2, 32, 8, 2048, True) == "fa_fwd_persistent"      # 512 items of up to 16 K/V tiles
+    assert kernel(4, 32, 32, 8192, True) == "fa_fwd_persistent"     # items of 64 K/V tiles
+    assert kernel(1, 32, 8, 16384, True) == "fa_fwd_persistent"     # 2048 items of up to 128 K/V tiles
+    assert kernel(1, 32, 8, 32768, True) == "fa_fwd_pair"           # items of 256 K/V tiles
+    assert binding.fa_plan(SMS, 1, 32, 8, 32768, 32768, 128, 128, True, flags=binding.FA_FLAG_LEGACY_PAIR_KERNEL)["kernel"] == "fa_fwd_pipelined"
     assert binding.fa_plan(SMS, 8, 16, 16, 2048, 2048, 64, 64, True)["kernel"] == "fa_fwd_persistent"   # d = 64: up to 16 tiles
     assert binding.fa_plan(SMS, 4, 16, 16, 4096, 4096, 64, 64, True)["kernel"] == "fa_fwd_pipelined"
 
@@ -100,7 +102,7 @@ def test_flags_and_configuration_override_the_choice():
 def test_packed_batches_and_head_size_192():
     assert binding.fa_plan(SMS, 2, 16, 4, 1024, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_pair"         # 128 items
     assert binding.fa_plan(SMS, 8, 16, 4, 1024, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_persistent"   # 512 items of up to 8 K/V tiles
-    assert binding.fa_plan(SMS, 4, 16, 4, 2048, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_pair"         # 512 items of up to 16
+    assert binding.fa_plan(SMS, 4, 16, 4, 2048, 1024, 128, 128, True, varlen=True)["kernel"] == "fa_fwd_persistent"   # 512 items of up to 16
     assert binding.fa_plan(SMS, 4, 16, 4, 2048, 1024, 192, 128, True, varlen=True)["kernel"] == "fa_fwd_stream"
     assert binding.fa_plan(SMS, 1, 16, 16, 2048, 2048, 192, 128, True)["kernel"] == "fa_fwd_stream"
 
@@ -120,7 +122,8 @@ def test_packed_batches_of_many_short_sequences():
     p = plan(64, 32, 8, 128)
     assert p["kernel"] == "fa_fwd_persistent" and p["ctas"] == SMS and p["kv_splits"] == 1, p
     assert plan(8, 32, 8, 128, S=1024)["kernel"] == "fa_fwd_persistent"
-    assert plan(8, 32, 8, 128, S=2048)["kernel"] == "fa_fwd_pair"
+    assert plan(8, 32, 8, 128, S=2048)["kernel"] == "fa_fwd_persistent"
+    assert plan(1, 32, 8, 128, S=32768)["kernel"] == "fa_fwd_pair"      # items of 256 K/V tiles
     # without it: single tiles of two heads of a group share a CTA of the pair kernel
     p = plan(64, 32, 8, 128, flags=binding.FA_FLAG_NO_PERSISTENT)
     assert p["kernel"] == "fa_fwd_pair" and p["ctas"] == 64 * 16 and p["kv_splits"] == 1, p
@@ -139,3 +142,14 @@ def test_head_size_64_long_items():
     assert kernel(16384, True) == "fa_fwd_pipelined"
     assert kernel(32768, True) == "fa_fwd_stream"
     assert kernel(8192, False) == "fa_fwd_stream"
+
+
+def test_two_cta_kernel_is_used_only_where_it_applies():
+    """Head size 64, packed batches and split-KV launches stay on the other kernels when the flag is set."""
+    flags = binding.FA_FLAG_TWO_CTA_KERNEL
+    assert binding.fa_plan(148, 1, 32, 8, 2048, 2048, 128, 128, True, flags=flags)["kernel"] == "fa_fwd_duo"
+    assert binding.fa_plan(148, 1, 32, 8, 2048, 2048, 128, 128, True, flags=flags)["ctas"] == 2 * 16 * 16
+    assert binding.fa_plan(148, 1, 128, 128, 4096, 4096, 192, 128, True, flags=flags)["kernel"] == "fa_fwd_duo"
+    assert binding.fa_plan(148, 1, 16, 16, 2048, 2048, 64, 64, True, flags=flags)["kernel"] != "fa_fwd_duo"
+    assert binding.fa_plan(148, 4, 16, 4, 1024, 1024, 128, 128, True, flags=flags, varlen=True)["kernel"] != "fa_fwd_duo"
+    assert binding.fa_plan(148, 1, 32, 32, 128, 32768, 128, 128, False, flags=flags)["kernel"] != "fa_fwd_duo"   # split-KV
