@@ -47,7 +47,7 @@ PAPER_SECONDS = {"llama3_8b_gqa_s2048": 34076e-6}
 NCU_DRAM_BYTES_PER_LAUNCH = {
     "bert_base_mha_s512": 2.42e6 + 0.0,
     "llama3_8b_gqa_s2048": 25.23e6 + 0.0,
-    "llama2_7b_mha_b4_s8192": 922.56e6 + 256.61e6,
+    "llama2_7b_mha_b4_s8192": 923.00e6 + 253.69e6,
     "deepseek_v2_mha_s4096_d192_128": 579.18e6 + 124.12e6,
     "long_context_gqa_s131072": 3.14e9 + 1.06e9,
 }
@@ -517,7 +517,7 @@ def plan_ab(binding, device, gpu_index):
     import torch
     variants = (("planned", 0), ("two_tiles_per_item", binding.FA_FLAG_NO_PERSISTENT | binding.FA_FLAG_NO_STREAM_KERNEL),
                 ("persistent", binding.FA_FLAG_FORCE_PERSISTENT | binding.FA_FLAG_NO_STREAM_KERNEL),
-                ("stream", binding.FA_FLAG_STREAM_KERNEL))
+                ("stream", binding.FA_FLAG_STREAM_KERNEL), ("two_cta", binding.FA_FLAG_TWO_CTA_KERNEL))
     handles = {name: binding.fa_create(device=device.index, flags=flags) for name, flags in variants}
     cases = list(workloads.CONFIGS)
     for (B, Hq, Hkv, S, causal) in ((64, 32, 8, 128, True), (32, 32, 8, 256, True), (16, 32, 8, 512, True), (8, 32, 8, 1024, True),
