@@ -271,10 +271,17 @@ fa_status fa_plan(int num_sms, const fa_config* cfg, int varlen,
 /*
  * The same operation with HOST buffers (same layouts and types): copies Q, K, V
  * to staging memory owned by the handle, runs fa_forward, copies O (and lse if
- * not NULL) back, all on `stream`, and synchronises `stream` before returning.
- * Pinned host buffers give the full copy bandwidth; pageable ones work.  The
- * staging buffers grow on demand (device allocation on the first call and
- * whenever a larger problem arrives) and are freed by fa_destroy.
+ * not NULL) back, and synchronises `stream` before returning.  Problems of 256 MiB
+ * and more (all five tensors) are cut into up to 16 chunks of whole (batch, K/V head)
+ * units, which are independent and contiguous in every tensor: the copies of the
+ * next chunk in and of the previous chunk out run on two copy streams of the handle
+ * under the kernel of the current chunk, which runs on `stream`; work queued on
+ * `stream` before the call precedes all of it, work queued after it follows all of
+ * it.  Smaller problems go through `stream` in one piece.  Pinned host buffers give
+ * the full copy bandwidth and the overlap; pageable ones work.  The staging buffers
+ * grow on demand (device allocation on the first call and whenever a larger problem
+ * arrives; the copy streams and events are created by the first large call) and are
+ * freed by fa_destroy.
  */
 fa_status fa_forward_host(fa_handle* h,
                           const void* Q_host, const void* K_host, const void* V_host,
