@@ -37,6 +37,7 @@
 
 #include "fa_common.cuh"
 #include "fa_fwd_pipelined.cuh"
+#include "fa_softmax_pass.cuh"
 #include "ptx.cuh"
 
 namespace fa {
@@ -61,18 +62,6 @@ struct PairCfg {
 // Registers per thread after the per-role reallocation (384 threads start with 168 each):
 // 256 softmax threads x 216 + 128 other threads x 72 = 64512.
 constexpr int kPairRegsSoftmax = 216, kPairRegsOther = 72;
-// Every kEmuEvery-th pair of exponentials is computed on the FMA pipe (0 = none).
-#ifndef FA_EMU_EVERY
-#define FA_EMU_EVERY 0
-#endif
-constexpr int kEmuEvery = FA_EMU_EVERY;
-// Chunks (of 32 keys) whose exponentials are issued against the carried reference maximum while the row maximum of
-// the tile is being reduced; the check of the maximum comes behind them.
-#ifndef FA_SPEC_CHUNKS
-#define FA_SPEC_CHUNKS 1
-#endif
-constexpr int kSpecChunks = FA_SPEC_CHUNKS;
-
 struct PairShared {
     uint64_t q_full[2];
     uint64_t k_full[4], k_empty[4];
@@ -269,7 +258,6 @@ fa_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q,
         const int row = tid & (kTileM - 1);
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1) + lane_sel;
-        const uint32_t tP = tS;
         const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1) + lane_sel;
         const uint32_t bar_s = smem_addr(&sh.s_full[t]);
         const uint32_t bar_pf = smem_addr(&sh.p_first[t]);
@@ -286,153 +274,15 @@ fa_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q,
         float m_ref = -INFINITY;   // reference maximum, raw score units
         float l = 0.f;
         bool ok = true;
-        FA_PHASE_DECL();      // phases: 0 wait for S, 1 load, 2 maximum + first chunk, 3 to the first hand-off, 4 to the second, 5 row sum
+        FA_PHASE_DECL();      // phases: 0 wait for S, 5 the pass
         for (int j = 0; j < nkv_t; ++j) {
             ok = __all_sync(0xffffffffu, mbar_wait(bar_s, j & 1, wctx, kSiteSoftmaxSFull));
             if (!ok) break;
             tc_fence_after_sync();
             FA_PHASE(0);
             const int j0 = (j_base + j) * kTileN;
-            const bool need_mask = (j0 + kTileN - 1 > kmax_row);
-
-            const float2 c2 = make_float2(c, c);
-            float2 nmc2;
-            float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
-            float alpha = 1.f;
-            uint32_t s[kTileN];
-            // One exponential per score.  The MUFU pipe does 16 per cycle and SM, which for a 128 x 128 tile is as
-            // long as the tile's two MMAs, so every kEmuEvery-th pair goes to the FMA pipe instead (ptx::exp2_poly2).
-            auto exp_pair = [&](int q, int e) {
-                const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[q * 32 + e]),
-                                                        __uint_as_float(s[q * 32 + e + 1])), c2, nmc2);
-                if (kEmuEvery > 0 && ((e / 2) % (kEmuEvery > 0 ? kEmuEvery : 1)) == (kEmuEvery - 1)) {
-                    const float2 r = exp2_poly2(x);
-                    s[q * 32 + e] = __float_as_uint(r.x);
-                    s[q * 32 + e + 1] = __float_as_uint(r.y);
-                } else {
-                    s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
-                    s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
-                }
-            };
-            auto exp_chunk = [&](int q) {
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) exp_pair(q, e);
-            };
-            // bf16 conversion and store of one chunk of P (over the first half of S), row sum of the chunk
-            auto emit_chunk = [&](int q) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    const float2 v0 = make_float2(__uint_as_float(s[q * 32 + e]), __uint_as_float(s[q * 32 + e + 1]));
-                    const float2 v1 = make_float2(__uint_as_float(s[q * 32 + e + 2]), __uint_as_float(s[q * 32 + e + 3]));
-                    pk[e / 2] = pack_bf16x2(v0.x, v0.y);
-                    pk[e / 2 + 1] = pack_bf16x2(v1.x, v1.y);
-                }
-                tmem_st_x16(tP + q * 16, pk);
-            };
-            auto sum_chunk = [&](int q) {
-#pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    sum_a = fadd2_ftz(sum_a, make_float2(__uint_as_float(s[q * 32 + e]), __uint_as_float(s[q * 32 + e + 1])));
-                    sum_b = fadd2_ftz(sum_b, make_float2(__uint_as_float(s[q * 32 + e + 2]), __uint_as_float(s[q * 32 + e + 3])));
-                }
-            };
-            // The exponentials do not wait for the row maximum: they start against the reference
-            // maximum carried over from earlier tiles while the maximum of this tile is reduced.
-            // Only if some row of the warp grew past the threshold (always on the first tile, rarely
-            // afterwards) is the reference advanced and the pass repeated; nothing has been stored
-            // yet at that point, so S is still intact in TMEM.
-#pragma unroll 1
-            for (;;) {
-                tmem_ld_x32(tS + 0, s + 0);
-                tmem_ld_x32(tS + 32, s + 32);
-                tmem_ld_x32(tS + 64, s + 64);
-                tmem_ld_x32(tS + 96, s + 96);
-                tc_wait_ld();
-                FA_PHASE(1);
-                if (need_mask) {
-#pragma unroll
-                    for (int e = 0; e < kTileN; ++e)
-                        if (j0 + e > kmax_row) s[e] = 0xff800000u;   // -inf
-                }
-                const float mc = (m_ref == -INFINITY) ? 0.f : m_ref * c;
-                nmc2 = make_float2(-mc, -mc);
-                float a[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) a[q] = -INFINITY;
-#ifdef FA_MAX_INTERLEAVE
-                // Row maximum and the first kSpecChunks chunks of exponentials in one stream: per pair of exponentials,
-                // the maximum of that pair's scores (before they are overwritten) and of pairs further on, so
-                // that the reduction sits on the ALU pipe under the MUFU time instead of ahead of it.
-#pragma unroll
-                for (int q = 0; q < kSpecChunks; ++q) {
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        const int g = (e / 2) & 7;
-#pragma unroll
-                        for (int r = q; r < 4; r += kSpecChunks)
-                            a[(g + r) & 7] = fmax3(a[(g + r) & 7], __uint_as_float(s[r * 32 + e]), __uint_as_float(s[r * 32 + e + 1]));
-                        exp_pair(q, e);
-                    }
-                }
-#else
-#pragma unroll
-                for (int e = 0; e < kTileN; e += 16) {
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        a[q] = fmax3(a[q], __uint_as_float(s[e + 2 * q]), __uint_as_float(s[e + 2 * q + 1]));
-                }
-#pragma unroll
-                for (int q = 0; q < kSpecChunks; ++q) exp_chunk(q);
-#endif
-                float mx = fmaxf(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]));
-                mx = fmax3(mx, a[6], a[7]);
-                const bool grow = mx > m_ref + tau_raw;
-                if (!__any_sync(0xffffffffu, grow)) break;
-                if (grow) {
-                    alpha = exp2_approx((m_ref - mx) * c);    // r = exp(u' - u); 0 on the first tile
-                    m_ref = mx;
-                }
-            }
-            // Rare: a reference maximum of this warp's rows moved, so its rows of O_t are rescaled here.
-            // PV_t(j-1) is complete (S_t(j) could not be visible otherwise) and PV_t(j) waits for p_first.
-            if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll 1
-                for (int cc = 0; cc < DV / 32; ++cc) {
-                    uint32_t r[32];
-                    tmem_ld_x32(tO + cc * 32, r);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-                    tmem_st_x32(tO + cc * 32, reinterpret_cast<uint32_t(&)[32]>(r));
-                }
-            }
-            FA_PHASE(2);
-            if (kSpecChunks < 2) exp_chunk(1);
-            emit_chunk(0);
-            exp_chunk(2);
-            emit_chunk(1);
-            emit_chunk(2);
-            // keys 0..95 of P are stored: the MMA thread may start O += P V on them
-            tc_wait_st();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_pf);
-            FA_PHASE(3);
-            exp_chunk(3);
-            emit_chunk(3);
-            tc_wait_st();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_pr);
-            FA_PHASE(4);
-            // the row sum is off the chain: it is taken after the hand-off
-            sum_chunk(0);
-            sum_chunk(1);
-            sum_chunk(2);
-            sum_chunk(3);
-            l = l * alpha + ((sum_a.x + sum_a.y) + (sum_b.x + sum_b.y));
+            softmax_pass_128<DV>(tS, tO, c, tau_raw, j0, kmax_row, j == 0, m_ref, l, lane,
+                                 [&]() { mbar_arrive(bar_pf); }, [&]() { mbar_arrive(bar_pr); });
             FA_PHASE(5);
         }
         FA_PHASE_STORE(6, nkv_t);

@@ -182,7 +182,6 @@ fa_fwd_pair_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
         const int row = tid & (kTileM - 1);
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + (t == 0 ? Cfg::kColS0 : Cfg::kColS1) + lane_sel;
-        const uint32_t tP = tS;
         const uint32_t tO = tmem_base + (t == 0 ? Cfg::kColO0 : Cfg::kColO1) + lane_sel;
         const uint32_t bar_s = smem_addr(&sh.s_full[t]);
         const uint32_t bar_pf = smem_addr(&sh.p_first[t]);
@@ -224,107 +223,8 @@ fa_fwd_pair_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 if (!ok) break;
                 FA_PHASE(1);
                 tc_fence_after_sync();
-                const int j0 = j * kTileN;
-                const bool need_mask = (j0 + kTileN - 1 > kmax_row);
-
-                const float2 c2 = make_float2(c, c);
-                float2 nmc2;
-                float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
-                float alpha = 1.f;
-                uint32_t s[kTileN];
-                auto exp_chunk = [&](int q) {
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[q * 32 + e]),
-                                                                __uint_as_float(s[q * 32 + e + 1])), c2, nmc2);
-                        s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
-                        s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
-                    }
-                };
-                auto emit_chunk = [&](int q) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2)
-                        pk[e / 2] = pack_bf16x2(__uint_as_float(s[q * 32 + e]), __uint_as_float(s[q * 32 + e + 1]));
-                    tmem_st_x16(tP + q * 16, pk);
-                };
-                auto sum_chunk = [&](int q) {
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        sum_a = fadd2_ftz(sum_a, make_float2(__uint_as_float(s[q * 32 + e]), __uint_as_float(s[q * 32 + e + 1])));
-                        sum_b = fadd2_ftz(sum_b, make_float2(__uint_as_float(s[q * 32 + e + 2]), __uint_as_float(s[q * 32 + e + 3])));
-                    }
-                };
-                // speculative first chunk of exponentials against the carried reference maximum: see fa_fwd_pair_kernel
-#pragma unroll 1
-                for (;;) {
-                    tmem_ld_x32(tS + 0, s + 0);
-                    tmem_ld_x32(tS + 32, s + 32);
-                    tmem_ld_x32(tS + 64, s + 64);
-                    tmem_ld_x32(tS + 96, s + 96);
-                    tc_wait_ld();
-                    if (need_mask) {
-#pragma unroll
-                        for (int e = 0; e < kTileN; ++e)
-                            if (j0 + e > kmax_row) s[e] = 0xff800000u;   // -inf
-                    }
-                    const float mc = (m_ref == -INFINITY) ? 0.f : m_ref * c;
-                    nmc2 = make_float2(-mc, -mc);
-                    float a[8];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) a[q] = -INFINITY;
-#pragma unroll
-                    for (int e = 0; e < kTileN; e += 16) {
-#pragma unroll
-                        for (int q = 0; q < 8; ++q)
-                            a[q] = fmax3(a[q], __uint_as_float(s[e + 2 * q]), __uint_as_float(s[e + 2 * q + 1]));
-                    }
-                    exp_chunk(0);
-                    float mx = fmaxf(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]));
-                    mx = fmax3(mx, a[6], a[7]);
-                    const bool grow = mx > m_ref + tau_raw;
-                    if (!__any_sync(0xffffffffu, grow)) break;
-                    if (grow) {
-                        alpha = exp2_approx((m_ref - mx) * c);    // r = exp(u' - u); 0 on the first tile
-                        m_ref = mx;
-                    }
-                }
-                // Rare: a reference maximum of this warp's rows moved, so its rows of O_t are rescaled here.
-                // PV_t(j-1) is complete (S_t(j) could not be visible otherwise) and PV_t(j) waits for p_first.
-                if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll 1
-                    for (int cc = 0; cc < DV / 32; ++cc) {
-                        uint32_t r[32];
-                        tmem_ld_x32(tO + cc * 32, r);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-                        tmem_st_x32(tO + cc * 32, reinterpret_cast<uint32_t(&)[32]>(r));
-                    }
-                }
-                exp_chunk(1);
-                emit_chunk(0);
-                exp_chunk(2);
-                emit_chunk(1);
-                emit_chunk(2);
-                // keys 0..95 of P are stored: the MMA thread may start O += P V on them
-                tc_wait_st();
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_pf);
-                exp_chunk(3);
-                emit_chunk(3);
-                tc_wait_st();
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_pr);
-                // the row sum is off the chain: it is taken after the hand-off
-                sum_chunk(0);
-                sum_chunk(1);
-                sum_chunk(2);
-                sum_chunk(3);
-                l = l * alpha + ((sum_a.x + sum_a.y) + (sum_b.x + sum_b.y));
+                softmax_pass_128<DV>(tS, tO, c, tau_raw, j * kTileN, kmax_row, j == 0, m_ref, l, lane,
+                                     [&]() { mbar_arrive(bar_pf); }, [&]() { mbar_arrive(bar_pr); });
                 FA_PHASE(2);
             }
             if (!ok) break;
