@@ -247,6 +247,33 @@ fa_status fa_forward_fp8(fa_handle* h,
                          int causal, float scale, void* stream);
 
 /*
+ * MX form of the 8-bit variant (microscaling: the closest counterpart on this GPU of a block
+ * floating-point format, Section 3 / Table 1 of the paper): e4m3 values with one e8m0 scale
+ * 2^(byte - 127) per 32 elements ALONG EACH CONTRACTION, applied inside the tensor-core instruction
+ * (tcgen05.mma kind::mxf8f6f4 with block scaling).  Q8, K8, V8 as for fa_forward_fp8.  The
+ * represented tensors are
+ *   Q[b,h,i,c] = 2^(eq - 127) * Q8[b,h,i,c]   eq = scale of (row i, columns 32*(c/32) .. +31)
+ *   K[b,h,j,c] = 2^(ek - 127) * K8[b,h,j,c]   ek = scale of (key j, columns 32*(c/32) .. +31)
+ *   V[b,h,j,c] = 2^(ev - 127) * V8[b,h,j,c]   ev = scale of (column c, keys 32*(j/32) .. +31)
+ * and the scales are passed in the layout the tensor core reads them in, one 512-byte atom per
+ * 128-row tile (DEVICE memory, 16-byte aligned, uint8):
+ *   q_sf [B, Hq,  ceil(Sq/128), 512]   byte (r%32)*16 + (r/32)*4 + kb : row 128*t + r, column block kb
+ *   k_sf [B, Hkv, ceil(Sk/128), 512]   byte (r%32)*16 + (r/32)*4 + kb : key 128*t + r, column block kb
+ *   v_sf [B, Hkv, ceil(Sk/128), 512]   byte (c%32)*16 + (c/32)*4 + kb : column c, keys 128*t + 32*kb .. +31
+ * (d = 64 uses kb = 0, 1 of Q and K and c < 64 of V; unused bytes, and those of rows past the end
+ * of a tensor, must still be valid scales, e.g. 127: 255 is NaN.)  The probabilities are rounded to
+ * e4m3 with scale 1 before the second contraction, as in fa_forward_fp8.  Runs on the stream tiling
+ * (one head per query tile, split-KV where the plan wants it).  O, lse, other arguments and errors
+ * as for fa_forward_fp8.
+ */
+fa_status fa_forward_mxfp8(fa_handle* h,
+                           const void* Q8, const void* K8, const void* V8,
+                           const uint8_t* q_sf, const uint8_t* k_sf, const uint8_t* v_sf,
+                           void* O, float* lse,
+                           int B, int Hq, int Hkv, int Sq, int Sk, int d,
+                           int causal, float scale, void* stream);
+
+/*
  * What the library would launch for a problem: which kernel (tiling), how many K/V splits, how
  * many CTAs, and the two run-time estimates behind the choice (0 when none was needed).  A pure
  * host function: no handle, no device, no CUDA call; `num_sms` is the SM count to plan for (148 on

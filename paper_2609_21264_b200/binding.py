@@ -31,7 +31,7 @@ FA_FLAG_NO_HEAD_PACKING = 128
 FA_FLAG_LEGACY_PAIR_KERNEL = 256
 FA_FLAG_TWO_CTA_KERNEL = 512
 
-EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_varlen", "fa_forward_fp8", "fa_plan", "fa_forward_host", "fa_last_status", "fa_destroy",
+EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_varlen", "fa_forward_fp8", "fa_forward_mxfp8", "fa_plan", "fa_forward_host", "fa_last_status", "fa_destroy",
            "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits",
            "fa_forward_split_noalloc", "fa_noalloc_scratch_bytes", "fa_noalloc_last_status", "fa_debug_set_drop_v_load")
 
@@ -84,6 +84,8 @@ def load():
     lib.fa_plan.argtypes = [i32, ctypes.POINTER(fa_config), i32] + [i32] * 8 + [ctypes.POINTER(fa_plan_info)]
     lib.fa_forward_fp8.restype = i32
     lib.fa_forward_fp8.argtypes = [vp] * 9 + [i32] * 7 + [f32, vp]
+    lib.fa_forward_mxfp8.restype = i32
+    lib.fa_forward_mxfp8.argtypes = [vp] * 9 + [i32] * 7 + [f32, vp]
     lib.fa_forward_strided.restype = i32
     lib.fa_forward_strided.argtypes = fwd_args[:-1] + [vp, vp, vp, vp, vp]
     lib.fa_last_status.restype = i32
@@ -305,4 +307,33 @@ def forward_fp8(h, q8, k8, v8, q_scale, k_scale, v_scale, *, causal: bool, scale
                         torch.cuda.current_stream(q8.device).cuda_stream)
     if st != FA_OK:
         raise FaError(st, "fa_forward_fp8")
+    return out, lse
+
+
+def fa_forward_mxfp8(h, Q8, K8, V8, q_sf, k_sf, v_sf, O, lse, B, Hq, Hkv, Sq, Sk, d, causal, scale, stream=0) -> int:
+    """Raw call of the MX form (e4m3 values, e8m0 scale atoms); device pointers as integers; returns the status code."""
+    return load().fa_forward_mxfp8(h, Q8, K8, V8, q_sf, k_sf, v_sf, O, lse, B, Hq, Hkv, Sq, Sk, d,
+                                   int(bool(causal)), float(scale), stream)
+
+
+def forward_mxfp8(h, q8, k8, v8, q_sf, k_sf, v_sf, *, causal: bool, scale: float = 0.0, want_lse=True):
+    """MX attention on torch CUDA tensors: q8/k8/v8 uint8 [B,H,S,d] with d = 64 or 128, scale atoms uint8
+    [B,H,ceil(S/128),512] in the layout of fa_forward_mxfp8.  Returns (O bf16 [B,Hq,Sq,d], lse fp32 [B,Hq,Sq])."""
+    import torch
+    for t in (q8, k8, v8, q_sf, k_sf, v_sf):
+        if t.element_size() != 1 or not t.is_cuda or not t.is_contiguous() or t.dim() != 4:
+            raise ValueError("codes and scale atoms must be contiguous 4-D one-byte CUDA tensors")
+    B, Hq, Sq, d = q8.shape
+    _, Hkv, Sk, _ = k8.shape
+    n_qt, n_kt = (Sq + 127) // 128, (Sk + 127) // 128
+    for t, shape in ((q_sf, (B, Hq, n_qt, 512)), (k_sf, (B, Hkv, n_kt, 512)), (v_sf, (B, Hkv, n_kt, 512))):
+        if tuple(t.shape) != shape:
+            raise ValueError("scale atoms must have shape %s" % (shape,))
+    out = torch.empty((B, Hq, Sq, d), dtype=torch.bfloat16, device=q8.device)
+    lse = torch.empty((B, Hq, Sq), dtype=torch.float32, device=q8.device) if want_lse else None
+    st = fa_forward_mxfp8(h, q8.data_ptr(), k8.data_ptr(), v8.data_ptr(), q_sf.data_ptr(), k_sf.data_ptr(), v_sf.data_ptr(),
+                          out.data_ptr(), lse.data_ptr() if lse is not None else None, B, Hq, Hkv, Sq, Sk, d, causal, scale,
+                          torch.cuda.current_stream(q8.device).cuda_stream)
+    if st != FA_OK:
+        raise FaError(st, "fa_forward_mxfp8")
     return out, lse

@@ -936,16 +936,21 @@ fa_status fa_forward_varlen(fa_handle* h, const void* Q, const void* K, const vo
                        cu_seqlens_q, cu_seqlens_k, total_q, pl, st);
 }
 
-fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const void* V8,
-                         const float* q_scale, const float* k_scale, const float* v_scale,
-                         void* O, float* lse, int B, int Hq, int Hkv, int Sq, int Sk, int d, int causal,
-                         float scale, void* stream) {
+// Both 8-bit entry points: fp32 scales per 128-row block (q_scale, k_scale, v_scale; each may be NULL), or, with
+// q_sf != NULL, the MX form with e8m0 scale atoms (q_sf, k_sf, v_sf).
+static fa_status forward_fp8_common(fa_handle* h, const void* Q8, const void* K8, const void* V8,
+                                    const float* q_scale, const float* k_scale, const float* v_scale,
+                                    const uint8_t* q_sf, const uint8_t* k_sf, const uint8_t* v_sf,
+                                    void* O, float* lse, int B, int Hq, int Hkv, int Sq, int Sk, int d, int causal,
+                                    float scale, void* stream) {
     if (!h) return FA_ERR_INVALID_ARG;
     if (d != 64 && d != 128) return (d > 0) ? FA_ERR_UNSUPPORTED : FA_ERR_INVALID_ARG;
+    const bool mx = q_sf != nullptr;
     fa_status s = check_args(Q8, K8, V8, O, lse, B, Hq, Hkv, Sq, Sk, d, d, scale, true);
     if (s != FA_OK) return s;
     if ((q_scale && misaligned(q_scale, 4)) || (k_scale && misaligned(k_scale, 4)) || (v_scale && misaligned(v_scale, 4)))
         return FA_ERR_INVALID_ARG;
+    if (mx && (!k_sf || !v_sf || misaligned(q_sf, 16) || misaligned(k_sf, 16) || misaligned(v_sf, 16))) return FA_ERR_INVALID_ARG;
     if (h->flags & FA_FLAG_SERIAL_KERNEL) return FA_ERR_UNSUPPORTED;
     DeviceGuard guard(h->device);
     if (!guard.ok()) return FA_ERR_CUDA;
@@ -955,7 +960,11 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     // The tiling is planned as for 16-bit operands of the same shape (the 8-bit kernels' per-CTA
     // costs are lower by a similar factor in both tilings).  Only the stream tiling splits K/V
     // and packs heads.
-    const LaunchPlan pl = plan_launch(h->num_sms, h->flags, h->kv_splits_cfg, h->scratch_bytes, false,
+    // (The MX form runs on the stream tiling with one head per query tile: its scale atoms follow the tile's rows.)
+    const uint32_t plan_flags = mx ? ((h->flags & ~(FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_FORCE_PERSISTENT | FA_FLAG_TWO_CTA_KERNEL)) |
+                                      FA_FLAG_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)
+                                   : h->flags;
+    const LaunchPlan pl = plan_launch(h->num_sms, plan_flags, h->kv_splits_cfg, h->scratch_bytes, false,
                                       B, Hq, Hkv, Sq, Sk, d, d, causal ? 1 : 0);
     const int q_box_rows = pl.pack_heads > 1 ? Sq : fa::kTileM;
     // an e4m3 row is d bytes: one box column of d bytes, swizzled over d bytes
@@ -987,6 +996,7 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     p.debug_drop_v_load = (h->flags & FA_FLAG_DEBUG_DROP_V_LOAD) ? 1 : 0;
     fa::Fp8Params f;
     f.q_scale = q_scale; f.k_scale = k_scale; f.v_scale = v_scale;
+    f.q_sf = q_sf; f.k_sf = k_sf; f.v_sf = v_sf;
     f.n_kv_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;
     const bool use_stream = pl.kernel == kPlanStream;
     p.kv_splits = use_stream ? pl.kv_splits : 1;
@@ -1010,7 +1020,8 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
         p.lse_part = p.o_part + static_cast<size_t>(n_partials) * B * Hq * Sq * d;
     }
     h->last_splits = p.kv_splits;
-    h->last_kernel = use_stream ? "fa_fwd_fp8_stream" : "fa_fwd_fp8";
+    h->last_kernel = use_stream ? (mx ? "fa_fwd_mxfp8_stream" : "fa_fwd_fp8_stream") : "fa_fwd_fp8";
+    if (mx && !use_stream) return FA_ERR_UNSUPPORTED;       // (cannot happen: the stream tiling was forced above)
 
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -1034,6 +1045,7 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
             {fa::fa_fwd_fp8_stream_kernel<128, false, 1>, fa::fa_fwd_fp8_stream_kernel<128, true, 1>,
              fa::fa_fwd_fp8_stream_kernel<128, true, 2>, fa::fa_fwd_fp8_stream_kernel<128, true, 4>}};
         Kernel kernel = kernels[d128 ? 1 : 0][variant];
+        if (mx) kernel = d128 ? fa::fa_fwd_fp8_stream_kernel<128, false, 1, true> : fa::fa_fwd_fp8_stream_kernel<64, false, 1, true>;
         if ((s = ensure_smem_attr(h, kernel, smem)) != FA_OK) return s;
         const long long n_ctas = (pack ? static_cast<long long>(Hq / pl.pack_heads) : static_cast<long long>(p.n_q_tiles) * Hq) * B * p.kv_splits;
         if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
@@ -1070,6 +1082,23 @@ fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const voi
     if (cudaLaunchKernelEx(&cfg, kernel, map_q, map_k, map_v, map_o, p, f) != cudaSuccess) return FA_ERR_CUDA;
     h->launches += 1;
     return FA_OK;
+}
+
+fa_status fa_forward_fp8(fa_handle* h, const void* Q8, const void* K8, const void* V8,
+                         const float* q_scale, const float* k_scale, const float* v_scale,
+                         void* O, float* lse, int B, int Hq, int Hkv, int Sq, int Sk, int d, int causal,
+                         float scale, void* stream) {
+    return forward_fp8_common(h, Q8, K8, V8, q_scale, k_scale, v_scale, nullptr, nullptr, nullptr, O, lse, B, Hq, Hkv, Sq, Sk, d,
+                              causal, scale, stream);
+}
+
+fa_status fa_forward_mxfp8(fa_handle* h, const void* Q8, const void* K8, const void* V8,
+                           const uint8_t* q_sf, const uint8_t* k_sf, const uint8_t* v_sf,
+                           void* O, float* lse, int B, int Hq, int Hkv, int Sq, int Sk, int d, int causal,
+                           float scale, void* stream) {
+    if (!q_sf || !k_sf || !v_sf) return FA_ERR_INVALID_ARG;
+    return forward_fp8_common(h, Q8, K8, V8, nullptr, nullptr, nullptr, q_sf, k_sf, v_sf, O, lse, B, Hq, Hkv, Sq, Sk, d,
+                              causal, scale, stream);
 }
 
 fa_status fa_plan(int num_sms, const fa_config* cfg, int varlen, int B, int Hq, int Hkv, int Sq, int Sk, int dqk, int dv,

@@ -54,6 +54,11 @@ struct Fp8Params {
     const float* k_scale;    // [B, Hkv, n_kv_tiles] or nullptr
     const float* v_scale;    // [B, Hkv] or nullptr
     int n_kv_tiles;          // ceil(Sk / 128)
+    // MX variant (e8m0 scales per 32 elements along the contraction; fa_fwd_fp8_stream_kernel with kMx): one
+    // 512-byte scale atom per 128-row tile, byte (r % 32) * 16 + (r / 32) * 4 + kb
+    const uint8_t* q_sf;     // [B, Hq, n_q_tiles, 512]: row r of the query tile, block kb of its d columns
+    const uint8_t* k_sf;     // [B, Hkv, n_kv_tiles, 512]: key r of the K tile, block kb of its d columns
+    const uint8_t* v_sf;     // [B, Hkv, n_kv_tiles, 512]: column r of V, block kb of the tile's 128 keys
 };
 
 template <int D>

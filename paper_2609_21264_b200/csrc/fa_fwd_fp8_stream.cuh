@@ -8,6 +8,15 @@
 // the stream tiling is planned: grids under a wave and decode-like shapes with split-KV
 // (attention over an 8-bit K/V cache).  Head sizes 64 and 128, fixed-length contiguous tensors.
 //   TMEM  S^0 [0,128)  S^1 [128,256)  O [256,384)  P^0 [384,416)  P^1 [448,480)
+//
+// kMx: the MX form of the operands (the closest counterpart of a block floating point format on this GPU): e4m3
+// codes with one e8m0 scale per 32 elements ALONG THE CONTRACTION, for Q and K per row and block of the head
+// dimension, for V per column and block of 32 keys, applied inside tcgen05.mma kind::mxf8f6f4.block_scale.
+// Nothing is folded into the exp2 constant then.  The scales of a 128-row tile arrive as one 512-byte atom next
+// to the tile (a plain bulk copy on the tile's mbarrier) and go from shared memory to TMEM columns
+// [416,440) with tcgen05.cp, issued by the MMA thread that uses them, just ahead of the tile's MMAs; P is
+// rounded to e4m3 as before and carries the scale 1 (one constant atom).
+//   TMEM  scales: Q [416,420)  K^0 [420,424)  K^1 [424,428)  P [428,432)  V^0 [432,436)  V^1 [436,440)
 #pragma once
 
 #include "fa_fwd_fp8.cuh"
@@ -22,7 +31,10 @@ struct Fp8StreamCfg {
     static constexpr int kOBytes = (D / kChunkCols) * kChunkBytes;      // bf16 output tile
     static constexpr int kKStages = 4;
     static constexpr int kVStages = 4;
-    static constexpr int kTileBytes = (1 + kKStages + kVStages) * kTile8 + kOBytes;
+    static constexpr int kSfAtom = 512;                  // scales of one 128-row tile (MX variant)
+    static constexpr int kSfBytes = (2 + kKStages + kVStages) * kSfAtom;     // Q, P (constant), K and V stages
+    static constexpr int kTileBytes = (1 + kKStages + kVStages) * kTile8 + kOBytes + kSfBytes;
+    static constexpr int kColSf = 416;
     static constexpr int kTmemCols = 512;
     static constexpr int kColS = 0, kColO = 256, kColP = 384;   // P^b at kColP + 64 b (32 columns used)
 };
@@ -40,7 +52,7 @@ constexpr int fp8_stream_smem_bytes() { return Fp8StreamCfg<D>::kTileBytes + sta
 // partials.  A softmax warp then issues 1 / kRep of the exponentials per K/V tile (an
 // instruction costs the same for one live row as for 32), which takes a few-row problem from the
 // MUFU bound to the bound of the K/V stream.
-template <int D, bool kPack = false, int kRep = 1>
+template <int D, bool kPack = false, int kRep = 1, bool kMx = false>
 __global__ void __launch_bounds__(512, 1)
 fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                      const __grid_constant__ CUtensorMap tm_k,
@@ -51,6 +63,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     constexpr int DV = Cfg::kD;
     constexpr int kTile8 = Cfg::kTile8;
     static_assert(kRep == 1 || (kPack && (kRep == 2 || kRep == 4)), "copies of the query rows need packed heads");
+    static_assert(!kMx || !kPack, "the MX variant has no packed heads (its scale atoms follow the query tile's rows)");
     constexpr int kRepRows = kTileM / kRep;      // rows of one copy of the pack
     constexpr int kCols = kTileN / kRep;         // keys of a K/V tile that one copy takes
     constexpr int kChunks = kCols / 32;
@@ -82,6 +95,10 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     const uint32_t sK = sQ + kTile8;
     const uint32_t sV = sK + NK * kTile8;
     const uint32_t sStage = sV + NV * kTile8;      // the bf16 output tile passes through here
+    const uint32_t sSfQ = sStage + Cfg::kOBytes;   // scale atoms (MX variant): Q, P, K stages, V stages
+    const uint32_t sSfP = sSfQ + Cfg::kSfAtom;
+    const uint32_t sSfK = sSfP + Cfg::kSfAtom;
+    const uint32_t sSfV = sSfK + NK * Cfg::kSfAtom;
 
     // 1-D grid: L2-sized groups of (batch, head) instances one after the other; inside a group
     // every head's last (with a causal mask: heaviest) query tile first.
@@ -152,6 +169,11 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         prefetch_tensormap(&tm_v);
         prefetch_tensormap(&tm_o);
     }
+    if constexpr (kMx) {
+        // P carries the scale 1 = 2^(127 - 127) in every block
+        if (tid < Cfg::kSfAtom / 16) st_shared_v4(sSfP + tid * 16, 0x7f7f7f7fu, 0x7f7f7f7fu, 0x7f7f7f7fu, 0x7f7f7f7fu);
+        fence_proxy_async_smem();
+    }
     if constexpr (kPack) {
         // the rows of the query tile past the pack's last row are never loaded: zero scores there
         for (int o = tid * 16; o < kTile8; o += 512 * 16) st_shared_v4(sQ + o, 0u, 0u, 0u, 0u);
@@ -193,8 +215,9 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         int kmax_row = Sk - 1;
         if (p.causal && i_glob + off < kmax_row) kmax_row = i_glob + off;
         // scale * log2 e * (scale of this query tile); the key tile's scale joins per tile
-        const float cq = p.scale_log2 * ((f.q_scale && row_valid) ? __ldg(f.q_scale + static_cast<size_t>(q_idx) * p.n_q_tiles + q_tile) : 1.f);
-        const float* k_scale = f.k_scale ? f.k_scale + static_cast<size_t>(kv_idx) * f.n_kv_tiles + j_base : nullptr;
+        // (MX variant: the scales are applied inside the MMAs)
+        const float cq = p.scale_log2 * ((!kMx && f.q_scale && row_valid) ? __ldg(f.q_scale + static_cast<size_t>(q_idx) * p.n_q_tiles + q_tile) : 1.f);
+        const float* k_scale = (!kMx && f.k_scale) ? f.k_scale + static_cast<size_t>(kv_idx) * f.n_kv_tiles + j_base : nullptr;
 
         if constexpr (kRep > 1) {
             // the columns of P^g that belong to the other copies' keys are never written: zero once
@@ -349,7 +372,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                     tc_fence_after_sync();
                     const float lt = sh.lsum[0][row] + sh.lsum[1][row];
                     const float m_fin = sh.mref[row];
-                    const float sv = f.v_scale ? __ldg(f.v_scale + kv_idx) : 1.f;
+                    const float sv = (!kMx && f.v_scale) ? __ldg(f.v_scale + kv_idx) : 1.f;
                     const float inv_l = (lt > 0.f) ? (sv / lt) : 0.f;
                     if (g == 0 && p.lse && row_valid && !partial_out)
                         p.lse[lse_row0 + i_glob] = (lt > 0.f) ? (m_fin * 0.6931471805599453f + logf(lt)) : -INFINITY;
@@ -452,6 +475,12 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
             auto desc = [](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(kDescHi) << 32) | lo; };
             bool ok = mbar_wait(smem_addr(&sh.q_full), 0, wctx, kSiteMmaQFull);
+            if constexpr (kMx) {
+                if (ok) {
+                    tc_fence_after_sync();
+                    tmem_cp_scales_32x16B(tmem_base + Cfg::kColSf, sSfQ);
+                }
+            }
             int sk = 0;
             uint32_t ph_k = 0;
             for (int j = 0; j < n_kv && ok; ++j) {
@@ -462,9 +491,18 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 tc_fence_after_sync();
                 const uint32_t tS = tmem_base + Cfg::kColS + (j & 1) * 128;
                 const uint32_t klo = k_lo0 + sk * (kTile8 >> 4);
+                if constexpr (kMx) {
+                    const uint32_t tSfK = tmem_base + Cfg::kColSf + 4 + (j & 1) * 4;
+                    tmem_cp_scales_32x16B(tSfK, sSfK + sk * Cfg::kSfAtom);
 #pragma unroll
-                for (int kk = 0; kk < Cfg::kD / 32; ++kk)      // k-steps of 32 elements = 32 bytes
-                    mma_ss_f8(tS, desc(q_lo + kk * 2), desc(klo + kk * 2), kIdescQK, kk > 0 ? 1u : 0u);
+                    for (int kk = 0; kk < Cfg::kD / 32; ++kk)      // K block kk of Q's rows and of K's rows
+                        mma_ss_mx(tS, desc(q_lo + kk * 2), desc(klo + kk * 2), make_idesc_mx_e4m3(kTileM, kTileN, false, kk, kk),
+                                  tmem_base + Cfg::kColSf, tSfK, kk > 0 ? 1u : 0u);
+                } else {
+#pragma unroll
+                    for (int kk = 0; kk < Cfg::kD / 32; ++kk)      // k-steps of 32 elements = 32 bytes
+                        mma_ss_f8(tS, desc(q_lo + kk * 2), desc(klo + kk * 2), kIdescQK, kk > 0 ? 1u : 0u);
+                }
                 tc_commit(smem_addr(&sh.s_full[j & 1]));
                 tc_commit(smem_addr(&sh.k_empty[sk]));
                 if (++sk == NK) { sk = 0; ph_k ^= 1u; }
@@ -482,6 +520,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             int sv = 0;
             uint32_t ph_v = 0;
             bool ok = true;
+            if constexpr (kMx) tmem_cp_scales_32x16B(tmem_base + Cfg::kColSf + 12, sSfP);     // (written before the set-up barrier)
             for (int j = 0; j < n_kv && ok; ++j) {
                 const uint32_t use = static_cast<uint32_t>(j >> 1);
                 ok = mbar_wait(smem_addr(&sh.v_full[sv]), ph_v, wctx, kSiteMmaKvFull);
@@ -490,9 +529,18 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 tc_fence_after_sync();
                 const uint32_t tP = tmem_base + Cfg::kColP + (j & 1) * 64;
                 const uint32_t vlo = v_lo0 + sv * (kTile8 >> 4);
+                if constexpr (kMx) {
+                    const uint32_t tSfV = tmem_base + Cfg::kColSf + 16 + (j & 1) * 4;
+                    tmem_cp_scales_32x16B(tSfV, sSfV + sv * Cfg::kSfAtom);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)                  // four k-steps of 32 keys: 8 P columns, 32 V rows of D bytes
-                    mma_ts_f8(tO, tP + kk * 8, desc(vlo + kk * Fp8Cfg<D>::kVStep), kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < 4; ++kk)              // block kk of the tile's keys: P's scale (1) and V's per column
+                        mma_ts_mx(tO, tP + kk * 8, desc(vlo + kk * Fp8Cfg<D>::kVStep), make_idesc_mx_e4m3(kTileM, DV, true, kk, kk),
+                                  tmem_base + Cfg::kColSf + 12, tSfV, (j > 0 || kk > 0) ? 1u : 0u);
+                } else {
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)              // four k-steps of 32 keys: 8 P columns, 32 V rows of D bytes
+                        mma_ts_f8(tO, tP + kk * 8, desc(vlo + kk * Fp8Cfg<D>::kVStep), kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+                }
                 tc_commit(smem_addr(&sh.p_free[j & 1]));
                 tc_commit(smem_addr(&sh.v_empty[sv]));
                 if (j + 1 == n_kv) tc_commit(smem_addr(&sh.o_final));
@@ -509,9 +557,12 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
             {
                 const uint32_t bar = smem_addr(&sh.q_full);
                 // with packed heads the box is Sq rows x pack_heads heads (row h * Sq + i of the tile)
-                mbar_arrive_expect_tx(bar, kPack ? static_cast<uint32_t>(kRep * p.pack_heads * Sq * D) : static_cast<uint32_t>(kTile8));
+                mbar_arrive_expect_tx(bar, (kPack ? static_cast<uint32_t>(kRep * p.pack_heads * Sq * D) : static_cast<uint32_t>(kTile8)) +
+                                               (kMx ? Cfg::kSfAtom : 0));
 #pragma unroll
                 for (int r = 0; r < kRep; ++r) tma_load_4d(sQ + r * kRepRows * D, &tm_q, bar, 0, i0, hq, b);
+                if constexpr (kMx)
+                    bulk_load_1d(sSfQ, f.q_sf + (static_cast<size_t>(b * p.Hq + hq) * p.n_q_tiles + q_tile) * Cfg::kSfAtom, Cfg::kSfAtom, bar);
             }
             bool ok = true;
             for (int j = 0; j < n_kv && ok; ++j) {
@@ -519,8 +570,11 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 ok = mbar_wait(smem_addr(&sh.k_empty[s]), ((j / NK) & 1) ^ 1, wctx, kSiteLoadKvEmpty);
                 if (!ok) break;
                 const uint32_t bar = smem_addr(&sh.k_full[s]);
-                mbar_arrive_expect_tx(bar, kTile8);
+                mbar_arrive_expect_tx(bar, kTile8 + (kMx ? Cfg::kSfAtom : 0));
                 tma_load_4d(sK + s * kTile8, &tm_k, bar, 0, (j_base + j) * kTileN, kvh, b);
+                if constexpr (kMx)
+                    bulk_load_1d(sSfK + s * Cfg::kSfAtom, f.k_sf + (static_cast<size_t>(kv_idx) * f.n_kv_tiles + j_base + j) * Cfg::kSfAtom,
+                                 Cfg::kSfAtom, bar);
             }
         }
     } else {
@@ -534,8 +588,11 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 ok = mbar_wait(smem_addr(&sh.v_empty[s]), ((j / NV) & 1) ^ 1, wctx, kSiteLoadKvEmpty);
                 if (!ok) break;
                 const uint32_t bar = smem_addr(&sh.v_full[s]);
-                mbar_arrive_expect_tx(bar, kTile8);
+                mbar_arrive_expect_tx(bar, kTile8 + (kMx ? Cfg::kSfAtom : 0));
                 tma_load_4d(sV + s * kTile8, &tm_v, bar, 0, (j_base + j) * kTileN, kvh, b);
+                if constexpr (kMx)
+                    bulk_load_1d(sSfV + s * Cfg::kSfAtom, f.v_sf + (static_cast<size_t>(kv_idx) * f.n_kv_tiles + j_base + j) * Cfg::kSfAtom,
+                                 Cfg::kSfAtom, bar);
             }
         }
     }

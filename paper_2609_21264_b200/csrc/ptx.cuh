@@ -383,6 +383,60 @@ FA_DEVI void mma_ts_f8(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32
         : "memory");
 }
 
+// Block-scaled 8-bit operands (kind::mxf8f6f4.block_scale): e4m3 data with one e8m0 scale (2^(byte - 127)) per
+// 32 elements along K, for every row of A and every column of B; one instruction covers K = 32, i.e. one scale
+// per row / column.  The scales sit in TMEM: a 128-row (or 128-column) operand takes 4 columns; lane l of every
+// 32-lane quadrant holds, in column g and byte kb, the scale of row l % 32 + 32 g for K block kb, and the
+// instruction descriptor names the byte (make_idesc_mx_e4m3's sf ids).  They get there from shared memory with
+// tcgen05.cp 32x128b.warpx4 (32 rows of 16 bytes, replicated to the four quadrants), source bytes at
+// (r % 32) * 16 + (r / 32) * 4 + kb.  Probed bit-exact on B200 with exactly representable data, both with A
+// from shared memory and with A from TMEM and an MN-major B.
+//   bits [4,6) B scale id   [7,10) A format (0 = e4m3)   [10,13) B format   15 / 16 A / B major
+//   [17,23) N >> 3   23 scale format (1 = e8m0)   [24,29) M >> 4   [29,31) A scale id
+__host__ __device__ constexpr uint32_t make_idesc_mx_e4m3(int m, int n, bool b_mn_major, uint32_t a_sf_id, uint32_t b_sf_id) {
+    return (b_sf_id << 4) | ((b_mn_major ? 1u : 0u) << 16) | (static_cast<uint32_t>(n >> 3) << 17) | (1u << 23) |
+           (static_cast<uint32_t>(m >> 4) << 24) | (a_sf_id << 29);
+}
+FA_DEVI void mma_ss_mx(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t sfa_tmem, uint32_t sfb_tmem,
+                       uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+        : "memory");
+}
+FA_DEVI void mma_ts_mx(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t sfa_tmem, uint32_t sfb_tmem,
+                       uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], [%1], %2, %3, [%5], [%6], p;\n"
+        "}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+        : "memory");
+}
+// 32 rows x 16 bytes from shared memory into 4 TMEM columns of all four lane quadrants; issued by ONE thread, in
+// order with that thread's MMAs (and covered by its next tcgen05.commit).  The source is described like a K-major
+// MMA operand without swizzle: 8-row x 16-byte core matrices 128 bytes apart.
+FA_DEVI void tmem_cp_scales_32x16B(uint32_t taddr, uint32_t saddr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>(16u >> 4) << 16;
+    d |= static_cast<uint64_t>(128u >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(d) : "memory");
+}
+// Plain (untiled) bulk copy global -> shared with completion on an mbarrier; both addresses 16-byte aligned,
+// size a multiple of 16.
+FA_DEVI void bulk_load_1d(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
+}
+
 // D[tmem] (+)= A[tmem] * B[smem]; A holds bf16 pairs packed in 32-bit columns.
 FA_DEVI void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                     uint32_t accumulate) {

@@ -172,3 +172,60 @@ def quantize_e4m3_blocks(x: np.ndarray, block_rows: int | None):
     codes = (xt / per_row).to(torch.float32).to(torch.float8_e4m3fn)
     deq = codes.to(torch.float64) * per_row
     return codes.view(torch.uint8).numpy(), scales.numpy(), deq.numpy()
+
+
+def quantize_mx_e4m3(x: np.ndarray, along: str):
+    """MX (microscaling) e4m3 form of a [B, H, S, d] float array: one e8m0 scale 2^(e - 127) per block of 32
+    elements, along the columns of a row (`along="cols"`: Q and K, whose contraction runs over d) or along the rows
+    of a column (`along="rows"`: V, whose contraction runs over the keys).
+
+    The scale of a block is the smallest power of two with amax / scale <= 448 (the largest e4m3 value; 2^0 for an
+    all-zero block), so nothing saturates; the codes are x / scale rounded to nearest-even e4m3.  Returns (codes uint8 [B,H,S,d],
+    exponent bytes uint8 [B,H,S,d/32] or [B,H,ceil(S/32),d], dequantised float64 [B,H,S,d] = codes * scale exactly).
+    """
+    import torch
+    B, H, S, d = x.shape
+    xt = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float64))
+    if along == "cols":
+        blocks = xt.view(B, H, S, d // 32, 32)
+        amax = blocks.abs().amax(dim=4)                                       # [B,H,S,d/32]
+    elif along == "rows":
+        nb = (S + 31) // 32
+        xp = torch.nn.functional.pad(xt, (0, 0, 0, nb * 32 - S))
+        amax = xp.view(B, H, nb, 32, d).abs().amax(dim=3)                     # [B,H,nb,d]
+    else:
+        raise ValueError(along)
+    e = torch.where(amax > 0, torch.ceil(torch.log2(torch.clamp(amax, min=1e-300) / 448.0)), torch.zeros_like(amax))
+    e = torch.clamp(e, -127.0, 127.0)
+    scale = torch.pow(torch.tensor(2.0, dtype=torch.float64), e)
+    if along == "cols":
+        per_elem = scale.repeat_interleave(32, dim=3)                         # [B,H,S,d]
+    else:
+        per_elem = scale.repeat_interleave(32, dim=2)[:, :, :S, :]
+    q = torch.clamp(xt / per_elem, -448.0, 448.0)
+    codes = q.to(torch.float32).to(torch.float8_e4m3fn)
+    deq = codes.to(torch.float64) * per_elem
+    return codes.view(torch.uint8).numpy(), (e + 127.0).to(torch.uint8).numpy(), deq.numpy()
+
+
+def mx_scale_atoms(exps: np.ndarray, along: str, S: int) -> np.ndarray:
+    """The exponent bytes of quantize_mx_e4m3 in the layout the tensor core reads: one 512-byte atom per 128-row
+    tile, [B, H, ceil(S/128), 512], byte (r % 32) * 16 + (r / 32) * 4 + kb.  `along="cols"`: r = row of the tile,
+    kb = block of 32 columns; `along="rows"`: r = column, kb = block of 32 rows of the tile.  Unused bytes hold 127
+    (scale 1)."""
+    B, H = exps.shape[:2]
+    nt = (S + 127) // 128
+    atoms = np.full((B, H, nt, 32, 4, 4), 127, dtype=np.uint8)                # [.., r % 32, r / 32, kb]
+    if along == "cols":
+        nkb = exps.shape[3]
+        pad = np.full((B, H, nt * 128, nkb), 127, dtype=np.uint8)
+        pad[:, :, :S] = exps
+        t = pad.reshape(B, H, nt, 4, 32, nkb)                                 # [.., r / 32, r % 32, kb]
+        atoms[..., :nkb] = t.transpose(0, 1, 2, 4, 3, 5)
+    else:
+        d = exps.shape[3]
+        pad = np.full((B, H, nt * 4, d), 127, dtype=np.uint8)
+        pad[:, :, :exps.shape[2]] = exps
+        t = pad.reshape(B, H, nt, 4, d // 32, 32)                             # [.., kb, c / 32, c % 32]
+        atoms[:, :, :, :, :d // 32, :] = t.transpose(0, 1, 2, 5, 4, 3)
+    return np.ascontiguousarray(atoms.reshape(B, H, nt, 512))

@@ -58,10 +58,11 @@ def _kernels():
         ("fa_fwd_duo", b.FA_FLAG_TWO_CTA_KERNEL, "bf16", (1, 4, 2, 300, 300, 192)),
         ("fa_fwd_fp8", b.FA_FLAG_NO_STREAM_KERNEL, "e4m3", (1, 2, 2, 256, 384, 128)),
         ("fa_fwd_fp8_stream", b.FA_FLAG_STREAM_KERNEL, "e4m3", (1, 2, 1, 200, 500, 128)),
+        ("fa_fwd_mxfp8_stream", 0, "mx", (1, 2, 1, 200, 500, 128)),
     ]
 
 
-@pytest.mark.parametrize("case", range(12))
+@pytest.mark.parametrize("case", range(13))
 def test_every_kernel_reports_a_wait_that_runs_out_and_the_handle_recovers(case):
     """The hook drops the first V tile of every CTA: the launch returns (every wait is bounded), the host reads
     FA_ERR_DEVICE_TIMEOUT with the site that gave up, and the NEXT launch through the same handle, with the hook off,
@@ -78,11 +79,21 @@ def test_every_kernel_reports_a_wait_that_runs_out_and_the_handle_recovers(case)
         q8, sq, qd = W.quantize_e4m3_blocks(W.bf16_bits_to_f64(Q), 128)
         k8, sk, kd = W.quantize_e4m3_blocks(W.bf16_bits_to_f64(K), 128)
         v8, sv, vd = W.quantize_e4m3_blocks(W.bf16_bits_to_f64(V), None)
+    if kind == "mx":
+        # e8m0 scales per 32 elements along each contraction, as scale atoms
+        q8, qe, qd = W.quantize_mx_e4m3(W.bf16_bits_to_f64(Q), "cols")
+        k8, ke, kd = W.quantize_mx_e4m3(W.bf16_bits_to_f64(K), "cols")
+        v8, ve, vd = W.quantize_mx_e4m3(W.bf16_bits_to_f64(V), "rows")
+        qa, ka, va = W.mx_scale_atoms(qe, "cols", Sq), W.mx_scale_atoms(ke, "cols", Sk), W.mx_scale_atoms(ve, "rows", Sk)
     h = b.fa_create(flags=flags | b.FA_FLAG_DEBUG_DROP_V_LOAD, wait_limit_ms=20, kv_splits=1)
     try:
         def launch():
             if kind == "bf16":
                 o, lse = b.forward(h, to_torch_bf16(Q), to_torch_bf16(K), to_torch_bf16(V), causal=True, scale=w.scale)
+            elif kind == "mx":
+                o, lse = b.forward_mxfp8(h, torch.from_numpy(q8).cuda(), torch.from_numpy(k8).cuda(), torch.from_numpy(v8).cuda(),
+                                         torch.from_numpy(qa).cuda(), torch.from_numpy(ka).cuda(), torch.from_numpy(va).cuda(),
+                                         causal=True, scale=w.scale)
             else:
                 o, lse = b.forward_fp8(h, torch.from_numpy(q8).cuda(), torch.from_numpy(k8).cuda(), torch.from_numpy(v8).cuda(),
                                        torch.from_numpy(sq).cuda(), torch.from_numpy(sk).cuda(), torch.from_numpy(sv).cuda(),
