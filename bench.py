@@ -652,8 +652,32 @@ def main():
         torch.cuda.synchronize()
         t8 = e0.elapsed_time(e1) * 1e-3 / k
         line["block_scaled_e4m3"] = {"workload": w.name, "us": t8 * 1e6, "tflops_algorithmic": fl_alg / t8 / 1e12,
-                                     "speedup_over_bf16": t_step / t8, "steps": k,
+                                     "speedup_over_bf16": t_step / t8, "steps": k, "kernel": binding.fa_last_kernel_name(h),
                                      "note": "fa_forward_fp8, N(0,sigma^2) rounded to e4m3, unit scales, one input set"}
+        # the MX form of the same operands (e8m0 scales per 32 elements inside the MMA; unit scale atoms here)
+        n_qt, n_kt = (w.Sq + 127) // 128, (w.Sk + 127) // 128
+        qa = torch.full((w.B, w.Hq, n_qt, 512), 127, dtype=torch.uint8, device=device)
+        ka = torch.full((w.B, w.Hkv, n_kt, 512), 127, dtype=torch.uint8, device=device)
+
+        def one_mx():
+            stx = binding.fa_forward_mxfp8(h, q8.data_ptr(), k8.data_ptr(), v8.data_ptr(), qa.data_ptr(), ka.data_ptr(), ka.data_ptr(),
+                                           o8.data_ptr(), l8.data_ptr(), w.B, w.Hq, w.Hkv, w.Sq, w.Sk, 128, w.causal, w.scale, cs)
+            if stx != binding.FA_OK:
+                raise binding.FaError(stx, "fa_forward_mxfp8")
+
+        for _ in range(3):
+            one_mx()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(k):
+            one_mx()
+        e1.record()
+        torch.cuda.synchronize()
+        tx = e0.elapsed_time(e1) * 1e-3 / k
+        line["mx_e4m3"] = {"workload": w.name, "us": tx * 1e6, "tflops_algorithmic": fl_alg / tx / 1e12,
+                           "speedup_over_bf16": t_step / tx, "steps": k, "kernel": binding.fa_last_kernel_name(h),
+                           "note": "fa_forward_mxfp8, the same codes with unit e8m0 scale atoms"}
+        del qa, ka
         del q8, k8, v8, o8, l8
 
     if not args.no_decode and world == 1:

@@ -103,3 +103,51 @@ def test_sigma_sweep_of_the_block_scaled_e4m3_path(d):
         binding.fa_destroy(h)
         for row in report:
             print("sigma %.2f  kernel MAE %.2e (paper's bf16 curve %.2e) min Pearson %.6f | with input quantisation MAE %.2e Pearson %.6f" % row)
+
+
+@pytest.mark.parametrize("d", [64, 128], ids=["d64_the_papers_shape", "d128"])
+def test_sigma_sweep_of_the_mx_path(d):
+    """The same protocol for the MX form (fa_forward_mxfp8): e8m0 scales per 32 elements along each contraction.
+    Kernel error against the oracle on the represented tensors, end-to-end error against the oracle on the original
+    inputs.  On these i.i.d. inputs every block has the same magnitude, so the figures equal those of one scale per
+    128-row block to two digits (measured, both tables are in the design document); what scales every 32 elements
+    buy shows on inputs whose rows and columns differ in magnitude (tests/test_gpu_mxfp8.py)."""
+    import torch
+    from paper_2609_21264_b200 import binding
+    g = json.load(open(GOLDEN))
+    H, S = g["shape"]["H"], g["shape"]["S"]
+    h = binding.fa_create()
+    report = []
+    try:
+        for sigma, mae_paper in zip(g["sigma"], g["mae_x1e-2"]):
+            w = W.Workload("sweep_mx", 1, H, H, S, S, d, d, True, d ** -0.5, sigma=sigma, seed=4321)
+            Q, K, V = (W.bf16_bits_to_f64(x) for x in W.make_inputs(w))
+            q8, qe, Qd = W.quantize_mx_e4m3(Q, "cols")
+            k8, ke, Kd = W.quantize_mx_e4m3(K, "cols")
+            v8, ve, Vd = W.quantize_mx_e4m3(V, "rows")
+            O_rep, lse_rep = oracle.attention(Qd, Kd, Vd, causal=True, scale=w.scale)
+            O_org, _ = oracle.attention(Q, K, V, causal=True, scale=w.scale)
+            dev = lambda a: torch.from_numpy(a).cuda()
+            o, lse = binding.forward_mxfp8(h, dev(q8), dev(k8), dev(v8), dev(W.mx_scale_atoms(qe, "cols", S)),
+                                           dev(W.mx_scale_atoms(ke, "cols", S)), dev(W.mx_scale_atoms(ve, "rows", S)),
+                                           causal=True, scale=w.scale)
+            torch.cuda.synchronize()
+            assert binding.fa_last_status(h)[0] == binding.FA_OK
+            O = o.double().cpu().numpy()
+            lse = lse.double().cpu().numpy()
+            mae_k = float(np.abs(O - O_rep).mean())
+            mae_e = float(np.abs(O - O_org).mean())
+            rho_k = min(float(np.corrcoef(O[0, i].ravel(), O_rep[0, i].ravel())[0, 1]) for i in range(H))
+            rho_e = min(float(np.corrcoef(O[0, i].ravel(), O_org[0, i].ravel())[0, 1]) for i in range(H))
+            report.append((sigma, mae_k, mae_paper * 1e-2, rho_k, mae_e, rho_e))
+            assert np.isfinite(O).all() and np.isfinite(lse).all()
+            assert np.abs(lse - lse_rep).max() <= 1e-3 * max(1.0, sigma ** 2), (sigma,)
+            # the kernel's own error is that of the e4m3 path (the same rounding of P): same bounds
+            assert mae_k <= mae_paper * 1e-2 * (2.0 if sigma < 1.0 else 1.0), (sigma, mae_k)
+            assert rho_k >= 0.9995, (sigma, rho_k)
+            assert mae_e <= 0.09 * sigma, (sigma, mae_e)
+            assert rho_e >= 0.98, (sigma, rho_e)
+    finally:
+        binding.fa_destroy(h)
+        for row in report:
+            print("sigma %.2f  kernel MAE %.2e (paper's bf16 curve %.2e) min Pearson %.6f | with input quantisation MAE %.2e Pearson %.6f" % row)
