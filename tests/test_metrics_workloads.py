@@ -112,3 +112,44 @@ def test_block_quantiser_of_the_8_bit_path():
         step = np.where(np.abs(y) < 2.0 ** -6, 2.0 ** -9, 2.0 ** (np.floor(np.log2(np.maximum(np.abs(y), 2.0 ** -6))) - 3))
         assert (np.abs(_decode_e4m3(codes) - y) <= 0.5 * step * (1 + 1e-6) + 1e-9).all()
         assert (np.abs(_decode_e4m3(codes)) <= 448.0).all()
+
+
+def test_mx_quantiser_and_scale_atoms():
+    """quantize_mx_e4m3: power-of-two scales per 32 elements, the smallest that avoids saturation, nearest-even codes;
+    mx_scale_atoms: byte (r % 32) * 16 + (r / 32) * 4 + kb of a tile's 512-byte atom, padding 127."""
+    rng = np.random.default_rng(12)
+    x = rng.standard_normal((2, 3, 300, 64)) * np.exp2(rng.integers(-12, 13, size=(2, 3, 300, 1)).astype(np.float64))
+    x[0, 0, 5, :32] = 0.0                                        # an all-zero block keeps the scale 2^0
+    for along in ("cols", "rows"):
+        codes, exps, deq = W.quantize_mx_e4m3(x, along)
+        assert codes.dtype == np.uint8 and exps.dtype == np.uint8 and codes.shape == x.shape
+        assert not np.isin(codes, (0x7f, 0xff)).any() and exps.max() < 255
+        if along == "cols":
+            assert exps.shape == (2, 3, 300, 2)
+            per_elem = np.repeat(np.exp2(exps.astype(np.float64) - 127.0), 32, axis=3)
+            amax = np.abs(x).reshape(2, 3, 300, 2, 32).max(axis=4)
+            assert exps[0, 0, 5, 0] == 127
+        else:
+            assert exps.shape == (2, 3, 10, 64)
+            per_elem = np.repeat(np.exp2(exps.astype(np.float64) - 127.0), 32, axis=2)[:, :, :300]
+            xp = np.concatenate([x, np.zeros((2, 3, 20, 64))], axis=2)
+            amax = np.abs(xp).reshape(2, 3, 10, 32, 64).max(axis=3)
+        assert np.array_equal(deq, _decode_e4m3(codes) * per_elem)
+        scale = np.exp2(exps.astype(np.float64) - 127.0)
+        nz = amax > 0
+        assert (amax[nz] / scale[nz] <= 448.0).all() and (amax[nz] / scale[nz] > 224.0).all()     # the smallest such power of two
+        y = x / per_elem
+        step = np.where(np.abs(y) < 2.0 ** -6, 2.0 ** -9, 2.0 ** (np.floor(np.log2(np.maximum(np.abs(y), 2.0 ** -6))) - 3))
+        assert (np.abs(_decode_e4m3(codes) - y) <= 0.5 * step * (1 + 1e-6) + 1e-9).all()
+        atoms = W.mx_scale_atoms(exps, along, 300)
+        assert atoms.shape == (2, 3, 3, 512) and atoms.dtype == np.uint8
+        for _ in range(200):
+            b, h, t, r, kb = rng.integers(2), rng.integers(3), rng.integers(3), rng.integers(128), rng.integers(4)
+            byte = atoms[b, h, t, (r % 32) * 16 + (r // 32) * 4 + kb]
+            if along == "cols":
+                row = 128 * t + r
+                want = exps[b, h, row, kb] if (row < 300 and kb < 2) else 127
+            else:
+                blk = 4 * t + kb
+                want = exps[b, h, blk, r] if (blk < 10 and r < 64) else 127
+            assert byte == want
