@@ -232,7 +232,9 @@ fa_status fa_forward_varlen(fa_handle* h,
  * run on the 8-bit tensor-core path with fp32 accumulation; the probabilities are rounded to e4m3
  * before the second one (the row sums use the unrounded values).  O is bf16 [B, Hq, Sq, d], lse
  * fp32 [B, Hq, Sq] or NULL, both of Eq. 1 applied to the represented Q, K, V.  Head sizes 64 and
- * 128; other sizes, and handles created with FA_FLAG_SERIAL_KERNEL, return FA_ERR_UNSUPPORTED.  The
+ * 128, and d = 192 for the 192/128 shapes (Q8 and K8 with 192 columns, V8 and O with 128; stream
+ * tiling with one head per query tile); other sizes, and handles created with FA_FLAG_SERIAL_KERNEL,
+ * return FA_ERR_UNSUPPORTED.  The
  * tiling is planned as for fa_forward (pair or stream tiling, split-KV and shared query tiles for
  * grouped heads on the stream tiling; the partials use the handle's scratch buffer); with shared
  * query tiles of at most 64 rows the rows are additionally processed as two or four copies that

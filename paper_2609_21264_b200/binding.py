@@ -288,18 +288,21 @@ def forward_varlen(h, q, k, v, cu_seqlens_q, cu_seqlens_k, max_sq: int, *, causa
 
 def forward_fp8(h, q8, k8, v8, q_scale, k_scale, v_scale, *, causal: bool, scale: float = 0.0, want_lse=True):
     """Block-scaled e4m3 attention on torch CUDA tensors: q8/k8/v8 uint8 (or float8_e4m3fn) [B,H,S,d]
-    with d = 64 or 128, scales fp32 CUDA tensors or None.  Returns (O bf16 [B,Hq,Sq,d], lse fp32 [B,Hq,Sq])."""
+    with d = 64 or 128 (or q8/k8 with d = 192 and v8 with 128), scales fp32 CUDA tensors or None.  Returns (O bf16 [B,Hq,Sq,d], lse fp32 [B,Hq,Sq])."""
     import torch
     for t in (q8, k8, v8):
         if t.element_size() != 1 or not t.is_cuda or not t.is_contiguous() or t.dim() != 4:
             raise ValueError("q8, k8, v8 must be contiguous 4-D one-byte CUDA tensors")
     B, Hq, Sq, d = q8.shape
     _, Hkv, Sk, _ = k8.shape
+    dv = 128 if d == 192 else d                 # the 192/128 shapes: V and O have head size 128
+    if v8.shape[-1] != dv:
+        raise ValueError("v8 must have head size %d" % dv)
     n_qt, n_kt = (Sq + 127) // 128, (Sk + 127) // 128
     for t, shape in ((q_scale, (B, Hq, n_qt)), (k_scale, (B, Hkv, n_kt)), (v_scale, (B, Hkv))):
         if t is not None and (t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != shape):
             raise ValueError("scale tensors must be contiguous fp32 CUDA tensors of shape %s" % (shape,))
-    out = torch.empty((B, Hq, Sq, d), dtype=torch.bfloat16, device=q8.device)
+    out = torch.empty((B, Hq, Sq, dv), dtype=torch.bfloat16, device=q8.device)
     lse = torch.empty((B, Hq, Sq), dtype=torch.float32, device=q8.device) if want_lse else None
     ptr = lambda t: t.data_ptr() if t is not None else None
     st = fa_forward_fp8(h, q8.data_ptr(), k8.data_ptr(), v8.data_ptr(), ptr(q_scale), ptr(k_scale), ptr(v_scale),

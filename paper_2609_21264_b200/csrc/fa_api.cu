@@ -944,9 +944,11 @@ static fa_status forward_fp8_common(fa_handle* h, const void* Q8, const void* K8
                                     void* O, float* lse, int B, int Hq, int Hkv, int Sq, int Sk, int d, int causal,
                                     float scale, void* stream) {
     if (!h) return FA_ERR_INVALID_ARG;
-    if (d != 64 && d != 128) return (d > 0) ? FA_ERR_UNSUPPORTED : FA_ERR_INVALID_ARG;
     const bool mx = q_sf != nullptr;
-    fa_status s = check_args(Q8, K8, V8, O, lse, B, Hq, Hkv, Sq, Sk, d, d, scale, true);
+    // d = 192: the 192/128 shapes (Q and K of head size 192, V and O of 128); fp32 block scales only
+    if (d != 64 && d != 128 && !(d == 192 && !mx)) return (d > 0) ? FA_ERR_UNSUPPORTED : FA_ERR_INVALID_ARG;
+    const int dv = (d == 192) ? 128 : d;
+    fa_status s = check_args(Q8, K8, V8, O, lse, B, Hq, Hkv, Sq, Sk, d, dv, scale, true);
     if (s != FA_OK) return s;
     if ((q_scale && misaligned(q_scale, 4)) || (k_scale && misaligned(k_scale, 4)) || (v_scale && misaligned(v_scale, 4)))
         return FA_ERR_INVALID_ARG;
@@ -961,36 +963,47 @@ static fa_status forward_fp8_common(fa_handle* h, const void* Q8, const void* K8
     // costs are lower by a similar factor in both tilings).  Only the stream tiling splits K/V
     // and packs heads.
     // (The MX form runs on the stream tiling with one head per query tile: its scale atoms follow the tile's rows.)
-    const uint32_t plan_flags = mx ? ((h->flags & ~(FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_FORCE_PERSISTENT | FA_FLAG_TWO_CTA_KERNEL)) |
-                                      FA_FLAG_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)
-                                   : h->flags;
+    // (So does head size 192/128: only the stream kernel has it.)
+    const uint32_t plan_flags = (mx || d == 192) ? ((h->flags & ~(FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_FORCE_PERSISTENT | FA_FLAG_TWO_CTA_KERNEL)) |
+                                                    FA_FLAG_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)
+                                                 : h->flags;
     const LaunchPlan pl = plan_launch(h->num_sms, plan_flags, h->kv_splits_cfg, h->scratch_bytes, false,
-                                      B, Hq, Hkv, Sq, Sk, d, d, causal ? 1 : 0);
+                                      B, Hq, Hkv, Sq, Sk, d, dv, causal ? 1 : 0);
     const int q_box_rows = pl.pack_heads > 1 ? Sq : fa::kTileM;
     // an e4m3 row is d bytes: one box column of d bytes, swizzled over d bytes
     const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;
     const long long hq_stride = static_cast<long long>(Sq) * d, hk_stride = static_cast<long long>(Sk) * d;
-    if ((s = get_map(h, Q8, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, q_box_rows, &mq, 1, pl.pack_heads, d)) != FA_OK) return s;
+    const long long ho_stride = static_cast<long long>(Sq) * dv, hv_stride = static_cast<long long>(Sk) * dv;
+    // (a row of 192 bytes is loaded as two boxes: 128 bytes with the 128-byte swizzle, 64 bytes with the 64-byte one)
+    const int sw_qk = (d == 64) ? 64 : 128;
+    if ((s = get_map(h, Q8, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, q_box_rows, &mq, 1, pl.pack_heads, sw_qk)) != FA_OK) return s;
     CUtensorMap map_q = *mq;
-    if ((s = get_map(h, K8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mk, 1, 1, d)) != FA_OK) return s;
+    if ((s = get_map(h, K8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mk, 1, 1, sw_qk)) != FA_OK) return s;
     CUtensorMap map_k = *mk;
-    if ((s = get_map(h, V8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mv, 1, 1, d)) != FA_OK) return s;
+    if ((s = get_map(h, V8, dv, Sk, Hkv, B, hv_stride * Hkv, hv_stride, dv, fa::kTileN, &mv, 1, 1, dv)) != FA_OK) return s;
     CUtensorMap map_v = *mv;
-    if ((s = get_map(h, O, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, q_box_rows, &mo, 2, pl.pack_heads)) != FA_OK) return s;
+    if ((s = get_map(h, O, dv, Sq, Hq, B, ho_stride * Hq, ho_stride, dv, q_box_rows, &mo, 2, pl.pack_heads)) != FA_OK) return s;
     CUtensorMap map_o = *mo;
+    CUtensorMap map_q2 = map_q, map_k2 = map_k;
+    if (d == 192) {
+        if ((s = get_map(h, Q8, d, Sq, Hq, B, hq_stride * Hq, hq_stride, d, q_box_rows, &mq, 1, 1, 64)) != FA_OK) return s;
+        map_q2 = *mq;
+        if ((s = get_map(h, K8, d, Sk, Hkv, B, hk_stride * Hkv, hk_stride, d, fa::kTileN, &mk, 1, 1, 64)) != FA_OK) return s;
+        map_k2 = *mk;
+    }
 
     fa::FwdParams p;
     memset(&p, 0, sizeof p);
     p.O = static_cast<__nv_bfloat16*>(O);
-    p.o_stride_b = hq_stride * Hq;
-    p.o_stride_h = hq_stride;
-    p.o_stride_s = d;
+    p.o_stride_b = ho_stride * Hq;
+    p.o_stride_h = ho_stride;
+    p.o_stride_s = dv;
     p.lse = lse;
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Sk = Sk;
     p.causal = causal ? 1 : 0;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
-    p.heads_per_group = heads_per_group(static_cast<long long>(Sk) * 2 * d, B, Hq, Hkv);      // one byte per element
+    p.heads_per_group = heads_per_group(static_cast<long long>(Sk) * (d + dv), B, Hq, Hkv);      // one byte per element
     p.status = h->status_dev;
     p.wait_limit_ns = h->wait_limit_ns;
     p.debug_drop_v_load = (h->flags & FA_FLAG_DEBUG_DROP_V_LOAD) ? 1 : 0;
@@ -1011,13 +1024,13 @@ static fa_status forward_fp8_common(fa_handle* h, const void* Q8, const void* K8
         // every copy is one more partial per split for the merge kernel to read: with many splits
         // (short CTAs, where the exponentials saved are few) the merge would cost more than it saves
         while (copies > 1 && copies * p.kv_splits > 32) copies /= 2;
-        const unsigned long long per_partial = static_cast<unsigned long long>(B) * Hq * Sq * (d + 1) * 4ull;
+        const unsigned long long per_partial = static_cast<unsigned long long>(B) * Hq * Sq * (dv + 1) * 4ull;
         while (copies > 1 && per_partial * p.kv_splits * copies > h->scratch_bytes) copies /= 2;
     }
     const int n_partials = p.kv_splits * copies;
     if (n_partials > 1) {
         p.o_part = static_cast<float*>(h->scratch);
-        p.lse_part = p.o_part + static_cast<size_t>(n_partials) * B * Hq * Sq * d;
+        p.lse_part = p.o_part + static_cast<size_t>(n_partials) * B * Hq * Sq * dv;
     }
     h->last_splits = p.kv_splits;
     h->last_kernel = use_stream ? (mx ? "fa_fwd_mxfp8_stream" : "fa_fwd_fp8_stream") : "fa_fwd_fp8";
@@ -1033,10 +1046,11 @@ static fa_status forward_fp8_common(fa_handle* h, const void* Q8, const void* K8
     cfg.numAttrs = (h->flags & FA_FLAG_NO_DEPENDENT_LAUNCH) ? 0 : 1;
     const bool d128 = (d == 128);
     if (use_stream) {
-        const int smem = d128 ? fa::fp8_stream_smem_bytes<128>() : fa::fp8_stream_smem_bytes<64>();
-        static_assert(fa::fp8_stream_smem_bytes<128>() <= 227 * 1024, "shared memory budget exceeded");
+        const int smem = d == 192 ? fa::fp8_stream_smem_bytes<192>() : (d128 ? fa::fp8_stream_smem_bytes<128>() : fa::fp8_stream_smem_bytes<64>());
+        static_assert(fa::fp8_stream_smem_bytes<128>() <= 227 * 1024 && fa::fp8_stream_smem_bytes<192>() <= 227 * 1024,
+                      "shared memory budget exceeded");
         const bool pack = pl.pack_heads > 1;
-        using Kernel = void (*)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, fa::FwdParams, fa::Fp8Params);
+        using Kernel = void (*)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, fa::FwdParams, fa::Fp8Params);
         // variant: 0 = one head per tile, 1..3 = packed heads with 1, 2, 4 copies of the rows
         const int variant = !pack ? 0 : (copies == 4 ? 3 : (copies == 2 ? 2 : 1));
         static const Kernel kernels[2][4] = {
@@ -1046,12 +1060,13 @@ static fa_status forward_fp8_common(fa_handle* h, const void* Q8, const void* K8
              fa::fa_fwd_fp8_stream_kernel<128, true, 2>, fa::fa_fwd_fp8_stream_kernel<128, true, 4>}};
         Kernel kernel = kernels[d128 ? 1 : 0][variant];
         if (mx) kernel = d128 ? fa::fa_fwd_fp8_stream_kernel<128, false, 1, true> : fa::fa_fwd_fp8_stream_kernel<64, false, 1, true>;
+        if (d == 192) kernel = fa::fa_fwd_fp8_stream_kernel<192, false, 1, false>;
         if ((s = ensure_smem_attr(h, kernel, smem)) != FA_OK) return s;
         const long long n_ctas = (pack ? static_cast<long long>(Hq / pl.pack_heads) : static_cast<long long>(p.n_q_tiles) * Hq) * B * p.kv_splits;
         if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
         cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
         cfg.dynamicSmemBytes = smem;
-        if (cudaLaunchKernelEx(&cfg, kernel, map_q, map_k, map_v, map_o, p, f) != cudaSuccess) return FA_ERR_CUDA;
+        if (cudaLaunchKernelEx(&cfg, kernel, map_q, map_k, map_v, map_o, map_q2, map_k2, p, f) != cudaSuccess) return FA_ERR_CUDA;
         h->launches += 1;
         if (n_partials > 1) {
             const long long n_rows = static_cast<long long>(B) * Hq * Sq;
@@ -1060,7 +1075,7 @@ static fa_status forward_fp8_common(fa_handle* h, const void* Q8, const void* K8
             cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
             cfg.blockDim = dim3(128, 1, 1);
             cfg.dynamicSmemBytes = 0;
-            auto combine = d128 ? fa::fa_combine_kernel<128> : fa::fa_combine_kernel<64>;
+            auto combine = dv == 128 ? fa::fa_combine_kernel<128> : fa::fa_combine_kernel<64>;
             if (cudaLaunchKernelEx(&cfg, combine, static_cast<const float*>(p.o_part),
                                    static_cast<const float*>(p.lse_part), p.O, p.lse, n_rows, n_partials, p.Hq, p.Sq,
                                    p.o_stride_b, p.o_stride_h, p.o_stride_s) != cudaSuccess) return FA_ERR_CUDA;

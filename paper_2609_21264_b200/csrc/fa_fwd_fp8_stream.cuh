@@ -6,7 +6,7 @@
 // tile and are folded into the exp2 constant of that tile, so the reference maximum that the
 // two warpgroups hand to each other is kept in scaled log2 units.  Used by fa_forward_fp8 where
 // the stream tiling is planned: grids under a wave and decode-like shapes with split-KV
-// (attention over an 8-bit K/V cache).  Head sizes 64 and 128, fixed-length contiguous tensors.
+// (attention over an 8-bit K/V cache).  Head sizes 64, 128 and 192/128, fixed-length contiguous tensors.
 //   TMEM  S^0 [0,128)  S^1 [128,256)  O [256,384)  P^0 [384,416)  P^1 [448,480)
 //
 // kMx: the MX form of the operands (the closest counterpart of a block floating point format on this GPU): e4m3
@@ -24,19 +24,32 @@
 
 namespace fa {
 
+// D = head size of Q and K; V and O have the same, except D = 192, where they have 128 (the 192/128 shapes).
+// A Q or K row of 192 bytes is two swizzled chunks: columns [0,128) with the 128-byte swizzle (16 KB per
+// 128-row tile) and columns [128,192) with the 64-byte swizzle (8 KB), each with a tensor map of its own.
 template <int D>
 struct Fp8StreamCfg {
+    static_assert(D == 64 || D == 128 || D == 192, "head sizes of the 8-bit stream kernel");
     static constexpr int kD = D;
-    static constexpr int kTile8 = kTileM * kD;           // one 128 x D e4m3 tile (16 or 8 KB), one swizzled chunk
-    static constexpr int kOBytes = (D / kChunkCols) * kChunkBytes;      // bf16 output tile
+    static constexpr int kDV = (D == 192) ? 128 : D;
+    static constexpr int kTile8 = kTileM * kD;           // one 128 x D e4m3 tile of Q or K (8, 16 or 24 KB)
+    static constexpr int kVTile8 = kTileM * kDV;         // one 128 x DV e4m3 tile of V
+    static constexpr int kOBytes = (kDV / kChunkCols) * kChunkBytes;      // bf16 output tile
     static constexpr int kKStages = 4;
     static constexpr int kVStages = 4;
     static constexpr int kSfAtom = 512;                  // scales of one 128-row tile (MX variant)
     static constexpr int kSfBytes = (2 + kKStages + kVStages) * kSfAtom;     // Q, P (constant), K and V stages
-    static constexpr int kTileBytes = (1 + kKStages + kVStages) * kTile8 + kOBytes + kSfBytes;
-    static constexpr int kColSf = 416;
+    static constexpr int kTileBytes = (1 + kKStages) * kTile8 + kVStages * kVTile8 + kOBytes + kSfBytes;
     static constexpr int kTmemCols = 512;
     static constexpr int kColS = 0, kColO = 256, kColP = 384;   // P^b at kColP + 64 b (32 columns used)
+    static constexpr int kColSf = 416;
+    // shared-memory descriptor high words (stride between 8-row groups, version, swizzle mode) of a chunk with
+    // 128-byte and with 64-byte rows
+    static constexpr uint32_t kDescHi128 = (1024u >> 4) | (1u << 14) | (2u << 29);
+    static constexpr uint32_t kDescHi64 = (512u >> 4) | (1u << 14) | (4u << 29);
+    static constexpr uint32_t kDescHiQK = (D == 64) ? kDescHi64 : kDescHi128;      // first chunk of Q and K
+    static constexpr uint32_t kDescHiV = (kDV == 64) ? kDescHi64 : kDescHi128;
+    static constexpr uint32_t kVStep = (32u * kDV) >> 4;  // 32 keys of V, in descriptor address units
 };
 
 template <int D>
@@ -58,10 +71,14 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                      const __grid_constant__ CUtensorMap tm_k,
                      const __grid_constant__ CUtensorMap tm_v,
                      const __grid_constant__ CUtensorMap tm_o,
+                     const __grid_constant__ CUtensorMap tm_q2,    // D = 192: columns [128,192) of Q and of K
+                     const __grid_constant__ CUtensorMap tm_k2,    // (64-byte swizzle); otherwise unused
                      const FwdParams p, const Fp8Params f) {
     using Cfg = Fp8StreamCfg<D>;
-    constexpr int DV = Cfg::kD;
+    constexpr int DV = Cfg::kDV;
     constexpr int kTile8 = Cfg::kTile8;
+    constexpr int kVTile8 = Cfg::kVTile8;
+    static_assert(D != 192 || (!kPack && !kMx), "192/128: one head per query tile, fp32 block scales");
     static_assert(kRep == 1 || (kPack && (kRep == 2 || kRep == 4)), "copies of the query rows need packed heads");
     static_assert(!kMx || !kPack, "the MX variant has no packed heads (its scale atoms follow the query tile's rows)");
     constexpr int kRepRows = kTileM / kRep;      // rows of one copy of the pack
@@ -94,7 +111,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
     const uint32_t sQ = smem_base;
     const uint32_t sK = sQ + kTile8;
     const uint32_t sV = sK + NK * kTile8;
-    const uint32_t sStage = sV + NV * kTile8;      // the bf16 output tile passes through here
+    const uint32_t sStage = sV + NV * kVTile8;     // the bf16 output tile passes through here
     const uint32_t sSfQ = sStage + Cfg::kOBytes;   // scale atoms (MX variant): Q, P, K stages, V stages
     const uint32_t sSfP = sSfQ + Cfg::kSfAtom;
     const uint32_t sSfK = sSfP + Cfg::kSfAtom;
@@ -470,10 +487,11 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         setmaxnreg_dec<kRegsOther>();
         if (elect_one() && n_kv > 0) {
             constexpr uint32_t kIdescQK = make_idesc_e4m3_f32(kTileM, kTileN, false, false);
-            constexpr uint32_t kDescHi = Fp8Cfg<D>::kDescHi;
+            constexpr uint32_t kDescHi = Cfg::kDescHiQK;
             const uint32_t q_lo = ((sQ & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
             auto desc = [](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(kDescHi) << 32) | lo; };
+            auto desc64 = [](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(Cfg::kDescHi64) << 32) | lo; };
             bool ok = mbar_wait(smem_addr(&sh.q_full), 0, wctx, kSiteMmaQFull);
             if constexpr (kMx) {
                 if (ok) {
@@ -500,8 +518,14 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                                   tmem_base + Cfg::kColSf, tSfK, kk > 0 ? 1u : 0u);
                 } else {
 #pragma unroll
-                    for (int kk = 0; kk < Cfg::kD / 32; ++kk)      // k-steps of 32 elements = 32 bytes
+                    for (int kk = 0; kk < (D == 192 ? 4 : Cfg::kD / 32); ++kk)      // k-steps of 32 elements = 32 bytes
                         mma_ss_f8(tS, desc(q_lo + kk * 2), desc(klo + kk * 2), kIdescQK, kk > 0 ? 1u : 0u);
+                    if constexpr (D == 192) {
+                        // columns [128,192): the second chunk of Q and of K (64-byte rows), 16 KB behind the first
+#pragma unroll
+                        for (int kk = 0; kk < 2; ++kk)
+                            mma_ss_f8(tS, desc64(q_lo + (16384 >> 4) + kk * 2), desc64(klo + (16384 >> 4) + kk * 2), kIdescQK, 1u);
+                    }
                 }
                 tc_commit(smem_addr(&sh.s_full[j & 1]));
                 tc_commit(smem_addr(&sh.k_empty[sk]));
@@ -513,7 +537,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
         setmaxnreg_dec<kRegsOther>();
         if (elect_one() && n_kv > 0) {
             constexpr uint32_t kIdescPV = make_idesc_e4m3_f32(kTileM, DV, false, true);
-            constexpr uint32_t kDescHi = Fp8Cfg<D>::kDescHi;
+            constexpr uint32_t kDescHi = Cfg::kDescHiV;
             const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((16384u >> 4) << 16);   // one swizzled row spans dv: the chunk stride is not used
             const uint32_t tO = tmem_base + Cfg::kColO;
             auto desc = [](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(kDescHi) << 32) | lo; };
@@ -528,18 +552,18 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t tP = tmem_base + Cfg::kColP + (j & 1) * 64;
-                const uint32_t vlo = v_lo0 + sv * (kTile8 >> 4);
+                const uint32_t vlo = v_lo0 + sv * (kVTile8 >> 4);
                 if constexpr (kMx) {
                     const uint32_t tSfV = tmem_base + Cfg::kColSf + 16 + (j & 1) * 4;
                     tmem_cp_scales_32x16B(tSfV, sSfV + sv * Cfg::kSfAtom);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)              // block kk of the tile's keys: P's scale (1) and V's per column
-                        mma_ts_mx(tO, tP + kk * 8, desc(vlo + kk * Fp8Cfg<D>::kVStep), make_idesc_mx_e4m3(kTileM, DV, true, kk, kk),
+                        mma_ts_mx(tO, tP + kk * 8, desc(vlo + kk * Cfg::kVStep), make_idesc_mx_e4m3(kTileM, DV, true, kk, kk),
                                   tmem_base + Cfg::kColSf + 12, tSfV, (j > 0 || kk > 0) ? 1u : 0u);
                 } else {
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)              // four k-steps of 32 keys: 8 P columns, 32 V rows of D bytes
-                        mma_ts_f8(tO, tP + kk * 8, desc(vlo + kk * Fp8Cfg<D>::kVStep), kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+                        mma_ts_f8(tO, tP + kk * 8, desc(vlo + kk * Cfg::kVStep), kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
                 }
                 tc_commit(smem_addr(&sh.p_free[j & 1]));
                 tc_commit(smem_addr(&sh.v_empty[sv]));
@@ -561,6 +585,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                (kMx ? Cfg::kSfAtom : 0));
 #pragma unroll
                 for (int r = 0; r < kRep; ++r) tma_load_4d(sQ + r * kRepRows * D, &tm_q, bar, 0, i0, hq, b);
+                if constexpr (D == 192) tma_load_4d(sQ + 16384, &tm_q2, bar, 128, i0, hq, b);
                 if constexpr (kMx)
                     bulk_load_1d(sSfQ, f.q_sf + (static_cast<size_t>(b * p.Hq + hq) * p.n_q_tiles + q_tile) * Cfg::kSfAtom, Cfg::kSfAtom, bar);
             }
@@ -572,6 +597,7 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 const uint32_t bar = smem_addr(&sh.k_full[s]);
                 mbar_arrive_expect_tx(bar, kTile8 + (kMx ? Cfg::kSfAtom : 0));
                 tma_load_4d(sK + s * kTile8, &tm_k, bar, 0, (j_base + j) * kTileN, kvh, b);
+                if constexpr (D == 192) tma_load_4d(sK + s * kTile8 + 16384, &tm_k2, bar, 128, (j_base + j) * kTileN, kvh, b);
                 if constexpr (kMx)
                     bulk_load_1d(sSfK + s * Cfg::kSfAtom, f.k_sf + (static_cast<size_t>(kv_idx) * f.n_kv_tiles + j_base + j) * Cfg::kSfAtom,
                                  Cfg::kSfAtom, bar);
@@ -588,8 +614,8 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 ok = mbar_wait(smem_addr(&sh.v_empty[s]), ((j / NV) & 1) ^ 1, wctx, kSiteLoadKvEmpty);
                 if (!ok) break;
                 const uint32_t bar = smem_addr(&sh.v_full[s]);
-                mbar_arrive_expect_tx(bar, kTile8 + (kMx ? Cfg::kSfAtom : 0));
-                tma_load_4d(sV + s * kTile8, &tm_v, bar, 0, (j_base + j) * kTileN, kvh, b);
+                mbar_arrive_expect_tx(bar, kVTile8 + (kMx ? Cfg::kSfAtom : 0));
+                tma_load_4d(sV + s * kVTile8, &tm_v, bar, 0, (j_base + j) * kTileN, kvh, b);
                 if constexpr (kMx)
                     bulk_load_1d(sSfV + s * Cfg::kSfAtom, f.v_sf + (static_cast<size_t>(kv_idx) * f.n_kv_tiles + j_base + j) * Cfg::kSfAtom,
                                  Cfg::kSfAtom, bar);

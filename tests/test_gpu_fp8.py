@@ -43,7 +43,7 @@ def _run(handle, w, q8, k8, v8, sq, sk, sv):
 
 
 def _wl(name, B, Hq, Hkv, Sq, Sk, causal, seed, sigma=1.0, d=128):
-    return W.Workload(name, B=B, Hq=Hq, Hkv=Hkv, Sq=Sq, Sk=Sk, dqk=d, dv=d, causal=causal, scale=d ** -0.5,
+    return W.Workload(name, B=B, Hq=Hq, Hkv=Hkv, Sq=Sq, Sk=Sk, dqk=d, dv=(128 if d == 192 else d), causal=causal, scale=d ** -0.5,
                       sigma=sigma, seed=seed)
 
 
@@ -69,6 +69,13 @@ CASES = [
     _wl("fp8_d64_group7_single_query", 2, 14, 2, 1, 3000, False, 1354, d=64),
     _wl("fp8_d64_group4_sq10_causal", 1, 8, 2, 10, 900, True, 1355, d=64),
     _wl("fp8_d64_group2_sq50", 1, 4, 2, 50, 640, True, 1356, d=64),
+    # head sizes 192/128 (stream tiling on either handle): rows of Q and K in two swizzled chunks, 128 + 64 bytes
+    _wl("fp8_d192_one_tile", 1, 1, 1, 128, 128, False, 1360, d=192),
+    _wl("fp8_d192_gqa_causal_ragged", 2, 8, 2, 333, 333, True, 1361, d=192),
+    _wl("fp8_d192_mha_full_sq_ne_sk", 1, 4, 4, 200, 457, False, 1362, d=192),
+    _wl("fp8_d192_deepseek_like_s1024", 1, 8, 8, 1024, 1024, True, 1363, d=192),
+    _wl("fp8_d192_one_tile_many_keys", 1, 2, 1, 100, 2100, False, 1364, d=192),      # split-KV
+    _wl("fp8_d192_grouped_single_query", 1, 8, 2, 1, 1500, False, 1365, d=192),      # one head per tile at this size
 ]
 
 
@@ -194,8 +201,31 @@ def test_fp8_default_handle_plans_both_tilings():
 def test_fp8_unsupported_head_size(handle):
     import torch
     from paper_2609_21264_b200 import binding
-    z = torch.zeros((1, 1, 128, 192), dtype=torch.uint8, device="cuda")
-    o = torch.zeros((1, 1, 128, 192), dtype=torch.bfloat16, device="cuda")
-    st = binding.fa_forward_fp8(handle, z.data_ptr(), z.data_ptr(), z.data_ptr(), None, None, None, o.data_ptr(), None,
-                                1, 1, 1, 128, 128, 192, False, 0.0)
-    assert st == binding.FA_ERR_UNSUPPORTED
+    z = torch.zeros((1, 1, 128, 256), dtype=torch.uint8, device="cuda")
+    o = torch.zeros((1, 1, 128, 256), dtype=torch.bfloat16, device="cuda")
+    for d in (96, 256):
+        st = binding.fa_forward_fp8(handle, z.data_ptr(), z.data_ptr(), z.data_ptr(), None, None, None, o.data_ptr(), None,
+                                    1, 1, 1, 128, 128, d, False, 0.0)
+        assert st == binding.FA_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("part", ["first_128_columns", "last_64_columns"])
+def test_fp8_d192_each_chunk_of_the_rows_on_its_own(handle, part):
+    """Head size 192: a row of Q or K lies in shared memory as two chunks with different swizzles (columns [0,128) and
+    [128,192)).  With all other columns zero the scores come from one chunk alone, so a k-step that reads the wrong
+    bytes of either shows in lse (1e-3) at once."""
+    w = _wl("fp8_d192_" + part, 1, 2, 2, 300, 420, True, 1370 + len(part), d=192)
+    rng = np.random.default_rng(w.seed)
+    Q = rng.standard_normal((1, 2, 300, 192)) * 1.5
+    K = rng.standard_normal((1, 2, 420, 192)) * 1.5
+    V = rng.standard_normal((1, 2, 420, 128))
+    cols = slice(128, 192) if part == "first_128_columns" else slice(0, 128)      # the columns that are zeroed
+    Q[..., cols] = 0.0
+    K[..., cols] = 0.0
+    q8, sq, Qd = W.quantize_e4m3_blocks(Q, 128)
+    k8, sk, Kd = W.quantize_e4m3_blocks(K, 128)
+    v8, sv, Vd = W.quantize_e4m3_blocks(V, None)
+    O_ref, lse_ref = oracle.attention(Qd, Kd, Vd, causal=True, scale=w.scale)
+    assert np.abs(lse_ref[np.isfinite(lse_ref)]).max() > 1.0                       # the scores matter
+    O, lse = _run(handle, w, q8, k8, v8, sq, sk, sv)
+    _check(w, O, lse, O_ref, lse_ref, Vd)
