@@ -563,6 +563,8 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the records of the other configurations (key 'per_config')")
     ap.add_argument("--table6", action="store_true",
                     help="also time the twelve attention shapes of the paper's Table 6 (key 'table6')")
+    ap.add_argument("--eight-bit", action="store_true",
+                    help="time the 8-bit variants on the workload (keys 'block_scaled_e4m3', 'mx_e4m3') even with --no-sweep")
     ap.add_argument("--no-decode", action="store_true", help="skip the grouped-head decode step and the packed batches (keys 'decode', 'packed_batches')")
     ap.add_argument("--plan-ab", action="store_true",
                     help="also time every configuration, and items of every length, with each kernel forced, next to the "
@@ -625,7 +627,7 @@ def main():
             "per_launch_us_min": rec["per_launch_us_min"], "per_launch_us_median": rec["per_launch_us_median"],
             "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches)}
 
-    if not args.no_sweep and world == 1 and w.dqk == 128 and w.dv == 128:
+    if (args.eight_bit or not args.no_sweep) and world == 1 and w.dqk == 128 and w.dv == 128:
         # the block-scaled e4m3 variant on the same shape (N(0, sigma^2) rounded to e4m3, unit scales), for context
         gen = torch.Generator(device=device).manual_seed(w.seed)
         q8, k8, v8 = (torch.randn(shape, generator=gen, device=device).mul_(w.sigma).to(torch.float8_e4m3fn).view(torch.uint8)
