@@ -49,6 +49,15 @@ struct Fp8Cfg {
     static constexpr int kThreads = 512;
 };
 
+// Share of the exponentials of the 8-bit kernels that is computed on the FMA pipe: every kFp8EmuEvery-th pair (0 = none).
+// Measured on B200 with Gaussian data (pair kernel, TFLOP/s, none / every 4th / 3rd / 2nd pair): causal S 2048 921 / 1033 /
+// 1029 / 966, B4 S 8192 1270 / 1377 / 1384 / 1303, S 32768 1422 / 1519 / 1546 / 1408, 64-round non-causal items 1321 /
+// 1611 / 1540 / 1402.
+#ifndef FA_FP8_EMU_EVERY
+#define FA_FP8_EMU_EVERY 4
+#endif
+constexpr int kFp8EmuEvery = FA_FP8_EMU_EVERY;
+
 struct Fp8Params {
     const float* q_scale;    // [B, Hq, n_q_tiles] or nullptr (= 1)
     const float* k_scale;    // [B, Hkv, n_kv_tiles] or nullptr
@@ -215,13 +224,22 @@ fa_fwd_fp8_kernel(const __grid_constant__ CUtensorMap tm_q,
             float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
             float alpha = 1.f;
             uint32_t s[kTileN];
+            // With 8-bit operands the MMAs of a tile take half the cycles of the exponentials (512 against 1024 on the
+            // MUFU at 16 per cycle and SM): the loop is MUFU-bound.  Every kFp8EmuEvery-th pair of exponentials therefore
+            // goes to the FMA pipe (ptx::exp2_poly2, relative error 7.5e-5 against e4m3's 2^-4 for P and 1e-3 for lse).
             auto exp_chunk = [&](int q) {
 #pragma unroll
                 for (int e = 0; e < 32; e += 2) {
                     const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[q * 32 + e]),
                                                             __uint_as_float(s[q * 32 + e + 1])), c2, nmc2);
-                    s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
-                    s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
+                    if (kFp8EmuEvery > 0 && ((e / 2) % (kFp8EmuEvery > 0 ? kFp8EmuEvery : 1)) == kFp8EmuEvery - 1) {
+                        const float2 r = exp2_poly2(x);
+                        s[q * 32 + e] = __float_as_uint(r.x);
+                        s[q * 32 + e + 1] = __float_as_uint(r.y);
+                    } else {
+                        s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
+                        s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
+                    }
                 }
             };
             // Row sum (of the unrounded values), e4m3 conversion and store of one 32-key chunk of P.

@@ -317,8 +317,15 @@ fa_fwd_fp8_stream_kernel(const __grid_constant__ CUtensorMap tm_q,
                 for (int e = 0; e < 32; e += 2) {
                     const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[q * 32 + e]),
                                                             __uint_as_float(s[q * 32 + e + 1])), c2, nmc2);
-                    s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
-                    s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
+                    // (every kFp8EmuEvery-th pair on the FMA pipe: the 8-bit loop is MUFU-bound, see fa_fwd_fp8.cuh)
+                    if (kFp8EmuEvery > 0 && ((e / 2) % (kFp8EmuEvery > 0 ? kFp8EmuEvery : 1)) == kFp8EmuEvery - 1) {
+                        const float2 r = exp2_poly2(x);
+                        s[q * 32 + e] = __float_as_uint(r.x);
+                        s[q * 32 + e + 1] = __float_as_uint(r.y);
+                    } else {
+                        s[q * 32 + e] = __float_as_uint(exp2_approx(x.x));
+                        s[q * 32 + e + 1] = __float_as_uint(exp2_approx(x.y));
+                    }
                 }
             };
             auto emit_chunk = [&](int q) {

@@ -44,14 +44,15 @@ FA_DEVI float exp2_approx(float x) {
 
 // exp2 of two values on the FMA pipe instead of the MUFU: the integer part n = floor(x) is taken with the
 // 1.5 * 2^23 trick (an addition rounded towards minus infinity leaves n in the low mantissa bits), the fraction
-// f = x - n in [0, 1) goes through a cubic (minimax fit of 2^f, relative error 7.5e-5, far below the bf16 rounding
-// of P that follows), and n is put back with a shift and an integer add into the exponent field.  Valid for
-// x < 127; x below -127 is clamped there and comes out as a denormal (below 1.2e-38), which the row sum's
-// flushing additions read as zero.
+// f = x - n in [0, 1) goes through a cubic (minimax fit of 2^f, relative error 7.5e-5, far below the rounding of P
+// to bf16 or e4m3 that follows), and n is put back with a shift and an integer add into the exponent field.
+// Valid for x < 127.  x below -125 (masked scores are -inf) is clamped there and comes out as about 2^-125, which
+// rounds to zero in P and vanishes in the row sum; the clamp must stay above -126, where the integer add would
+// carry out of the exponent field and produce a NaN pattern.
 FA_DEVI float2 exp2_poly2(float2 x) {
     const float kMagic = 12582912.f;
-    x.x = fmaxf(x.x, -127.f);
-    x.y = fmaxf(x.y, -127.f);
+    x.x = fmaxf(x.x, -125.f);
+    x.y = fmaxf(x.y, -125.f);
     unsigned long long xb, yb, mb;
     asm("mov.b64 %0, {%1, %2};" : "=l"(xb) : "f"(x.x), "f"(x.y));
     asm("mov.b64 %0, {%1, %1};" : "=l"(mb) : "f"(kMagic));

@@ -112,7 +112,8 @@ def test_fp8_uniform_scores_give_exact_column_means(handle):
     ref = np.cumsum(Vd[0, 0], axis=0) / np.arange(1, w.Sk + 1)[:, None]
     for h in range(w.Hq):
         assert np.abs(O[0, h] - ref).max() <= 2.0 ** -8 * np.abs(ref).max() + 1e-6
-        assert np.abs(lse[0, h] - np.log(np.arange(1, w.Sq + 1))).max() <= 1e-5
+        # (a quarter of the exponentials come from the FMA-pipe polynomial, relative error 7.5e-5: 2^0 is 0.999925 there)
+        assert np.abs(lse[0, h] - np.log(np.arange(1, w.Sq + 1))).max() <= 5e-5
 
 
 def test_fp8_scales_are_applied_per_block(handle):

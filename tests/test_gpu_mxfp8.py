@@ -130,7 +130,8 @@ def test_mx_uniform_scores_give_exact_column_means(handle, d):
     ref = np.cumsum(Vd[0, 0], axis=0) / np.arange(1, 301)[:, None]
     for h in range(2):
         assert (np.abs(O[0, h] - ref) <= 2.0 ** -8 * np.abs(ref) + 2.0 ** -20 * np.abs(Vd[0, 0]).max(axis=0)[None, :] + 1e-7).all()
-        assert np.abs(lse[0, h] - np.log(np.arange(1, 301))).max() <= 1e-5
+        # (a quarter of the exponentials come from the FMA-pipe polynomial, relative error 7.5e-5: 2^0 is 0.999925 there)
+        assert np.abs(lse[0, h] - np.log(np.arange(1, 301))).max() <= 5e-5
 
 
 def test_mx_powers_of_two_move_between_codes_and_scales(handle):
