@@ -23,8 +23,8 @@
 //   q_full, k_full[], v_full[], p_first[], p_rest[]   live in the leader: TMA loads of both CTAs complete
 //       their bytes there (cp.async.bulk.tensor with .cta_group::2), softmax warps of both CTAs arrive there
 //       (mbarrier.arrive on the mapped shared::cluster address);
-//   s_full[], k_empty[], v_empty[], o_final            exist in both CTAs and are signalled in both by one
-//       tcgen05.commit.cta_group::2 with a CTA mask;
+//   s_full[], k_empty[], v_empty[], o_final            exist in both CTAs and are signalled in both by a pair of
+//       tcgen05.commit.cta_group::2, one per CTA (the partner's barrier through its mapped address);
 //   every wait is bounded as elsewhere; a wait that runs out raises the abort flag of both CTAs.
 // A CTA must not exit while its partner can still touch its shared memory or TMEM: all threads of the
 // cluster meet at a cluster barrier before TMEM is freed.  (barrier.cluster.wait only waits for threads
@@ -339,7 +339,6 @@ fa_fwd_duo_kernel(const __grid_constant__ CUtensorMap tm_q,
             // k-step k of Q (chunks of 128 rows) and of this CTA's half of K (chunks of 64 rows)
             auto qoff = [](int k) -> uint32_t { return static_cast<uint32_t>(((k / 4) * kChunkBytes + (k % 4) * 32) >> 4); };
             auto koff = [](int k) -> uint32_t { return static_cast<uint32_t>(((k / 4) * Cfg::kKHalfChunkBytes + (k % 4) * 32) >> 4); };
-            constexpr uint16_t kBoth = 3;
             // a barrier whose phase 0 completed long ago and which never moves again: filler for unused probe slots
             const uint32_t bar_always = smem_addr(&sh.q_full);
 
@@ -355,8 +354,8 @@ fa_fwd_duo_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                         for (int k = 0; k < kKSteps; ++k)
                             mma2_ss(tS, desc(q_lo + qoff(k)), desc(klo + koff(k)), kIdescQK, k > 0 ? 1u : 0u);
-                        tc_commit_2cta(smem_addr(&sh.s_full[t]), kBoth);
-                        tc_commit_2cta(smem_addr(&sh.k_empty[t]), kBoth);
+                        tc_commit_2cta(smem_addr(&sh.s_full[t]), mapa_shared(smem_addr(&sh.s_full[t]), 1u));
+                        tc_commit_2cta(smem_addr(&sh.k_empty[t]), mapa_shared(smem_addr(&sh.k_empty[t]), 1u));
                     }
                 }
             }
@@ -412,10 +411,10 @@ fa_fwd_duo_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                     for (int k = 7; k < kKSteps; ++k)
                         mma2_ss(tS, desc(q_lo + qoff(k)), desc(klo + koff(k)), kIdescQK, 1u);
-                    tc_commit_2cta(smem_addr(&sh.s_full[bsel]), kBoth);
+                    tc_commit_2cta(smem_addr(&sh.s_full[bsel]), mapa_shared(smem_addr(&sh.s_full[bsel]), 1u));
                 }
-                tc_commit_2cta(smem_addr(&sh.v_empty[sv]), kBoth);
-                if (more) tc_commit_2cta(smem_addr(&sh.k_empty[sk]), kBoth);
+                tc_commit_2cta(smem_addr(&sh.v_empty[sv]), mapa_shared(smem_addr(&sh.v_empty[sv]), 1u));
+                if (more) tc_commit_2cta(smem_addr(&sh.k_empty[sk]), mapa_shared(smem_addr(&sh.k_empty[sk]), 1u));
                 sv = sv_n; ph_v = ph_v_n; sk = sk_n; ph_k = ph_k_n;
                 return true;
             };
@@ -424,7 +423,7 @@ fa_fwd_duo_kernel(const __grid_constant__ CUtensorMap tm_q,
                 ok = tile_block(IntC<0>{}, j);
                 if (ok && j + 1 < n_kv) ok = tile_block(IntC<1>{}, j + 1);
             }
-            if (ok) tc_commit_2cta(smem_addr(&sh.o_final), kBoth);
+            if (ok) tc_commit_2cta(smem_addr(&sh.o_final), mapa_shared(smem_addr(&sh.o_final), 1u));
         }
     } else if (warp == 9) {
         // ============================================================ TMA loads: this CTA's Q tile and its halves of K_j, V_j

@@ -551,7 +551,7 @@ FA_DEVI void st_shared_cluster_u32(uint32_t addr_cluster, uint32_t v) {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr_cluster), "r"(v) : "memory");
 }
 // 4-D tiled load into this CTA's shared memory whose bytes are counted on an mbarrier that may sit in the partner
-// CTA (shared::cluster address).  No multicast: every CTA fetches its own box.
+// CTA (shared::cluster address).  Every CTA fetches its own box into its own shared memory.
 FA_DEVI void tma_load_4d_2cta(uint32_t dst_smem, const CUtensorMap* map, uint32_t bar_cluster,
                               int c0, int c1, int c2, int c3) {
     asm volatile(
@@ -573,11 +573,11 @@ FA_DEVI void tmem_dealloc_2cta(uint32_t taddr, uint32_t ncols) {
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
                  : "memory");
 }
-// Arrive (count 1) on the mbarrier at this offset in every CTA of `cta_mask` once every tcgen05 async op
-// issued so far by this thread has completed.
-FA_DEVI void tc_commit_2cta(uint32_t bar, uint16_t cta_mask) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"(cta_mask) : "memory");
+// Arrive (count 1) on the mbarrier at this offset in BOTH CTAs of the pair once every tcgen05 async op issued so far
+// by this thread has completed: one commit per CTA, the partner's barrier through its mapped address.
+FA_DEVI void tc_commit_2cta(uint32_t bar, uint32_t bar_in_partner) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_in_partner) : "memory");
 }
 // 256 x N x 16 MMAs over a CTA pair, issued by ONE thread of the even CTA: rows 0..127 of A and D belong to the
 // even CTA, rows 128..255 to the odd one; each CTA supplies N/2 columns of B from its own shared memory (same
