@@ -194,3 +194,48 @@ def test_mx_argument_errors(handle):
                                     None, *args, 128, False, 0.0) == binding.FA_OK
     torch.cuda.synchronize()
     assert binding.fa_last_status(handle) == (binding.FA_OK, 0)
+
+
+def test_fuzz_mx_and_8bit_192(handle):
+    """Seeded random problems through the two newest 8-bit forms (the MX entry at head sizes 64 and 128, and
+    fa_forward_fp8 at 192/128), whatever split count the library plans for them, each against the oracle on the
+    represented tensors."""
+    import torch
+    from paper_2609_21264_b200 import binding
+    rng = np.random.default_rng(20261205)
+    dev = lambda a: torch.from_numpy(a).cuda()
+    splits_seen = set()
+    for it in range(48):
+        mx = bool(it % 2)
+        d = int(rng.choice([64, 128])) if mx else 192
+        dv = 128 if d == 192 else d
+        hkv, gqa, B = int(rng.integers(1, 4)), int(rng.choice([1, 2, 4, 6])), int(rng.integers(1, 3))
+        causal = bool(rng.integers(0, 2))
+        shape = int(rng.integers(0, 4))
+        if shape == 0:
+            sq, sk = int(rng.integers(1, 65)), int(rng.integers(1, 5000))        # decode-like
+        elif shape == 1:
+            sq = sk = int(rng.integers(1, 900))
+        elif shape == 2:
+            sq, sk = int(rng.integers(100, 700)), int(rng.integers(1, 300))      # more queries than keys
+        else:
+            sq, sk = int(rng.integers(65, 300)), int(rng.integers(1000, 4000))
+        name = "case%d %s b%d h%dx%d %dx%d d%d %s" % (it, "mx" if mx else "e4m3", B, hkv, gqa, sq, sk, d, "causal" if causal else "full")
+        w = W.Workload(name, B=B, Hq=hkv * gqa, Hkv=hkv, Sq=sq, Sk=sk, dqk=d, dv=dv, causal=causal, scale=d ** -0.5, seed=31000 + it)
+        Q = rng.standard_normal((B, w.Hq, sq, d)); K = rng.standard_normal((B, hkv, sk, d)); V = rng.standard_normal((B, hkv, sk, dv))
+        if mx:
+            (q8, k8, v8, qa, ka, va), (Qd, Kd, Vd) = _quantise(w, Q, K, V)
+            o, lse = binding.forward_mxfp8(handle, dev(q8), dev(k8), dev(v8), dev(qa), dev(ka), dev(va), causal=causal, scale=w.scale)
+        else:
+            q8, sqs, Qd = W.quantize_e4m3_blocks(Q, 128)
+            k8, sks, Kd = W.quantize_e4m3_blocks(K, 128)
+            v8, svs, Vd = W.quantize_e4m3_blocks(V, None)
+            o, lse = binding.forward_fp8(handle, dev(q8), dev(k8), dev(v8), dev(sqs), dev(sks), dev(svs), causal=causal, scale=w.scale)
+        torch.cuda.synchronize()
+        st, detail = binding.fa_last_status(handle)
+        assert st == binding.FA_OK, (name, st, hex(detail))
+        assert binding.fa_last_kernel_name(handle) == ("fa_fwd_mxfp8_stream" if mx else "fa_fwd_fp8_stream"), name
+        splits_seen.add((mx, binding.fa_last_kv_splits(handle) > 1))
+        O_ref, lse_ref = oracle.attention(Qd, Kd, Vd, causal=causal, scale=w.scale)
+        _check(w, bf16_tensor_to_f64(o), lse.double().cpu().numpy(), O_ref, lse_ref, Vd, mean_bound=1e-2)
+    assert splits_seen == {(True, False), (True, True), (False, False), (False, True)}, splits_seen
