@@ -109,6 +109,10 @@ typedef enum fa_status {
  * warpgroups keep separate partial results for the even and the odd K/V tiles and merge them at
  * the end, so its output agrees with the other kernels' to rounding, not bit for bit. */
 #define FA_FLAG_TWO_CTA_KERNEL 512u
+/* fa_config.flags: run the same class of problems on the kernel that gives a pair of SMs FOUR query tiles (two
+ * per CTA, as in the pair kernels, every MMA a two-CTA tcgen05.mma over one tile of each CTA): csrc/fa_fwd_quad.cuh.
+ * Takes precedence over FA_FLAG_TWO_CTA_KERNEL. */
+#define FA_FLAG_QUAD_KERNEL 1024u
 
 /* Optional creation parameters.  Zero-initialise, set struct_size = sizeof(fa_config). */
 typedef struct fa_config {

@@ -30,6 +30,7 @@ FA_FLAG_NO_STREAM_KERNEL = 64
 FA_FLAG_NO_HEAD_PACKING = 128
 FA_FLAG_LEGACY_PAIR_KERNEL = 256
 FA_FLAG_TWO_CTA_KERNEL = 512
+FA_FLAG_QUAD_KERNEL = 1024
 
 EXPORTS = ("fa_create", "fa_forward", "fa_forward_strided", "fa_forward_varlen", "fa_forward_fp8", "fa_forward_mxfp8", "fa_plan", "fa_forward_host", "fa_last_status", "fa_destroy",
            "fa_strerror", "fa_launch_count", "fa_last_kernel_name", "fa_last_kv_splits",

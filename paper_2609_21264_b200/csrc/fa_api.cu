@@ -15,6 +15,7 @@
 #include "fa_fwd_pipelined.cuh"
 #include "fa_fwd_pair.cuh"
 #include "fa_fwd_duo.cuh"
+#include "fa_fwd_quad.cuh"
 #include "fa_fwd_pair_persistent.cuh"
 #include "fa_fwd_persistent.cuh"
 #include "fa_fwd_stream.cuh"
@@ -253,6 +254,33 @@ fa_status launch_duo(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& mk,
     return FA_OK;
 }
 
+// Four query tiles per pair of CTAs (clusters of two, two-CTA MMAs, two tiles per CTA): fa_fwd_quad.cuh.
+template <int DQK, int DV, int kMode>
+fa_status launch_quad(fa_handle* h, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                      const CUtensorMap& mo, const fa::FwdParams& p, cudaStream_t st) {
+    constexpr int smem = fa::quad_smem_bytes<DQK, DV>();
+    static_assert(smem <= 227 * 1024, "shared memory budget exceeded");
+    auto kernel = fa::fa_fwd_quad_kernel<DQK, DV, kMode>;
+    fa_status s = ensure_smem_attr(h, kernel, smem);
+    if (s != FA_OK) return s;
+    constexpr int heads = kMode == 0 ? 1 : (kMode == 1 ? 2 : 4);      // heads of an item; 4 / heads adjacent tiles of each
+    const long long n_ctas = 2ll * ((p.n_q_tiles + 4 / heads - 1) / (4 / heads)) * (p.Hq / heads) * p.B;
+    if (n_ctas > 0x7fffffffLL) return FA_ERR_UNSUPPORTED;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);       // the kernel carries __cluster_dims__(2, 1, 1)
+    cfg.blockDim = dim3(fa::QuadCfg<DQK, DV>::kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = (h->flags & FA_FLAG_NO_DEPENDENT_LAUNCH) ? 0 : 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mo, p) != cudaSuccess) return FA_ERR_CUDA;
+    h->launches += 1;
+    return FA_OK;
+}
+
 // Number of K/V splits for a problem: 1 unless the query tiles alone leave most SMs idle and the
 // K/V range is long enough to cut; never more than the scratch buffer can hold partials for.
 int choose_kv_splits(int num_sms, uint32_t kv_splits_cfg, size_t scratch_bytes, int B, int Hq, int Sq, int Sk, int dv,
@@ -456,12 +484,13 @@ TilingEstimate estimate_tilings(int num_sms, int B, int Hq, int Sq, int Sk, int 
 
 // Which kernel a launch uses and how its K/V range is split: a pure function of the problem, the
 // handle's configuration and the SM count (fa_plan exposes it).
-enum PlanKernel { kPlanSerial = 0, kPlanPair = 1, kPlanPersistent = 2, kPlanStream = 3, kPlanDuo = 4 };
+enum PlanKernel { kPlanSerial = 0, kPlanPair = 1, kPlanPersistent = 2, kPlanStream = 3, kPlanDuo = 4, kPlanQuad = 5 };
 struct LaunchPlan {
     int kernel;
     int kv_splits;
     int tiles_per_split;
     int pack_heads;                // > 1: stream kernel with that many query heads of a K/V head per query tile
+    int quad_mode;                 // quad kernel: which four tiles a cluster takes (fa_fwd_quad.cuh)
     bool head_pair;                // pair kernel: the CTA's two tiles are one query tile of two adjacent heads of a group
     double pair_us, stream_us;     // the two estimates (0 when no estimate was needed)
 };
@@ -474,6 +503,7 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     pl.tiles_per_split = 0x3fffffff;
     pl.pack_heads = 1;
     pl.head_pair = false;
+    pl.quad_mode = 0;
     pl.pair_us = pl.stream_us = 0.0;
     const int n_q_tiles = (Sq + fa::kTileM - 1) / fa::kTileM;
     int max_tiles = (Sk + fa::kTileN - 1) / fa::kTileN;           // K/V tiles of the longest query tile
@@ -565,7 +595,11 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
     const bool duo_ok = !varlen && dqk != 64 && pair_splits == 1 && stream_splits == 1;
     bool duo = false;
     if ((flags & FA_FLAG_TWO_CTA_KERNEL) && duo_ok) duo = true;
-    if (duo) {
+    if ((flags & FA_FLAG_QUAD_KERNEL) && duo_ok) {
+        pl.kernel = kPlanQuad;
+        const int gqa = Hq / Hkv;
+        pl.quad_mode = (flags & FA_FLAG_NO_HEAD_PACKING) ? 0 : (gqa % 4 == 0 ? 2 : (gqa % 2 == 0 ? 1 : 0));
+    } else if (duo) {
         pl.kernel = kPlanDuo;
         pl.head_pair = head_pair_ok;
     } else if (stream) {
@@ -676,6 +710,17 @@ fa_status run_forward(fa_handle* h, const CUtensorMap& map_q, const CUtensorMap&
         if (dqk == 128) return launch_pipelined<128, 128, false>(h, map_q, map_k, map_v, map_o, p, st);
         return launch_pipelined<192, 128, false>(h, map_q, map_k, map_v, map_o, p, st);
     }
+    if (pl.kernel == kPlanQuad) {
+        h->last_kernel = "fa_fwd_quad";
+        if (dqk == 128) {
+            if (pl.quad_mode == 2) return launch_quad<128, 128, 2>(h, map_q, map_k, map_v, map_o, p, st);
+            if (pl.quad_mode == 1) return launch_quad<128, 128, 1>(h, map_q, map_k, map_v, map_o, p, st);
+            return launch_quad<128, 128, 0>(h, map_q, map_k, map_v, map_o, p, st);
+        }
+        if (pl.quad_mode == 2) return launch_quad<192, 128, 2>(h, map_q, map_k, map_v, map_o, p, st);
+        if (pl.quad_mode == 1) return launch_quad<192, 128, 1>(h, map_q, map_k, map_v, map_o, p, st);
+        return launch_quad<192, 128, 0>(h, map_q, map_k, map_v, map_o, p, st);
+    }
     if (pl.kernel == kPlanDuo) {
         h->last_kernel = "fa_fwd_duo";
         if (pl.head_pair) {
@@ -726,7 +771,7 @@ fa_status fa_create(fa_handle** out, const fa_config* cfg) {
         if (flags & ~(FA_FLAG_SERIAL_KERNEL | FA_FLAG_DEBUG_DROP_V_LOAD | FA_FLAG_NO_DEPENDENT_LAUNCH |
                       FA_FLAG_NO_PERSISTENT | FA_FLAG_FORCE_PERSISTENT | FA_FLAG_STREAM_KERNEL |
                       FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING | FA_FLAG_LEGACY_PAIR_KERNEL |
-                      FA_FLAG_TWO_CTA_KERNEL)) return FA_ERR_INVALID_ARG;
+                      FA_FLAG_TWO_CTA_KERNEL | FA_FLAG_QUAD_KERNEL)) return FA_ERR_INVALID_ARG;
         if (kv_splits_cfg > 256) return FA_ERR_INVALID_ARG;
     }
     if (scratch_bytes == 0) scratch_bytes = 32ull << 20;
@@ -874,7 +919,7 @@ fa_status fa_forward_strided(fa_handle* h, const void* Q, const void* K, const v
     if ((s = get_map(h, Q, dqk, Sq, Hq, B, q_strides[0], q_strides[1], q_strides[2], q_box_rows, &mq, 2, pl.pack_heads)) != FA_OK) return s;
     CUtensorMap map_q = *mq;   // copies: a later insertion may evict or move cache entries
     // (the two-CTA kernel loads K in boxes of 64 keys: each CTA of a pair keeps half of a K tile)
-    const int k_box_rows = pl.kernel == kPlanDuo ? fa::kTileN / 2 : fa::kTileN;
+    const int k_box_rows = (pl.kernel == kPlanDuo || pl.kernel == kPlanQuad) ? fa::kTileN / 2 : fa::kTileN;
     if ((s = get_map(h, K, dqk, Sk, Hkv, B, k_strides[0], k_strides[1], k_strides[2], k_box_rows, &mk)) != FA_OK) return s;
     CUtensorMap map_k = *mk;
     if ((s = get_map(h, V, dv, Sk, Hkv, B, v_strides[0], v_strides[1], v_strides[2], fa::kTileN, &mv)) != FA_OK) return s;
@@ -1131,7 +1176,7 @@ fa_status fa_plan(int num_sms, const fa_config* cfg, int varlen, int B, int Hq, 
     }
     const LaunchPlan pl = plan_launch(num_sms, flags, splits_cfg, static_cast<size_t>(scratch), varlen != 0,
                                       B, Hq, Hkv, Sq, Sk, dqk, dv, causal ? 1 : 0);
-    static const char* const names[5] = {"fa_fwd_simple", "fa_fwd_pipelined", "fa_fwd_persistent", "fa_fwd_stream", "fa_fwd_duo"};
+    static const char* const names[6] = {"fa_fwd_simple", "fa_fwd_pipelined", "fa_fwd_persistent", "fa_fwd_stream", "fa_fwd_duo", "fa_fwd_quad"};
     out->kernel = names[pl.kernel];
     // the one-item-per-CTA tiling with two query tiles has a kernel of its own at head size 128
     if (pl.kernel == kPlanPair && dqk == 128 && dv == 128 && !(flags & FA_FLAG_LEGACY_PAIR_KERNEL)) out->kernel = "fa_fwd_pair";
@@ -1142,6 +1187,11 @@ fa_status fa_plan(int num_sms, const fa_config* cfg, int varlen, int B, int Hq, 
     switch (pl.kernel) {
         case kPlanSerial: ctas = n_q_tiles * Hq * B; break;
         case kPlanPair: ctas = (pl.head_pair ? n_q_tiles * (Hq / 2) : ((n_q_tiles + 1) / 2) * Hq) * B * pl.kv_splits; break;
+        case kPlanQuad: {
+            const int heads = pl.quad_mode == 0 ? 1 : (pl.quad_mode == 1 ? 2 : 4);
+            ctas = 2 * ((n_q_tiles + 4 / heads - 1) / (4 / heads)) * (Hq / heads) * B;
+            break;
+        }
         case kPlanDuo: ctas = 2 * (pl.head_pair ? n_q_tiles * (Hq / 2) : ((n_q_tiles + 1) / 2) * Hq) * B; break;
         case kPlanPersistent:
             ctas = (pl.head_pair ? n_q_tiles * (Hq / 2) : ((n_q_tiles + 1) / 2) * Hq) * B;

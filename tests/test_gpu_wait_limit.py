@@ -56,13 +56,15 @@ def _kernels():
         ("fa_fwd_persistent", b.FA_FLAG_FORCE_PERSISTENT | b.FA_FLAG_NO_STREAM_KERNEL | b.FA_FLAG_LEGACY_PAIR_KERNEL, "bf16", (2, 4, 2, 300, 300, 128)),
         ("fa_fwd_duo", b.FA_FLAG_TWO_CTA_KERNEL, "bf16", (1, 2, 2, 256, 384, 128)),
         ("fa_fwd_duo", b.FA_FLAG_TWO_CTA_KERNEL, "bf16", (1, 4, 2, 300, 300, 192)),
+        ("fa_fwd_quad", b.FA_FLAG_QUAD_KERNEL, "bf16", (1, 4, 1, 600, 700, 128)),
+        ("fa_fwd_quad", b.FA_FLAG_QUAD_KERNEL, "bf16", (1, 3, 3, 300, 300, 192)),
         ("fa_fwd_fp8", b.FA_FLAG_NO_STREAM_KERNEL, "e4m3", (1, 2, 2, 256, 384, 128)),
         ("fa_fwd_fp8_stream", b.FA_FLAG_STREAM_KERNEL, "e4m3", (1, 2, 1, 200, 500, 128)),
         ("fa_fwd_mxfp8_stream", 0, "mx", (1, 2, 1, 200, 500, 128)),
     ]
 
 
-@pytest.mark.parametrize("case", range(13))
+@pytest.mark.parametrize("case", range(15))
 def test_every_kernel_reports_a_wait_that_runs_out_and_the_handle_recovers(case):
     """The hook drops the first V tile of every CTA: the launch returns (every wait is bounded), the host reads
     FA_ERR_DEVICE_TIMEOUT with the site that gave up, and the NEXT launch through the same handle, with the hook off,

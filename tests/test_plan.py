@@ -153,3 +153,17 @@ def test_two_cta_kernel_is_used_only_where_it_applies():
     assert binding.fa_plan(148, 1, 16, 16, 2048, 2048, 64, 64, True, flags=flags)["kernel"] != "fa_fwd_duo"
     assert binding.fa_plan(148, 4, 16, 4, 1024, 1024, 128, 128, True, flags=flags, varlen=True)["kernel"] != "fa_fwd_duo"
     assert binding.fa_plan(148, 1, 32, 32, 128, 32768, 128, 128, False, flags=flags)["kernel"] != "fa_fwd_duo"   # split-KV
+
+
+def test_quad_kernel_is_used_only_where_it_applies_and_picks_its_tiles_by_group_size():
+    flags = binding.FA_FLAG_QUAD_KERNEL
+    pl = binding.fa_plan(148, 1, 32, 8, 2048, 2048, 128, 128, True, flags=flags)
+    assert pl["kernel"] == "fa_fwd_quad" and pl["ctas"] == 2 * 16 * 8            # four heads x one tile per cluster
+    pl = binding.fa_plan(148, 1, 32, 16, 2048, 2048, 128, 128, True, flags=flags)
+    assert pl["kernel"] == "fa_fwd_quad" and pl["ctas"] == 2 * 8 * 16            # two heads x two adjacent tiles
+    pl = binding.fa_plan(148, 1, 128, 128, 4096 + 128, 4096 + 128, 192, 128, True, flags=flags)
+    assert pl["kernel"] == "fa_fwd_quad" and pl["ctas"] == 2 * 9 * 128           # one head x four tiles, 33 tiles -> 9 clusters
+    assert binding.fa_plan(148, 1, 16, 16, 2048, 2048, 64, 64, True, flags=flags)["kernel"] != "fa_fwd_quad"
+    assert binding.fa_plan(148, 4, 16, 4, 1024, 1024, 128, 128, True, flags=flags, varlen=True)["kernel"] != "fa_fwd_quad"
+    assert binding.fa_plan(148, 1, 32, 32, 128, 32768, 128, 128, False, flags=flags)["kernel"] != "fa_fwd_quad"   # split-KV
+
