@@ -298,7 +298,7 @@ def oracle_timed(w, budget_s=20.0, host=None):
 DECODE_SHAPES = ((8, 32, 8, 1, 8192, 128), (64, 32, 8, 1, 4096, 128), (1, 32, 8, 16, 131072, 128), (4, 32, 8, 128, 8192, 128))
 
 
-def time_libraries(binding, h, device):
+def time_libraries(binding, h, device, only=None):
     """Library attention kernels on the same GPU and shapes, for context: PyTorch's
     scaled_dot_product_attention with each of its fused back ends, and flash_attn where it is
     installed.  One input set per shape (the library kernels and ours see the same L2 state);
@@ -352,6 +352,10 @@ def time_libraries(binding, h, device):
         return row
 
     rows = []
+    if only is not None:            # a custom shape: that shape alone
+        fa, _, _ = workload_numbers(only)
+        return [one_shape(only.name, only.B, only.Hq, only.Hkv, only.Sq, only.Sk, only.dqk, only.dv, only.causal, only.scale, fa,
+                          2 * only.B * only.Hkv * only.Sk * (only.dqk + only.dv))]
     for wc in workloads.CONFIGS:
         fa, _, _ = workload_numbers(wc)
         rows.append(one_shape(wc.name, wc.B, wc.Hq, wc.Hkv, wc.Sq, wc.Sk, wc.dqk, wc.dv, wc.causal, wc.scale, fa,
@@ -517,7 +521,8 @@ def plan_ab(binding, device, gpu_index):
     import torch
     variants = (("planned", 0), ("two_tiles_per_item", binding.FA_FLAG_NO_PERSISTENT | binding.FA_FLAG_NO_STREAM_KERNEL),
                 ("persistent", binding.FA_FLAG_FORCE_PERSISTENT | binding.FA_FLAG_NO_STREAM_KERNEL),
-                ("stream", binding.FA_FLAG_STREAM_KERNEL), ("two_cta", binding.FA_FLAG_TWO_CTA_KERNEL))
+                ("stream", binding.FA_FLAG_STREAM_KERNEL), ("two_cta", binding.FA_FLAG_TWO_CTA_KERNEL),
+                ("two_cta_four_tiles", binding.FA_FLAG_QUAD_KERNEL))
     handles = {name: binding.fa_create(device=device.index, flags=flags) for name, flags in variants}
     cases = list(workloads.CONFIGS)
     for (B, Hq, Hkv, S, causal) in ((64, 32, 8, 128, True), (32, 32, 8, 256, True), (16, 32, 8, 512, True), (8, 32, 8, 1024, True),
@@ -572,6 +577,9 @@ def main():
     ap.add_argument("--libraries", action="store_true",
                     help="also time the attention kernels of the libraries in the image (torch SDPA back ends, flash_attn) "
                          "on the five configurations and a few decode shapes, for context (key 'libraries')")
+    ap.add_argument("--flags", type=int, default=0,
+                    help="fa_config.flags of the handle that runs the workload (FA_FLAG_* bits, e.g. 1024 for the kernel with "
+                         "four query tiles per pair of SMs); for A/B timing and ncu captures of a kernel the planner does not pick")
     args = ap.parse_args()
     w = workloads.config(args.config)
     if args.shape:
@@ -609,8 +617,8 @@ def main():
 
     gpu_index = physical_gpu_index(local)
     peaks = load_peaks()
-    h = binding.fa_create(device=local)
-    h_plain = binding.fa_create(device=local, flags=binding.FA_FLAG_NO_DEPENDENT_LAUNCH)
+    h = binding.fa_create(device=local, flags=args.flags)
+    h_plain = binding.fa_create(device=local, flags=args.flags | binding.FA_FLAG_NO_DEPENDENT_LAUNCH)
     rec, roofline, seconds, launches, steps, warmup = measure_config(binding, h, h_plain, w, device, peaks, gpu_index, steps, warmup, world)
     t_step = seconds / steps
     clocks = rec["clocks"]
@@ -626,6 +634,8 @@ def main():
             "paper_context": "3.62 TFLOP_GEMM/s on XDNA 2 (paper's headline, other hardware and shape)",
             "per_launch_us_min": rec["per_launch_us_min"], "per_launch_us_median": rec["per_launch_us_median"],
             "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches)}
+    if args.flags:
+        line["config"]["handle_flags"] = args.flags
 
     if (args.eight_bit or not args.no_sweep) and world == 1 and w.dqk == 128 and w.dv == 128:
         # the block-scaled e4m3 variant on the same shape (N(0, sigma^2) rounded to e4m3, unit scales), for context
@@ -807,7 +817,7 @@ def main():
         line["table6"] = rows
 
     if args.libraries and world == 1:
-        line["libraries"] = time_libraries(binding, h, device)
+        line["libraries"] = time_libraries(binding, h, device, only=w if args.shape else None)
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = oracle_timed(w, host=host)
