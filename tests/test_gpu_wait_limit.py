@@ -51,6 +51,7 @@ def _kernels():
         ("fa_fwd_pipelined", b.FA_FLAG_NO_STREAM_KERNEL | b.FA_FLAG_NO_PERSISTENT, "bf16", (1, 2, 2, 256, 384, 64)),
         ("fa_fwd_stream", b.FA_FLAG_STREAM_KERNEL, "bf16", (1, 2, 1, 200, 500, 128)),
         ("fa_fwd_stream", b.FA_FLAG_STREAM_KERNEL, "bf16", (1, 2, 2, 130, 300, 192)),
+        ("fa_fwd_stream_persistent", b.FA_FLAG_STREAM_KERNEL, "bf16", (8, 16, 4, 512, 640, 192)),
         ("fa_fwd_persistent", b.FA_FLAG_FORCE_PERSISTENT | b.FA_FLAG_NO_STREAM_KERNEL, "bf16", (2, 4, 2, 300, 300, 128)),
         ("fa_fwd_persistent", b.FA_FLAG_FORCE_PERSISTENT | b.FA_FLAG_NO_STREAM_KERNEL, "bf16", (2, 4, 4, 300, 300, 64)),
         ("fa_fwd_persistent", b.FA_FLAG_FORCE_PERSISTENT | b.FA_FLAG_NO_STREAM_KERNEL | b.FA_FLAG_LEGACY_PAIR_KERNEL, "bf16", (2, 4, 2, 300, 300, 128)),
@@ -64,7 +65,7 @@ def _kernels():
     ]
 
 
-@pytest.mark.parametrize("case", range(15))
+@pytest.mark.parametrize("case", range(16))
 def test_every_kernel_reports_a_wait_that_runs_out_and_the_handle_recovers(case):
     """The hook drops the first V tile of every CTA: the launch returns (every wait is bounded), the host reads
     FA_ERR_DEVICE_TIMEOUT with the site that gave up, and the NEXT launch through the same handle, with the hook off,

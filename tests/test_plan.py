@@ -14,8 +14,9 @@ def plan(w, **kw):
 
 
 def test_benchmark_configurations():
-    # (config 3: 4096 items of up to 64 K/V tiles, 27 per SM: the persistent kernel; config 5: items of 1024 tiles)
-    expect = ["fa_fwd_stream", "fa_fwd_pair", "fa_fwd_persistent", "fa_fwd_stream", "fa_fwd_pair"]
+    # (config 3: 4096 items of up to 64 K/V tiles, 27 per SM: the persistent kernel; config 4: 4096 one-tile items of up
+    #  to 32 K/V tiles at 192/128: the stream kernel's persistent form; config 5: items of 1024 tiles)
+    expect = ["fa_fwd_stream", "fa_fwd_pair", "fa_fwd_persistent", "fa_fwd_stream_persistent", "fa_fwd_pair"]
     for w, kernel in zip(W.CONFIGS, expect):
         p = plan(w)
         assert p["kernel"] == kernel, (w.name, p)
@@ -23,7 +24,8 @@ def test_benchmark_configurations():
     # grid sizes: one CTA per query tile or per pair of query tiles
     assert plan(W.CONFIGS[0])["ctas"] == 12 * 4
     assert plan(W.CONFIGS[1])["ctas"] == 32 * 8
-    assert plan(W.CONFIGS[3])["ctas"] == 128 * 32
+    assert plan(W.CONFIGS[3])["ctas"] == SMS                  # one CTA per SM walks the 128 * 32 items
+    assert plan(W.CONFIGS[3], flags=binding.FA_FLAG_NO_PERSISTENT)["ctas"] == 128 * 32
 
 
 def test_table6_rows():
@@ -87,7 +89,8 @@ def test_few_queries_with_grouped_heads_share_a_query_tile():
 
 def test_flags_and_configuration_override_the_choice():
     w = W.CONFIGS[1]
-    assert plan(w, flags=binding.FA_FLAG_STREAM_KERNEL)["kernel"] == "fa_fwd_stream"
+    assert plan(w, flags=binding.FA_FLAG_STREAM_KERNEL)["kernel"] == "fa_fwd_stream_persistent"     # 512 one-tile items
+    assert plan(w, flags=binding.FA_FLAG_STREAM_KERNEL | binding.FA_FLAG_NO_PERSISTENT)["kernel"] == "fa_fwd_stream"
     assert plan(w, flags=binding.FA_FLAG_FORCE_PERSISTENT | binding.FA_FLAG_NO_STREAM_KERNEL)["kernel"] == "fa_fwd_persistent"
     assert plan(w, flags=binding.FA_FLAG_SERIAL_KERNEL)["kernel"] == "fa_fwd_simple"
     assert plan(W.CONFIGS[0], flags=binding.FA_FLAG_NO_STREAM_KERNEL)["kernel"] == "fa_fwd_pipelined"
@@ -166,4 +169,16 @@ def test_quad_kernel_is_used_only_where_it_applies_and_picks_its_tiles_by_group_
     assert binding.fa_plan(148, 1, 16, 16, 2048, 2048, 64, 64, True, flags=flags)["kernel"] != "fa_fwd_quad"
     assert binding.fa_plan(148, 4, 16, 4, 1024, 1024, 128, 128, True, flags=flags, varlen=True)["kernel"] != "fa_fwd_quad"
     assert binding.fa_plan(148, 1, 32, 32, 128, 32768, 128, 128, False, flags=flags)["kernel"] != "fa_fwd_quad"   # split-KV
+
+
+def test_persistent_stream_kernel_takes_short_one_tile_items_only():
+    kernel = lambda B, H, S, causal, **kw: binding.fa_plan(SMS, B, H, H, S, S, 192, 128, causal, **kw)["kernel"]
+    assert kernel(4, 128, 2048, True) == "fa_fwd_stream_persistent"       # 8192 items of up to 16 K/V tiles
+    assert kernel(1, 128, 4096, True) == "fa_fwd_stream_persistent"       # up to 32
+    assert kernel(1, 128, 8192, True) == "fa_fwd_stream"                  # longer items: no gain measured
+    assert kernel(1, 8, 2048, True) == "fa_fwd_stream"                    # 128 items: under three per SM
+    assert kernel(4, 128, 2048, True, flags=binding.FA_FLAG_NO_PERSISTENT) == "fa_fwd_stream"
+    assert kernel(1, 128, 8192, True, flags=binding.FA_FLAG_FORCE_PERSISTENT | binding.FA_FLAG_STREAM_KERNEL) == "fa_fwd_stream_persistent"
+    # packed batches and split-KV stay on the one-item kernel
+    assert binding.fa_plan(SMS, 64, 128, 128, 512, 512, 192, 128, True, varlen=True)["kernel"] == "fa_fwd_stream"
 
