@@ -521,7 +521,9 @@ def plan_ab(binding, device, gpu_index):
     import torch
     variants = (("planned", 0), ("two_tiles_per_item", binding.FA_FLAG_NO_PERSISTENT | binding.FA_FLAG_NO_STREAM_KERNEL),
                 ("persistent", binding.FA_FLAG_FORCE_PERSISTENT | binding.FA_FLAG_NO_STREAM_KERNEL),
-                ("stream", binding.FA_FLAG_STREAM_KERNEL), ("two_cta", binding.FA_FLAG_TWO_CTA_KERNEL),
+                ("stream", binding.FA_FLAG_STREAM_KERNEL | binding.FA_FLAG_NO_PERSISTENT),
+                ("stream_persistent", binding.FA_FLAG_STREAM_KERNEL | binding.FA_FLAG_FORCE_PERSISTENT),
+                ("two_cta", binding.FA_FLAG_TWO_CTA_KERNEL),
                 ("two_cta_four_tiles", binding.FA_FLAG_QUAD_KERNEL))
     handles = {name: binding.fa_create(device=device.index, flags=flags) for name, flags in variants}
     cases = list(workloads.CONFIGS)

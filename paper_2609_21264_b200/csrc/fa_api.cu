@@ -1054,8 +1054,9 @@ static fa_status forward_fp8_common(fa_handle* h, const void* Q8, const void* K8
     const uint32_t plan_flags = (mx || d == 192) ? ((h->flags & ~(FA_FLAG_NO_STREAM_KERNEL | FA_FLAG_FORCE_PERSISTENT | FA_FLAG_TWO_CTA_KERNEL)) |
                                                     FA_FLAG_STREAM_KERNEL | FA_FLAG_NO_HEAD_PACKING)
                                                  : h->flags;
-    const LaunchPlan pl = plan_launch(h->num_sms, plan_flags, h->kv_splits_cfg, h->scratch_bytes, false,
-                                      B, Hq, Hkv, Sq, Sk, d, dv, causal ? 1 : 0);
+    LaunchPlan pl = plan_launch(h->num_sms, plan_flags, h->kv_splits_cfg, h->scratch_bytes, false,
+                                B, Hq, Hkv, Sq, Sk, d, dv, causal ? 1 : 0);
+    if (pl.kernel == kPlanStreamPersistent) pl.kernel = kPlanStream;      // (the 8-bit stream kernel has no persistent form)
     const int q_box_rows = pl.pack_heads > 1 ? Sq : fa::kTileM;
     // an e4m3 row is d bytes: one box column of d bytes, swizzled over d bytes
     const CUtensorMap *mq = nullptr, *mk = nullptr, *mv = nullptr, *mo = nullptr;

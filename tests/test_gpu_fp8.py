@@ -199,6 +199,33 @@ def test_fp8_default_handle_plans_both_tilings():
         binding.fa_destroy(h)
 
 
+def test_fp8_many_short_items_stay_on_the_8bit_stream_kernel():
+    """Where the 16-bit planner would pick the persistent form of its stream kernel (many one-tile items, here 512 of up
+    to four K/V tiles at 192/128 and in MX form), the 8-bit entries, which have no such form, run their stream kernel
+    and match a second launch whose planner is told not to use persistent kernels at all."""
+    from paper_2609_21264_b200 import binding
+    import torch
+    # (the 8-bit entries force the stream tiling at 192/128)
+    assert binding.fa_plan(148, 4, 32, 32, 512, 512, 192, 128, True, flags=binding.FA_FLAG_STREAM_KERNEL)["kernel"] == "fa_fwd_stream_persistent"
+    g = torch.Generator(device="cuda").manual_seed(1340)
+    mk = lambda *shape: torch.randn(shape, generator=g, device="cuda").to(torch.float8_e4m3fn).view(torch.uint8)
+    outs = []
+    for flags in (0, binding.FA_FLAG_NO_PERSISTENT):
+        h = binding.fa_create(flags=flags)
+        try:
+            q8, k8, v8 = mk(4, 32, 512, 192), mk(4, 32, 512, 192), mk(4, 32, 512, 128)
+            o, lse = binding.forward_fp8(h, q8, k8, v8, None, None, None, causal=True, scale=192 ** -0.5)
+            torch.cuda.synchronize()
+            assert binding.fa_last_status(h) == (binding.FA_OK, 0)
+            assert binding.fa_last_kernel_name(h) == "fa_fwd_fp8_stream"
+            outs.append((o.clone(), lse.clone()))
+            g.manual_seed(1340)
+        finally:
+            binding.fa_destroy(h)
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    assert torch.isfinite(outs[0][0].float()).all()
+
+
 def test_fp8_unsupported_head_size(handle):
     import torch
     from paper_2609_21264_b200 import binding
