@@ -19,9 +19,11 @@
 //     tiles have gone through the rings, and how many items it has finished;
 //   * the O accumulator: the first PV product of an item (accumulate = 0) waits until the epilogue of the item before
 //     has read O out of TMEM (o_read);
-//   * the output is staged for its TMA store in a stage of the K ring (an O tile is never larger than a K tile): every
-//     item takes one more ring position than it has K tiles, the one after its last K tile, which nothing is loaded
-//     into and whose "empty" arrival comes from the storing thread instead of an MMA commit.  So the query tile's
+//   * the output is staged for its TMA store in a stage of the V ring (an O tile is exactly as large as a V tile): every
+//     item takes one more ring position than it has V tiles, the one after its last V tile, which nothing is loaded
+//     into and whose "empty" arrival comes from the storing thread instead of an MMA commit.  (The V ring, not the K
+//     ring: with two stages of each at 192/128 the stage comes back only when the store has read it, and the next
+//     item's second V tile is needed a softmax pass later than its second K tile.)  So the query tile's
 //     space is free as soon as the item's last score MMA is complete (q_free, a commit), and the next item's Q and
 //     first K/V tiles are loaded, and its first scores computed, under the last softmax passes, the last PV products
 //     and the epilogue of the current item.
@@ -195,7 +197,7 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
         const float tau_raw = kRescaleThresholdLog2 / c;
         uint32_t u_own = 0, u_other = 0;      // uses of this warpgroup's / the other one's buffers before the current item
         uint32_t itc = 0;                     // items with K/V tiles finished so far
-        uint32_t kt = 0;                      // K ring positions taken before the current item
+        uint32_t vt = 0;                      // V ring positions taken before the current item
         bool ok = true;
 
         for (uint32_t k = 0; ok; ++k) {
@@ -373,12 +375,12 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             const float inv_l = (lt > 0.f) ? (1.f / lt) : 0.f;
             if (g == 0 && p.lse && row_valid)
                 p.lse[lse_row0 + i_glob] = (lt > 0.f) ? (m_fin * c * 0.6931471805599453f + logf(lt)) : -INFINITY;
-            // warpgroup g converts columns [g*DV/2, (g+1)*DV/2) of O into the staging tile (the K stage after the
-            // item's last K tile: its previous tile was read by a score MMA that is long complete), then one thread
+            // warpgroup g converts columns [g*DV/2, (g+1)*DV/2) of O into the staging tile (the V stage after the
+            // item's last V tile: its previous tile was read by a PV product that is complete), then one thread
             // stores it with TMA; rows past Sq are clipped
             const uint32_t tO = tmem_base + Cfg::kColO + lane_sel;
-            const int s_stage = static_cast<int>((kt + static_cast<uint32_t>(n_kv)) % NK);
-            const uint32_t s_tile = sK + s_stage * Cfg::kKBytes;
+            const int s_stage = static_cast<int>((vt + static_cast<uint32_t>(n_kv)) % NV);
+            const uint32_t s_tile = sV + s_stage * Cfg::kVBytes;
             const uint32_t sO = s_tile + row * 128;
 #pragma unroll 1
             for (int cc = g * (DV / 64); cc < (g + 1) * (DV / 64); ++cc) {
@@ -410,11 +412,11 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                     for (int ch = 0; ch < DV / kChunkCols; ++ch)
                         tma_store_4d(&tm_o, s_tile + ch * kChunkBytes, ch * kChunkCols, i0, it.hq, it.b);
                     tma_store_commit();
-                    tma_store_wait_read_all();     // the staging tile goes back to the K ring
-                    mbar_arrive(smem_addr(&sh.k_empty[s_stage]));
+                    tma_store_wait_read_all();     // the staging tile goes back to the V ring
+                    mbar_arrive(smem_addr(&sh.v_empty[s_stage]));
                 }
             }
-            kt += static_cast<uint32_t>(n_kv) + 1u;
+            vt += static_cast<uint32_t>(n_kv) + 1u;
             u_own += static_cast<uint32_t>((n_kv + 1 - g) >> 1);        // tiles j = g, g+2, ... < n_kv
             u_other += static_cast<uint32_t>((n_kv + g) >> 1);          // the other warpgroup's: j = g^1, ...
             ++itc;
@@ -509,7 +511,6 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                     if (j + 1 == n_kv) tc_commit(smem_addr(&sh.q_free));
                     if (++sk == NK) { sk = 0; ph_k ^= 1u; }
                 }
-                if (++sk == NK) { sk = 0; ph_k ^= 1u; }       // the ring position of the item's staging tile
                 u[0] += static_cast<uint32_t>((n_kv + 1) >> 1);
                 u[1] += static_cast<uint32_t>(n_kv >> 1);
                 ++itc;
@@ -555,6 +556,7 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                     if (j + 1 == n_kv) tc_commit(smem_addr(&sh.o_final));
                     if (++sv == NV) { sv = 0; ph_v ^= 1u; }
                 }
+                if (++sv == NV) { sv = 0; ph_v ^= 1u; }       // the ring position of the item's staging tile
                 u[0] += static_cast<uint32_t>((n_kv + 1) >> 1);
                 u[1] += static_cast<uint32_t>(n_kv >> 1);
                 ++itc;
@@ -597,8 +599,9 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 }
                 if (it.n_kv == 0) continue;
                 const int n_kv = it.n_kv;
-                // the first K tile goes ahead of Q: its stage is free before the query tile's space is
-                const int ahead = 1;
+                // the first K tiles go ahead of Q: their stages are free before the query tile's space is (the last one
+                // of the ring comes free with it: both were read by the last score MMA of the item before)
+                const int ahead = n_kv < NK - 1 ? n_kv : NK - 1;
                 for (int j = 0; j < ahead && ok; ++j) ok = load_k(it, j);
                 if (!ok) break;
                 // the last score MMA of the item before has read the query tile
@@ -612,17 +615,6 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                         tma_load_4d(sQ + cc * kChunkBytes, &tm_q, bar, cc * kChunkCols, it.i0, it.hq, it.b);
                 }
                 for (int j = ahead; j < n_kv && ok; ++j) ok = load_k(it, j);
-                if (!ok) break;
-                {
-                    // The ring position of the item's staging tile: nothing to load, but the stage's barriers move on
-                    // in step with the positions (a plain arrival completes the phase of k_full that a load would
-                    // have; it may only be made once the stage's previous phase is over, i.e. its tile consumed).
-                    const int s = static_cast<int>(kt % NK);
-                    ok = mbar_wait(smem_addr(&sh.k_empty[s]), ((kt / NK) & 1u) ^ 1u, wctx, kSiteLoadKvEmpty);
-                    if (!ok) break;
-                    mbar_arrive(smem_addr(&sh.k_full[s]));
-                    ++kt;
-                }
                 ++itc;
             }
         }
@@ -650,6 +642,17 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
 #pragma unroll
                     for (int cc = 0; cc < Cfg::kVChunks; ++cc)
                         tma_load_4d(sV + s * Cfg::kVBytes + cc * kChunkBytes, &tm_v, bar, cc * kChunkCols, j * kTileN, it.kvh, it.b);
+                    ++vt;
+                }
+                if (!ok) break;
+                {
+                    // The ring position of the item's staging tile: nothing to load, but the stage's barriers move on
+                    // in step with the positions (a plain arrival completes the phase of v_full that a load would
+                    // have; it may only be made once the stage's previous phase is over, i.e. its tile consumed).
+                    const int s = static_cast<int>(vt % NV);
+                    ok = mbar_wait(smem_addr(&sh.v_empty[s]), ((vt / NV) & 1u) ^ 1u, wctx, kSiteLoadKvEmpty);
+                    if (!ok) break;
+                    mbar_arrive(smem_addr(&sh.v_full[s]));
                     ++vt;
                 }
             }
