@@ -77,8 +77,8 @@ typedef enum fa_status {
  * kernel (one CTA per SM walking a list of items) and everything else on the one-item-per-CTA kernel.  These two flags override the choice where
  * both kernels apply (head sizes 64 and 128, no split-KV); results are bit-identical.  The stream kernel
  * (FA_FLAG_STREAM_KERNEL below) has a persistent form of its own for fixed-length launches with at least three
- * one-tile items per SM of at most 32 K/V tiles each (csrc/fa_fwd_stream_persistent.cuh; any length with
- * FA_FLAG_FORCE_PERSISTENT), under the same two flags and with the same guarantee. */
+ * one-tile items per SM of at most 32 K/V tiles each (csrc/fa_fwd_stream_persistent.cuh; any number and length of
+ * items with FA_FLAG_FORCE_PERSISTENT), under the same two flags and with the same guarantee. */
 #define FA_FLAG_NO_PERSISTENT 8u
 #define FA_FLAG_FORCE_PERSISTENT 16u
 /* A third tiling: one query tile per CTA with its K/V tiles streamed through both softmax

@@ -631,8 +631,8 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
         pl.kernel = kPlanDuo;
         pl.head_pair = head_pair_ok;
     } else if (stream && !varlen && stream_splits == 1 && !(flags & FA_FLAG_NO_PERSISTENT) &&
-               static_cast<long long>(n_q_tiles) * Hq * B >= 3ll * num_sms &&
-               (longest <= 32 || (flags & FA_FLAG_FORCE_PERSISTENT))) {
+               ((static_cast<long long>(n_q_tiles) * Hq * B >= 3ll * num_sms && longest <= 32) ||
+                (flags & FA_FLAG_FORCE_PERSISTENT))) {
         // Many short one-tile items per SM: the stream kernel's persistent form (a CTA's fixed cost once per SM, the
         // next item's loads and first scores under the current item's tail).  Measured on B200 at 192/128 against the
         // one-item stream kernel: +13 % on items of 8 K/V tiles (no mask), +7 % on causal items of up to 16, +2 %
