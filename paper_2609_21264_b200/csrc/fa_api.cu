@@ -635,8 +635,8 @@ LaunchPlan plan_launch(int num_sms, uint32_t flags, uint32_t kv_splits_cfg, size
                 (flags & FA_FLAG_FORCE_PERSISTENT))) {
         // Many short one-tile items per SM: the stream kernel's persistent form (a CTA's fixed cost once per SM, the
         // next item's loads and first scores under the current item's tail).  Measured on B200 at 192/128 against the
-        // one-item stream kernel: +13 % on items of 8 K/V tiles (no mask), +7 % on causal items of up to 16, +2 %
-        // up to 24, level up to 32 (config 4) and on longer items.
+        // one-item stream kernel: +18 % on items of 8 K/V tiles (no mask), +10 % on causal items of up to 16, +4.5 %
+        // up to 24, +2.6 % up to 32 (config 4), within 1 % on longer items.
         pl.kernel = kPlanStreamPersistent;
     } else if (stream) {
         pl.kernel = kPlanStream;

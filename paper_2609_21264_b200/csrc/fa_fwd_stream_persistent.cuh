@@ -27,6 +27,10 @@
 //     space is free as soon as the item's last score MMA is complete (q_free, a commit), and the next item's Q and
 //     first K/V tiles are loaded, and its first scores computed, under the last softmax passes, the last PV products
 //     and the epilogue of the current item.
+//   * the epilogue belongs to the correction warps, which have nothing else to do then (one thread per query row,
+//     as for the rescale): they take the two warpgroups' partial row sums, wait for the item's last PV product, read O
+//     out of TMEM, normalise, stage and store it.  The softmax warps publish their sums and go straight on to the next
+//     item, whose first passes run under the last PV product and the epilogue of this one.
 // Items without a visible key (more queries than keys under a causal mask) have no loads, no MMAs and no barrier
 // traffic: the softmax warps write their zeros and -inf and every role moves on.
 #pragma once
@@ -42,9 +46,10 @@ struct StreamPersistShared {
     uint64_t v_full[4], v_empty[4];
     uint64_t s_full[2], s_free[2], st_full[2], p_ready[2], p_free[2];      // as in StreamShared
     uint64_t o_final;        // PV MMA -> epilogue: the item's last PV product is complete
-    uint64_t o_read;         // softmax warps -> PV MMA: the epilogue has read O out of TMEM
-    uint64_t l_ready;        // softmax warps -> epilogue: partial row sums published
-    uint64_t o_staged;       // softmax warps -> storing thread
+    uint64_t o_read;         // correction warps -> PV MMA: the epilogue has read O out of TMEM
+    uint64_t l_ready;        // softmax warps -> correction warps: partial row sums (and the final u) published
+    uint64_t state_read;     // correction warps -> softmax warps: the epilogue has read them
+    uint64_t o_staged;       // correction warps -> storing thread
     uint64_t item_full[4];   // loader -> every other role: ring slot holds the index of the CTA's next item (-1: none)
     uint64_t item_empty[4];  // the 15 consumers (8 softmax warps, 4 correction warps, 2 MMA threads, V loader) -> loader
     int item_ring[4];
@@ -132,9 +137,10 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
         mbar_init(smem_addr(&sh.q_full), 1);
         mbar_init(smem_addr(&sh.q_free), 1);
         mbar_init(smem_addr(&sh.o_final), 1);
-        mbar_init(smem_addr(&sh.o_read), 8);
+        mbar_init(smem_addr(&sh.o_read), 4);
         mbar_init(smem_addr(&sh.l_ready), 8);
-        mbar_init(smem_addr(&sh.o_staged), 8);
+        mbar_init(smem_addr(&sh.state_read), 4);
+        mbar_init(smem_addr(&sh.o_staged), 4);
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_addr(&sh.s_full[i]), 1);
@@ -197,7 +203,6 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
         const float tau_raw = kRescaleThresholdLog2 / c;
         uint32_t u_own = 0, u_other = 0;      // uses of this warpgroup's / the other one's buffers before the current item
         uint32_t itc = 0;                     // items with K/V tiles finished so far
-        uint32_t vt = 0;                      // V ring positions taken before the current item
         bool ok = true;
 
         for (uint32_t k = 0; ok; ++k) {
@@ -231,10 +236,10 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 continue;
             }
 
-            // every warp has finished the epilogue of the item before (its reads of the row state in shared memory)
-            // before any warp publishes the state of this item's tiles; normally long complete
+            // the epilogue of the item before has read the row state in shared memory before any warp publishes the
+            // state of this item's tiles; normally long complete
             if (itc >= 1u) {
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.o_read), (itc - 1u) & 1u, wctx, kSiteEpiStaged));
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.state_read), (itc - 1u) & 1u, wctx, kSiteEpiState));
                 if (!ok) break;
             }
             float l = 0.f;             // this warpgroup's partial row sum, relative to the current u
@@ -341,82 +346,18 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             }
             if (!ok) break;
 
-            // ---- epilogue of the item: O = G' / s (bf16), lse = u * scale + ln s
-            // (the item is decoded again here instead of keeping its fields in registers through the loop above)
-            StreamItem it;
-            {
-                int idx_again = idx;
-                asm volatile("" : "+r"(idx_again));
-                decode(idx_again, it);
-            }
-            const int i0 = it.i0;
-            const int i_glob = i0 + row;
-            const bool row_valid = i_glob < Sq;
-            const size_t lse_row0 = static_cast<size_t>(it.b * p.Hq + it.hq) * p.Sq;
+            // ---- end of the item: the partial row sum goes to the correction warps, which run the epilogue
             const int last = n_kv - 1;
-            const uint32_t ipar = itc & 1u;
             // The warpgroup that did not run the last tile still has to apply its r.
             if ((last & 1) != g && last >= 1) {
                 const uint32_t use_last = u_other + static_cast<uint32_t>(last >> 1);
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_st_other, use_last & 1u, wctx, kSiteSoftmaxCorrFree));
                 if (ok) l *= sh.alpha[last & 1][row];
             }
-            if (ok) {
-                sh.lsum[g][row] = (g <= last) ? l : 0.f;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_addr(&sh.l_ready));
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.l_ready), ipar, wctx, kSiteEpiStaged));
-            }
-            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.o_final), ipar, wctx, kSiteEpiOFull));
             if (!ok) break;
-            tc_fence_after_sync();
-            const float lt = sh.lsum[0][row] + sh.lsum[1][row];
-            const float m_fin = sh.mref[row];
-            const float inv_l = (lt > 0.f) ? (1.f / lt) : 0.f;
-            if (g == 0 && p.lse && row_valid)
-                p.lse[lse_row0 + i_glob] = (lt > 0.f) ? (m_fin * c * 0.6931471805599453f + logf(lt)) : -INFINITY;
-            // warpgroup g converts columns [g*DV/2, (g+1)*DV/2) of O into the staging tile (the V stage after the
-            // item's last V tile: its previous tile was read by a PV product that is complete), then one thread
-            // stores it with TMA; rows past Sq are clipped
-            const uint32_t tO = tmem_base + Cfg::kColO + lane_sel;
-            const int s_stage = static_cast<int>((vt + static_cast<uint32_t>(n_kv)) % NV);
-            const uint32_t s_tile = sV + s_stage * Cfg::kVBytes;
-            const uint32_t sO = s_tile + row * 128;
-#pragma unroll 1
-            for (int cc = g * (DV / 64); cc < (g + 1) * (DV / 64); ++cc) {
-                uint32_t r[32];
-                tmem_ld_x32(tO + cc * 32, r);
-                tc_wait_ld();
-                const uint32_t chunk = sO + (cc >> 1) * kChunkBytes;
-#pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    const uint32_t piece = static_cast<uint32_t>(((cc & 1) * 4 + v) ^ (row & 7)) << 4;
-                    st_shared_v4(chunk + piece,
-                                 pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
-                                 pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
-                                 pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
-                                 pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
-                }
-            }
-            // O is out of TMEM: the next item's first PV product may overwrite it
-            tc_fence_before_sync();
-            fence_proxy_async_smem();
+            sh.lsum[g][row] = (g <= last) ? l : 0.f;
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(smem_addr(&sh.o_read));
-                mbar_arrive(smem_addr(&sh.o_staged));
-            }
-            if (warp == 0 && lane == 0) {
-                if (mbar_wait(smem_addr(&sh.o_staged), ipar, wctx, kSiteEpiStaged)) {
-#pragma unroll
-                    for (int ch = 0; ch < DV / kChunkCols; ++ch)
-                        tma_store_4d(&tm_o, s_tile + ch * kChunkBytes, ch * kChunkCols, i0, it.hq, it.b);
-                    tma_store_commit();
-                    tma_store_wait_read_all();     // the staging tile goes back to the V ring
-                    mbar_arrive(smem_addr(&sh.v_empty[s_stage]));
-                }
-            }
-            vt += static_cast<uint32_t>(n_kv) + 1u;
+            if (lane == 0) mbar_arrive(smem_addr(&sh.l_ready));
             u_own += static_cast<uint32_t>((n_kv + 1 - g) >> 1);        // tiles j = g, g+2, ... < n_kv
             u_other += static_cast<uint32_t>((n_kv + g) >> 1);          // the other warpgroup's: j = g^1, ...
             ++itc;
@@ -428,6 +369,7 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tO = tmem_base + Cfg::kColO + lane_sel;
         uint32_t u[2] = {0u, 0u};             // uses of buffer pair 0 / 1 before the current item
+        uint32_t vt = 0, itc = 0;             // V ring positions taken and items finished before the current item
         bool ok = true;
         for (uint32_t k = 0; ok; ++k) {
             int idx = item_wait(k);
@@ -466,6 +408,66 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_addr(&sh.p_ready[j & 1]));
             }
+            if (!ok) break;
+
+            // ---- epilogue of the item: O = G' / s (bf16), lse = u * scale + ln s
+            const uint32_t ipar = itc & 1u;
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.l_ready), ipar, wctx, kSiteEpiStaged));
+            if (!ok) break;
+            const float lt = sh.lsum[0][row] + sh.lsum[1][row];
+            const float m_fin = sh.mref[row];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_addr(&sh.state_read));        // the softmax warps may publish the next item's state
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.o_final), ipar, wctx, kSiteEpiOFull));
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int i_glob = it.i0 + row;
+            const float inv_l = (lt > 0.f) ? (1.f / lt) : 0.f;
+            if (p.lse && i_glob < Sq)
+                p.lse[static_cast<size_t>(it.b * p.Hq + it.hq) * p.Sq + i_glob] =
+                    (lt > 0.f) ? (m_fin * c * 0.6931471805599453f + logf(lt)) : -INFINITY;
+            // O goes into the staging tile (the V stage after the item's last V tile: its previous tile was read by a PV
+            // product that is complete), then one thread stores it with TMA; rows past Sq are clipped
+            const int s_stage = static_cast<int>((vt + static_cast<uint32_t>(n_kv)) % NV);
+            const uint32_t s_tile = sV + s_stage * Cfg::kVBytes;
+            const uint32_t sO = s_tile + row * 128;
+#pragma unroll 1
+            for (int cc = 0; cc < DV / 32; ++cc) {
+                uint32_t r[32];
+                tmem_ld_x32(tO + cc * 32, r);
+                tc_wait_ld();
+                const uint32_t chunk = sO + (cc >> 1) * kChunkBytes;
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    const uint32_t piece = static_cast<uint32_t>(((cc & 1) * 4 + v) ^ (row & 7)) << 4;
+                    st_shared_v4(chunk + piece,
+                                 pack_bf16x2(__uint_as_float(r[8 * v]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l),
+                                 pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l),
+                                 pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l),
+                                 pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l));
+                }
+            }
+            // O is out of TMEM: the next item's first PV product may overwrite it
+            tc_fence_before_sync();
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(smem_addr(&sh.o_read));
+                mbar_arrive(smem_addr(&sh.o_staged));
+            }
+            if (warp == 8 && lane == 0) {
+                if (mbar_wait(smem_addr(&sh.o_staged), ipar, wctx, kSiteEpiStaged)) {
+#pragma unroll
+                    for (int ch = 0; ch < DV / kChunkCols; ++ch)
+                        tma_store_4d(&tm_o, s_tile + ch * kChunkBytes, ch * kChunkCols, it.i0, it.hq, it.b);
+                    tma_store_commit();
+                    tma_store_wait_read_all();     // the staging tile goes back to the V ring
+                    mbar_arrive(smem_addr(&sh.v_empty[s_stage]));
+                }
+            }
+            __syncwarp();
+            vt += static_cast<uint32_t>(n_kv) + 1u;
+            ++itc;
             u[0] += static_cast<uint32_t>((n_kv + 1) >> 1);
             u[1] += static_cast<uint32_t>(n_kv >> 1);
         }
