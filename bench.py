@@ -48,7 +48,7 @@ NCU_DRAM_BYTES_PER_LAUNCH = {
     "bert_base_mha_s512": 2.42e6 + 0.0,
     "llama3_8b_gqa_s2048": 25.23e6 + 0.0,
     "llama2_7b_mha_b4_s8192": 923.00e6 + 253.69e6,
-    "deepseek_v2_mha_s4096_d192_128": 571.05e6 + 122.52e6,
+    "deepseek_v2_mha_s4096_d192_128": 569.05e6 + 121.60e6,
     "long_context_gqa_s131072": 3.14e9 + 1.06e9,
 }
 
