@@ -63,3 +63,37 @@ def test_persistent_stream_kernel_matches_the_oracle_and_the_one_item_kernel(w):
     finally:
         assert binding.fa_destroy(h) == binding.FA_OK
         assert binding.fa_destroy(h1) == binding.FA_OK
+
+
+def test_back_to_back_launches_of_varied_shapes_equal_the_one_item_kernel():
+    """Hundreds of launches through one handle without a synchronisation in between, shapes changing every 25 launches
+    (the ticket counter and the tensor-map cache carry over): every result equals the one-item kernel's bit for bit
+    and no wait runs out."""
+    import random
+    import torch
+    from paper_2609_21264_b200 import binding
+    rnd = random.Random(2310)
+    h = binding.fa_create(wait_limit_ms=2000)
+    h1 = binding.fa_create(flags=binding.FA_FLAG_NO_PERSISTENT, wait_limit_ms=2000)
+    try:
+        gen = torch.Generator(device="cuda").manual_seed(2310)
+        persistent = 0
+        for it in range(12):
+            B, H = rnd.choice([1, 2, 4]), rnd.choice([32, 64, 128])
+            S = rnd.choice([384, 512, 1024, 1536, 2048, 3072])
+            Sk = S + rnd.choice([0, 0, 128, 700])
+            causal = rnd.random() < 0.7
+            q = torch.randn((B, H, S, 192), generator=gen, device="cuda").bfloat16()
+            k = torch.randn((B, H, Sk, 192), generator=gen, device="cuda").bfloat16()
+            v = torch.randn((B, H, Sk, 128), generator=gen, device="cuda").bfloat16()
+            o_ref, l_ref = binding.forward(h1, q, k, v, causal=causal)
+            for _ in range(25):
+                o, l = binding.forward(h, q, k, v, causal=causal)
+            torch.cuda.synchronize()
+            assert binding.fa_last_status(h) == (binding.FA_OK, 0)
+            persistent += binding.fa_last_kernel_name(h) == "fa_fwd_stream_persistent"
+            assert torch.equal(o, o_ref) and torch.equal(l, l_ref), (it, B, H, S, Sk, causal)
+        assert persistent >= 4          # the draw reaches the kernel this test is about
+    finally:
+        assert binding.fa_destroy(h) == binding.FA_OK
+        assert binding.fa_destroy(h1) == binding.FA_OK
