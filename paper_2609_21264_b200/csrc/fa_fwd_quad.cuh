@@ -36,14 +36,8 @@
 namespace fa {
 
 namespace ptx {
-// Arrive (count 1) on the mbarrier at this shared-memory offset in BOTH CTAs of the pair once every tcgen05
-// operation issued so far by this thread has completed (one instruction; its cost to the issuing thread is
-// about that of an MMA, so the loop uses as few as it can).
-FA_DEVI void tc_commit_pair_both(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
-}
-// The same on this CTA's barrier only.
+// Arrive (count 1) on this CTA's barrier only once every tcgen05 operation issued so far by this thread has completed
+// (the two-CTA form of the commit; ptx::tc_commit_2cta signals the barrier at the same offset in both CTAs).
 FA_DEVI void tc_commit_pair_local(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -291,7 +285,7 @@ fa_fwd_quad_kernel(const __grid_constant__ CUtensorMap tm_q,
             // k-step k of a query tile (chunks of 128 rows) and of this CTA's half of K (chunks of 64 rows)
             auto qoff = [](int k) -> uint32_t { return static_cast<uint32_t>(((k / 4) * kChunkBytes + (k % 4) * 32) >> 4); };
             auto koff = [](int k) -> uint32_t { return static_cast<uint32_t>(((k / 4) * Cfg::kKHalfChunkBytes + (k % 4) * 32) >> 4); };
-            auto commit_all = [](uint32_t bar) { tc_commit_pair_both(bar); };
+            auto commit_all = [](uint32_t bar) { tc_commit_2cta(bar, mapa_shared(bar, 1u)); };
             // a barrier whose phase 0 completed long ago and which never moves again: filler for unused probe slots
             const uint32_t bar_always = smem_addr(&sh.q_full[nkv_0 > 0 ? 0 : 1]);
 
