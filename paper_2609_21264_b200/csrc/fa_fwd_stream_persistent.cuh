@@ -14,9 +14,11 @@
 // shared memory (item_full / item_empty).
 //
 // What carries over from item to item:
-//   * every mbarrier keeps running: a role tracks how often each S/P buffer pair has been used (tile j of an item
-//     uses buffer j & 1, so an item with an odd number of tiles leaves the two counts one apart), how many K and V
-//     tiles have gone through the rings, and how many items it has finished;
+//   * every mbarrier keeps running: a role counts the K/V tiles of all its items (tile j of an item whose
+//     predecessors had T tiles is tile T + j of the CTA: it uses S/P buffer pair (T + j) & 1, for the
+//     ((T + j) >> 1)-th time, and belongs to softmax warpgroup (T + j) & 1, so that the two warpgroups keep
+//     alternating across items with odd numbers of tiles and an item's first tile goes to the warpgroup that did not
+//     run the last tile of the item before), the ring positions of K and V, and the items it has finished;
 //   * the O accumulator: the first PV product of an item (accumulate = 0) waits until the epilogue of the item before
 //     has read O out of TMEM (o_read);
 //   * the output is staged for its TMA store in a stage of the V ring (an O tile is exactly as large as a V tile): every
@@ -201,7 +203,7 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
         const uint32_t bar_pr = smem_addr(&sh.p_ready[g]);
         const uint32_t bar_pf = smem_addr(&sh.p_free[g]);
         const float tau_raw = kRescaleThresholdLog2 / c;
-        uint32_t u_own = 0, u_other = 0;      // uses of this warpgroup's / the other one's buffers before the current item
+        uint32_t T = 0;                       // K/V tiles of the items before the current one
         uint32_t itc = 0;                     // items with K/V tiles finished so far
         bool ok = true;
 
@@ -243,8 +245,8 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 if (!ok) break;
             }
             float l = 0.f;             // this warpgroup's partial row sum, relative to the current u
-            for (int j = g; j < n_kv; j += 2) {
-                const uint32_t use = u_own + static_cast<uint32_t>(j >> 1);      // n-th use of this warpgroup's buffers
+            for (int j = static_cast<int>((static_cast<uint32_t>(g) ^ T) & 1u); j < n_kv; j += 2) {      // tiles with (T + j) & 1 == g
+                const uint32_t use = (T + static_cast<uint32_t>(j)) >> 1;       // n-th use of this warpgroup's buffers
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_s, use & 1u, wctx, kSiteSoftmaxSFull));
                 if (!ok) break;
                 tc_fence_after_sync();
@@ -281,11 +283,11 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 // Row state of tile j-1 (the other warpgroup's): u, and the factor r it applied.
                 float m_ref = -INFINITY, r_prev = 1.f;
                 if (j > 0) {
-                    const uint32_t use_prev = u_other + static_cast<uint32_t>((j - 1) >> 1);
+                    const uint32_t use_prev = (T + static_cast<uint32_t>(j - 1)) >> 1;
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_st_other, use_prev & 1u, wctx, kSiteSoftmaxCorrFree));
                     if (!ok) break;
                     m_ref = sh.mref[row];
-                    r_prev = sh.alpha[(j - 1) & 1][row];
+                    r_prev = sh.alpha[g ^ 1][row];
                 }
                 // P^g and the slot of this tile's r are reused: the PV MMA of the buffer's previous use (two tiles
                 // ago, or in the item before) must be complete, which also means that the correction warps have
@@ -300,7 +302,7 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                     m_ref = mx;
                 }
                 sh.mref[row] = m_ref;
-                sh.alpha[j & 1][row] = alpha;
+                sh.alpha[g][row] = alpha;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_st);
 
@@ -349,17 +351,17 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             // ---- end of the item: the partial row sum goes to the correction warps, which run the epilogue
             const int last = n_kv - 1;
             // The warpgroup that did not run the last tile still has to apply its r.
-            if ((last & 1) != g && last >= 1) {
-                const uint32_t use_last = u_other + static_cast<uint32_t>(last >> 1);
+            const int g_last = static_cast<int>((T + static_cast<uint32_t>(last)) & 1u);      // the warpgroup of the last tile
+            if (g_last != g && last >= 1) {
+                const uint32_t use_last = (T + static_cast<uint32_t>(last)) >> 1;
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_st_other, use_last & 1u, wctx, kSiteSoftmaxCorrFree));
-                if (ok) l *= sh.alpha[last & 1][row];
+                if (ok) l *= sh.alpha[g_last][row];
             }
             if (!ok) break;
-            sh.lsum[g][row] = (g <= last) ? l : 0.f;
+            sh.lsum[g][row] = (last >= 1 || g_last == g) ? l : 0.f;       // (a single tile belongs to one warpgroup only)
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_addr(&sh.l_ready));
-            u_own += static_cast<uint32_t>((n_kv + 1 - g) >> 1);        // tiles j = g, g+2, ... < n_kv
-            u_other += static_cast<uint32_t>((n_kv + g) >> 1);          // the other warpgroup's: j = g^1, ...
+            T += static_cast<uint32_t>(n_kv);
             ++itc;
         }
     } else if (warp < 12) {
@@ -368,7 +370,7 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
         const int row = tid & (kTileM - 1);
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tO = tmem_base + Cfg::kColO + lane_sel;
-        uint32_t u[2] = {0u, 0u};             // uses of buffer pair 0 / 1 before the current item
+        uint32_t T = 0;                       // K/V tiles of the items before the current one
         uint32_t vt = 0, itc = 0;             // V ring positions taken and items finished before the current item
         bool ok = true;
         for (uint32_t k = 0; ok; ++k) {
@@ -382,14 +384,14 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             if (it.n_kv == 0) continue;
             const int n_kv = it.n_kv;
             for (int j = 0; j < n_kv && ok; ++j) {
-                const uint32_t use = u[j & 1] + static_cast<uint32_t>(j >> 1);
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.st_full[j & 1]), use & 1u, wctx, kSiteCorrScale));
+                const uint32_t gj = T + static_cast<uint32_t>(j), bsel = gj & 1u, use = gj >> 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.st_full[bsel]), use & 1u, wctx, kSiteCorrScale));
                 if (!ok) break;
-                const float alpha = sh.alpha[j & 1][row];
+                const float alpha = sh.alpha[bsel][row];
                 if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
                     // O must hold the complete sum up to tile j-1 before it is rescaled
-                    const uint32_t use_prev = u[(j - 1) & 1] + static_cast<uint32_t>((j - 1) >> 1);
-                    ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.p_free[(j - 1) & 1]), use_prev & 1u, wctx, kSiteCorrPvDone));
+                    const uint32_t use_prev = (gj - 1u) >> 1;
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.p_free[bsel ^ 1u]), use_prev & 1u, wctx, kSiteCorrPvDone));
                     if (!ok) break;
                     tc_fence_after_sync();
 #pragma unroll 1
@@ -406,7 +408,7 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                     tc_fence_before_sync();
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_addr(&sh.p_ready[j & 1]));
+                if (lane == 0) mbar_arrive(smem_addr(&sh.p_ready[bsel]));
             }
             if (!ok) break;
 
@@ -468,8 +470,7 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             __syncwarp();
             vt += static_cast<uint32_t>(n_kv) + 1u;
             ++itc;
-            u[0] += static_cast<uint32_t>((n_kv + 1) >> 1);
-            u[1] += static_cast<uint32_t>(n_kv >> 1);
+            T += static_cast<uint32_t>(n_kv);
         }
     } else if (warp == 12) {
         // ============================================================ score MMAs: S^(j&1) = Q K_j^T
@@ -480,7 +481,7 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             const uint32_t q_lo = ((sQ & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
             auto desc = [](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(kDescHi) << 32) | lo; };
-            uint32_t u[2] = {0u, 0u};
+            uint32_t T = 0;
             uint32_t itc = 0;
             int sk = 0;
             uint32_t ph_k = 0;
@@ -495,26 +496,25 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 const int n_kv = it.n_kv;
                 ok = mbar_wait(smem_addr(&sh.q_full), itc & 1u, wctx, kSiteMmaQFull);
                 for (int j = 0; j < n_kv && ok; ++j) {
-                    const uint32_t use = u[j & 1] + static_cast<uint32_t>(j >> 1);
+                    const uint32_t gj = T + static_cast<uint32_t>(j), bsel = gj & 1u, use = gj >> 1;
                     ok = mbar_wait(smem_addr(&sh.k_full[sk]), ph_k, wctx, kSiteMmaKvFull);
                     // the softmax warps have read the buffer's previous S (two tiles ago, or in the item before)
-                    if (ok && use >= 1u) ok = mbar_wait(smem_addr(&sh.s_free[j & 1]), (use - 1u) & 1u, wctx, kSiteMmaSFree);
+                    if (ok && use >= 1u) ok = mbar_wait(smem_addr(&sh.s_free[bsel]), (use - 1u) & 1u, wctx, kSiteMmaSFree);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t tS = tmem_base + Cfg::kColS + (j & 1) * 128;
+                    const uint32_t tS = tmem_base + Cfg::kColS + bsel * 128;
                     const uint32_t klo = k_lo0 + sk * (Cfg::kKBytes >> 4);
 #pragma unroll
                     for (int k = 0; k < DQK / 16; ++k) {
                         const uint32_t koff = ((k / 4) * kChunkBytes + (k % 4) * 32) >> 4;
                         mma_ss(tS, desc(q_lo + koff), desc(klo + koff), kIdescQK, k > 0 ? 1u : 0u);
                     }
-                    tc_commit(smem_addr(&sh.s_full[j & 1]));
+                    tc_commit(smem_addr(&sh.s_full[bsel]));
                     tc_commit(smem_addr(&sh.k_empty[sk]));
                     if (j + 1 == n_kv) tc_commit(smem_addr(&sh.q_free));
                     if (++sk == NK) { sk = 0; ph_k ^= 1u; }
                 }
-                u[0] += static_cast<uint32_t>((n_kv + 1) >> 1);
-                u[1] += static_cast<uint32_t>(n_kv >> 1);
+                T += static_cast<uint32_t>(n_kv);
                 ++itc;
             }
         }
@@ -527,7 +527,7 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
             const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((static_cast<uint32_t>(kChunkBytes) >> 4) << 16);
             const uint32_t tO = tmem_base + Cfg::kColO;
             auto desc = [](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(kDescHi) << 32) | lo; };
-            uint32_t u[2] = {0u, 0u};
+            uint32_t T = 0;
             uint32_t itc = 0;
             int sv = 0;
             uint32_t ph_v = 0;
@@ -543,24 +543,23 @@ fa_fwd_stream_persistent_kernel(const __grid_constant__ CUtensorMap tm_q,
                 // the epilogue of the item before has read O out of TMEM
                 if (itc >= 1u) ok = mbar_wait(smem_addr(&sh.o_read), (itc - 1u) & 1u, wctx, kSiteMmaSFree);
                 for (int j = 0; j < n_kv && ok; ++j) {
-                    const uint32_t use = u[j & 1] + static_cast<uint32_t>(j >> 1);
+                    const uint32_t gj = T + static_cast<uint32_t>(j), bsel = gj & 1u, use = gj >> 1;
                     ok = mbar_wait(smem_addr(&sh.v_full[sv]), ph_v, wctx, kSiteMmaKvFull);
-                    if (ok) ok = mbar_wait(smem_addr(&sh.p_ready[j & 1]), use & 1u, wctx, kSiteMmaPFull);
+                    if (ok) ok = mbar_wait(smem_addr(&sh.p_ready[bsel]), use & 1u, wctx, kSiteMmaPFull);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t tP = tmem_base + Cfg::kColP + (j & 1) * 64;
+                    const uint32_t tP = tmem_base + Cfg::kColP + bsel * 64;
                     const uint32_t vlo = v_lo0 + sv * (Cfg::kVBytes >> 4);
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
                         mma_ts(tO, tP + kk * 8, desc(vlo + kk * (2048 >> 4)), kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
-                    tc_commit(smem_addr(&sh.p_free[j & 1]));
+                    tc_commit(smem_addr(&sh.p_free[bsel]));
                     tc_commit(smem_addr(&sh.v_empty[sv]));
                     if (j + 1 == n_kv) tc_commit(smem_addr(&sh.o_final));
                     if (++sv == NV) { sv = 0; ph_v ^= 1u; }
                 }
                 if (++sv == NV) { sv = 0; ph_v ^= 1u; }       // the ring position of the item's staging tile
-                u[0] += static_cast<uint32_t>((n_kv + 1) >> 1);
-                u[1] += static_cast<uint32_t>(n_kv >> 1);
+                T += static_cast<uint32_t>(n_kv);
                 ++itc;
             }
         }
